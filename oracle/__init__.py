@@ -1,0 +1,216 @@
+"""fp64 CPU oracle for the Cool-SD verify-and-resample round -- TEST INFRASTRUCTURE.
+
+A thin ``ctypes`` wrapper around ``csd_oracle.c`` (plain C, fp64).  Only the
+tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package; the product (``paper_2601_09212_b200``) never does, and this package
+never imports the product.
+
+The wrapper does marshalling only; all arithmetic lives in the C file, which
+cites the passages of the paper it follows (Algorithm 1, Eq. relax, Eq. sdar,
+Eq. opt_G).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "csd_oracle.c")
+_LIB = os.path.join(_HERE, "libcsd_oracle.so")
+
+F32, BF16, F64 = 0, 1, 2
+STATUS_BADROW, STATUS_BADTOKEN, STATUS_ZFALLBACK = 1, 2, 4
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP on, no fast-math, no contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
+               "-fno-fast-math", "-Wall", "-Wextra", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+class _Params(C.Structure):
+    _fields_ = [
+        ("target_logits", C.c_void_p), ("draft_logits", C.c_void_p),
+        ("target_uncond", C.c_void_p), ("draft_uncond", C.c_void_p),
+        ("dtype", C.c_int32), ("cfg_scale", C.c_float), ("top_k", C.c_int32),
+        ("B", C.c_int32), ("gamma", C.c_int32), ("V", C.c_int32), ("target_rows", C.c_int32),
+        ("target_batch_stride", C.c_int64), ("draft_batch_stride", C.c_int64),
+        ("draft_tokens", C.c_void_p), ("uniforms", C.c_void_p), ("relax_schedule", C.c_void_p),
+        ("out_tokens", C.c_void_p), ("out_accept_len", C.c_void_p), ("out_status", C.c_void_p),
+        ("p", C.c_void_p), ("q", C.c_void_p), ("f", C.c_void_p), ("G", C.c_void_p),
+        ("margin_accept", C.c_void_p), ("margin_cdf", C.c_void_p),
+    ]
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        lib = C.CDLL(_LIB)
+        lib.orc_num_threads.restype = C.c_int
+        lib.orc_set_num_threads.argtypes = [C.c_int]
+        lib.orc_make_schedule.argtypes = [C.c_int, C.c_double, C.c_double, C.c_int, C.c_void_p]
+        lib.orc_make_schedule.restype = C.c_int
+        lib.orc_accept_prob.argtypes = [C.c_double, C.c_double, C.c_double]
+        lib.orc_accept_prob.restype = C.c_double
+        lib.orc_softmax.argtypes = [C.c_void_p, C.c_int, C.c_void_p]
+        lib.orc_softmax.restype = C.c_int
+        lib.orc_resample_weights.argtypes = [C.c_void_p, C.c_void_p, C.c_double, C.c_int, C.c_void_p]
+        lib.orc_resample_weights.restype = C.c_double
+        lib.orc_resample_dist.argtypes = [C.c_void_p, C.c_void_p, C.c_double, C.c_int, C.c_void_p]
+        lib.orc_resample_dist.restype = C.c_double
+        lib.orc_inverse_cdf.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_void_p]
+        lib.orc_inverse_cdf.restype = C.c_int
+        lib.orc_prepare_row.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int,
+                                        C.c_float, C.c_int, C.c_void_p, C.c_void_p]
+        lib.orc_prepare_row.restype = None
+        lib.orc_verify.argtypes = [C.POINTER(_Params)]
+        lib.orc_verify.restype = C.c_int
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().orc_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    _load().orc_set_num_threads(int(n))
+
+
+def _f64(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def make_schedule(kind: int, delta: float, nu_or_ell: float, L: int) -> np.ndarray:
+    """omega_1..omega_L; kind 0 uniform, 1 exponential (Eq. sdar), 2 linear."""
+    out = np.empty(max(L, 0), dtype=np.float64)
+    rc = _load().orc_make_schedule(int(kind), float(delta), float(nu_or_ell), int(L), _ptr(out))
+    if rc != 0:
+        raise ValueError("orc_make_schedule: bad arguments")
+    return out
+
+
+def accept_prob(p: float, q: float, omega: float) -> float:
+    """Eq. relax at one token."""
+    return float(_load().orc_accept_prob(float(p), float(q), float(omega)))
+
+
+def softmax(z) -> Optional[np.ndarray]:
+    z = _f64(z)
+    P = np.empty_like(z)
+    ok = _load().orc_softmax(_ptr(z), int(z.size), _ptr(P))
+    return P if ok else None
+
+
+def resample_weights(P, Q, omega: float):
+    """Unnormalised Eq. opt_G and its total Z."""
+    P, Q = _f64(P), _f64(Q)
+    g = np.empty_like(P)
+    Z = _load().orc_resample_weights(_ptr(P), _ptr(Q), float(omega), int(P.size), _ptr(g))
+    return g, float(Z)
+
+
+def resample_dist(P, Q, omega: float) -> np.ndarray:
+    """Eq. opt_G (falls back to P when the positive part is empty)."""
+    P, Q = _f64(P), _f64(Q)
+    G = np.empty_like(P)
+    _load().orc_resample_dist(_ptr(P), _ptr(Q), float(omega), int(P.size), _ptr(G))
+    return G
+
+
+def inverse_cdf(g, Z: float, u: float):
+    g = _f64(g)
+    margin = C.c_double(0.0)
+    tok = _load().orc_inverse_cdf(_ptr(g), int(g.size), float(Z), float(u), C.byref(margin))
+    return int(tok), float(margin.value)
+
+
+def _raw(a: np.ndarray, dtype: int) -> np.ndarray:
+    """Stored logits as the bytes the C side reads (bf16 travels as uint16)."""
+    want = {F32: np.float32, BF16: np.uint16, F64: np.float64}[dtype]
+    a = np.ascontiguousarray(a)
+    if a.dtype != want:
+        raise TypeError(f"logits must be {want} for dtype code {dtype}, got {a.dtype}")
+    return a
+
+
+def prepare_row(cond, uncond, dtype: int, cfg_scale: float, top_k: int) -> np.ndarray:
+    cond = _raw(cond, dtype)
+    un = None if uncond is None else _raw(uncond, dtype)
+    V = int(cond.size)
+    z = np.empty(V, dtype=np.float64)
+    scratch = np.empty(V, dtype=np.float64)
+    _load().orc_prepare_row(_ptr(cond), _ptr(un), int(dtype), 0, V, float(cfg_scale), int(top_k),
+                            _ptr(z), _ptr(scratch))
+    return z
+
+
+@dataclass
+class VerifyResult:
+    tokens: np.ndarray        # [B, gamma+1] int32, -1 padded
+    accept_len: np.ndarray    # [B] int32
+    status: np.ndarray        # [B] int32
+    p: np.ndarray             # [B, gamma] float64
+    q: np.ndarray
+    f: np.ndarray
+    G: Optional[np.ndarray]   # [B, V] float64 (distribution drawn from; zeros if none)
+    margin_accept: np.ndarray  # [B, gamma]
+    margin_cdf: np.ndarray     # [B]
+
+
+def verify(target_logits, draft_logits, draft_tokens, uniforms, relax_schedule, *,
+           dtype: int = F32, target_uncond=None, draft_uncond=None, cfg_scale: float = 1.0,
+           top_k: int = 0, want_G: bool = True, want_pqf: bool = True) -> VerifyResult:
+    """One verification round for B sequences (Algorithm 1, verification stage).
+
+    target_logits [B, T, V] with T in {gamma, gamma+1}; draft_logits [B, gamma, V];
+    draft_tokens [B, gamma] int32; uniforms [B, gamma+1] float32 (columns
+    0..gamma-1 are r_i, column gamma is the resample / bonus draw);
+    relax_schedule [gamma] float32.
+    """
+    t = _raw(target_logits, dtype)
+    d = _raw(draft_logits, dtype)
+    B, T, V = t.shape
+    gamma = d.shape[1]
+    assert d.shape == (B, gamma, V) and T in (gamma, gamma + 1)
+    tu = None if target_uncond is None else _raw(target_uncond, dtype)
+    du = None if draft_uncond is None else _raw(draft_uncond, dtype)
+    if (tu is None) != (du is None):
+        raise ValueError("guidance needs both unconditional arrays")
+    tok = np.ascontiguousarray(draft_tokens, dtype=np.int32)
+    uni = np.ascontiguousarray(uniforms, dtype=np.float32)
+    om = np.ascontiguousarray(relax_schedule, dtype=np.float32)
+    assert tok.shape == (B, gamma) and uni.shape == (B, gamma + 1) and om.shape == (gamma,)
+    res = VerifyResult(
+        tokens=np.empty((B, gamma + 1), np.int32), accept_len=np.empty(B, np.int32),
+        status=np.zeros(B, np.int32),
+        p=np.empty((B, gamma)), q=np.empty((B, gamma)), f=np.empty((B, gamma)),
+        G=np.zeros((B, V)) if want_G else None,
+        margin_accept=np.empty((B, gamma)), margin_cdf=np.empty(B))
+    prm = _Params(
+        _ptr(t), _ptr(d), _ptr(tu), _ptr(du), int(dtype), float(cfg_scale), int(top_k),
+        B, gamma, V, T, T * V, gamma * V, _ptr(tok), _ptr(uni), _ptr(om),
+        _ptr(res.tokens), _ptr(res.accept_len), _ptr(res.status),
+        _ptr(res.p) if want_pqf else None, _ptr(res.q) if want_pqf else None,
+        _ptr(res.f) if want_pqf else None, _ptr(res.G),
+        _ptr(res.margin_accept), _ptr(res.margin_cdf))
+    rc = _load().orc_verify(C.byref(prm))
+    if rc != 0:
+        raise RuntimeError(f"orc_verify failed with code {rc}")
+    return res

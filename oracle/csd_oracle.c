@@ -1,0 +1,429 @@
+/*
+ * csd_oracle.c -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * A plain, slow, fp64 CPU statement of one verification round of relaxed
+ * speculative decoding with annealed relaxation (Cool-SD): Algorithm 1 of the
+ * paper (verification stage), the relaxed acceptance probability (Eq. relax),
+ * the annealing schedules (UniformRSD, Eq. sdar, and the linear variant of the
+ * schedule ablation), and the bound-minimising resampling distribution
+ * (Eq. opt_G, Theorem 2 / Proposition LP).
+ *
+ * It shares no code with the CUDA library.  Only the tests, the smoke check and
+ * the benchmark's CPU-baseline leg may call it.  Everything is written as the
+ * paper writes it: one sequence at a time, a sequential for/break over the
+ * draft positions, full V-length distributions formed explicitly.  There is no
+ * blocking, fusion or reordering.  OpenMP (if compiled in) only runs different
+ * sequences on different cores.
+ *
+ * Readings of points the paper leaves open (each is the build's choice and is
+ * mirrored, not shared, by the CUDA side):
+ *   - index base of the schedule: i = 1..L (Eq. sdar is stated for i in [L]).
+ *   - 0/0 := 1 (Notations appendix): q = 0 gives f = 1; p = 0 < q gives f = 0.
+ *   - G* is always Eq. opt_G, Norm([P - Q f]_+), also where omega_i < 1.
+ *   - sampling from G* is by inverse CDF in token-id order with ONE supplied
+ *     uniform u per sequence: smallest x with C(x) > u*Z; if rounding leaves no
+ *     such x, the last x with positive mass.
+ *   - Z = 0 (only when P == Q and omega >= 1): fall back to G := P.
+ *   - the bonus token (tau = L) uses the same u and needs an (L+1)-th target
+ *     row; without it the slot is -1.
+ *   - guidance mix (not in the paper's verify step; an input-preparation
+ *     reading): z = fmaf(s, c - u, u) evaluated in fp32, then everything in fp64.
+ *   - top-k (not in the paper): keep every logit >= the k-th largest of the row.
+ *   - rows holding NaN or +inf, or with no finite entry, are "invalid": the
+ *     position rejects (f := 0); an invalid drafter row resamples from P (the
+ *     value of Eq. opt_G at f = 0); an invalid target row emits -1.
+ *   - a draft token outside [0, V) rejects (f := 0) and is flagged.
+ *
+ * Pins (tests/test_oracle_*.py): Theorem 1 by exact enumeration and chi-square,
+ * Theorem 2's expectation and TV bound by brute force on tiny alphabets,
+ * Proposition LP's closed form against random and grid search over G,
+ * Proposition 2, the schedule's normalisation, and textbook routines
+ * (log-sum-exp, partition, cumsum/searchsorted) for the building blocks.
+ * Parity unpinned: nothing -- the paper prints no worked numeric example, so
+ * there is no printed value to pin to; every function has an analytic pin.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORC_F32 0
+#define ORC_BF16 1
+#define ORC_F64 2
+
+#define ORC_STATUS_BADROW 1
+#define ORC_STATUS_BADTOKEN 2
+#define ORC_STATUS_ZFALLBACK 4
+
+typedef struct {
+  const void *target_logits; /* [B, target_rows, V] (batch stride below) */
+  const void *draft_logits;  /* [B, gamma, V] */
+  const void *target_uncond; /* NULL: no guidance mix */
+  const void *draft_uncond;
+  int32_t dtype; /* ORC_F32 / ORC_BF16 / ORC_F64 */
+  float cfg_scale;
+  int32_t top_k; /* 0: off */
+  int32_t B, gamma, V, target_rows;
+  int64_t target_batch_stride, draft_batch_stride; /* in elements */
+  const int32_t *draft_tokens; /* [B, gamma] */
+  const float *uniforms;       /* [B, gamma+1] */
+  const float *relax_schedule; /* [gamma] omega_i */
+  int32_t *out_tokens;         /* [B, gamma+1] */
+  int32_t *out_accept_len;     /* [B] */
+  int32_t *out_status;         /* [B] or NULL */
+  double *p, *q, *f;           /* [B, gamma] or NULL: all positions, for comparison */
+  double *G;                   /* [B, V] or NULL: distribution drawn from */
+  double *margin_accept;       /* [B, gamma] or NULL: |r_i - f_i| where the test ran, else +inf */
+  double *margin_cdf;          /* [B] or NULL: distance of u to the nearest CDF boundary of the pick */
+} orc_params;
+
+int orc_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+void orc_set_num_threads(int n) {
+#ifdef _OPENMP
+  if (n > 0) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
+
+/* ---- stored value -> the fp32 value it encodes ---------------------------- */
+static float bf16_to_float(uint16_t h) {
+  uint32_t w = ((uint32_t)h) << 16;
+  float f;
+  memcpy(&f, &w, sizeof f);
+  return f;
+}
+
+static double load_value(const void *base, int dtype, int64_t idx) {
+  if (dtype == ORC_F32) return (double)((const float *)base)[idx];
+  if (dtype == ORC_BF16) return (double)bf16_to_float(((const uint16_t *)base)[idx]);
+  return ((const double *)base)[idx];
+}
+
+/* ---- schedules ------------------------------------------------------------ */
+/* kind 0: UniformRSD, omega_i = delta.
+ * kind 1: Eq. sdar, omega_i = delta * exp(-nu*i - mu), mu fixed by
+ *         sum_{i=1..L} exp(-nu*i - mu) = L.
+ * kind 2: linear variant, omega_i = delta * L * w_i / sum_j w_j with
+ *         w_i = (ell - i) / (ell (ell + 1)), clamped at 0 for i >= ell.
+ * Returns 0, or -1 on bad arguments. */
+int orc_make_schedule(int kind, double delta, double nu_or_ell, int L, double *omega) {
+  if (L < 1 || !omega || !(delta >= 0.0)) return -1;
+  if (kind == 0) {
+    for (int i = 1; i <= L; ++i) omega[i - 1] = delta;
+    return 0;
+  }
+  if (kind == 1) {
+    double nu = nu_or_ell;
+    if (!(nu >= 0.0)) return -1;
+    double total = 0.0;
+    for (int i = 1; i <= L; ++i) total += exp(-nu * (double)i);
+    double mu = log(total / (double)L); /* sum_i exp(-nu i - mu) = L */
+    for (int i = 1; i <= L; ++i) omega[i - 1] = delta * exp(-nu * (double)i - mu);
+    return 0;
+  }
+  if (kind == 2) {
+    double ell = nu_or_ell;
+    if (!(ell > 1.0)) return -1;
+    double total = 0.0;
+    for (int i = 1; i <= L; ++i) {
+      double w = (ell - (double)i) / (ell * (ell + 1.0));
+      if (w < 0.0) w = 0.0;
+      omega[i - 1] = w;
+      total += w;
+    }
+    if (!(total > 0.0)) return -1;
+    for (int i = 1; i <= L; ++i) omega[i - 1] = delta * (double)L * omega[i - 1] / total;
+    return 0;
+  }
+  return -1;
+}
+
+/* ---- building blocks -------------------------------------------------------*/
+
+/* Relaxed acceptance probability, Eq. relax: min{1, omega p / q}, 0/0 := 1. */
+double orc_accept_prob(double p, double q, double omega) {
+  if (q == 0.0) return 1.0; /* p/q = +inf for p > 0, and 0/0 := 1 */
+  if (p == 0.0) return 0.0;
+  double ratio = omega * p / q;
+  return ratio < 1.0 ? ratio : 1.0;
+}
+
+/* Softmax of a V-vector of logits.  Returns 1 if the row is valid. */
+int orc_softmax(const double *z, int V, double *P) {
+  double m = -INFINITY;
+  for (int x = 0; x < V; ++x) {
+    if (isnan(z[x]) || z[x] == INFINITY) return 0;
+    if (z[x] > m) m = z[x];
+  }
+  if (m == -INFINITY) return 0;
+  double S = 0.0;
+  for (int x = 0; x < V; ++x) S += exp(z[x] - m);
+  for (int x = 0; x < V; ++x) P[x] = exp(z[x] - m) / S;
+  return 1;
+}
+
+/* Unnormalised Eq. opt_G: g(x) = [P(x) - Q(x) f(x)]_+ with
+ * f(x) = min{1, omega P(x)/Q(x)} (Eq. relax evaluated at candidate x).
+ * Returns Z = sum_x g(x). */
+double orc_resample_weights(const double *P, const double *Q, double omega, int V, double *g) {
+  double Z = 0.0;
+  for (int x = 0; x < V; ++x) {
+    double fx = orc_accept_prob(P[x], Q[x], omega);
+    double v = P[x] - Q[x] * fx;
+    if (!(v > 0.0)) v = 0.0;
+    g[x] = v;
+    Z += v;
+  }
+  return Z;
+}
+
+/* Eq. opt_G normalised; falls back to P when Z = 0.  Returns Z. */
+double orc_resample_dist(const double *P, const double *Q, double omega, int V, double *G) {
+  double Z = orc_resample_weights(P, Q, omega, V, G);
+  if (Z > 0.0) {
+    for (int x = 0; x < V; ++x) G[x] /= Z;
+  } else {
+    for (int x = 0; x < V; ++x) G[x] = P[x];
+  }
+  return Z;
+}
+
+/* Inverse-CDF draw from unnormalised non-negative weights g with total Z:
+ * smallest x with C(x) > u Z; else the last x with g(x) > 0.  *margin gets the
+ * distance (in probability units) from u to the nearest boundary of the picked
+ * token's CDF interval that separates it from another token of positive mass. */
+int orc_inverse_cdf(const double *g, int V, double Z, double u, double *margin) {
+  double target = u * Z;
+  double c = 0.0, c_lo = 0.0, c_hi = 0.0;
+  int tok = -1, last_pos = -1, first_pos = -1;
+  for (int x = 0; x < V; ++x) {
+    double c_prev = c;
+    c += g[x];
+    if (g[x] > 0.0) {
+      last_pos = x;
+      if (first_pos < 0) first_pos = x;
+    }
+    if (tok < 0 && c > target) {
+      tok = x;
+      c_lo = c_prev;
+      c_hi = c;
+    }
+  }
+  if (tok < 0) {
+    tok = last_pos;
+    if (margin) *margin = 0.0; /* decided by rounding alone */
+    return tok;
+  }
+  if (margin) {
+    double mg = INFINITY;
+    if (tok != first_pos) mg = fabs(u - c_lo / Z);
+    if (tok != last_pos) {
+      double d = fabs(u - c_hi / Z);
+      if (d < mg) mg = d;
+    }
+    *margin = mg;
+  }
+  return tok;
+}
+
+/* Row preparation: stored values -> fp64 logits, optional guidance mix (fp32
+ * fmaf, see header) and optional top-k mask. */
+static int cmp_desc(const void *a, const void *b) {
+  double x = *(const double *)a, y = *(const double *)b;
+  return (x < y) - (x > y);
+}
+
+void orc_prepare_row(const void *cond, const void *uncond, int dtype, int64_t offset, int V,
+                     float cfg_scale, int top_k, double *z, double *scratch) {
+  for (int x = 0; x < V; ++x) {
+    if (uncond) {
+      volatile float c = (float)load_value(cond, dtype, offset + x);
+      volatile float un = (float)load_value(uncond, dtype, offset + x);
+      volatile float d = c - un; /* rounded to fp32 */
+      float mixed = fmaf(cfg_scale, d, un);
+      z[x] = (double)mixed;
+    } else {
+      z[x] = load_value(cond, dtype, offset + x);
+    }
+  }
+  if (top_k > 0 && top_k < V) {
+    int has_nan = 0;
+    for (int x = 0; x < V; ++x) has_nan |= isnan(z[x]);
+    if (!has_nan) {
+      memcpy(scratch, z, (size_t)V * sizeof(double));
+      qsort(scratch, (size_t)V, sizeof(double), cmp_desc);
+      double kth = scratch[top_k - 1];
+      for (int x = 0; x < V; ++x)
+        if (z[x] < kth) z[x] = -INFINITY;
+    }
+  }
+}
+
+/* ---- Algorithm 1, verification stage, one sequence ------------------------ */
+static void verify_one(const orc_params *a, int b, double *zt, double *zd, double *P, double *Q,
+                       double *g, double *scratch) {
+  const int L = a->gamma, V = a->V;
+  const int32_t *tok = a->draft_tokens + (int64_t)b * L;
+  const float *unif = a->uniforms + (int64_t)b * (L + 1);
+  int32_t *out = a->out_tokens + (int64_t)b * (L + 1);
+  for (int i = 0; i <= L; ++i) out[i] = -1;
+  if (a->margin_accept)
+    for (int i = 0; i < L; ++i) a->margin_accept[(int64_t)b * L + i] = INFINITY;
+  if (a->margin_cdf) a->margin_cdf[b] = INFINITY;
+  if (a->G)
+    for (int x = 0; x < V; ++x) a->G[(int64_t)b * V + x] = 0.0;
+
+  int status = 0;
+  int tau = 0;
+  int emitted = 0; /* set once the (tau+1)-th token slot has been decided */
+  const double u = (double)unif[L];
+
+  for (int i = 1; i <= L; ++i) {
+    const int64_t t_off = (int64_t)b * a->target_batch_stride + (int64_t)(i - 1) * V;
+    const int64_t d_off = (int64_t)b * a->draft_batch_stride + (int64_t)(i - 1) * V;
+    orc_prepare_row(a->target_logits, a->target_uncond, a->dtype, t_off, V, a->cfg_scale, a->top_k,
+                    zt, scratch);
+    orc_prepare_row(a->draft_logits, a->draft_uncond, a->dtype, d_off, V, a->cfg_scale, a->top_k,
+                    zd, scratch);
+    const int t_ok = orc_softmax(zt, V, P);
+    const int d_ok = orc_softmax(zd, V, Q);
+    const double omega = (double)a->relax_schedule[i - 1];
+    const int x_i = tok[i - 1];
+    const int tok_ok = (x_i >= 0 && x_i < V);
+    double f;
+    if (!t_ok || !d_ok) {
+      f = 0.0;
+      status |= ORC_STATUS_BADROW;
+    } else if (!tok_ok) {
+      f = 0.0;
+      status |= ORC_STATUS_BADTOKEN;
+    } else {
+      f = orc_accept_prob(P[x_i], Q[x_i], omega);
+    }
+    const double r = (double)unif[i - 1];
+    if (a->margin_accept && t_ok && d_ok && tok_ok)
+      a->margin_accept[(int64_t)b * L + (i - 1)] = fabs(r - f);
+    if (r <= f) {
+      tau = i;
+      out[i - 1] = x_i;
+    } else {
+      /* rejected at position i: draw x_i from G*_i */
+      if (!t_ok) {
+        out[i - 1] = -1;
+      } else {
+        double Z;
+        if (d_ok) {
+          Z = orc_resample_weights(P, Q, omega, V, g);
+        } else { /* f == 0 for every candidate: Eq. opt_G gives P */
+          Z = 0.0;
+          for (int x = 0; x < V; ++x) {
+            g[x] = P[x];
+            Z += P[x];
+          }
+        }
+        if (!(Z > 0.0)) {
+          status |= ORC_STATUS_ZFALLBACK;
+          Z = 0.0;
+          for (int x = 0; x < V; ++x) {
+            g[x] = P[x];
+            Z += P[x];
+          }
+        }
+        double mg = INFINITY;
+        out[i - 1] = orc_inverse_cdf(g, V, Z, u, &mg);
+        if (a->margin_cdf) a->margin_cdf[b] = mg;
+        if (a->G)
+          for (int x = 0; x < V; ++x) a->G[(int64_t)b * V + x] = g[x] / Z;
+      }
+      emitted = 1;
+      break;
+    }
+  }
+
+  if (!emitted && tau == L && a->target_rows == L + 1) {
+    /* bonus token x_{L+1} ~ P(. | x_{1:L}) */
+    const int64_t t_off = (int64_t)b * a->target_batch_stride + (int64_t)L * V;
+    orc_prepare_row(a->target_logits, a->target_uncond, a->dtype, t_off, V, a->cfg_scale, a->top_k,
+                    zt, scratch);
+    if (orc_softmax(zt, V, P)) {
+      double Z = 0.0;
+      for (int x = 0; x < V; ++x) Z += P[x];
+      double mg = INFINITY;
+      out[L] = orc_inverse_cdf(P, V, Z, u, &mg);
+      if (a->margin_cdf) a->margin_cdf[b] = mg;
+      if (a->G)
+        for (int x = 0; x < V; ++x) a->G[(int64_t)b * V + x] = P[x] / Z;
+    } else {
+      status |= ORC_STATUS_BADROW;
+      out[L] = -1;
+    }
+  }
+  a->out_accept_len[b] = tau;
+  if (a->out_status) a->out_status[b] = status;
+
+  /* Diagnostics for comparison only (not part of the procedure): p, q, f at
+   * every position, including those after the first rejection. */
+  if (a->p || a->q || a->f) {
+    for (int i = 1; i <= L; ++i) {
+      const int64_t t_off = (int64_t)b * a->target_batch_stride + (int64_t)(i - 1) * V;
+      const int64_t d_off = (int64_t)b * a->draft_batch_stride + (int64_t)(i - 1) * V;
+      orc_prepare_row(a->target_logits, a->target_uncond, a->dtype, t_off, V, a->cfg_scale,
+                      a->top_k, zt, scratch);
+      orc_prepare_row(a->draft_logits, a->draft_uncond, a->dtype, d_off, V, a->cfg_scale, a->top_k,
+                      zd, scratch);
+      const int t_ok = orc_softmax(zt, V, P);
+      const int d_ok = orc_softmax(zd, V, Q);
+      const int x_i = tok[i - 1];
+      const int ok = t_ok && d_ok && x_i >= 0 && x_i < V;
+      const int64_t o = (int64_t)b * L + (i - 1);
+      const double pv = ok ? P[x_i] : NAN, qv = ok ? Q[x_i] : NAN;
+      if (a->p) a->p[o] = pv;
+      if (a->q) a->q[o] = qv;
+      if (a->f) a->f[o] = ok ? orc_accept_prob(pv, qv, (double)a->relax_schedule[i - 1]) : 0.0;
+    }
+  }
+}
+
+/* Batched driver: sequences are independent.  Returns 0, or -1 on bad shapes,
+ * -2 if memory could not be had. */
+int orc_verify(const orc_params *a) {
+  if (!a || a->B < 1 || a->gamma < 1 || a->V < 2) return -1;
+  if (a->target_rows != a->gamma && a->target_rows != a->gamma + 1) return -1;
+  int failed = 0;
+#ifdef _OPENMP
+#pragma omp parallel
+#endif
+  {
+    const size_t V = (size_t)a->V;
+    double *buf = (double *)malloc(6 * V * sizeof(double));
+    if (!buf) {
+#ifdef _OPENMP
+#pragma omp atomic write
+#endif
+      failed = 1;
+    }
+#ifdef _OPENMP
+#pragma omp barrier
+#endif
+    if (!failed) {
+#ifdef _OPENMP
+#pragma omp for schedule(dynamic, 1)
+#endif
+      for (int b = 0; b < a->B; ++b)
+        verify_one(a, b, buf, buf + V, buf + 2 * V, buf + 3 * V, buf + 4 * V, buf + 5 * V);
+    }
+    free(buf);
+  }
+  return failed ? -2 : 0;
+}
