@@ -1,0 +1,185 @@
+/*
+ * csd.h -- C ABI of libcsd: the batched verify-and-resample round of Cool-SD
+ * (annealed relaxation of speculative decoding) on one NVIDIA B200 (sm_100a).
+ *
+ * What one call computes, for B independent sequences with gamma drafted
+ * tokens each (Algorithm 1, verification stage):
+ *   1. softmax statistics of every target and drafter logit row (Algorithm 1,
+ *      "calculate P(x~_i | ...) in parallel");
+ *   2. the relaxed acceptance probability f_i = min{1, omega_i P(x~_i)/Q(x~_i)}
+ *      (Eq. relax; 0/0 := 1 per the Notations appendix) and the accept test
+ *      r_i <= f_i for every position;
+ *   3. tau = number of leading accepted positions (the for/break of Algorithm 1);
+ *   4. at the first rejected position j = tau + 1 the bound-minimising
+ *      resampling distribution G*_j = Norm([P_j - Q_j f_j(.)]_+) (Eq. opt_G,
+ *      Theorem 2) and one inverse-CDF draw from it; if every position was
+ *      accepted, the bonus token from P_{gamma+1} (Algorithm 1, last step);
+ *   5. the emitted block x_{1:tau+1}.
+ * The schedule omega_1..omega_gamma is an input (csd_make_schedule builds the
+ * paper's: UniformRSD, Eq. sdar, and the linear variant of the ablation).
+ *
+ * Conventions
+ *   - All data pointers are DEVICE pointers owned by the caller unless a
+ *     parameter says HOST.  The library reads inputs, writes outputs and the
+ *     caller's workspace, and nothing else.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     legacy default stream) of the CURRENT device; calls return without
+ *     synchronising.  Outputs are valid once the stream has reached that point.
+ *   - Return value: CSD_OK (0) or a negative csd_error.  Errors found on the
+ *     host are reported before anything is enqueued.  Problems in the DATA
+ *     never trap or hang: they set bits in out_status[b] and give a defined
+ *     result (see csd_status_bits).
+ *   - Layout: row-major, V contiguous.  Row (b, i) of target_logits starts at
+ *     element b*target_batch_stride + i*V, of draft_logits at
+ *     b*draft_batch_stride + i*V.  The fast path needs 16-byte aligned base
+ *     pointers and V*sizeof(element) and the batch strides in bytes to be
+ *     multiples of 16; anything else takes a slower scalar path with the same
+ *     results.
+ *   - Inverse-CDF convention: token = smallest x with C(x) > u*Z in token-id
+ *     order (C the running sum of the unnormalised weights, Z their total); if
+ *     rounding leaves none, the last x with positive weight.  One uniform per
+ *     sequence (uniforms[b][gamma]) serves the resample or the bonus draw.
+ *   - If the positive part in Eq. opt_G is empty (P == Q, omega >= 1; reachable
+ *     only through rounding) the draw falls back to G := P_j.
+ */
+#ifndef CSD_H_
+#define CSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { CSD_F32 = 0, CSD_BF16 = 1 } csd_dtype;
+
+typedef enum {
+  CSD_OK = 0,
+  CSD_ERR_NULL = -1,      /* a required pointer is NULL */
+  CSD_ERR_SHAPE = -2,     /* B < 1, gamma outside [1,32], V outside [2, 2^20], bad target_rows/stride */
+  CSD_ERR_DTYPE = -3,     /* unknown csd_dtype */
+  CSD_ERR_WORKSPACE = -4, /* workspace NULL, misaligned (256 B) or smaller than csd_workspace_size */
+  CSD_ERR_ARG = -5,       /* inconsistent options (one unconditional array without the other, top_k < 0, ...) */
+  CSD_ERR_LAUNCH = -6,    /* the CUDA runtime refused a launch or copy; see cudaGetLastError */
+  CSD_ERR_ALLOC = -7      /* csd_verify only: its internal workspace could not be allocated */
+} csd_error;
+
+/* Bits of out_status[b]; they refer only to positions the algorithm looked at
+ * (1..tau+1 and the bonus row), like the sequential loop of Algorithm 1. */
+typedef enum {
+  CSD_STATUS_BADROW = 1,   /* a row held NaN or +inf, or no finite entry: that position
+                              rejects (f := 0).  An unusable drafter row resamples from
+                              P_j (Eq. opt_G at f = 0); an unusable target row emits -1. */
+  CSD_STATUS_BADTOKEN = 2, /* draft token outside [0, V): that position rejects */
+  CSD_STATUS_ZFALLBACK = 4 /* empty positive part: drew from P_j instead */
+} csd_status_bits;
+
+/*
+ * Simple form (Algorithm 1, verification stage; Eq. relax; Eq. opt_G):
+ * fp32 logits, contiguous [B, gamma, V] arrays, no bonus row (slot gamma of a
+ * fully accepted sequence is -1), no guidance mix, no top-k.
+ *
+ *   target_logits  [B, gamma, V]  device, read
+ *   draft_logits   [B, gamma, V]  device, read
+ *   draft_tokens   [B, gamma]     device, read; each in [0, V)
+ *   uniforms       [B, gamma+1]   device, read; in (0,1); columns 0..gamma-1 are the
+ *                                 accept draws r_i, column gamma the resample draw u
+ *   relax_schedule [gamma]        device, read; omega_i >= 0 (all 1.0 = vanilla
+ *                                 speculative decoding); negative or NaN counts as 0
+ *   out_tokens     [B, gamma+1]   device, written; x_{1:tau+1}, then -1
+ *   out_accept_len [B]            device, written; tau in [0, gamma]
+ *
+ * Scratch: this form keeps one workspace per device inside the library,
+ * allocated with cudaMalloc on first use and grown when a larger problem
+ * arrives (so the first call of a given size must not be inside a stream
+ * capture, and concurrent calls on different streams of one device must use
+ * csd_verify_ex with their own workspaces instead).
+ */
+int csd_verify(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
+               const float* uniforms, const float* relax_schedule, int B, int gamma, int V,
+               int32_t* out_tokens, int32_t* out_accept_len, void* stream);
+
+/*
+ * Full form.  Adds: bf16 logits; an optional (gamma+1)-th target row for the
+ * bonus token (Algorithm 1, last step); batch strides; guidance mixing fused
+ * into the load, z = fmaf(cfg_scale, cond - uncond, uncond) evaluated in fp32
+ * with the difference rounded to fp32 first (the drafter-side classifier-free
+ * guidance of the paper's Additional Implementation Details, applied here to
+ * both models' rows when the unconditional arrays are given); top-k filtering
+ * before the softmax (keep every logit >= the k-th largest of its row, ties
+ * kept; not in the paper, part of the benchmark definition); per-sequence
+ * status; optional diagnostic outputs.
+ */
+typedef struct csd_params {
+  const void* target_logits; /* [B, target_rows, V] conditional (or only) rows     */
+  const void* draft_logits;  /* [B, gamma, V]                                      */
+  const void* target_uncond; /* same layout as target_logits, or NULL               */
+  const void* draft_uncond;  /* same layout as draft_logits; NULL iff target_uncond */
+  float cfg_scale;           /* s in uncond + s*(cond - uncond); unused without uncond */
+  int32_t top_k;             /* 0 or >= V: off                                      */
+  int32_t dtype;             /* csd_dtype of all four logit arrays                  */
+  int32_t B, gamma, V;
+  int32_t target_rows;         /* gamma or gamma + 1                                */
+  int64_t target_batch_stride; /* elements; 0 means target_rows * V                 */
+  int64_t draft_batch_stride;  /* elements; 0 means gamma * V                       */
+  const int32_t* draft_tokens; /* [B, gamma]                                        */
+  const float* uniforms;       /* [B, gamma+1]                                      */
+  const float* relax_schedule; /* [gamma]                                           */
+  int32_t* out_tokens;         /* [B, gamma+1]                                      */
+  int32_t* out_accept_len;     /* [B]                                               */
+  int32_t* out_status;         /* [B] or NULL; csd_status_bits                      */
+  float* dbg_p;                /* [B, gamma] or NULL: P_i(x~_i)                     */
+  float* dbg_q;                /* [B, gamma] or NULL: Q_i(x~_i)                     */
+  float* dbg_f;                /* [B, gamma] or NULL: f_i (0 where the row or token is unusable) */
+  float* dbg_G;                /* [B, V] or NULL: the distribution the emitted token was drawn
+                                  from (G*_j, or P for the bonus draw / fallbacks); zeros if none */
+  void* workspace;             /* >= csd_workspace_size(...) bytes, 256-byte aligned; contents
+                                  need no initialisation and are garbage afterwards.  Two calls
+                                  that may overlap on the GPU need different workspaces.    */
+  size_t workspace_bytes;
+  void* stream;
+} csd_params;
+
+int csd_verify_ex(const csd_params* p);
+
+/* Bytes of workspace that csd_verify_ex needs for any call with these sizes
+ * (any target_rows, guidance and top-k setting).  0 if the sizes are invalid. */
+size_t csd_workspace_size(int B, int gamma, int V, int dtype);
+
+/*
+ * Host-buffer form: the same round for a caller whose logits, tokens, uniforms
+ * and schedule sit in HOST memory (pinned memory makes the copies asynchronous).
+ * Every data pointer of `host` (inputs, outputs, optional diagnostics) is a
+ * HOST pointer; host->workspace / workspace_bytes are ignored.  `staging` is a
+ * DEVICE buffer of at least csd_host_staging_size(host) bytes, 256-byte
+ * aligned, that the library uses for the device copies of inputs and outputs
+ * and for its workspace.  The call enqueues host->device copies, the kernels and
+ * device->host copies of out_tokens / out_accept_len / out_status (and any
+ * diagnostics requested) on host->stream and returns; results are in the host
+ * arrays once the stream has been synchronised.
+ */
+int csd_verify_host(const csd_params* host, void* staging, size_t staging_bytes);
+size_t csd_host_staging_size(const csd_params* host);
+
+/*
+ * Relaxation schedules, written to HOST memory out_host[0..L-1] = omega_1..omega_L.
+ *   kind 0  UniformRSD: omega_i = delta.
+ *   kind 1  Cool-SD, Eq. sdar: omega_i = delta * exp(-nu*i - mu) with mu fixed by
+ *           sum_{i=1..L} exp(-nu*i - mu) = L  (nu_or_ell = nu >= 0).
+ *   kind 2  linear variant of the schedule ablation: omega_i = delta * L * w_i / sum_j w_j,
+ *           w_i = (ell - i) / (ell (ell + 1)), clamped at 0 for i >= ell (nu_or_ell = ell > 1).
+ * Returns CSD_OK, CSD_ERR_NULL or CSD_ERR_ARG.
+ */
+int csd_make_schedule(int kind, double delta, double nu_or_ell, int L, float* out_host);
+
+/* Static, NUL-terminated description of a csd_error value. */
+const char* csd_error_string(int code);
+
+/* Version of this ABI: major*10000 + minor*100 + patch. */
+int csd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CSD_H_ */

@@ -1,0 +1,411 @@
+// Host side of libcsd: argument checks, workspace layout, launch configuration.
+// Every step of the method runs in the kernels of csd_kernels.cuh; nothing here
+// touches logits.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "../../include/csd.h"
+#include "csd_kernels.cuh"
+
+namespace {
+
+using namespace csd;
+
+constexpr int kMaxV = 1 << 20;
+constexpr int kMaxDevices = 64;
+constexpr size_t kAlign = 256;
+
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+inline int elem_size(int dtype) { return dtype == CSD_F32 ? 4 : 2; }
+inline int vec_width(int dtype) { return 16 / elem_size(dtype); }
+
+struct DeviceInfo {
+  int sms = 0;
+};
+DeviceInfo g_dev[kMaxDevices];
+std::mutex g_mutex;
+
+int device_sms(int* dev_out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+  if (dev_out) *dev_out = dev;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (g_dev[dev].sms == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    g_dev[dev].sms = n;
+  }
+  return g_dev[dev].sms;
+}
+
+bool shape_ok(int B, int gamma, int V) {
+  return B >= 1 && gamma >= 1 && gamma <= kMaxGamma && V >= 2 && V <= kMaxV;
+}
+
+// Workspace: [partials: rows * max_parts float2][thresholds: rows float]
+struct Layout {
+  size_t rows, max_parts, partials_off, thresholds_off, total;
+};
+Layout layout_for(int B, int gamma, int V, int dtype) {
+  Layout l;
+  l.rows = (size_t)B * (size_t)(2 * gamma + 1);
+  const size_t min_part = (size_t)kStatsThreads * vec_width(dtype);  // U = 1
+  l.max_parts = ((size_t)V + min_part - 1) / min_part;
+  l.partials_off = 0;
+  l.thresholds_off = align_up(l.rows * l.max_parts * sizeof(float2));
+  l.total = l.thresholds_off + align_up(l.rows * sizeof(float));
+  return l;
+}
+
+template <typename T, bool CFG, int U>
+cudaError_t launch_stats(const StatsArgs& a, int sms, cudaStream_t stream) {
+  auto kern = row_stats_kernel<T, CFG, U>;
+  int per_sm = 0;
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kStatsThreads, 0);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) per_sm = 1;
+  long long grid = (long long)sms * per_sm;
+  if (grid > a.n_items) grid = a.n_items;
+  kern<<<(unsigned)grid, kStatsThreads, 0, stream>>>(a);
+  return cudaGetLastError();
+}
+
+template <typename T, bool CFG>
+cudaError_t launch_stats_u(const StatsArgs& a, int U, int sms, cudaStream_t stream) {
+  switch (U) {
+    case 8: return launch_stats<T, CFG, 8>(a, sms, stream);
+    case 4: return launch_stats<T, CFG, 4>(a, sms, stream);
+    case 2: return launch_stats<T, CFG, 2>(a, sms, stream);
+    default: return launch_stats<T, CFG, 1>(a, sms, stream);
+  }
+}
+
+template <typename T, bool CFG>
+cudaError_t launch_finish(const FinishArgs& a, cudaStream_t stream) {
+  auto kern = finish_kernel<T, CFG>;
+  constexpr int TILE = 32 * Elem<T>::kVec;
+  const size_t smem = (size_t)((a.V + TILE - 1) / TILE) * sizeof(double);
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3((unsigned)a.B);
+  cfg.blockDim = dim3(kFinishThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+int verify_impl(const csd_params& p) {
+  if (!p.target_logits || !p.draft_logits || !p.draft_tokens || !p.uniforms || !p.relax_schedule ||
+      !p.out_tokens || !p.out_accept_len)
+    return CSD_ERR_NULL;
+  if (p.dtype != CSD_F32 && p.dtype != CSD_BF16) return CSD_ERR_DTYPE;
+  if (!shape_ok(p.B, p.gamma, p.V)) return CSD_ERR_SHAPE;
+  if (p.target_rows != p.gamma && p.target_rows != p.gamma + 1) return CSD_ERR_SHAPE;
+  const int64_t tstride = p.target_batch_stride ? p.target_batch_stride : (int64_t)p.target_rows * p.V;
+  const int64_t dstride = p.draft_batch_stride ? p.draft_batch_stride : (int64_t)p.gamma * p.V;
+  if (tstride < (int64_t)p.target_rows * p.V || dstride < (int64_t)p.gamma * p.V) return CSD_ERR_SHAPE;
+  const bool cfg = p.target_uncond != nullptr;
+  if ((p.target_uncond == nullptr) != (p.draft_uncond == nullptr)) return CSD_ERR_ARG;
+  if (p.top_k < 0) return CSD_ERR_ARG;
+  if (cfg && !isfinite(p.cfg_scale)) return CSD_ERR_ARG;
+  const bool topk = p.top_k > 0 && p.top_k < p.V;
+  if (topk) return CSD_ERR_ARG;  // not built yet
+  const Layout lay = layout_for(p.B, p.gamma, p.V, p.dtype);
+  if (!p.workspace || ((uintptr_t)p.workspace % kAlign) != 0 || p.workspace_bytes < lay.total)
+    return CSD_ERR_WORKSPACE;
+  int dev = 0;
+  const int sms = device_sms(&dev);
+  if (sms <= 0) return CSD_ERR_LAUNCH;
+
+  const int es = elem_size(p.dtype), vw = vec_width(p.dtype);
+  auto aligned16 = [](const void* q) { return ((uintptr_t)q & 15u) == 0; };
+  bool vec_ok = (p.V % vw) == 0 && (tstride * es) % 16 == 0 && (dstride * es) % 16 == 0 &&
+                aligned16(p.target_logits) && aligned16(p.draft_logits);
+  if (cfg) vec_ok = vec_ok && aligned16(p.target_uncond) && aligned16(p.draft_uncond);
+
+  cudaStream_t stream = (cudaStream_t)p.stream;
+  const int rows_per_seq = p.target_rows + p.gamma;
+  const long long rows = (long long)p.B * rows_per_seq;
+
+  // part size: the largest that still leaves every SM several blocks to work on
+  int U = cfg ? 4 : 8;
+  auto parts_for = [&](int u) { return (p.V + kStatsThreads * u * vw - 1) / (kStatsThreads * u * vw); };
+  while (U > 1 && rows * parts_for(U) < 4LL * sms) U >>= 1;
+
+  StatsArgs sa;
+  sa.target = p.target_logits; sa.draft = p.draft_logits;
+  sa.target_uncond = p.target_uncond; sa.draft_uncond = p.draft_uncond;
+  sa.cfg_scale = p.cfg_scale;
+  sa.B = p.B; sa.gamma = p.gamma; sa.T = p.target_rows; sa.V = p.V;
+  sa.tstride = tstride; sa.dstride = dstride;
+  sa.parts = parts_for(U);
+  sa.part_elems = kStatsThreads * U * vw;
+  sa.n_items = (int)(rows * sa.parts);
+  sa.vec_ok = vec_ok ? 1 : 0;
+  sa.partials = reinterpret_cast<float2*>((char*)p.workspace + lay.partials_off);
+
+  FinishArgs fa;
+  fa.target = p.target_logits; fa.draft = p.draft_logits;
+  fa.target_uncond = p.target_uncond; fa.draft_uncond = p.draft_uncond;
+  fa.cfg_scale = p.cfg_scale;
+  fa.B = p.B; fa.gamma = p.gamma; fa.T = p.target_rows; fa.V = p.V;
+  fa.tstride = tstride; fa.dstride = dstride;
+  fa.parts = sa.parts;
+  fa.vec_ok = sa.vec_ok;
+  fa.use_topk = topk ? 1 : 0;
+  fa.partials = sa.partials;
+  fa.thresholds = reinterpret_cast<const float*>((char*)p.workspace + lay.thresholds_off);
+  fa.tokens = p.draft_tokens; fa.uniforms = p.uniforms; fa.schedule = p.relax_schedule;
+  fa.out_tokens = p.out_tokens; fa.out_accept_len = p.out_accept_len; fa.out_status = p.out_status;
+  fa.dbg_p = p.dbg_p; fa.dbg_q = p.dbg_q; fa.dbg_f = p.dbg_f; fa.dbg_G = p.dbg_G;
+
+  cudaError_t e;
+  if (p.dtype == CSD_F32) {
+    e = cfg ? launch_stats_u<float, true>(sa, U, sms, stream) : launch_stats_u<float, false>(sa, U, sms, stream);
+    if (e == cudaSuccess) e = cfg ? launch_finish<float, true>(fa, stream) : launch_finish<float, false>(fa, stream);
+  } else {
+    e = cfg ? launch_stats_u<__nv_bfloat16, true>(sa, U, sms, stream)
+            : launch_stats_u<__nv_bfloat16, false>(sa, U, sms, stream);
+    if (e == cudaSuccess)
+      e = cfg ? launch_finish<__nv_bfloat16, true>(fa, stream) : launch_finish<__nv_bfloat16, false>(fa, stream);
+  }
+  return e == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
+}
+
+// internal workspace of the simple form, one per device
+struct OwnedWorkspace {
+  void* ptr = nullptr;
+  size_t bytes = 0;
+};
+OwnedWorkspace g_ws[kMaxDevices];
+
+}  // namespace
+
+extern "C" {
+
+size_t csd_workspace_size(int B, int gamma, int V, int dtype) {
+  if (!shape_ok(B, gamma, V) || (dtype != CSD_F32 && dtype != CSD_BF16)) return 0;
+  return layout_for(B, gamma, V, dtype).total;
+}
+
+int csd_verify_ex(const csd_params* p) {
+  if (!p) return CSD_ERR_NULL;
+  return verify_impl(*p);
+}
+
+int csd_verify(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
+               const float* uniforms, const float* relax_schedule, int B, int gamma, int V,
+               int32_t* out_tokens, int32_t* out_accept_len, void* stream) {
+  if (!shape_ok(B, gamma, V)) return CSD_ERR_SHAPE;
+  const size_t need = csd_workspace_size(B, gamma, V, CSD_F32);
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CSD_ERR_LAUNCH;
+  void* ws = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    OwnedWorkspace& w = g_ws[dev];
+    if (w.bytes < need) {
+      // earlier calls may still be using the old buffer
+      if (w.ptr) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return CSD_ERR_LAUNCH;
+        cudaFree(w.ptr);
+        w.ptr = nullptr;
+        w.bytes = 0;
+      }
+      if (cudaMalloc(&w.ptr, need) != cudaSuccess) {
+        w.ptr = nullptr;
+        (void)cudaGetLastError();
+        return CSD_ERR_ALLOC;
+      }
+      w.bytes = need;
+    }
+    ws = w.ptr;
+  }
+  csd_params p;
+  memset(&p, 0, sizeof p);
+  p.target_logits = target_logits; p.draft_logits = draft_logits;
+  p.cfg_scale = 1.0f; p.top_k = 0; p.dtype = CSD_F32;
+  p.B = B; p.gamma = gamma; p.V = V; p.target_rows = gamma;
+  p.draft_tokens = draft_tokens; p.uniforms = uniforms; p.relax_schedule = relax_schedule;
+  p.out_tokens = out_tokens; p.out_accept_len = out_accept_len;
+  p.workspace = ws; p.workspace_bytes = need;
+  p.stream = stream;
+  return verify_impl(p);
+}
+
+// ---- host-buffer form -----------------------------------------------------------
+namespace {
+struct HostPlan {
+  size_t logits_t, logits_d, tokens, uniforms, schedule, out_tokens, out_len, out_status;
+  size_t dbg_pqf, dbg_G;
+  size_t off_t, off_d, off_tu, off_du, off_tok, off_uni, off_sched, off_otok, off_olen, off_ostat;
+  size_t off_p, off_q, off_f, off_G, off_ws, ws_bytes, total;
+  int64_t tstride, dstride;
+};
+bool host_plan(const csd_params& h, HostPlan& pl) {
+  if (!shape_ok(h.B, h.gamma, h.V) || (h.dtype != CSD_F32 && h.dtype != CSD_BF16)) return false;
+  if (h.target_rows != h.gamma && h.target_rows != h.gamma + 1) return false;
+  pl.tstride = h.target_batch_stride ? h.target_batch_stride : (int64_t)h.target_rows * h.V;
+  pl.dstride = h.draft_batch_stride ? h.draft_batch_stride : (int64_t)h.gamma * h.V;
+  if (pl.tstride < (int64_t)h.target_rows * h.V || pl.dstride < (int64_t)h.gamma * h.V) return false;
+  const size_t es = elem_size(h.dtype);
+  pl.logits_t = (size_t)h.B * pl.tstride * es;
+  pl.logits_d = (size_t)h.B * pl.dstride * es;
+  pl.tokens = (size_t)h.B * h.gamma * 4;
+  pl.uniforms = (size_t)h.B * (h.gamma + 1) * 4;
+  pl.schedule = (size_t)h.gamma * 4;
+  pl.out_tokens = (size_t)h.B * (h.gamma + 1) * 4;
+  pl.out_len = (size_t)h.B * 4;
+  pl.out_status = (size_t)h.B * 4;
+  pl.dbg_pqf = (size_t)h.B * h.gamma * 4;
+  pl.dbg_G = (size_t)h.B * h.V * 4;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += align_up(bytes); return o; };
+  pl.off_t = take(pl.logits_t);
+  pl.off_d = take(pl.logits_d);
+  pl.off_tu = take(h.target_uncond ? pl.logits_t : 0);
+  pl.off_du = take(h.draft_uncond ? pl.logits_d : 0);
+  pl.off_tok = take(pl.tokens);
+  pl.off_uni = take(pl.uniforms);
+  pl.off_sched = take(pl.schedule);
+  pl.off_otok = take(pl.out_tokens);
+  pl.off_olen = take(pl.out_len);
+  pl.off_ostat = take(pl.out_status);
+  pl.off_p = take(h.dbg_p ? pl.dbg_pqf : 0);
+  pl.off_q = take(h.dbg_q ? pl.dbg_pqf : 0);
+  pl.off_f = take(h.dbg_f ? pl.dbg_pqf : 0);
+  pl.off_G = take(h.dbg_G ? pl.dbg_G : 0);
+  pl.ws_bytes = layout_for(h.B, h.gamma, h.V, h.dtype).total;
+  pl.off_ws = take(pl.ws_bytes);
+  pl.total = off;
+  return true;
+}
+}  // namespace
+
+size_t csd_host_staging_size(const csd_params* host) {
+  HostPlan pl;
+  if (!host || !host_plan(*host, pl)) return 0;
+  return pl.total;
+}
+
+int csd_verify_host(const csd_params* host, void* staging, size_t staging_bytes) {
+  if (!host) return CSD_ERR_NULL;
+  const csd_params& h = *host;
+  if (!h.target_logits || !h.draft_logits || !h.draft_tokens || !h.uniforms || !h.relax_schedule ||
+      !h.out_tokens || !h.out_accept_len)
+    return CSD_ERR_NULL;
+  if (h.dtype != CSD_F32 && h.dtype != CSD_BF16) return CSD_ERR_DTYPE;
+  if ((h.target_uncond == nullptr) != (h.draft_uncond == nullptr)) return CSD_ERR_ARG;
+  HostPlan pl;
+  if (!host_plan(h, pl)) return CSD_ERR_SHAPE;
+  if (!staging || ((uintptr_t)staging % kAlign) != 0 || staging_bytes < pl.total) return CSD_ERR_WORKSPACE;
+  char* base = (char*)staging;
+  cudaStream_t stream = (cudaStream_t)h.stream;
+  auto h2d = [&](size_t off, const void* src, size_t bytes) {
+    return cudaMemcpyAsync(base + off, src, bytes, cudaMemcpyHostToDevice, stream);
+  };
+  auto d2h = [&](void* dst, size_t off, size_t bytes) {
+    return cudaMemcpyAsync(dst, base + off, bytes, cudaMemcpyDeviceToHost, stream);
+  };
+  cudaError_t e = h2d(pl.off_t, h.target_logits, pl.logits_t);
+  if (e == cudaSuccess) e = h2d(pl.off_d, h.draft_logits, pl.logits_d);
+  if (e == cudaSuccess && h.target_uncond) e = h2d(pl.off_tu, h.target_uncond, pl.logits_t);
+  if (e == cudaSuccess && h.draft_uncond) e = h2d(pl.off_du, h.draft_uncond, pl.logits_d);
+  if (e == cudaSuccess) e = h2d(pl.off_tok, h.draft_tokens, pl.tokens);
+  if (e == cudaSuccess) e = h2d(pl.off_uni, h.uniforms, pl.uniforms);
+  if (e == cudaSuccess) e = h2d(pl.off_sched, h.relax_schedule, pl.schedule);
+  if (e != cudaSuccess) return CSD_ERR_LAUNCH;
+
+  csd_params d = h;
+  d.target_logits = base + pl.off_t;
+  d.draft_logits = base + pl.off_d;
+  d.target_uncond = h.target_uncond ? base + pl.off_tu : nullptr;
+  d.draft_uncond = h.draft_uncond ? base + pl.off_du : nullptr;
+  d.target_batch_stride = pl.tstride;
+  d.draft_batch_stride = pl.dstride;
+  d.draft_tokens = (const int32_t*)(base + pl.off_tok);
+  d.uniforms = (const float*)(base + pl.off_uni);
+  d.relax_schedule = (const float*)(base + pl.off_sched);
+  d.out_tokens = (int32_t*)(base + pl.off_otok);
+  d.out_accept_len = (int32_t*)(base + pl.off_olen);
+  d.out_status = (int32_t*)(base + pl.off_ostat);
+  d.dbg_p = h.dbg_p ? (float*)(base + pl.off_p) : nullptr;
+  d.dbg_q = h.dbg_q ? (float*)(base + pl.off_q) : nullptr;
+  d.dbg_f = h.dbg_f ? (float*)(base + pl.off_f) : nullptr;
+  d.dbg_G = h.dbg_G ? (float*)(base + pl.off_G) : nullptr;
+  d.workspace = base + pl.off_ws;
+  d.workspace_bytes = pl.ws_bytes;
+  const int rc = verify_impl(d);
+  if (rc != CSD_OK) return rc;
+
+  e = d2h(h.out_tokens, pl.off_otok, pl.out_tokens);
+  if (e == cudaSuccess) e = d2h(h.out_accept_len, pl.off_olen, pl.out_len);
+  if (e == cudaSuccess && h.out_status) e = d2h(h.out_status, pl.off_ostat, pl.out_status);
+  if (e == cudaSuccess && h.dbg_p) e = d2h(h.dbg_p, pl.off_p, pl.dbg_pqf);
+  if (e == cudaSuccess && h.dbg_q) e = d2h(h.dbg_q, pl.off_q, pl.dbg_pqf);
+  if (e == cudaSuccess && h.dbg_f) e = d2h(h.dbg_f, pl.off_f, pl.dbg_pqf);
+  if (e == cudaSuccess && h.dbg_G) e = d2h(h.dbg_G, pl.off_G, pl.dbg_G);
+  return e == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
+}
+
+// ---- schedules (host arithmetic, fp64, rounded once to fp32) -------------------------
+int csd_make_schedule(int kind, double delta, double nu_or_ell, int L, float* out_host) {
+  if (!out_host) return CSD_ERR_NULL;
+  if (L < 1 || !(delta >= 0.0) || !isfinite(delta)) return CSD_ERR_ARG;
+  if (kind == 0) {
+    for (int i = 0; i < L; ++i) out_host[i] = (float)delta;
+    return CSD_OK;
+  }
+  if (kind == 1) {
+    const double nu = nu_or_ell;
+    if (!(nu >= 0.0) || !isfinite(nu)) return CSD_ERR_ARG;
+    // geometric weights exp(-nu (i-1)), normalised so that the multipliers average delta
+    double norm = 0.0, w = 1.0;
+    const double ratio = exp(-nu);
+    for (int i = 0; i < L; ++i) { norm += w; w *= ratio; }
+    w = delta * (double)L / norm;
+    for (int i = 0; i < L; ++i) { out_host[i] = (float)w; w *= ratio; }
+    return CSD_OK;
+  }
+  if (kind == 2) {
+    const double ell = nu_or_ell;
+    if (!(ell > 1.0) || !isfinite(ell)) return CSD_ERR_ARG;
+    double norm = 0.0;
+    for (int i = 1; i <= L; ++i) norm += fmax(0.0, ell - (double)i);
+    if (!(norm > 0.0)) return CSD_ERR_ARG;
+    for (int i = 1; i <= L; ++i) out_host[i - 1] = (float)(delta * (double)L * fmax(0.0, ell - (double)i) / norm);
+    return CSD_OK;
+  }
+  return CSD_ERR_ARG;
+}
+
+const char* csd_error_string(int code) {
+  switch (code) {
+    case CSD_OK: return "ok";
+    case CSD_ERR_NULL: return "a required pointer is NULL";
+    case CSD_ERR_SHAPE: return "bad shape: need B >= 1, 1 <= gamma <= 32, 2 <= V <= 2^20, target_rows in {gamma, gamma+1}, strides covering the rows";
+    case CSD_ERR_DTYPE: return "unknown dtype (CSD_F32 or CSD_BF16)";
+    case CSD_ERR_WORKSPACE: return "workspace missing, not 256-byte aligned, or too small";
+    case CSD_ERR_ARG: return "inconsistent or unsupported options";
+    case CSD_ERR_LAUNCH: return "CUDA runtime error while enqueueing work";
+    case CSD_ERR_ALLOC: return "could not allocate the internal workspace";
+    default: return "unknown error code";
+  }
+}
+
+int csd_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,536 @@
+// Device code of libcsd: the verify-and-resample round of Cool-SD on sm_100a.
+//
+// Two kernels per call, the second launched with programmatic dependent launch
+// so that its blocks are resident and waiting when the first one drains:
+//
+//   row_stats_kernel   streams every logit row once from HBM (the only HBM
+//                      traffic of the call) and leaves, per (row, part), the pair
+//                      (m, s) with  sum_x exp(z_x) = (1 + s) * exp(m)  over that part:
+//                      m the maximum, s the sum of exp(z - m) over all OTHER
+//                      entries.  Keeping the "1 +" out of the fp32 sum preserves the
+//                      relative accuracy of 1 - P(argmax) on sharply peaked rows.
+//   finish_kernel      one block per sequence: merges the parts, gathers the
+//                      drafted tokens' logits, evaluates Eq. relax and the accept
+//                      tests, finds tau, re-reads the two rows of position tau+1
+//                      (L2 hits at the sizes of interest), forms Eq. opt_G, and
+//                      draws by inverse CDF with fp64 running sums.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace csd {
+
+constexpr int kStatsThreads = 256;
+constexpr int kFinishThreads = 1024;
+constexpr int kMaxGamma = 32;
+constexpr float kLog2e = 1.4426950408889634f;
+#define CSD_NEG_INF (__int_as_float(0xff800000))
+#define CSD_POS_INF (__int_as_float(0x7f800000))
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// ---- (m, s) algebra ---------------------------------------------------------
+// identity: m = -inf, s = -1 (so that 1 + s = 0)
+__device__ __forceinline__ void stat_merge(float& m, float& s, float m2, float s2) {
+  if (m2 > m) {
+    float t = m; m = m2; m2 = t;
+    t = s; s = s2; s2 = t;
+  }
+  if (m2 != CSD_NEG_INF) s += (1.0f + s2) * ex2f((m2 - m) * kLog2e);
+}
+
+__device__ __forceinline__ void stat_warp_allreduce(float& m, float& s) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    float m2 = __shfl_xor_sync(0xffffffffu, m, off);
+    float s2 = __shfl_xor_sync(0xffffffffu, s, off);
+    stat_merge(m, s, m2, s2);
+  }
+}
+
+// (m, s) of n register-resident values
+template <int N>
+__device__ __forceinline__ void stat_of_values(const float (&z)[N], float& m, float& s) {
+  m = CSD_NEG_INF;
+#pragma unroll
+  for (int k = 0; k < N; ++k) m = fmaxf(m, z[k]);
+  float acc = 0.0f;
+  int cnt = 0;
+#pragma unroll
+  for (int k = 0; k < N; ++k) {
+    float e = ex2f((z[k] - m) * kLog2e);
+    if (z[k] == m) cnt += 1; else acc += e;   // NaN entries poison acc, which marks the row
+  }
+  s = acc + (float)(cnt - 1);
+}
+
+// ---- element access -----------------------------------------------------------
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+  static constexpr int kVec = 4;
+  __device__ static __forceinline__ void load_vec(const float* p, float (&out)[4]) {
+    float4 v = __ldg(reinterpret_cast<const float4*>(p));
+    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+  }
+  __device__ static __forceinline__ float load_one(const float* p) { return __ldg(p); }
+};
+template <> struct Elem<__nv_bfloat16> {
+  static constexpr int kVec = 8;
+  __device__ static __forceinline__ void load_vec(const __nv_bfloat16* p, float (&out)[8]) {
+    uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      out[2 * k] = __uint_as_float(w[k] << 16);
+      out[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+    }
+  }
+  __device__ static __forceinline__ float load_one(const __nv_bfloat16* p) {
+    return __uint_as_float(((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
+  }
+};
+
+// guidance mix: the difference is rounded to fp32, then one fused multiply-add
+__device__ __forceinline__ float cfg_mix(float c, float u, float s) {
+  return __fmaf_rn(s, __fsub_rn(c, u), u);
+}
+
+// One logical row: conditional array, optional unconditional array, optional
+// top-k threshold.  Loads VEC consecutive logits starting at element x0.
+template <typename T, bool CFG>
+struct Row {
+  const T* cond;
+  const T* uncond;
+  float scale;
+  float thr;  // entries below thr become -inf (thr = -inf: no filter)
+  static constexpr int kVec = Elem<T>::kVec;
+
+  __device__ __forceinline__ void load_vec(int x0, float (&z)[Elem<T>::kVec]) const {
+    Elem<T>::load_vec(cond + x0, z);
+    if (CFG) {
+      float u[kVec];
+      Elem<T>::load_vec(uncond + x0, u);
+#pragma unroll
+      for (int k = 0; k < kVec; ++k) z[k] = cfg_mix(z[k], u[k], scale);
+    }
+  }
+  __device__ __forceinline__ float load_one(int x) const {
+    float z = Elem<T>::load_one(cond + x);
+    if (CFG) z = cfg_mix(z, Elem<T>::load_one(uncond + x), scale);
+    return z;
+  }
+  // vector when allowed, otherwise bounds-checked scalars; out-of-range -> -inf
+  __device__ __forceinline__ void load_tile(int x0, int V, bool vec_ok, float (&z)[Elem<T>::kVec]) const {
+    if (vec_ok) {
+      if (x0 < V) load_vec(x0, z);
+      else {
+#pragma unroll
+        for (int k = 0; k < kVec; ++k) z[k] = CSD_NEG_INF;
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < kVec; ++k) z[k] = (x0 + k < V) ? load_one(x0 + k) : CSD_NEG_INF;
+    }
+  }
+  __device__ __forceinline__ float filter(float z) const { return z < thr ? CSD_NEG_INF : z; }
+};
+
+// ============================ kernel 1: row statistics ==========================
+struct StatsArgs {
+  const void* target;
+  const void* draft;
+  const void* target_uncond;
+  const void* draft_uncond;
+  float cfg_scale;
+  int B, gamma, T, V;
+  int64_t tstride, dstride;  // elements
+  int parts;                 // parts per row
+  int part_elems;            // elements per part (multiple of the vector width)
+  int n_items;               // B * (T + gamma) * parts
+  int vec_ok;
+  float2* partials;          // [B * (T + gamma)][parts]
+};
+
+// U = 16-byte loads per thread per array per item
+template <typename T, bool CFG, int U>
+__global__ void __launch_bounds__(kStatsThreads) row_stats_kernel(const StatsArgs a) {
+  constexpr int VEC = Elem<T>::kVec;
+  __shared__ float sh_m[2][kStatsThreads / 32];
+  __shared__ float sh_s[2][kStatsThreads / 32];
+  pdl_launch_dependents();  // the finishing kernel may become resident as soon as blocks retire
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rows_per_seq = a.T + a.gamma;
+  int buf = 0;
+  for (int item = blockIdx.x; item < a.n_items; item += gridDim.x, buf ^= 1) {
+    const int part = item % a.parts;
+    const int row_id = item / a.parts;
+    const int b = row_id / rows_per_seq;
+    const int r = row_id - b * rows_per_seq;
+    Row<T, CFG> row;
+    row.scale = a.cfg_scale;
+    row.thr = CSD_NEG_INF;
+    if (r < a.T) {
+      const int64_t off = (int64_t)b * a.tstride + (int64_t)r * a.V;
+      row.cond = reinterpret_cast<const T*>(a.target) + off;
+      row.uncond = CFG ? reinterpret_cast<const T*>(a.target_uncond) + off : nullptr;
+    } else {
+      const int64_t off = (int64_t)b * a.dstride + (int64_t)(r - a.T) * a.V;
+      row.cond = reinterpret_cast<const T*>(a.draft) + off;
+      row.uncond = CFG ? reinterpret_cast<const T*>(a.draft_uncond) + off : nullptr;
+    }
+    const int x_begin = part * a.part_elems;
+    const int x_end = min(a.V, x_begin + a.part_elems);
+
+    float m, s;
+    if (a.vec_ok) {
+      float z[U][VEC];
+#pragma unroll
+      for (int k = 0; k < U; ++k) {
+        const int x0 = x_begin + (k * kStatsThreads + tid) * VEC;
+        if (x0 < x_end) row.load_vec(x0, z[k]);
+        else {
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) z[k][e] = CSD_NEG_INF;
+        }
+      }
+      // all loads are in flight before the first use
+      float flat[U * VEC];
+#pragma unroll
+      for (int k = 0; k < U; ++k)
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) flat[k * VEC + e] = z[k][e];
+      stat_of_values(flat, m, s);
+      // a thread whose slots were all padding reports the identity
+      // (padding entries are -inf and contribute exp(-inf) = 0 next to real values)
+      if (x_begin + tid * VEC >= x_end) { m = CSD_NEG_INF; s = -1.0f; }
+    } else {
+      m = CSD_NEG_INF; s = -1.0f;
+      for (int x = x_begin + tid; x < x_end; x += kStatsThreads) {
+        float one[1] = {row.load_one(x)};
+        float m1, s1;
+        stat_of_values(one, m1, s1);
+        stat_merge(m, s, m1, s1);
+      }
+    }
+    stat_warp_allreduce(m, s);
+    if (lane == 0) { sh_m[buf][warp] = m; sh_s[buf][warp] = s; }
+    __syncthreads();
+    if (warp == 0) {
+      float mm = lane < kStatsThreads / 32 ? sh_m[buf][lane] : CSD_NEG_INF;
+      float ss = lane < kStatsThreads / 32 ? sh_s[buf][lane] : -1.0f;
+#pragma unroll
+      for (int off = kStatsThreads / 64; off > 0; off >>= 1) {
+        float m2 = __shfl_xor_sync(0xffffffffu, mm, off);
+        float s2 = __shfl_xor_sync(0xffffffffu, ss, off);
+        stat_merge(mm, ss, m2, s2);
+      }
+      if (lane == 0) a.partials[(int64_t)row_id * a.parts + part] = make_float2(mm, ss);
+    }
+    // double-buffered staging: the next item writes the other buffer, and the
+    // barrier of that item orders this item's reads before the buffer's reuse
+  }
+}
+
+// ============================ kernel 2: per-sequence finish =====================
+struct FinishArgs {
+  const void* target;
+  const void* draft;
+  const void* target_uncond;
+  const void* draft_uncond;
+  float cfg_scale;
+  int B, gamma, T, V;
+  int64_t tstride, dstride;
+  int parts;
+  int vec_ok;
+  int use_topk;
+  const float2* partials;   // [B*(T+gamma)][parts]
+  const float* thresholds;  // [B*(T+gamma)] (top-k only)
+  const int32_t* tokens;
+  const float* uniforms;
+  const float* schedule;
+  int32_t* out_tokens;
+  int32_t* out_accept_len;
+  int32_t* out_status;
+  float* dbg_p;
+  float* dbg_q;
+  float* dbg_f;
+  float* dbg_G;
+};
+
+struct PairCtx {  // what Eq. opt_G needs at one position
+  float Mt, St, Md, Sd;   // (m, s) of the target and drafter rows
+  float inv_t;            // 1 / (1 + St)
+  float inv_den;          // 1 / ((1 + St)(1 + Sd))
+  float one_minus_omega;
+  int mode;               // 0: Eq. opt_G; 1: weights = P (bonus draw, unusable drafter row, Z fallback)
+};
+
+// unnormalised weight of one candidate token.  P - Q is formed as
+// ((et - ed) + (et*Sd - ed*St)) / ((1+St)(1+Sd)), which has no cancellation
+// beyond that of the inputs when both rows peak on the same token.
+__device__ __forceinline__ float weight_of(float zt, float zd, const PairCtx& c) {
+  const float et = ex2f((zt - c.Mt) * kLog2e);
+  if (c.mode == 1) return et * c.inv_t;
+  const float ed = ex2f((zd - c.Md) * kLog2e);
+  const float pq = ((et - ed) + (et * c.Sd - ed * c.St)) * c.inv_den;  // P - Q
+  const float alt = c.one_minus_omega * et * c.inv_t;                    // (1 - omega) P
+  return fmaxf(0.0f, fmaxf(pq, alt));
+}
+
+__device__ __forceinline__ double warp_sum_double(double v) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  return v;
+}
+__device__ __forceinline__ double warp_incl_scan_double(double v, int lane) {
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    double t = __shfl_up_sync(0xffffffffu, v, off);
+    if (lane >= off) v += t;
+  }
+  return v;
+}
+
+template <typename T, bool CFG>
+__global__ void __launch_bounds__(kFinishThreads, 1) finish_kernel(const FinishArgs a) {
+  constexpr int VEC = Elem<T>::kVec;
+  constexpr int TILE = 32 * VEC;
+  extern __shared__ double tile_sums[];  // one fp64 sum per tile of TILE tokens
+  __shared__ float sh_M[2][kMaxGamma + 1], sh_S[2][kMaxGamma + 1], sh_thr[2][kMaxGamma + 1];
+  __shared__ int sh_acc[kMaxGamma], sh_flag[kMaxGamma + 1], sh_valid[2][kMaxGamma + 1];
+  __shared__ int sh_pick_tile;
+  __shared__ double sh_pick_prefix, sh_Z;
+  __shared__ int sh_token;
+
+  const int b = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int L = a.gamma, V = a.V;
+  const int rows_per_seq = a.T + L;
+  const T* tgt = reinterpret_cast<const T*>(a.target) + (int64_t)b * a.tstride;
+  const T* dft = reinterpret_cast<const T*>(a.draft) + (int64_t)b * a.dstride;
+  const T* tgt_u = CFG ? reinterpret_cast<const T*>(a.target_uncond) + (int64_t)b * a.tstride : nullptr;
+  const T* dft_u = CFG ? reinterpret_cast<const T*>(a.draft_uncond) + (int64_t)b * a.dstride : nullptr;
+
+  pdl_wait();  // everything the statistics kernel wrote is visible from here on
+
+  // ---- 1. per position: merge parts, gather, Eq. relax, accept test ------------
+  for (int i = warp; i <= L; i += kFinishThreads / 32) {
+    const bool has_t = i < a.T, has_d = i < L;
+    float M[2] = {CSD_NEG_INF, CSD_NEG_INF}, S[2] = {-1.0f, -1.0f};
+    float thr[2] = {CSD_NEG_INF, CSD_NEG_INF};
+#pragma unroll
+    for (int which = 0; which < 2; ++which) {
+      if (which == 0 ? !has_t : !has_d) continue;
+      const int64_t row_id = (int64_t)b * rows_per_seq + (which == 0 ? i : a.T + i);
+      float m = CSD_NEG_INF, s = -1.0f;
+      for (int p = lane; p < a.parts; p += 32) {
+        const float2 v = a.partials[row_id * a.parts + p];
+        stat_merge(m, s, v.x, v.y);
+      }
+      stat_warp_allreduce(m, s);
+      M[which] = m; S[which] = s;
+      if (a.use_topk) thr[which] = a.thresholds[row_id];
+    }
+    if (lane == 0) {
+      const bool t_ok = has_t && M[0] > CSD_NEG_INF && M[0] < CSD_POS_INF && S[0] >= 0.0f && S[0] < CSD_POS_INF;
+      const bool d_ok = has_d && M[1] > CSD_NEG_INF && M[1] < CSD_POS_INF && S[1] >= 0.0f && S[1] < CSD_POS_INF;
+      sh_M[0][i] = M[0]; sh_S[0][i] = S[0]; sh_thr[0][i] = thr[0];
+      sh_M[1][i] = M[1]; sh_S[1][i] = S[1]; sh_thr[1][i] = thr[1];
+      sh_valid[0][i] = t_ok; sh_valid[1][i] = d_ok;
+      int flag = 0;
+      if (i < L) {
+        const int tok = a.tokens[(int64_t)b * L + i];
+        const bool tok_ok = tok >= 0 && tok < V;
+        float omega = a.schedule[i];
+        omega = omega >= 0.0f ? omega : 0.0f;
+        float f = 0.0f, p = __int_as_float(0x7fc00000), q = p;
+        if (!t_ok || !d_ok) flag = 1;
+        else if (!tok_ok) flag = 2;
+        else {
+          Row<T, CFG> rt{tgt + (int64_t)i * V, CFG ? tgt_u + (int64_t)i * V : nullptr, a.cfg_scale, thr[0]};
+          Row<T, CFG> rd{dft + (int64_t)i * V, CFG ? dft_u + (int64_t)i * V : nullptr, a.cfg_scale, thr[1]};
+          const float dt = rt.filter(rt.load_one(tok)) - M[0];
+          const float dd = rd.filter(rd.load_one(tok)) - M[1];
+          p = ex2f(dt * kLog2e) / (1.0f + S[0]);
+          q = ex2f(dd * kLog2e) / (1.0f + S[1]);
+          if (dd == CSD_NEG_INF) f = 1.0f;         // q = 0: p/q = +inf, and 0/0 := 1
+          else if (dt == CSD_NEG_INF) f = 0.0f;    // p = 0 < q
+          else f = fminf(1.0f, omega * ex2f((dt - dd) * kLog2e) * ((1.0f + S[1]) / (1.0f + S[0])));
+        }
+        const float r = a.uniforms[(int64_t)b * (L + 1) + i];
+        sh_acc[i] = (r <= f) ? 1 : 0;
+        if (a.dbg_p) a.dbg_p[(int64_t)b * L + i] = p;
+        if (a.dbg_q) a.dbg_q[(int64_t)b * L + i] = q;
+        if (a.dbg_f) a.dbg_f[(int64_t)b * L + i] = f;
+      }
+      sh_flag[i] = flag;
+    }
+  }
+  __syncthreads();
+
+  // ---- 2. tau = number of leading accepts (the for/break of Algorithm 1) --------
+  int tau = 0;
+  while (tau < L && sh_acc[tau]) ++tau;
+  int status = 0;
+  for (int i = 0; i <= min(tau, L - 1); ++i) status |= sh_flag[i];
+
+  // ---- 3. which row to draw from -------------------------------------------------
+  const int j = tau;  // 0-based row index of position tau+1 (j == L: bonus row)
+  PairCtx ctx;
+  bool draw = true;
+  if (j < L) {
+    if (!sh_valid[0][j]) draw = false;
+    ctx.mode = sh_valid[1][j] ? 0 : 1;
+  } else {
+    if (a.T == L + 1) {
+      ctx.mode = 1;
+      if (!sh_valid[0][L]) { draw = false; status |= 1; }
+    } else draw = false;
+  }
+  float* G_out = a.dbg_G ? a.dbg_G + (int64_t)b * V : nullptr;
+  const int ntiles = (V + TILE - 1) / TILE;
+  int token = -1;
+
+  if (draw) {
+    ctx.Mt = sh_M[0][j]; ctx.St = sh_S[0][j];
+    ctx.Md = j < L ? sh_M[1][j] : 0.0f; ctx.Sd = j < L ? sh_S[1][j] : 0.0f;
+    ctx.inv_t = 1.0f / (1.0f + ctx.St);
+    ctx.inv_den = ctx.inv_t / (1.0f + ctx.Sd);
+    float omega = j < L ? a.schedule[j] : 0.0f;
+    omega = omega >= 0.0f ? omega : 0.0f;
+    ctx.one_minus_omega = 1.0f - omega;
+    Row<T, CFG> rt{tgt + (int64_t)j * V, CFG ? tgt_u + (int64_t)j * V : nullptr, a.cfg_scale, sh_thr[0][j]};
+    Row<T, CFG> rd = rt;
+    if (j < L) rd = Row<T, CFG>{dft + (int64_t)j * V, CFG ? dft_u + (int64_t)j * V : nullptr, a.cfg_scale, sh_thr[1][j]};
+    const float u = a.uniforms[(int64_t)b * (L + 1) + L];
+
+    for (int attempt = 0; attempt < 2; ++attempt) {
+      // ---- 4. Eq. opt_G weights, one fp64 sum per tile ---------------------------
+      for (int tile = warp; tile < ntiles; tile += kFinishThreads / 32) {
+        const int x0 = tile * TILE + lane * VEC;
+        float zt[VEC], zd[VEC];
+        rt.load_tile(x0, V, a.vec_ok, zt);
+        if (ctx.mode == 0) rd.load_tile(x0, V, a.vec_ok, zd);
+        float acc = 0.0f;
+#pragma unroll
+        for (int k = 0; k < VEC; ++k)
+          acc += weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
+        const double tsum = warp_sum_double((double)acc);
+        if (lane == 0) tile_sums[tile] = tsum;
+      }
+      __syncthreads();
+      // ---- 5. locate the tile that holds the crossing C(x) > u Z ------------------
+      if (warp == 0) {
+        const int chunk = (ntiles + 31) / 32;
+        const int t0 = lane * chunk, t1 = min(ntiles, t0 + chunk);
+        double local = 0.0;
+        for (int t = t0; t < t1; ++t) local += tile_sums[t];
+        const double incl = warp_incl_scan_double(local, lane);
+        const double Z = __shfl_sync(0xffffffffu, incl, 31);
+        const double target = (double)u * Z;
+        const bool mine = incl > target && local > 0.0;
+        const unsigned ballot = __ballot_sync(0xffffffffu, mine);
+        if (lane == 0) { sh_Z = Z; sh_pick_tile = -1; }
+        __syncwarp();
+        if (ballot != 0 && lane == __ffs(ballot) - 1) {
+          double c = incl - local, c_pick = c;
+          int pick = t0;
+          for (int t = t0; t < t1; ++t) {
+            const double v = tile_sums[t];
+            if (v > 0.0) { pick = t; c_pick = c; }   // last tile with mass seen so far
+            if (c + v > target && v > 0.0) break;
+            c += v;
+          }
+          sh_pick_tile = pick;
+          sh_pick_prefix = c_pick;
+        }
+      }
+      __syncthreads();
+      const double Z = sh_Z;
+      if (!(Z > 0.0) || !(Z < (double)CSD_POS_INF)) {
+        if (attempt == 0 && ctx.mode == 0) {  // empty positive part: fall back to G := P_j
+          ctx.mode = 1;
+          status |= 4;
+          __syncthreads();
+          continue;
+        }
+        break;  // nothing to draw from
+      }
+      // ---- 6. scan inside that tile -------------------------------------------------
+      if (warp == 0) {
+        const int tile = sh_pick_tile;
+        const double target = (double)u * Z;
+        const int x0 = tile * TILE + lane * VEC;
+        float zt[VEC], zd[VEC];
+        rt.load_tile(x0, V, a.vec_ok, zt);
+        if (ctx.mode == 0) rd.load_tile(x0, V, a.vec_ok, zd);
+        double run[VEC];
+        double acc = 0.0;
+        int last_pos = -1;
+        unsigned posmask = 0;
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+          const float g = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
+          if (g > 0.0f) { last_pos = k; posmask |= 1u << k; }
+          acc += (double)g;
+          run[k] = acc;
+        }
+        const double before = sh_pick_prefix + (warp_incl_scan_double(acc, lane) - acc);
+        int first = -1;
+#pragma unroll
+        for (int k = VEC - 1; k >= 0; --k)
+          if (before + run[k] > target && ((posmask >> k) & 1u)) first = k;
+        const unsigned hit = __ballot_sync(0xffffffffu, first >= 0);
+        const unsigned pos = __ballot_sync(0xffffffffu, last_pos >= 0);
+        if (hit != 0) {
+          if (lane == __ffs(hit) - 1) sh_token = x0 + first;
+        } else if (pos != 0) {  // rounding left no crossing: last token with positive weight
+          if (lane == 31 - __clz(pos)) sh_token = x0 + last_pos;
+        } else if (lane == 0) sh_token = -1;
+      }
+      __syncthreads();
+      token = sh_token;
+      // ---- 7. optional: write the distribution drawn from ------------------------------
+      if (G_out) {
+        const float invZ = (float)(1.0 / Z);
+        for (int tile = warp; tile < ntiles; tile += kFinishThreads / 32) {
+          const int x0 = tile * TILE + lane * VEC;
+          float zt[VEC], zd[VEC];
+          rt.load_tile(x0, V, a.vec_ok, zt);
+          if (ctx.mode == 0) rd.load_tile(x0, V, a.vec_ok, zd);
+#pragma unroll
+          for (int k = 0; k < VEC; ++k)
+            if (x0 + k < V)
+              G_out[x0 + k] = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx) * invZ;
+        }
+      }
+      break;
+    }
+  }
+  if (G_out && token < 0)
+    for (int x = tid; x < V; x += kFinishThreads) G_out[x] = 0.0f;
+
+  // ---- 8. emit x_{1:tau+1} ---------------------------------------------------------
+  if (tid <= L) {
+    int v = -1;
+    if (tid < tau) v = a.tokens[(int64_t)b * L + tid];
+    else if (tid == tau) v = token;
+    a.out_tokens[(int64_t)b * (L + 1) + tid] = v;
+  }
+  if (tid == 0) {
+    a.out_accept_len[b] = tau;
+    if (a.out_status) a.out_status[b] = status;
+  }
+}
+
+}  // namespace csd

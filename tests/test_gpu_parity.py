@@ -1,0 +1,249 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same
+seeded inputs and the same supplied uniforms.  Accepted lengths and tokens must be identical
+except for decisions the oracle flags as within 1e-6 of a threshold (counted); probabilities and
+the resampling distribution within 1e-5 (fp32 logits) / 2e-3 (bf16 logits) absolute."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+import oracle
+import paper_2601_09212_b200 as csd
+from paper_2601_09212_b200 import workloads as W
+from gpu_util import check, run_gpu, run_oracle
+
+DEV = "cuda"
+
+
+def sched(L, kind="exp"):
+    if kind == "vanilla":
+        return np.ones(L, np.float32)
+    return csd.csd_make_schedule(1, 1.1, 0.7, L)
+
+
+def assert_ok(rep, max_near_frac=0.02):
+    assert rep.ok, rep.summary() + " :: " + str(rep.unexplained[:5])
+    assert rep.tau_mismatch_near + rep.token_mismatch_near <= max(2, max_near_frac * rep.n_seq), rep.summary()
+
+
+@pytest.mark.parametrize("dtype", [W.F32, W.BF16])
+@pytest.mark.parametrize("V", [2, 8, 33, 1000, 1024, 4100, 16384, 20000])
+@pytest.mark.parametrize("bonus", [False, True])
+def test_shapes_small(dtype, V, bonus):
+    L = 5
+    w = W.make("t", B=7, gamma=L, V=V, dtype=dtype, rho=0.8, bonus_row=bonus, schedule=sched(L),
+               seed=V, device=DEV)
+    rep, got, ref = check(w)
+    assert_ok(rep)
+
+
+@pytest.mark.parametrize("L", [1, 2, 16, 31, 32])
+def test_gamma_range(L):
+    w = W.make("t", B=5, gamma=L, V=2048, rho=0.95, bonus_row=True,
+               schedule=csd.csd_make_schedule(0, 1.5, 0.0, L), seed=L, device=DEV)
+    rep, got, ref = check(w)
+    assert_ok(rep)
+    assert got["accept_len"].max() > 2 or L <= 2
+
+
+@pytest.mark.parametrize("name,rho,kind", [("C1", 0.9, "exp"), ("C2", 0.7, "vanilla"), ("C2", 0.9, "exp"),
+                                           ("C2", 0.97, "vanilla"), ("C2", 0.97, "exp")])
+def test_config_c1_c2(name, rho, kind):
+    L = W.CONFIGS[name]["gamma"]
+    reps = []
+    for step in range(3):
+        w = W.config(name, step=step, rho=rho, schedule=sched(L, kind), device=DEV)
+        rep, got, ref = check(w)
+        assert_ok(rep)
+        reps.append(rep)
+    print(name, rho, kind, reps[0].summary())
+
+
+def test_vanilla_schedule_matches_plain_sd_on_gpu():
+    """omega == 1: the distribution drawn from is Norm([P - Q]_+) (Proposition 2)."""
+    w = W.make("t", B=32, gamma=4, V=4096, rho=0.8, schedule=sched(4, "vanilla"), seed=5, device=DEV)
+    got = run_gpu(w)
+    P = torch.softmax(w.target_logits.double(), -1).cpu().numpy()
+    Q = torch.softmax(w.draft_logits.double(), -1).cpu().numpy()
+    n = 0
+    for b in range(32):
+        j = got["accept_len"][b]
+        if j < 4:
+            van = np.maximum(P[b, j] - Q[b, j], 0)
+            assert np.abs(got["G"][b] - van / van.sum()).max() < 1e-5
+            n += 1
+    assert n > 0
+    assert abs(got["G"].sum(-1)[got["accept_len"] < 4] - 1).max() < 1e-4
+
+
+def test_bf16_large_batch_c4_sampled():
+    """Full-size heavy-tailed config: oracle on a sample of sequences."""
+    L = W.CONFIGS["C4"]["gamma"]
+    w = W.config("C4", step=0, schedule=sched(L), device=DEV)
+    rows = np.arange(0, 256, 8)
+    rep, got, ref = check(w, rows=rows, want_dbg=True)
+    assert_ok(rep)
+    # properties that hold for every sequence
+    tau = got["accept_len"]
+    assert tau.min() >= 0 and tau.max() <= L
+    tok = w.draft_tokens.cpu().numpy()
+    for b in range(256):
+        assert np.array_equal(got["tokens"][b, :tau[b]], tok[b, :tau[b]])
+        assert np.all(got["tokens"][b, tau[b] + 1:] == -1)
+        if tau[b] < L:
+            assert 0 <= got["tokens"][b, tau[b]] < w.V
+            assert abs(got["G"][b].sum() - 1) < 1e-3 and got["G"][b].min() >= 0
+            assert got["G"][b, got["tokens"][b, tau[b]]] > 0
+
+
+def test_cfg_mix_fused():
+    L = 6
+    for dtype in (W.F32, W.BF16):
+        w = W.make("t", B=9, gamma=L, V=3000 if dtype == W.F32 else 4096, dtype=dtype, cfg=True,
+                   cfg_scale=4.0, rho=0.9, bonus_row=True, schedule=sched(L), seed=11, device=DEV)
+        rep, got, ref = check(w)
+        assert_ok(rep)
+
+
+def test_batch_strides_and_unaligned_views():
+    """Rows embedded in a larger buffer (batch stride > rows*V) and a base pointer that is
+    only element-aligned (forces the scalar path)."""
+    L, V, B = 4, 1000, 6
+    w = W.make("t", B=B, gamma=L, V=V, rho=0.85, bonus_row=True, schedule=sched(L), seed=2, device=DEV)
+    ref_rep, got_plain, ref = check(w)
+    assert_ok(ref_rep)
+    pad = 24
+    big_t = torch.zeros(B, (L + 1) * V + pad, device=DEV)
+    big_d = torch.zeros(B, L * V + pad, device=DEV)
+    big_t[:, :(L + 1) * V] = w.target_logits.reshape(B, -1)
+    big_d[:, :L * V] = w.draft_logits.reshape(B, -1)
+    out_t = torch.empty(B, L + 1, dtype=torch.int32, device=DEV)
+    out_l = torch.empty(B, dtype=torch.int32, device=DEV)
+    prm = csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
+                          out_t, out_l, workspace=csd.new_workspace(B, L, V, w.dtype))
+    prm.target_logits = big_t.data_ptr()
+    prm.draft_logits = big_d.data_ptr()
+    prm.target_batch_stride = big_t.shape[1]
+    prm.draft_batch_stride = big_d.shape[1]
+    csd.csd_verify_ex(prm)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_t.cpu().numpy(), got_plain["tokens"])
+    assert np.array_equal(out_l.cpu().numpy(), got_plain["accept_len"])
+    # element-aligned only: shift everything by one float
+    flat_t = torch.zeros(B * (L + 1) * V + 1, device=DEV)
+    flat_d = torch.zeros(B * L * V + 1, device=DEV)
+    flat_t[1:] = w.target_logits.reshape(-1)
+    flat_d[1:] = w.draft_logits.reshape(-1)
+    prm.target_logits = flat_t.data_ptr() + 4
+    prm.draft_logits = flat_d.data_ptr() + 4
+    prm.target_batch_stride = (L + 1) * V
+    prm.draft_batch_stride = L * V
+    csd.csd_verify_ex(prm)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_t.cpu().numpy(), got_plain["tokens"])
+    assert np.array_equal(out_l.cpu().numpy(), got_plain["accept_len"])
+
+
+def test_bad_data_is_reported_not_trapped():
+    B, L, V = 5, 3, 64
+    w = W.make("t", B=B, gamma=L, V=V, rho=0.9, bonus_row=True, schedule=np.full(L, 1e6, np.float32),
+               seed=2, device=DEV)
+    w.draft_logits[0, 1, 5] = float("nan")
+    w.target_logits[1, 0, 7] = float("inf")
+    w.draft_tokens[2, 2] = V
+    w.draft_tokens[3, 0] = -1
+    rep, got, ref = check(w)
+    assert_ok(rep)
+    assert got["accept_len"].tolist() == [1, 0, 2, 0, 3]
+    assert got["status"].tolist() == [1, 1, 2, 2, 0]
+    assert got["tokens"][1, 0] == -1
+    # -inf entries are legal (masked tokens); a row of only -inf is not
+    w2 = W.make("t", B=2, gamma=2, V=40, rho=0.9, schedule=sched(2), seed=3, device=DEV)
+    w2.target_logits[0, 0, :20] = float("-inf")
+    w2.draft_logits[0, 1, 3] = float("-inf")
+    w2.target_logits[1, 0, :] = float("-inf")
+    rep, got, ref = check(w2)
+    assert_ok(rep)
+    assert got["status"][1] == 1
+
+
+def test_identical_models_and_zero_omega():
+    L = 3
+    w = W.make("t", B=16, gamma=L, V=512, rho=1.0, schedule=np.array([1.0, 0.3, 0.0], np.float32),
+               seed=6, device=DEV)
+    w.draft_logits.copy_(w.target_logits[:, :L])
+    rep, got, ref = check(w)
+    assert_ok(rep)
+    assert np.all(got["accept_len"] >= 1) and np.all(got["accept_len"] <= 2)
+
+
+def test_simple_form_and_determinism():
+    L, V, B = 8, 16384, 16
+    w = W.config("C2", step=1, schedule=sched(L), device=DEV)
+    out_t = torch.empty(B, L + 1, dtype=torch.int32, device=DEV)
+    out_l = torch.empty(B, dtype=torch.int32, device=DEV)
+    csd.csd_verify(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
+                   out_t, out_l)
+    torch.cuda.synchronize()
+    got = run_gpu(w, want_dbg=False)
+    assert np.array_equal(out_t.cpu().numpy(), got["tokens"])
+    assert np.array_equal(out_l.cpu().numpy(), got["accept_len"])
+    for _ in range(3):      # same inputs, same outputs
+        again = run_gpu(w, want_dbg=False)
+        assert np.array_equal(again["tokens"], got["tokens"])
+    # a second, larger problem grows the internal workspace
+    w2 = W.make("t", B=40, gamma=8, V=16384, rho=0.9, schedule=sched(8), seed=9, device=DEV)
+    out_t2 = torch.empty(40, 9, dtype=torch.int32, device=DEV)
+    out_l2 = torch.empty(40, dtype=torch.int32, device=DEV)
+    csd.csd_verify(w2.target_logits, w2.draft_logits, w2.draft_tokens, w2.uniforms, w2.relax_schedule,
+                   out_t2, out_l2)
+    torch.cuda.synchronize()
+    got2 = run_gpu(w2, want_dbg=False)
+    assert np.array_equal(out_t2.cpu().numpy(), got2["tokens"])
+
+
+def test_host_buffer_form():
+    L, V, B = 4, 4096, 8
+    w = W.make("t", B=B, gamma=L, V=V, dtype=W.BF16, rho=0.9, bonus_row=True, schedule=sched(L), seed=4,
+               device=DEV)
+    got = run_gpu(w, want_dbg=False)
+    pin = lambda t: t.cpu().pin_memory()
+    h = dict(t=pin(w.target_logits), d=pin(w.draft_logits), tok=pin(w.draft_tokens), u=pin(w.uniforms),
+             s=pin(w.relax_schedule))
+    out_t = torch.empty(B, L + 1, dtype=torch.int32).pin_memory()
+    out_l = torch.empty(B, dtype=torch.int32).pin_memory()
+    out_s = torch.empty(B, dtype=torch.int32).pin_memory()
+    prm = csd.make_params(h["t"], h["d"], h["tok"], h["u"], h["s"], out_t, out_l, out_status=out_s, host=True)
+    n = csd.csd_host_staging_size(prm)
+    assert n > w.logits_bytes()
+    staging = torch.empty(n, dtype=torch.uint8, device=DEV)
+    csd.csd_verify_host(prm, staging)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_t.numpy(), got["tokens"])
+    assert np.array_equal(out_l.numpy(), got["accept_len"])
+    assert np.array_equal(out_s.numpy(), got["status"])
+
+
+def test_argument_errors():
+    w = W.make("t", B=2, gamma=2, V=64, schedule=sched(2), device=DEV)
+    out_t = torch.empty(2, 3, dtype=torch.int32, device=DEV)
+    out_l = torch.empty(2, dtype=torch.int32, device=DEV)
+    prm = csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
+                          out_t, out_l, workspace=csd.new_workspace(2, 2, 64, 0))
+    lib = csd.library()
+    import ctypes as C
+    bad = csd.csd_params.from_buffer_copy(prm); bad.workspace_bytes = 16
+    assert lib.csd_verify_ex(C.byref(bad)) == -4
+    bad = csd.csd_params.from_buffer_copy(prm); bad.gamma = 33
+    assert lib.csd_verify_ex(C.byref(bad)) == -2
+    bad = csd.csd_params.from_buffer_copy(prm); bad.dtype = 5
+    assert lib.csd_verify_ex(C.byref(bad)) == -3
+    bad = csd.csd_params.from_buffer_copy(prm); bad.out_tokens = None
+    assert lib.csd_verify_ex(C.byref(bad)) == -1
+    bad = csd.csd_params.from_buffer_copy(prm); bad.target_uncond = prm.target_logits
+    assert lib.csd_verify_ex(C.byref(bad)) == -5
+    assert lib.csd_verify_ex(None) == -1
