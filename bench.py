@@ -1,0 +1,419 @@
+#!/usr/bin/env python
+"""Throughput of the batched verify-and-resample round of Cool-SD on B200.
+
+A "step" is one call of the whole path (row statistics, relaxed acceptance test, first
+rejection, optimal resampling distribution, inverse-CDF draw, emit) over one batch of
+synthetic logits.  Default workload: B=64 sequences x gamma=8 drafted positions x V=16384
+image tokens, bf16 logits, conditional/unconditional rows mixed on load (scale 4) and top-k
+1000 before the softmax, annealed schedule delta=1.1, nu=0.7.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl native|reference] [--workload C3]
+
+One JSON line on stdout (rank 0).  `value` is verified draft tokens per second with the inputs
+resident in HBM (a ring of distinct step inputs larger than L2, replayed as a CUDA graph);
+`e2e` is the same metric through the host-buffer entry point, host->device and device->host
+copies inside the timed region; `roofline` compares the step's algorithmic bytes with the
+measured HBM copy bandwidth; `cpu_baseline` is the fp64 CPU oracle timed on a bounded sample.
+With N > 1 every rank runs the same batch shape on its own GPU (sequences are independent: no
+exchange step, weak scaling).  `--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "verified_draft_tokens_per_sec"
+UNIT = "tokens/s"
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
+# one ncu capture, see profiles/).  Valid only for the kernel sources with this digest.
+NCU_TRAFFIC = {"sources_sha256": None, "workload": None, "bytes_per_launch": None}
+
+
+def sources_digest() -> str:
+    h = hashlib.sha256()
+    d = os.path.join(ROOT, "paper_2601_09212_b200", "csrc")
+    for name in sorted(os.listdir(d)):
+        with open(os.path.join(d, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks: NVML polled from a thread while the timed region runs (reading only)
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, pci_bus_id: str, period_s: float = 0.002):
+        self.index, self.period = pci_bus_id, period_s
+        self.samples, self.reasons, self.power = [], set(), []
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._nvml = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nvml = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByPciBusId(pci_bus_id.encode())
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nvml = None
+
+    def sample_once(self):
+        if self._nvml is None:
+            return
+        n = self._nvml
+        try:
+            self.samples.append(int(n.nvmlDeviceGetClockInfo(self._h, n.NVML_CLOCK_SM)))
+            r = int(n.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+            for bit, name in self.REASONS.items():
+                if r & bit:
+                    self.reasons.add(name)
+            self.power.append(n.nvmlDeviceGetPowerUsage(self._h) / 1000.0)
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self.sample_once()
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self._nvml is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self) -> dict:
+        if self._nvml is None or not self.samples:
+            return self._smi_fallback()
+        return {"sm_mhz": int(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w_max": round(max(self.power), 1) if self.power else None, "source": "nvml"}
+
+    def _smi_fallback(self) -> dict:
+        try:
+            out = subprocess.run(
+                ["nvidia-smi", f"--id={self.index}", "--query-gpu=clocks.sm,clocks.max.sm,"
+                 "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+                 "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap",
+                 "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=20).stdout
+            f = [x.strip() for x in out.strip().split(",")]
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            return {"sm_mhz": int(f[0]), "sm_max_mhz": int(f[1]),
+                    "reasons": [n for n, v in zip(names, f[2:6]) if v.lower().startswith("active")],
+                    "samples": 1, "source": "nvidia-smi after the timed region"}
+        except Exception as e:  # noqa: BLE001
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "source": f"unavailable: {e}"}
+
+
+# ---------------------------------------------------------------------------------------------
+def workload_kwargs(name: str) -> dict:
+    from paper_2601_09212_b200 import workloads as W
+    kw = dict(W.CONFIGS[name])
+    kw.pop("steps", None)
+    return kw
+
+
+def describe(name: str, kw: dict, sched_desc: str) -> dict:
+    from paper_2601_09212_b200 import workloads as W
+    d = {"workload": name, "B": kw["B"], "gamma": kw["gamma"], "V": kw["V"],
+         "logits": "bf16" if kw.get("dtype", W.F32) == W.BF16 else "fp32",
+         "guidance_mix": bool(kw.get("cfg", False)), "cfg_scale": kw.get("cfg_scale", 1.0) if kw.get("cfg") else None,
+         "top_k": kw.get("top_k", 0), "rho": kw.get("rho"), "law": kw.get("law", "gauss"),
+         "schedule": sched_desc, "target_rows": kw["gamma"]}
+    return d
+
+
+def algorithmic_bytes(kw: dict) -> int:
+    """Bytes one step must move: every stored logit once, plus tokens, uniforms, schedule, outputs."""
+    from paper_2601_09212_b200 import workloads as W
+    e = 2 if kw.get("dtype", W.F32) == W.BF16 else 4
+    A = 2 if kw.get("cfg") else 1
+    B, L, V = kw["B"], kw["gamma"], kw["V"]
+    return e * V * B * A * (L + L) + 4 * B * L + 4 * B * (L + 1) + 4 * L + 4 * B * (L + 2)
+
+
+def oracle_schedule(L: int):
+    import oracle
+    return oracle.make_schedule(1, 1.1, 0.7, L).astype(np.float32)
+
+
+def time_oracle(name: str, kw: dict, n_steps: int, seqs_per_step: int, warm: int = 0, seed: int = 0,
+                device="cpu", ring: int = 4):
+    """Times the CPU oracle as it stands on `n_steps` steps of `seqs_per_step` sequences each, drawn
+    from a small ring of seeded batches with the workload's recipe (generated outside the timed
+    region).  Returns (seconds, sequences processed, threads)."""
+    import oracle
+    from paper_2601_09212_b200 import workloads as W
+    oracle.build()
+    L = kw["gamma"]
+    sched = oracle_schedule(L)
+    kw = dict(kw, B=int(seqs_per_step))
+    batches = []
+    for s in range(min(ring, warm + n_steps)):
+        w = W.make(name, seed=1000 + seed, step=s, schedule=sched, device=device, **kw)
+        batches.append((w, w.host_arrays()))
+    total_t, total_seq = 0.0, 0
+    for s in range(warm + n_steps):
+        w, h = batches[s % len(batches)]
+        t0 = time.perf_counter()
+        oracle.verify(h["target_logits"], h["draft_logits"], h["draft_tokens"], h["uniforms"],
+                      h["relax_schedule"], dtype=w.dtype, target_uncond=h["target_uncond"],
+                      draft_uncond=h["draft_uncond"], cfg_scale=w.cfg_scale, top_k=w.top_k,
+                      want_G=False, want_pqf=False)
+        dt = time.perf_counter() - t0
+        if s >= warm:
+            total_t += dt
+            total_seq += int(seqs_per_step)
+    return total_t, total_seq, oracle.num_threads()
+
+
+def run_reference(args) -> None:
+    """The CPU oracle as the reference arm: K timed steps, each a bounded sample of the workload
+    (a batch of fewer sequences, same recipe), sized so that the run takes about two minutes."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    name = args.workload
+    kw = workload_kwargs(name)
+    oracle.build()
+    threads = oracle.num_threads()
+    L, B = kw["gamma"], kw["B"]
+    side = min(B, threads)                     # sequences that run side by side, one per thread
+    t_round, _, _ = time_oracle(name, kw, 1, side, warm=1)
+    budget = 120.0
+    rounds = max(1, int(budget / (args.steps + args.warmup) / max(t_round, 1e-6)))
+    seqs = int(min(B, rounds * side))
+    t, nseq, _ = time_oracle(name, kw, args.steps, seqs, warm=args.warmup)
+    value = nseq * L / t
+    sample = (f"{seqs} of {B} sequences per step, {args.steps} steps over a ring of 4 seeded batches "
+              f"of the workload's recipe")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": describe(name, kw, "exp delta=1.1 nu=0.7"),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------
+def run_native(args) -> None:
+    import torch
+    import paper_2601_09212_b200 as csd
+    from paper_2601_09212_b200 import _build, workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    _build.build_library()
+    csd.library()
+
+    name = args.workload
+    kw = workload_kwargs(name)
+    B, L, V, dtype = kw["B"], kw["gamma"], kw["V"], kw.get("dtype", W.F32)
+    sched = csd.csd_make_schedule(1, 1.1, 0.7, L)
+    step_bytes = algorithmic_bytes(kw)
+    ring_n = max(4, -(-4 * L2_BYTES // step_bytes))          # ring of distinct inputs >= 4 x L2
+    ring_n = min(ring_n, 64)
+    ring = [W.make(name, seed=1 + rank, step=s, schedule=sched, device=dev, **kw) for s in range(ring_n)]
+    outs = [dict(tok=torch.empty(B, L + 1, dtype=torch.int32, device=dev),
+                 tau=torch.empty(B, dtype=torch.int32, device=dev),
+                 st=torch.empty(B, dtype=torch.int32, device=dev),
+                 ws=csd.new_workspace(B, L, V, dtype, dev)) for _ in range(ring_n)]
+    stream = torch.cuda.Stream(device=dev)
+    prms = [csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
+                            o["tok"], o["tau"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
+                            cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=o["st"], workspace=o["ws"],
+                            stream=stream) for w, o in zip(ring, outs)]
+    kernels_per_step = 3 if (0 < kw.get("top_k", 0) < V) else 2
+
+    def enqueue(i):
+        csd.csd_verify_ex(prms[i % ring_n])
+
+    # one lap of the ring as a CUDA graph: the launches inside are the library's own
+    with torch.cuda.stream(stream):
+        for i in range(ring_n):
+            enqueue(i)
+    stream.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        for i in range(ring_n):
+            enqueue(i)
+
+    def run_steps(k):
+        laps, rest = divmod(k, ring_n)
+        with torch.cuda.stream(stream):
+            for _ in range(laps):
+                graph.replay()
+            for i in range(rest):
+                enqueue(i)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    run_steps(max(args.warmup, 3))
+    barrier()
+    props = torch.cuda.get_device_properties(dev)
+    sampler = ClockSampler(f"{props.pci_domain_id:08x}:{props.pci_bus_id:02x}:{props.pci_device_id:02x}.0")
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    e0.record(stream)
+    run_steps(args.steps)
+    e1.record(stream)
+    sampler.sample_once()
+    barrier()
+    sampler.stop()
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+
+    # accepted lengths of the last lap (a property of the synthetic drafter, reported for context)
+    mean_emit = float(np.mean([o["tau"].float().mean().item() + 1.0 for o in outs]))
+
+    # ---- end to end: host buffers in, host results out, copies inside the timed region ----------
+    e2e_steps = max(1, min(args.steps, 48))
+    host_n = 2
+    pin = lambda t: None if t is None else t.cpu().pin_memory()
+    hprm, hkeep = [], []
+    for w in ring[:host_n]:
+        hb = dict(t=pin(w.target_logits), d=pin(w.draft_logits), tu=pin(w.target_uncond), du=pin(w.draft_uncond),
+                  tok=pin(w.draft_tokens), u=pin(w.uniforms), s=pin(w.relax_schedule),
+                  ot=torch.empty(B, L + 1, dtype=torch.int32).pin_memory(),
+                  ol=torch.empty(B, dtype=torch.int32).pin_memory(),
+                  os=torch.empty(B, dtype=torch.int32).pin_memory())
+        p = csd.make_params(hb["t"], hb["d"], hb["tok"], hb["u"], hb["s"], hb["ot"], hb["ol"],
+                            target_uncond=hb["tu"], draft_uncond=hb["du"], cfg_scale=w.cfg_scale, top_k=w.top_k,
+                            out_status=hb["os"], stream=stream, host=True)
+        hprm.append(p)
+        hkeep.append(hb)
+    staging = [torch.empty(csd.csd_host_staging_size(p), dtype=torch.uint8, device=dev) for p in hprm]
+    h2d = sum(t.numel() * t.element_size() for k, t in hkeep[0].items()
+              if t is not None and k in ("t", "d", "tu", "du", "tok", "u", "s"))
+    d2h = sum(hkeep[0][k].numel() * 4 for k in ("ot", "ol", "os"))
+    for i in range(3):
+        csd.csd_verify_host(hprm[i % host_n], staging[i % host_n])
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for i in range(e2e_steps):
+        csd.csd_verify_host(hprm[i % host_n], staging[i % host_n])
+    f1.record(stream)
+    barrier()
+    e2e_ms = f0.elapsed_time(f1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    # the host arrays now hold the last step's results; they must equal the device-resident run's
+    last = (e2e_steps - 1) % host_n
+    same = bool(np.array_equal(hkeep[last]["ot"].numpy(), outs[last]["tok"].cpu().numpy()))
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    tokens = B * L * args.steps * world
+    value = tokens / (ms * 1e-3)
+    peak, peak_kind = measured_peak()
+    step_s = ms * 1e-3 / args.steps
+    achieved = step_bytes / step_s / 1e9
+    digest = sources_digest()
+    traffic = None
+    if NCU_TRAFFIC["sources_sha256"] == digest and NCU_TRAFFIC["workload"] == name:
+        traffic = NCU_TRAFFIC["bytes_per_launch"]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": dict(describe(name, kw, "exp delta=1.1 nu=0.7"),
+                       parallelism=f"dp{world} (independent sequences, no exchange)",
+                       l2=f"ring of {ring_n} distinct step inputs, {ring_n * step_bytes / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2",
+                       launch="CUDA graph of one ring lap, replayed"),
+        "clocks": sampler.summary(),
+        "e2e": {"value": B * L * e2e_steps * world / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": e2e_steps, "entry": "csd_verify_host (pinned host buffers)",
+                "matches_device_run": same},
+        "gpu_launches": kernels_per_step * args.steps,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": traffic, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+                     "bytes_per_launch": step_bytes,
+                     "duration_us": step_s * 1e6,
+                     "note": "duration = timed region / steps: all kernels of a step, an upper bound on the row-statistics kernel"},
+        "emitted_tokens_per_step_mean": B * mean_emit,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        t1, n1, threads = time_oracle(name, kw, 1, B, device=dev)
+        n = int(min(64, max(1, round(12.0 / max(t1, 1e-3)))))
+        t, nseq, threads = time_oracle(name, kw, n, B, seed=7, device=dev)
+        line["cpu_baseline"] = {"value": nseq * L / t, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"{n} full steps ({nseq} sequences, ring of 4 seeded batches) of the "
+                                          f"same workload, {t:.1f} s wall"}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5760)
+    ap.add_argument("--warmup", type=int, default=64)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--workload", default="C3")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_native(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -61,13 +61,17 @@ Layout layout_for(int B, int gamma, int V, int dtype) {
   return l;
 }
 
-template <typename T, bool CFG, int U>
+template <typename T, bool CFG, int U, bool TOPK>
 cudaError_t launch_stats(const StatsArgs& a, int sms, cudaStream_t stream) {
-  auto kern = row_stats_kernel<T, CFG, U>;
-  int per_sm = 0;
-  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kStatsThreads, 0);
-  if (e != cudaSuccess) return e;
-  if (per_sm < 1) per_sm = 1;
+  auto kern = row_stats_kernel<T, CFG, U, TOPK>;
+  static int cached_per_sm = 0;  // a property of the kernel, the same on every B200
+  int per_sm = cached_per_sm;
+  if (per_sm == 0) {
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kStatsThreads, 0);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    cached_per_sm = per_sm;
+  }
   long long grid = (long long)sms * per_sm;
   if (grid > a.n_items) grid = a.n_items;
   kern<<<(unsigned)grid, kStatsThreads, 0, stream>>>(a);
@@ -75,13 +79,25 @@ cudaError_t launch_stats(const StatsArgs& a, int sms, cudaStream_t stream) {
 }
 
 template <typename T, bool CFG>
-cudaError_t launch_stats_u(const StatsArgs& a, int U, int sms, cudaStream_t stream) {
-  switch (U) {
-    case 8: return launch_stats<T, CFG, 8>(a, sms, stream);
-    case 4: return launch_stats<T, CFG, 4>(a, sms, stream);
-    case 2: return launch_stats<T, CFG, 2>(a, sms, stream);
-    default: return launch_stats<T, CFG, 1>(a, sms, stream);
+cudaError_t launch_stats_u(const StatsArgs& a, int U, bool topk, int sms, cudaStream_t stream) {
+  if (topk) {  // U is 1 or 4 here
+    return U == 4 ? launch_stats<T, CFG, 4, true>(a, sms, stream) : launch_stats<T, CFG, 1, true>(a, sms, stream);
   }
+  switch (U) {
+    case 8: return launch_stats<T, CFG, 8, false>(a, sms, stream);
+    case 4: return launch_stats<T, CFG, 4, false>(a, sms, stream);
+    case 2: return launch_stats<T, CFG, 2, false>(a, sms, stream);
+    default: return launch_stats<T, CFG, 1, false>(a, sms, stream);
+  }
+}
+
+template <typename T, bool CFG>
+cudaError_t launch_select(const SelectArgs& a, int sms, cudaStream_t stream) {
+  const long long rows = (long long)a.B * (a.T + a.gamma);
+  long long grid = 2LL * sms;
+  if (grid > rows) grid = rows;
+  topk_threshold_kernel<T, CFG><<<(unsigned)grid, kSelectThreads, 0, stream>>>(a);
+  return cudaGetLastError();
 }
 
 template <typename T, bool CFG>
@@ -122,7 +138,6 @@ int verify_impl(const csd_params& p) {
   if (p.top_k < 0) return CSD_ERR_ARG;
   if (cfg && !isfinite(p.cfg_scale)) return CSD_ERR_ARG;
   const bool topk = p.top_k > 0 && p.top_k < p.V;
-  if (topk) return CSD_ERR_ARG;  // not built yet
   const Layout lay = layout_for(p.B, p.gamma, p.V, p.dtype);
   if (!p.workspace || ((uintptr_t)p.workspace % kAlign) != 0 || p.workspace_bytes < lay.total)
     return CSD_ERR_WORKSPACE;
@@ -141,9 +156,10 @@ int verify_impl(const csd_params& p) {
   const long long rows = (long long)p.B * rows_per_seq;
 
   // part size: the largest that still leaves every SM several blocks to work on
-  int U = cfg ? 4 : 8;
+  int U = (cfg || topk) ? 4 : 8;
   auto parts_for = [&](int u) { return (p.V + kStatsThreads * u * vw - 1) / (kStatsThreads * u * vw); };
   while (U > 1 && rows * parts_for(U) < 4LL * sms) U >>= 1;
+  if (topk && U == 2) U = 1;
 
   StatsArgs sa;
   sa.target = p.target_logits; sa.draft = p.draft_logits;
@@ -156,6 +172,17 @@ int verify_impl(const csd_params& p) {
   sa.n_items = (int)(rows * sa.parts);
   sa.vec_ok = vec_ok ? 1 : 0;
   sa.partials = reinterpret_cast<float2*>((char*)p.workspace + lay.partials_off);
+  sa.thresholds = reinterpret_cast<const float*>((char*)p.workspace + lay.thresholds_off);
+
+  SelectArgs se;
+  se.target = p.target_logits; se.draft = p.draft_logits;
+  se.target_uncond = p.target_uncond; se.draft_uncond = p.draft_uncond;
+  se.cfg_scale = p.cfg_scale;
+  se.B = p.B; se.gamma = p.gamma; se.T = p.target_rows; se.V = p.V;
+  se.tstride = tstride; se.dstride = dstride;
+  se.vec_ok = sa.vec_ok;
+  se.top_k = p.top_k;
+  se.thresholds = reinterpret_cast<float*>((char*)p.workspace + lay.thresholds_off);
 
   FinishArgs fa;
   fa.target = p.target_logits; fa.draft = p.draft_logits;
@@ -172,13 +199,18 @@ int verify_impl(const csd_params& p) {
   fa.out_tokens = p.out_tokens; fa.out_accept_len = p.out_accept_len; fa.out_status = p.out_status;
   fa.dbg_p = p.dbg_p; fa.dbg_q = p.dbg_q; fa.dbg_f = p.dbg_f; fa.dbg_G = p.dbg_G;
 
-  cudaError_t e;
+  cudaError_t e = cudaSuccess;
   if (p.dtype == CSD_F32) {
-    e = cfg ? launch_stats_u<float, true>(sa, U, sms, stream) : launch_stats_u<float, false>(sa, U, sms, stream);
+    if (topk) e = cfg ? launch_select<float, true>(se, sms, stream) : launch_select<float, false>(se, sms, stream);
+    if (e == cudaSuccess)
+      e = cfg ? launch_stats_u<float, true>(sa, U, topk, sms, stream) : launch_stats_u<float, false>(sa, U, topk, sms, stream);
     if (e == cudaSuccess) e = cfg ? launch_finish<float, true>(fa, stream) : launch_finish<float, false>(fa, stream);
   } else {
-    e = cfg ? launch_stats_u<__nv_bfloat16, true>(sa, U, sms, stream)
-            : launch_stats_u<__nv_bfloat16, false>(sa, U, sms, stream);
+    if (topk)
+      e = cfg ? launch_select<__nv_bfloat16, true>(se, sms, stream) : launch_select<__nv_bfloat16, false>(se, sms, stream);
+    if (e == cudaSuccess)
+      e = cfg ? launch_stats_u<__nv_bfloat16, true>(sa, U, topk, sms, stream)
+              : launch_stats_u<__nv_bfloat16, false>(sa, U, topk, sms, stream);
     if (e == cudaSuccess)
       e = cfg ? launch_finish<__nv_bfloat16, true>(fa, stream) : launch_finish<__nv_bfloat16, false>(fa, stream);
   }

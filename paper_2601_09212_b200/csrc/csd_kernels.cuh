@@ -1,8 +1,11 @@
 // Device code of libcsd: the verify-and-resample round of Cool-SD on sm_100a.
 //
-// Two kernels per call, the second launched with programmatic dependent launch
-// so that its blocks are resident and waiting when the first one drains:
+// Two kernels per call (three with top-k filtering), the last launched with
+// programmatic dependent launch so that its blocks are resident and waiting
+// when the statistics kernel drains:
 //
+//   topk_threshold_kernel  (top-k only) exact k-th largest value of every row by
+//                      radix select; the value is the filter threshold.
 //   row_stats_kernel   streams every logit row once from HBM (the only HBM
 //                      traffic of the call) and leaves, per (row, part), the pair
 //                      (m, s) with  sum_x exp(z_x) = (1 + s) * exp(m)  over that part:
@@ -158,10 +161,11 @@ struct StatsArgs {
   int n_items;               // B * (T + gamma) * parts
   int vec_ok;
   float2* partials;          // [B * (T + gamma)][parts]
+  const float* thresholds;   // [B * (T + gamma)], read only by the TOPK variants
 };
 
 // U = 16-byte loads per thread per array per item
-template <typename T, bool CFG, int U>
+template <typename T, bool CFG, int U, bool TOPK>
 __global__ void __launch_bounds__(kStatsThreads) row_stats_kernel(const StatsArgs a) {
   constexpr int VEC = Elem<T>::kVec;
   __shared__ float sh_m[2][kStatsThreads / 32];
@@ -178,7 +182,7 @@ __global__ void __launch_bounds__(kStatsThreads) row_stats_kernel(const StatsArg
     const int r = row_id - b * rows_per_seq;
     Row<T, CFG> row;
     row.scale = a.cfg_scale;
-    row.thr = CSD_NEG_INF;
+    row.thr = TOPK ? a.thresholds[row_id] : CSD_NEG_INF;
     if (r < a.T) {
       const int64_t off = (int64_t)b * a.tstride + (int64_t)r * a.V;
       row.cond = reinterpret_cast<const T*>(a.target) + off;
@@ -197,8 +201,13 @@ __global__ void __launch_bounds__(kStatsThreads) row_stats_kernel(const StatsArg
 #pragma unroll
       for (int k = 0; k < U; ++k) {
         const int x0 = x_begin + (k * kStatsThreads + tid) * VEC;
-        if (x0 < x_end) row.load_vec(x0, z[k]);
-        else {
+        if (x0 < x_end) {
+          row.load_vec(x0, z[k]);
+          if (TOPK) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) z[k][e] = row.filter(z[k][e]);
+          }
+        } else {
 #pragma unroll
           for (int e = 0; e < VEC; ++e) z[k][e] = CSD_NEG_INF;
         }
@@ -216,7 +225,7 @@ __global__ void __launch_bounds__(kStatsThreads) row_stats_kernel(const StatsArg
     } else {
       m = CSD_NEG_INF; s = -1.0f;
       for (int x = x_begin + tid; x < x_end; x += kStatsThreads) {
-        float one[1] = {row.load_one(x)};
+        float one[1] = {TOPK ? row.filter(row.load_one(x)) : row.load_one(x)};
         float m1, s1;
         stat_of_values(one, m1, s1);
         stat_merge(m, s, m1, s1);
@@ -238,6 +247,127 @@ __global__ void __launch_bounds__(kStatsThreads) row_stats_kernel(const StatsArg
     }
     // double-buffered staging: the next item writes the other buffer, and the
     // barrier of that item orders this item's reads before the buffer's reuse
+  }
+}
+
+
+// ============================ kernel 0: top-k thresholds (any V) ===================
+// Exact k-th largest value of every (mixed) row by a most-significant-digit-first
+// radix select over order-preserving 32-bit keys: three passes over the row with
+// digits of 11, 11 and 10 bits.  The value itself is the threshold, so ties with
+// the k-th largest are kept whatever their position.
+constexpr int kSelectThreads = 1024;
+constexpr int kSelectBins = 2048;
+
+__device__ __forceinline__ uint32_t order_key(float z) {
+  const uint32_t b = __float_as_uint(z);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float order_value(uint32_t key) {
+  return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
+}
+
+struct SelectArgs {
+  const void* target;
+  const void* draft;
+  const void* target_uncond;
+  const void* draft_uncond;
+  float cfg_scale;
+  int B, gamma, T, V;
+  int64_t tstride, dstride;
+  int vec_ok;
+  int top_k;          // 1 <= top_k < V
+  float* thresholds;  // [B * (T + gamma)]
+};
+
+// Walks a histogram from its top bin down and returns the bin that holds the
+// k-th largest key; *above gets the number of keys in higher bins.  One warp.
+__device__ __forceinline__ int select_bin_from_top(const int* hist, int nbins, int k, int lane, int* above) {
+  const int chunk = nbins / 32;                     // nbins is a multiple of 32
+  const int hi = nbins - lane * chunk;              // lane 0 owns the top chunk
+  int local = 0;
+  for (int d = hi - 1; d >= hi - chunk; --d) local += hist[d];
+  int incl = local;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += t;
+  }
+  const unsigned ballot = __ballot_sync(0xffffffffu, incl >= k);
+  const int owner = ballot ? __ffs(ballot) - 1 : 31;  // fewer than k keys: the lowest chunk
+  int bin = 0, cnt_above = 0;
+  if (lane == owner) {
+    int c = incl - local;
+    bin = hi - chunk;
+    cnt_above = c;
+    for (int d = hi - 1; d >= hi - chunk; --d) {
+      if (c + hist[d] >= k) { bin = d; cnt_above = c; break; }
+      c += hist[d];
+      cnt_above = c;
+    }
+  }
+  bin = __shfl_sync(0xffffffffu, bin, owner);
+  *above = __shfl_sync(0xffffffffu, cnt_above, owner);
+  return bin;
+}
+
+template <typename T, bool CFG>
+__global__ void __launch_bounds__(kSelectThreads) topk_threshold_kernel(const SelectArgs a) {
+  constexpr int VEC = Elem<T>::kVec;
+  __shared__ int hist[kSelectBins];
+  __shared__ uint32_t sh_prefix;
+  __shared__ int sh_k;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rows_per_seq = a.T + a.gamma;
+  const int n_rows = a.B * rows_per_seq;
+  for (int row_id = blockIdx.x; row_id < n_rows; row_id += gridDim.x) {
+    const int b = row_id / rows_per_seq;
+    const int r = row_id - b * rows_per_seq;
+    Row<T, CFG> row;
+    row.scale = a.cfg_scale;
+    row.thr = CSD_NEG_INF;
+    if (r < a.T) {
+      const int64_t off = (int64_t)b * a.tstride + (int64_t)r * a.V;
+      row.cond = reinterpret_cast<const T*>(a.target) + off;
+      row.uncond = CFG ? reinterpret_cast<const T*>(a.target_uncond) + off : nullptr;
+    } else {
+      const int64_t off = (int64_t)b * a.dstride + (int64_t)(r - a.T) * a.V;
+      row.cond = reinterpret_cast<const T*>(a.draft) + off;
+      row.uncond = CFG ? reinterpret_cast<const T*>(a.draft_uncond) + off : nullptr;
+    }
+    uint32_t prefix = 0, mask = 0;
+    int k = a.top_k;
+#pragma unroll 1
+    for (int pass = 0; pass < 3; ++pass) {
+      const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+      const int nbins = pass == 2 ? 1024 : 2048;
+      for (int d = tid; d < nbins; d += kSelectThreads) hist[d] = 0;
+      __syncthreads();
+      for (int x0 = tid * VEC; x0 < a.V; x0 += kSelectThreads * VEC) {
+        float z[VEC];
+        row.load_tile(x0, a.V, a.vec_ok, z);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+          const uint32_t key = order_key(z[e]);
+          if (x0 + e < a.V && (key & mask) == prefix) atomicAdd(&hist[(key >> shift) & (nbins - 1)], 1);
+        }
+      }
+      __syncthreads();
+      if (warp == 0) {
+        int above;
+        const int bin = select_bin_from_top(hist, nbins, k, lane, &above);
+        if (lane == 0) {
+          sh_prefix = prefix | ((uint32_t)bin << shift);
+          sh_k = k - above;
+        }
+      }
+      __syncthreads();
+      prefix = sh_prefix;
+      k = sh_k;
+      mask |= (uint32_t)(nbins - 1) << shift;
+    }
+    if (tid == 0) a.thresholds[row_id] = order_value(prefix);
+    __syncthreads();
   }
 }
 

@@ -109,6 +109,52 @@ def test_cfg_mix_fused():
         assert_ok(rep)
 
 
+@pytest.mark.parametrize("dtype", [W.F32, W.BF16])
+@pytest.mark.parametrize("V,k", [(64, 1), (64, 63), (1000, 10), (4096, 1000), (5000, 4999), (16384, 1000),
+                                 (20000, 50), (70000, 1000)])
+def test_topk_filter(dtype, V, k):
+    """Top-k before the softmax (keep every logit >= the k-th largest of its row), with and
+    without the guidance mix; bf16 rows hold many tied values, which the tie rule must keep."""
+    L = 4
+    for cfg in (False, True):
+        w = W.make("t", B=5, gamma=L, V=V, dtype=dtype, rho=0.9, bonus_row=True, cfg=cfg, top_k=k,
+                   schedule=sched(L), seed=V + k, device=DEV)
+        rep, got, ref = check(w)
+        assert_ok(rep)
+        live = got["accept_len"] < L
+        # the distribution drawn from has at most the kept tokens in its support
+        assert ((got["G"] > 0).sum(-1) >= 1).all()
+        if dtype == W.F32 and not cfg:
+            assert ((got["G"] > 0).sum(-1) <= k).all()
+
+
+def test_topk_with_masked_and_tied_rows():
+    """Rows with fewer than k finite entries (threshold -inf: nothing more is removed) and rows
+    where the k-th largest value is shared by many tokens."""
+    B, L, V, k = 4, 3, 512, 100
+    w = W.make("t", B=B, gamma=L, V=V, rho=0.9, bonus_row=True, top_k=k, schedule=sched(L), seed=1, device=DEV)
+    w.target_logits[0, 0, 50:] = float("-inf")
+    w.draft_logits[0, 0, 50:] = float("-inf")
+    w.draft_tokens[0, 0] = 7
+    w.target_logits[1, :, :] = torch.round(w.target_logits[1, :, :])       # heavy ties
+    w.draft_logits[1, :, :] = torch.round(w.draft_logits[1, :, :])
+    w.target_logits[2, 1, :] = 0.0                                         # all equal: everything kept
+    w.target_logits[3, 0, 5] = -0.0
+    w.target_logits[3, 0, 6] = 0.0
+    rep, got, ref = check(w)
+    assert_ok(rep)
+
+
+def test_config_c3_guidance_and_topk():
+    """B=64, gamma=8, V=16384, bf16, guidance mix s=4 fused into the load, top-k 1000."""
+    L = W.CONFIGS["C3"]["gamma"]
+    for step in range(2):
+        w = W.config("C3", step=step, schedule=sched(L), device=DEV)
+        rep, got, ref = check(w)
+        assert_ok(rep)
+        print("C3", rep.summary())
+
+
 def test_batch_strides_and_unaligned_views():
     """Rows embedded in a larger buffer (batch stride > rows*V) and a base pointer that is
     only element-aligned (forces the scalar path)."""
