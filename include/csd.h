@@ -62,7 +62,9 @@ typedef enum {
   CSD_ERR_WORKSPACE = -4, /* workspace NULL, misaligned (256 B) or smaller than csd_workspace_size */
   CSD_ERR_ARG = -5,       /* inconsistent options (one unconditional array without the other, top_k < 0, ...) */
   CSD_ERR_LAUNCH = -6,    /* the CUDA runtime refused a launch or copy; see cudaGetLastError */
-  CSD_ERR_ALLOC = -7      /* csd_verify only: its internal workspace could not be allocated */
+  CSD_ERR_ALLOC = -7,     /* csd_verify only: its internal workspace could not be allocated */
+  CSD_ERR_STATIC_LIMIT = -8 /* csd_verify_static only: the problem needs more scratch than the
+                               built-in CSD_STATIC_SCRATCH_BYTES */
 } csd_error;
 
 /* Bits of out_status[b]; they refer only to positions the algorithm looked at
@@ -99,6 +101,45 @@ typedef enum {
 int csd_verify(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
                const float* uniforms, const float* relax_schedule, int B, int gamma, int V,
                int32_t* out_tokens, int32_t* out_accept_len, void* stream);
+
+/*
+ * Allocation-free form of csd_verify.  (The paper has no counterpart: this entry
+ * point exists for the sake of callers, not of the method.)
+ *
+ * Some callers must not trigger a device allocation when they call into the
+ * library: code running between cudaStreamBeginCapture and EndCapture, a
+ * serving loop whose memory pool owns every byte of the device and treats a
+ * stray cudaMalloc as a bug, a real-time thread that cannot afford the implicit
+ * device synchronisation cudaMalloc/cudaFree may bring, or a process that is
+ * simply not allowed to grow.  csd_verify allocates (and may re-allocate) its
+ * scratch internally and csd_verify_ex wants the caller to provide it; this form
+ * does neither.  Its scratch is a fixed array of CSD_STATIC_SCRATCH_BYTES that is
+ * part of the library's device image, so every GPU on which the library is
+ * loaded holds those bytes from load until the process exits, whether or not
+ * this function is ever called.
+ *
+ * Arguments, results and conventions are exactly those of csd_verify (fp32
+ * logits, contiguous [B, gamma, V], no bonus row).  Differences:
+ *   - No cudaMalloc, cudaFree or other allocating call is made, ever.
+ *   - Problems whose csd_workspace_size(B, gamma, V, CSD_F32) exceeds
+ *     CSD_STATIC_SCRATCH_BYTES are refused with CSD_ERR_STATIC_LIMIT before
+ *     anything is enqueued (for scale: B=256, gamma=16, V=16384 needs about
+ *     1.1 MB and fits; B=256, gamma=16, V=65536 does not).
+ *   - The first call on each device looks up the device address of the array
+ *     (a cudaGetSymbolAddress call, made with that device current) and keeps
+ *     it; make that first call outside any stream capture.
+ *   - All calls on one device share the one array.  Nothing in it has to start
+ *     at zero -- each call overwrites every byte it later reads -- so no
+ *     clearing is needed between calls, and what a call leaves behind is
+ *     meaningless.  Two calls that may run on the GPU at the same time (different
+ *     streams, no ordering between them) would overwrite each other's scratch:
+ *     keep calls on one device ordered, or use csd_verify_ex with separate
+ *     workspaces for the concurrent ones.
+ */
+#define CSD_STATIC_SCRATCH_BYTES (2u * 1024u * 1024u)
+int csd_verify_static(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
+                      const float* uniforms, const float* relax_schedule, int B, int gamma, int V,
+                      int32_t* out_tokens, int32_t* out_accept_len, void* stream);
 
 /*
  * Full form.  Adds: bf16 logits; an optional (gamma+1)-th target row for the

@@ -19,7 +19,8 @@ from ._build import LIB_PATH
 
 CSD_F32, CSD_BF16 = 0, 1
 CSD_STATUS_BADROW, CSD_STATUS_BADTOKEN, CSD_STATUS_ZFALLBACK = 1, 2, 4
-EXPORTS = ("csd_verify", "csd_verify_ex", "csd_workspace_size", "csd_verify_host",
+CSD_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
+EXPORTS = ("csd_verify", "csd_verify_static", "csd_verify_ex", "csd_workspace_size", "csd_verify_host",
            "csd_host_staging_size", "csd_make_schedule", "csd_error_string", "csd_version")
 
 
@@ -58,6 +59,8 @@ def library() -> C.CDLL:
         lib = C.CDLL(LIB_PATH)
         lib.csd_verify.argtypes = [C.c_void_p] * 5 + [C.c_int] * 3 + [C.c_void_p] * 3
         lib.csd_verify.restype = C.c_int
+        lib.csd_verify_static.argtypes = lib.csd_verify.argtypes
+        lib.csd_verify_static.restype = C.c_int
         lib.csd_verify_ex.argtypes = [C.POINTER(csd_params)]
         lib.csd_verify_ex.restype = C.c_int
         lib.csd_workspace_size.argtypes = [C.c_int] * 4
@@ -160,6 +163,30 @@ def csd_verify(target_logits, draft_logits, draft_tokens, uniforms, relax_schedu
         _stream_handle(stream))
     if rc != 0:
         raise CsdError(rc, "csd_verify")
+
+
+def csd_verify_static(target_logits, draft_logits, draft_tokens, uniforms, relax_schedule, out_tokens,
+                      out_accept_len, stream=None) -> None:
+    """``csd_verify`` for callers that must not allocate on the device (inside a stream capture,
+    under a memory pool that owns the whole GPU, on a latency-critical thread): same arguments
+    and results, scratch taken from a fixed array inside the library, so nothing is allocated.
+    Raises ``CsdError`` (code -8) when the problem needs more than ``CSD_STATIC_SCRATCH_BYTES``;
+    calls on one device share that array and must not overlap on the GPU."""
+    B, gamma, V = target_logits.shape
+    if draft_logits.shape != (B, gamma, V):
+        raise ValueError("target_logits and draft_logits must both be [B, gamma, V]")
+    rc = library().csd_verify_static(
+        _dev_ptr(target_logits, "target_logits", torch.float32),
+        _dev_ptr(draft_logits, "draft_logits", torch.float32),
+        _dev_ptr(draft_tokens, "draft_tokens", torch.int32),
+        _dev_ptr(uniforms, "uniforms", torch.float32),
+        _dev_ptr(relax_schedule, "relax_schedule", torch.float32),
+        B, gamma, V,
+        _dev_ptr(out_tokens, "out_tokens", torch.int32),
+        _dev_ptr(out_accept_len, "out_accept_len", torch.int32),
+        _stream_handle(stream))
+    if rc != 0:
+        raise CsdError(rc, "csd_verify_static")
 
 
 def make_params(target_logits, draft_logits, draft_tokens, uniforms, relax_schedule, out_tokens,

@@ -278,6 +278,54 @@ int csd_verify(const float* target_logits, const float* draft_logits, const int3
   return verify_impl(p);
 }
 
+// ---- allocation-free form -------------------------------------------------------------
+// Scratch that lives in the library's device image.  In host code the name below
+// is only a handle for cudaGetSymbolAddress, never a device address: the kernels
+// get the address that call returns.
+static __device__ __align__(256) unsigned char g_static_scratch[CSD_STATIC_SCRATCH_BYTES];
+
+namespace {
+void* g_static_scratch_addr[kMaxDevices];  // per device, filled on first use
+
+// Device address of g_static_scratch on the current device; no allocation.
+int static_scratch_address(void** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CSD_ERR_LAUNCH;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (g_static_scratch_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) {
+      (void)cudaGetLastError();
+      return CSD_ERR_LAUNCH;
+    }
+    g_static_scratch_addr[dev] = ptr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return CSD_OK;
+}
+}  // namespace
+
+int csd_verify_static(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
+                      const float* uniforms, const float* relax_schedule, int B, int gamma, int V,
+                      int32_t* out_tokens, int32_t* out_accept_len, void* stream) {
+  if (!shape_ok(B, gamma, V)) return CSD_ERR_SHAPE;
+  const size_t need = csd_workspace_size(B, gamma, V, CSD_F32);
+  if (need > (size_t)CSD_STATIC_SCRATCH_BYTES) return CSD_ERR_STATIC_LIMIT;
+  void* scratch = nullptr;
+  const int rc = static_scratch_address(&scratch);
+  if (rc != CSD_OK) return rc;
+  csd_params p;
+  memset(&p, 0, sizeof p);
+  p.target_logits = target_logits; p.draft_logits = draft_logits;
+  p.cfg_scale = 1.0f; p.top_k = 0; p.dtype = CSD_F32;
+  p.B = B; p.gamma = gamma; p.V = V; p.target_rows = gamma;
+  p.draft_tokens = draft_tokens; p.uniforms = uniforms; p.relax_schedule = relax_schedule;
+  p.out_tokens = out_tokens; p.out_accept_len = out_accept_len;
+  p.workspace = scratch; p.workspace_bytes = CSD_STATIC_SCRATCH_BYTES;
+  p.stream = stream;
+  return verify_impl(p);
+}
+
 // ---- host-buffer form -----------------------------------------------------------
 namespace {
 struct HostPlan {
@@ -434,6 +482,7 @@ const char* csd_error_string(int code) {
     case CSD_ERR_ARG: return "inconsistent or unsupported options";
     case CSD_ERR_LAUNCH: return "CUDA runtime error while enqueueing work";
     case CSD_ERR_ALLOC: return "could not allocate the internal workspace";
+    case CSD_ERR_STATIC_LIMIT: return "problem too large for the built-in scratch of csd_verify_static (CSD_STATIC_SCRATCH_BYTES); use csd_verify_ex with a caller workspace";
     default: return "unknown error code";
   }
 }
