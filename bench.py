@@ -139,9 +139,32 @@ class ClockSampler:
 
 # ---------------------------------------------------------------------------------------------
 def workload_kwargs(name: str) -> dict:
+    """A named configuration (C1..C4) or a sweep point such as "B=64,gamma=8,V=16384,dtype=bf16"
+    (optional keys: rho, law, cfg, cfg_scale, top_k)."""
     from paper_2601_09212_b200 import workloads as W
-    kw = dict(W.CONFIGS[name])
-    kw.pop("steps", None)
+    if name in W.CONFIGS:
+        kw = dict(W.CONFIGS[name])
+        kw.pop("steps", None)
+        return kw
+    kw = dict(rho=0.9)
+    for item in name.split(","):
+        k, v = item.split("=")
+        k = k.strip()
+        if k == "dtype":
+            kw[k] = {"bf16": W.BF16, "fp32": W.F32, "f32": W.F32}[v.strip()]
+        elif k in ("B", "gamma", "V", "top_k"):
+            kw[k] = int(v)
+        elif k in ("rho", "cfg_scale", "scale"):
+            kw[k] = float(v)
+        elif k == "cfg":
+            kw[k] = v.strip() in ("1", "true", "True")
+        elif k == "law":
+            kw[k] = v.strip()
+        else:
+            raise SystemExit(f"unknown workload key {k}")
+    for need in ("B", "gamma", "V"):
+        if need not in kw:
+            raise SystemExit(f"workload needs {need}")
     return kw
 
 
@@ -267,7 +290,7 @@ def run_native(args) -> None:
                             o["tok"], o["tau"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
                             cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=o["st"], workspace=o["ws"],
                             stream=stream) for w, o in zip(ring, outs)]
-    kernels_per_step = 3 if (0 < kw.get("top_k", 0) < V) else 2
+    kernels_per_step = csd.csd_launch_count(prms[0])
 
     def enqueue(i):
         csd.csd_verify_ex(prms[i % ring_n])

@@ -74,7 +74,10 @@ typedef enum {
                               rejects (f := 0).  An unusable drafter row resamples from
                               P_j (Eq. opt_G at f = 0); an unusable target row emits -1. */
   CSD_STATUS_BADTOKEN = 2, /* draft token outside [0, V): that position rejects */
-  CSD_STATUS_ZFALLBACK = 4 /* empty positive part: drew from P_j instead */
+  CSD_STATUS_ZFALLBACK = 4, /* empty positive part: drew from P_j instead */
+  CSD_STATUS_TIMEOUT = 8    /* a bounded wait inside the kernel gave up (a copy into shared memory did
+                               not arrive within about a second): results of this call are unreliable.
+                               The condition stays set in the workspace until csd_workspace_init. */
 } csd_status_bits;
 
 /*
@@ -129,9 +132,10 @@ int csd_verify(const float* target_logits, const float* draft_logits, const int3
  *     (a cudaGetSymbolAddress call, made with that device current) and keeps
  *     it; make that first call outside any stream capture.
  *   - All calls on one device share the one array.  Nothing in it has to start
- *     at zero -- each call overwrites every byte it later reads -- so no
- *     clearing is needed between calls, and what a call leaves behind is
- *     meaningless.  Two calls that may run on the GPU at the same time (different
+ *     at a value the caller provides -- each call overwrites what it later reads -- so no
+ *     clearing is needed between calls (the few words that must be zero are zero
+ *     when the library is loaded and every call puts them back), and what a call
+ *     leaves behind is otherwise meaningless.  Two calls that may run on the GPU at the same time (different
  *     streams, no ordering between them) would overwrite each other's scratch:
  *     keep calls on one device ordered, or use csd_verify_ex with separate
  *     workspaces for the concurrent ones.
@@ -175,9 +179,10 @@ typedef struct csd_params {
   float* dbg_f;                /* [B, gamma] or NULL: f_i (0 where the row or token is unusable) */
   float* dbg_G;                /* [B, V] or NULL: the distribution the emitted token was drawn
                                   from (G*_j, or P for the bonus draw / fallbacks); zeros if none */
-  void* workspace;             /* >= csd_workspace_size(...) bytes, 256-byte aligned; contents
-                                  need no initialisation and are garbage afterwards.  Two calls
-                                  that may overlap on the GPU need different workspaces.    */
+  void* workspace;             /* >= csd_workspace_size(...) bytes, 256-byte aligned, zero-filled
+                                  once before its first use (csd_workspace_init or any memset);
+                                  every call leaves it ready for the next.  Two calls that may
+                                  overlap on the GPU need different workspaces.             */
   size_t workspace_bytes;
   void* stream;
 } csd_params;
@@ -187,6 +192,15 @@ int csd_verify_ex(const csd_params* p);
 /* Bytes of workspace that csd_verify_ex needs for any call with these sizes
  * (any target_rows, guidance and top-k setting).  0 if the sizes are invalid. */
 size_t csd_workspace_size(int B, int gamma, int V, int dtype);
+
+/* Number of kernels csd_verify_ex(p) would enqueue (1 on the fused path; 2, or 3 with
+ * top-k, on the path for unaligned or very small rows), or a negative csd_error.
+ * Validates like csd_verify_ex and enqueues nothing. */
+int csd_launch_count(const csd_params* p);
+
+/* Zero-fills a workspace on `stream` (needed once, before its first use; also the
+ * way to clear the sticky CSD_STATUS_TIMEOUT condition). */
+int csd_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Host-buffer form: the same round for a caller whose logits, tokens, uniforms

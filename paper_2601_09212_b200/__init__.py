@@ -18,9 +18,9 @@ import torch
 from ._build import LIB_PATH
 
 CSD_F32, CSD_BF16 = 0, 1
-CSD_STATUS_BADROW, CSD_STATUS_BADTOKEN, CSD_STATUS_ZFALLBACK = 1, 2, 4
+CSD_STATUS_BADROW, CSD_STATUS_BADTOKEN, CSD_STATUS_ZFALLBACK, CSD_STATUS_TIMEOUT = 1, 2, 4, 8
 CSD_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
-EXPORTS = ("csd_verify", "csd_verify_static", "csd_verify_ex", "csd_workspace_size", "csd_verify_host",
+EXPORTS = ("csd_verify", "csd_verify_static", "csd_verify_ex", "csd_workspace_size", "csd_workspace_init", "csd_launch_count", "csd_verify_host",
            "csd_host_staging_size", "csd_make_schedule", "csd_error_string", "csd_version")
 
 
@@ -65,6 +65,10 @@ def library() -> C.CDLL:
         lib.csd_verify_ex.restype = C.c_int
         lib.csd_workspace_size.argtypes = [C.c_int] * 4
         lib.csd_workspace_size.restype = C.c_size_t
+        lib.csd_launch_count.argtypes = [C.POINTER(csd_params)]
+        lib.csd_launch_count.restype = C.c_int
+        lib.csd_workspace_init.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
+        lib.csd_workspace_init.restype = C.c_int
         lib.csd_verify_host.argtypes = [C.POINTER(csd_params), C.c_void_p, C.c_size_t]
         lib.csd_verify_host.restype = C.c_int
         lib.csd_host_staging_size.argtypes = [C.POINTER(csd_params)]
@@ -235,6 +239,13 @@ def csd_verify_ex(params: csd_params) -> None:
         raise CsdError(rc, "csd_verify_ex")
 
 
+def csd_launch_count(params: csd_params) -> int:
+    n = library().csd_launch_count(C.byref(params))
+    if n < 0:
+        raise CsdError(n, "csd_launch_count")
+    return int(n)
+
+
 def csd_host_staging_size(params: csd_params) -> int:
     return int(library().csd_host_staging_size(C.byref(params)))
 
@@ -247,8 +258,16 @@ def csd_verify_host(params: csd_params, staging: torch.Tensor) -> None:
 
 
 def new_workspace(B: int, gamma: int, V: int, dtype: int, device="cuda") -> torch.Tensor:
-    """A device buffer of the size csd_verify_ex asks for (torch's allocator gives 512-byte alignment)."""
+    """A zero-filled device buffer of the size csd_verify_ex asks for (torch's allocator gives
+    512-byte alignment)."""
     n = csd_workspace_size(B, gamma, V, dtype)
     if n == 0:
         raise CsdError(-2, "csd_workspace_size")
-    return torch.empty(n, dtype=torch.uint8, device=device)
+    return torch.zeros(n, dtype=torch.uint8, device=device)
+
+
+def csd_workspace_init(workspace: torch.Tensor, stream=None) -> None:
+    rc = library().csd_workspace_init(_dev_ptr(workspace, "workspace"),
+                                      workspace.numel() * workspace.element_size(), _stream_handle(stream))
+    if rc != 0:
+        raise CsdError(rc, "csd_workspace_init")

@@ -15,6 +15,9 @@ namespace {
 
 using namespace csd;
 
+static_assert(sizeof(FusedSmem) <= 113 * 1024 && sizeof(PlainSmem) <= 113 * 1024, "two blocks per SM must fit");
+static_assert(sizeof(FusedSmem::ring) == kRingBytes && sizeof(PlainSmem::ring) == kRingBytes, "the finish uses the ring as 64 KB");
+
 constexpr int kMaxV = 1 << 20;
 constexpr int kMaxDevices = 64;
 constexpr size_t kAlign = 256;
@@ -46,19 +49,87 @@ bool shape_ok(int B, int gamma, int V) {
   return B >= 1 && gamma >= 1 && gamma <= kMaxGamma && V >= 2 && V <= kMaxV;
 }
 
-// Workspace: [partials: rows * max_parts float2][thresholds: rows float]
+// Workspace: [header: error flag][counters: B int][partials: rows * max_parts float2][thresholds: rows float]
+//            [token logits: rows float]
+// The header and the counters must be zero before the first call; every call leaves them zero.
 struct Layout {
-  size_t rows, max_parts, partials_off, thresholds_off, total;
+  size_t rows, max_parts, header_off, counters_off, partials_off, thresholds_off, tok_logit_off, zero_bytes, total;
 };
 Layout layout_for(int B, int gamma, int V, int dtype) {
   Layout l;
   l.rows = (size_t)B * (size_t)(2 * gamma + 1);
-  const size_t min_part = (size_t)kStatsThreads * vec_width(dtype);  // U = 1
+  // finest split any path uses: one warp stage of the plain kernel with guidance (fp32: 256 elements)
+  const size_t min_part = (size_t)kWStageBytes / (2 * (size_t)elem_size(dtype));
   l.max_parts = ((size_t)V + min_part - 1) / min_part;
-  l.partials_off = 0;
-  l.thresholds_off = align_up(l.rows * l.max_parts * sizeof(float2));
-  l.total = l.thresholds_off + align_up(l.rows * sizeof(float));
+  l.header_off = 0;
+  l.counters_off = kAlign;
+  l.partials_off = l.counters_off + align_up((size_t)B * sizeof(int));
+  l.zero_bytes = l.partials_off;
+  l.thresholds_off = l.partials_off + align_up(l.rows * l.max_parts * sizeof(float2));
+  l.tok_logit_off = l.thresholds_off + align_up(l.rows * sizeof(float));
+  l.total = l.tok_logit_off + align_up(l.rows * sizeof(float));
   return l;
+}
+
+// c with P(N(0,1) > c) = tail, by bisection on erfc (host, called once per call; 60 steps)
+double normal_upper_quantile(double tail) {
+  double lo = -8.0, hi = 8.0;
+  for (int it = 0; it < 60; ++it) {
+    const double mid = 0.5 * (lo + hi);
+    if (0.5 * erfc(mid / sqrt(2.0)) > tail) lo = mid; else hi = mid;
+  }
+  return 0.5 * (lo + hi);
+}
+
+template <typename T, bool CFG>
+cudaError_t launch_fused(const FusedArgs& a, int grid, cudaStream_t stream) {
+  auto kern = verify_topk_kernel<T, CFG>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FusedSmem));
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kFusedThreads);
+  cfg.dynamicSmemBytes = sizeof(FusedSmem);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+template <typename T, bool CFG>
+cudaError_t launch_plain(const FusedArgs& a, int grid, cudaStream_t stream) {
+  auto kern = verify_plain_kernel<T, CFG>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PlainSmem));
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kFusedThreads);
+  cfg.dynamicSmemBytes = sizeof(PlainSmem);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+template <typename T, bool CFG>
+cudaError_t launch_fused_t(const FusedArgs& a, bool topk, int grid, cudaStream_t stream) {
+  return topk ? launch_fused<T, CFG>(a, grid, stream) : launch_plain<T, CFG>(a, grid, stream);
 }
 
 template <typename T, bool CFG, int U, bool TOPK>
@@ -123,7 +194,7 @@ cudaError_t launch_finish(const FinishArgs& a, cudaStream_t stream) {
   return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
-int verify_impl(const csd_params& p) {
+int verify_impl(const csd_params& p, int* plan_only = nullptr) {
   if (!p.target_logits || !p.draft_logits || !p.draft_tokens || !p.uniforms || !p.relax_schedule ||
       !p.out_tokens || !p.out_accept_len)
     return CSD_ERR_NULL;
@@ -199,6 +270,72 @@ int verify_impl(const csd_params& p) {
   fa.out_tokens = p.out_tokens; fa.out_accept_len = p.out_accept_len; fa.out_status = p.out_status;
   fa.dbg_p = p.dbg_p; fa.dbg_q = p.dbg_q; fa.dbg_f = p.dbg_f; fa.dbg_G = p.dbg_G;
 
+  // ---- fused single-launch path: aligned rows of at least 512 bytes; with top-k, rows that fit the registers
+  const bool fused = vec_ok && (size_t)p.V * es >= 512 && (!topk || p.V <= kTopkMaxV) &&
+                     (p.V + 32 * vw - 1) / (32 * vw) <= kFinTiles;
+  if (plan_only) {  // number of kernels this call would enqueue
+    *plan_only = fused ? 1 : (topk ? 3 : 2);
+    return CSD_OK;
+  }
+  if (fused) {
+    FusedArgs ua;
+    ua.fin = fa;
+    ua.top_k = p.top_k;
+    ua.lo_sigmas = nanf("");
+    ua.tok_logit = reinterpret_cast<float*>((char*)p.workspace + lay.tok_logit_off);
+    ua.counters = reinterpret_cast<int*>((char*)p.workspace + lay.counters_off);
+    ua.error_flag = reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
+    long long grid, n_items;
+    if (topk) {
+      // one block-wide item per row
+      const int eps = kStageBytes / (es * (cfg ? 2 : 1));
+      ua.chunks_per_row = (p.V + eps - 1) / eps;
+      ua.chunks_per_part = ua.chunks_per_row;
+      ua.parts_per_row = 1;
+      ua.fin.parts = 1;
+      n_items = rows;
+      const double k = p.top_k, v = p.V;
+      const double tail = 1.25 * k / v + 4.0 * sqrt(k) / v + 16.0 / v;
+      if (tail < 0.45 && tail * v < 0.8 * kListCap) ua.lo_sigmas = (float)normal_upper_quantile(tail);
+      grid = sms;
+      if (grid > n_items) grid = n_items;
+      const long long need = (n_items + kStashItems - 1) / kStashItems;
+      if (grid < need) grid = need;
+    } else {
+      // warp-wide items: parts of rows, sized so that every warp of the grid gets several
+      const int eps = kWStageBytes / (es * (cfg ? 2 : 1));
+      const long long cpr = (p.V + eps - 1) / eps;
+      grid = 2LL * sms;
+      const long long warps = grid * kPlainWarps;
+      long long cpp = rows * cpr / (4 * warps);
+      if (cpp < 1) cpp = 1;
+      if (cpp > 8) cpp = 8;
+      // the finish stages a sequence's partials in the 64 KB ring: at most 8192 of them
+      const long long max_parts = (kRingBytes / (long long)sizeof(float2)) / rows_per_seq;
+      const long long min_cpp = (cpr + max_parts - 1) / max_parts;
+      if (cpp < min_cpp) cpp = min_cpp;
+      if (cpp > cpr) cpp = cpr;
+      ua.chunks_per_row = (int)cpr;
+      ua.chunks_per_part = (int)cpp;
+      ua.parts_per_row = (int)((cpr + cpp - 1) / cpp);
+      ua.fin.parts = ua.parts_per_row;
+      n_items = rows * ua.parts_per_row;
+      if (n_items > 0x7fffffffLL) return CSD_ERR_SHAPE;
+      if (grid * kPlainWarps > n_items) grid = (n_items + kPlainWarps - 1) / kPlainWarps;
+      const long long need = (n_items + (long long)kPlainWarps * kWarpStash - 1) / ((long long)kPlainWarps * kWarpStash);
+      if (grid < need) grid = need;
+    }
+    ua.n_items = (int)n_items;
+    ua.items_per_seq = (int)(n_items / p.B);
+    cudaError_t fe;
+    if (p.dtype == CSD_F32)
+      fe = cfg ? launch_fused_t<float, true>(ua, topk, (int)grid, stream) : launch_fused_t<float, false>(ua, topk, (int)grid, stream);
+    else
+      fe = cfg ? launch_fused_t<__nv_bfloat16, true>(ua, topk, (int)grid, stream)
+               : launch_fused_t<__nv_bfloat16, false>(ua, topk, (int)grid, stream);
+    return fe == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
+  }
+
   cudaError_t e = cudaSuccess;
   if (p.dtype == CSD_F32) {
     if (topk) e = cfg ? launch_select<float, true>(se, sms, stream) : launch_select<float, false>(se, sms, stream);
@@ -233,6 +370,19 @@ size_t csd_workspace_size(int B, int gamma, int V, int dtype) {
   return layout_for(B, gamma, V, dtype).total;
 }
 
+int csd_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  if (!workspace) return CSD_ERR_NULL;
+  if (((uintptr_t)workspace % kAlign) != 0 || workspace_bytes == 0) return CSD_ERR_WORKSPACE;
+  return cudaMemsetAsync(workspace, 0, workspace_bytes, (cudaStream_t)stream) == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
+}
+
+int csd_launch_count(const csd_params* p) {
+  if (!p) return CSD_ERR_NULL;
+  int n = 0;
+  const int rc = verify_impl(*p, &n);
+  return rc == CSD_OK ? n : rc;
+}
+
 int csd_verify_ex(const csd_params* p) {
   if (!p) return CSD_ERR_NULL;
   return verify_impl(*p);
@@ -263,6 +413,7 @@ int csd_verify(const float* target_logits, const float* draft_logits, const int3
         return CSD_ERR_ALLOC;
       }
       w.bytes = need;
+      if (cudaMemsetAsync(w.ptr, 0, need, (cudaStream_t)stream) != cudaSuccess) return CSD_ERR_LAUNCH;
     }
     ws = w.ptr;
   }
@@ -428,6 +579,8 @@ int csd_verify_host(const csd_params* host, void* staging, size_t staging_bytes)
   d.dbg_G = h.dbg_G ? (float*)(base + pl.off_G) : nullptr;
   d.workspace = base + pl.off_ws;
   d.workspace_bytes = pl.ws_bytes;
+  if (cudaMemsetAsync(d.workspace, 0, layout_for(h.B, h.gamma, h.V, h.dtype).zero_bytes, stream) != cudaSuccess)
+    return CSD_ERR_LAUNCH;
   const int rc = verify_impl(d);
   if (rc != CSD_OK) return rc;
 
@@ -487,6 +640,6 @@ const char* csd_error_string(int code) {
   }
 }
 
-int csd_version(void) { return 100; }
+int csd_version(void) { return 200; }
 
 }  // extern "C"
