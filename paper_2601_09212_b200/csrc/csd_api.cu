@@ -10,13 +10,14 @@
 
 #include "../../include/csd.h"
 #include "csd_kernels.cuh"
+#include "csd_fused.cuh"
 
 namespace {
 
 using namespace csd;
 
-static_assert(sizeof(FusedSmem) <= 113 * 1024 && sizeof(PlainSmem) <= 113 * 1024, "two blocks per SM must fit");
-static_assert(sizeof(FusedSmem::ring) == kRingBytes && sizeof(PlainSmem::ring) == kRingBytes, "the finish uses the ring as 64 KB");
+static_assert(sizeof(TopkSmem) <= 55 * 1024, "four blocks of the top-k kernel per SM must fit");
+static_assert(sizeof(PlainSmem) <= 74 * 1024, "three blocks of the plain kernel per SM must fit");
 
 constexpr int kMaxV = 1 << 20;
 constexpr int kMaxDevices = 64;
@@ -86,7 +87,7 @@ cudaError_t launch_fused(const FusedArgs& a, int grid, cudaStream_t stream) {
   auto kern = verify_topk_kernel<T, CFG>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(FusedSmem));
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TopkSmem));
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -94,7 +95,7 @@ cudaError_t launch_fused(const FusedArgs& a, int grid, cudaStream_t stream) {
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3(kFusedThreads);
-  cfg.dynamicSmemBytes = sizeof(FusedSmem);
+  cfg.dynamicSmemBytes = sizeof(TopkSmem);
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -271,8 +272,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
   fa.dbg_p = p.dbg_p; fa.dbg_q = p.dbg_q; fa.dbg_f = p.dbg_f; fa.dbg_G = p.dbg_G;
 
   // ---- fused single-launch path: aligned rows of at least 512 bytes; with top-k, rows that fit the registers
-  const bool fused = vec_ok && (size_t)p.V * es >= 512 && (!topk || p.V <= kTopkMaxV) &&
-                     (p.V + 32 * vw - 1) / (32 * vw) <= kFinTiles;
+  const bool fused = vec_ok && (size_t)p.V * es >= 512 && (p.V + 32 * vw - 1) / (32 * vw) <= kFinTiles;
   if (plan_only) {  // number of kernels this call would enqueue
     *plan_only = fused ? 1 : (topk ? 3 : 2);
     return CSD_OK;
@@ -287,42 +287,39 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
     ua.error_flag = reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
     long long grid, n_items;
     if (topk) {
-      // one block-wide item per row
-      const int eps = kStageBytes / (es * (cfg ? 2 : 1));
-      ua.chunks_per_row = (p.V + eps - 1) / eps;
-      ua.chunks_per_part = ua.chunks_per_row;
+      // one block-wide item per row, streamed in stages
+      ua.chunks_per_part = 0;
       ua.parts_per_row = 1;
       ua.fin.parts = 1;
       n_items = rows;
       const double k = p.top_k, v = p.V;
       const double tail = 1.25 * k / v + 4.0 * sqrt(k) / v + 16.0 / v;
       if (tail < 0.45 && tail * v < 0.8 * kListCap) ua.lo_sigmas = (float)normal_upper_quantile(tail);
-      grid = sms;
+      grid = 2LL * sms;
       if (grid > n_items) grid = n_items;
-      const long long need = (n_items + kStashItems - 1) / kStashItems;
+      const long long need = (n_items + kTkStash - 1) / kTkStash;
       if (grid < need) grid = need;
     } else {
       // warp-wide items: parts of rows, sized so that every warp of the grid gets several
       const int eps = kWStageBytes / (es * (cfg ? 2 : 1));
       const long long cpr = (p.V + eps - 1) / eps;
-      grid = 2LL * sms;
-      const long long warps = grid * kPlainWarps;
+      grid = 3LL * sms;
+      const long long warps = grid * kFusedWarps;
       long long cpp = rows * cpr / (4 * warps);
       if (cpp < 1) cpp = 1;
       if (cpp > 8) cpp = 8;
-      // the finish stages a sequence's partials in the 64 KB ring: at most 8192 of them
-      const long long max_parts = (kRingBytes / (long long)sizeof(float2)) / rows_per_seq;
+      // the finish stages a sequence's partials in the ring: 8 bytes each
+      const long long max_parts = (kPlainRingBytes / (long long)sizeof(float2)) / rows_per_seq;
       const long long min_cpp = (cpr + max_parts - 1) / max_parts;
       if (cpp < min_cpp) cpp = min_cpp;
       if (cpp > cpr) cpp = cpr;
-      ua.chunks_per_row = (int)cpr;
       ua.chunks_per_part = (int)cpp;
       ua.parts_per_row = (int)((cpr + cpp - 1) / cpp);
       ua.fin.parts = ua.parts_per_row;
       n_items = rows * ua.parts_per_row;
       if (n_items > 0x7fffffffLL) return CSD_ERR_SHAPE;
-      if (grid * kPlainWarps > n_items) grid = (n_items + kPlainWarps - 1) / kPlainWarps;
-      const long long need = (n_items + (long long)kPlainWarps * kWarpStash - 1) / ((long long)kPlainWarps * kWarpStash);
+      if (grid * kFusedWarps > n_items) grid = (n_items + kFusedWarps - 1) / kFusedWarps;
+      const long long need = (n_items + (long long)kFusedWarps * kWarpStash - 1) / ((long long)kFusedWarps * kWarpStash);
       if (grid < need) grid = need;
     }
     ua.n_items = (int)n_items;

@@ -1,0 +1,1129 @@
+// Single-launch path of libcsd (sm_100a): one persistent kernel per call.
+//
+// Phase 1 streams this block's share of the logit rows through rings of
+// shared-memory stages filled by bulk asynchronous copies (mbarrier completion)
+// and keeps the per-item results in shared memory; nothing is written to global
+// memory yet, so phase 1 may overlap the previous call on the stream
+// (programmatic dependent launch).  After griddepcontrol.wait, phase 2 publishes
+// the results, counts arrivals per sequence, and the block that completes a
+// sequence runs its finish: accept tests, tau, Eq. opt_G at position tau+1 with
+// the two rows brought back through the ring, inverse-CDF draw, emit.  No block
+// ever waits for another block; every wait on a copy is bounded.
+//
+//   verify_plain_kernel  every warp streams its own parts of rows through its own
+//                        ring and keeps a running (m, s) per lane.
+//   verify_topk_kernel   a block streams whole rows; the first stage of a row is
+//                        the sample for a mean/deviation guess `lo` of a value a
+//                        little below the k-th largest; values >= lo are gathered
+//                        as they stream by; one histogram over them finds the bin
+//                        of the k-th largest and an exact rank among that bin's
+//                        few values gives the threshold.  When the guess does not
+//                        bracket the answer the row is re-read from global memory
+//                        and selected exactly by radix, so the result never
+//                        depends on the guess.
+#pragma once
+#include "csd_kernels.cuh"
+
+namespace csd {
+
+constexpr int kFusedThreads = 256;
+constexpr int kFusedWarps = kFusedThreads / 32;
+constexpr long long kWaitCycles = 1ll << 31;  // about a second: then give up and flag it
+constexpr int kFinTiles = 1024;               // tiles of 32 lanes x 16 bytes: V <= 131072 (fp32) / 262144 (bf16)
+
+// ---- mbarrier and bulk-copy primitives -----------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_addr(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within kWaitCycles.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > kWaitCycles) return false;
+  }
+  return true;
+}
+// global -> shared bulk copy of `bytes` (multiple of 16; both addresses 16-byte aligned),
+// completion counted in bytes on `bar`
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_addr(dst)),
+               "l"(src), "r"(bytes), "r"(smem_addr(bar))
+               : "memory");
+}
+// orders this thread's earlier shared-memory accesses before a bulk copy it issues next
+__device__ __forceinline__ void fence_before_bulk() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// maximum that returns NaN when either operand is NaN (fmaxf would drop it)
+__device__ __forceinline__ float max_nan(float x, float y) {
+  float r;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(x), "f"(y));
+  return r;
+}
+
+template <typename T>
+__device__ __forceinline__ void unpack_vec(const unsigned char* p, float (&out)[Elem<T>::kVec]);
+template <>
+__device__ __forceinline__ void unpack_vec<float>(const unsigned char* p, float (&out)[4]) {
+  const float4 v = *reinterpret_cast<const float4*>(p);
+  out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+}
+template <>
+__device__ __forceinline__ void unpack_vec<__nv_bfloat16>(const unsigned char* p, float (&out)[8]) {
+  const uint4 v = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    out[2 * k] = __uint_as_float(w[k] << 16);
+    out[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+  }
+}
+template <typename T>
+__device__ __forceinline__ float load_scalar_smem(const unsigned char* p);
+template <>
+__device__ __forceinline__ float load_scalar_smem<float>(const unsigned char* p) {
+  return *reinterpret_cast<const float*>(p);
+}
+template <>
+__device__ __forceinline__ float load_scalar_smem<__nv_bfloat16>(const unsigned char* p) {
+  return __uint_as_float(((uint32_t) * reinterpret_cast<const unsigned short*>(p)) << 16);
+}
+
+struct FusedArgs {
+  FinishArgs fin;       // inputs, outputs, partials [rows][fin.parts], thresholds [rows]
+  int n_items;          // plain: rows * parts_per_row; top-k: rows
+  int chunks_per_part;  // plain kernel: warp stages per part
+  int parts_per_row;    // plain kernel
+  int items_per_seq;
+  int top_k;
+  float lo_sigmas;      // top-k guess: lo = mean + lo_sigmas * deviation (NaN: always select exactly)
+  float* tok_logit;     // [rows] (mixed, unfiltered) logit of the row's drafted token, written in phase 2
+  int* counters;        // [B] arrivals per sequence; zero before the first call, left zero by every call
+  int* error_flag;      // set when a bounded wait gave up
+};
+
+// ---- finish with everything staged in shared memory ---------------------------------
+// Few dependent round trips to global memory: one brings the sequence's partials,
+// thresholds, drafted tokens with their logits (found in phase 1 while the rows
+// streamed by), uniforms and multipliers into shared memory; after the accept tests,
+// bulk copies bring the two rows of position tau+1 into the ring, a segment at a
+// time, and Eq. opt_G is summed from there.
+struct FinishStage {
+  int tok[kMaxGamma + 1];
+  float uni[kMaxGamma + 1];
+  float omega[kMaxGamma];
+  float tokz[2 * kMaxGamma + 1];
+  float thr_row[2 * kMaxGamma + 1];
+  alignas(8) uint64_t bar;
+};
+
+// both (m, s) pairs reduced over the warp in one interleaved loop
+__device__ __forceinline__ void stat_warp_allreduce2(float& m0, float& s0, float& m1, float& s1) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float a0 = __shfl_xor_sync(0xffffffffu, m0, off);
+    const float b0 = __shfl_xor_sync(0xffffffffu, s0, off);
+    const float a1 = __shfl_xor_sync(0xffffffffu, m1, off);
+    const float b1 = __shfl_xor_sync(0xffffffffu, s1, off);
+    stat_merge(m0, s0, a0, b0);
+    stat_merge(m1, s1, a1, b1);
+  }
+}
+
+// ring: `ring_bytes` of shared memory (multiple of 4 KB) that nothing else uses meanwhile;
+// tile_sums: kFinTiles doubles, likewise.
+template <typename T, bool CFG>
+__device__ void finish_sequence_staged(const FusedArgs& ua, const int b, const int tid, unsigned char* ring,
+                                       const int ring_bytes, double* tile_sums, FinishSmem& sm, FinishStage& st,
+                                       uint32_t& phase, const int extra_status) {
+  constexpr int NT = kFusedThreads;
+  constexpr int VEC = Elem<T>::kVec;
+  constexpr int TILE = 32 * VEC;
+  constexpr int ARR = CFG ? 2 : 1;
+  constexpr int ES = (int)sizeof(T);
+  const FinishArgs& a = ua.fin;
+  const int lane = tid & 31, warp = tid >> 5;
+  const int L = a.gamma, V = a.V;
+  const int rows_per_seq = a.T + L;
+  const T* tgt = reinterpret_cast<const T*>(a.target) + (int64_t)b * a.tstride;
+  const T* dft = reinterpret_cast<const T*>(a.draft) + (int64_t)b * a.dstride;
+  const T* tgt_u = CFG ? reinterpret_cast<const T*>(a.target_uncond) + (int64_t)b * a.tstride : nullptr;
+  const T* dft_u = CFG ? reinterpret_cast<const T*>(a.draft_uncond) + (int64_t)b * a.dstride : nullptr;
+
+  // ---- 0. one round trip: everything the accept tests need ----------------------------
+  const int n_entries = rows_per_seq * a.parts;   // the host keeps this within the ring
+  float2* staged = reinterpret_cast<float2*>(ring);
+  {
+    const float2* src = a.partials + (int64_t)b * n_entries;
+    for (int idx = tid; idx < n_entries; idx += NT) staged[idx] = __ldcg(src + idx);
+    if (tid < L) {
+      st.tok[tid] = a.tokens[(int64_t)b * L + tid];
+      const float om = a.schedule[tid];
+      st.omega[tid] = om >= 0.0f ? om : 0.0f;
+    }
+    if (tid <= L) st.uni[tid] = a.uniforms[(int64_t)b * (L + 1) + tid];
+    if (tid < rows_per_seq) {
+      st.thr_row[tid] = a.use_topk ? __ldcg(a.thresholds + (int64_t)b * rows_per_seq + tid) : CSD_NEG_INF;
+      st.tokz[tid] = __ldcg(ua.tok_logit + (int64_t)b * rows_per_seq + tid);
+    }
+  }
+  __syncthreads();
+
+  // ---- 1. per position: merge parts, Eq. relax, accept test ------------------------------
+  const int n_pos = a.T > L ? L + 1 : L;   // the bonus position only if its row exists
+  if (tid == 0 && n_pos == L) { sm.valid[0][L] = 0; sm.valid[1][L] = 0; sm.flag[L] = 0; }
+  for (int i = warp; i < n_pos; i += NT / 32) {
+    const bool has_d = i < L;   // has_t always holds here
+    float M[2] = {CSD_NEG_INF, CSD_NEG_INF}, S[2] = {-1.0f, -1.0f};
+    for (int p = lane; p < a.parts; p += 32) {
+      const float2 v = staged[i * a.parts + p];
+      stat_merge(M[0], S[0], v.x, v.y);
+      if (has_d) {
+        const float2 w = staged[(a.T + i) * a.parts + p];
+        stat_merge(M[1], S[1], w.x, w.y);
+      }
+    }
+    stat_warp_allreduce2(M[0], S[0], M[1], S[1]);
+    if (lane == 0) {
+      const float thr0 = st.thr_row[i], thr1 = has_d ? st.thr_row[a.T + i] : CSD_NEG_INF;
+      const bool t_ok = M[0] > CSD_NEG_INF && M[0] < CSD_POS_INF && S[0] >= 0.0f && S[0] < CSD_POS_INF;
+      const bool d_ok = has_d && M[1] > CSD_NEG_INF && M[1] < CSD_POS_INF && S[1] >= 0.0f && S[1] < CSD_POS_INF;
+      sm.M[0][i] = M[0]; sm.S[0][i] = S[0]; sm.thr[0][i] = thr0;
+      sm.M[1][i] = M[1]; sm.S[1][i] = S[1]; sm.thr[1][i] = thr1;
+      sm.valid[0][i] = t_ok; sm.valid[1][i] = d_ok;
+      int flag = 0;
+      if (i < L) {
+        const int tok = st.tok[i];
+        const bool tok_ok = tok >= 0 && tok < V;
+        const float omega = st.omega[i];
+        float f = 0.0f, p = __int_as_float(0x7fc00000), q = p;
+        if (!t_ok || !d_ok) flag = 1;
+        else if (!tok_ok) flag = 2;
+        else {
+          const float zt = st.tokz[i], zd = st.tokz[a.T + i];
+          const float dt = (zt < thr0 ? CSD_NEG_INF : zt) - M[0];
+          const float dd = (zd < thr1 ? CSD_NEG_INF : zd) - M[1];
+          p = ex2f(dt * kLog2e) / (1.0f + S[0]);
+          q = ex2f(dd * kLog2e) / (1.0f + S[1]);
+          if (dd == CSD_NEG_INF) f = 1.0f;         // q = 0: p/q = +inf, and 0/0 := 1
+          else if (dt == CSD_NEG_INF) f = 0.0f;    // p = 0 < q
+          else f = fminf(1.0f, omega * ex2f((dt - dd) * kLog2e) * ((1.0f + S[1]) / (1.0f + S[0])));
+        }
+        sm.acc[i] = (st.uni[i] <= f) ? 1 : 0;
+        if (a.dbg_p) a.dbg_p[(int64_t)b * L + i] = p;
+        if (a.dbg_q) a.dbg_q[(int64_t)b * L + i] = q;
+        if (a.dbg_f) a.dbg_f[(int64_t)b * L + i] = f;
+      }
+      sm.flag[i] = flag;
+    }
+  }
+  __syncthreads();
+
+  // ---- 2. tau = number of leading accepts (the for/break of Algorithm 1) --------
+  int tau = 0;
+  while (tau < L && sm.acc[tau]) ++tau;
+  int status = extra_status;
+  for (int i = 0; i <= min(tau, L - 1); ++i) status |= sm.flag[i];
+
+  // ---- 3. which row to draw from -------------------------------------------------
+  const int j = tau;  // 0-based row index of position tau+1 (j == L: bonus row)
+  PairCtx ctx;
+  bool draw = true;
+  if (j < L) {
+    if (!sm.valid[0][j]) draw = false;
+    ctx.mode = sm.valid[1][j] ? 0 : 1;
+  } else {
+    if (a.T == L + 1) {
+      ctx.mode = 1;
+      if (!sm.valid[0][L]) { draw = false; status |= 1; }
+    } else draw = false;
+  }
+  float* G_out = a.dbg_G ? a.dbg_G + (int64_t)b * V : nullptr;
+  const int ntiles = (V + TILE - 1) / TILE;
+  int token = -1;
+
+  if (draw) {
+    ctx.Mt = sm.M[0][j]; ctx.St = sm.S[0][j];
+    ctx.Md = j < L ? sm.M[1][j] : 0.0f; ctx.Sd = j < L ? sm.S[1][j] : 0.0f;
+    ctx.inv_t = 1.0f / (1.0f + ctx.St);
+    ctx.inv_den = ctx.inv_t / (1.0f + ctx.Sd);
+    ctx.one_minus_omega = 1.0f - (j < L ? st.omega[j] : 0.0f);
+    Row<T, CFG> rt{tgt + (int64_t)j * V, CFG ? tgt_u + (int64_t)j * V : nullptr, a.cfg_scale, sm.thr[0][j]};
+    Row<T, CFG> rd = rt;
+    if (j < L) rd = Row<T, CFG>{dft + (int64_t)j * V, CFG ? dft_u + (int64_t)j * V : nullptr, a.cfg_scale, sm.thr[1][j]};
+    const float u = st.uni[L];
+
+    for (int attempt = 0; attempt < 2; ++attempt) {
+      // ---- 4. Eq. opt_G weights: the rows come through the ring, one fp64 sum per tile ------
+      const int n_arr = (ctx.mode == 0 ? 2 : 1) * ARR;
+      const int seg_elems = (ring_bytes / n_arr / (TILE * ES)) * TILE;   // elements of each array per segment
+      const int slot_bytes = seg_elems * ES;
+      for (int x0 = 0; x0 < V; x0 += seg_elems) {
+        __syncthreads();   // everybody is done with what the ring held
+        const int n = min(seg_elems, V - x0);
+        if (tid == 0) {
+          fence_before_bulk();
+          const uint32_t bytes = (uint32_t)(n * ES);
+          mbar_expect_tx(&st.bar, bytes * n_arr);
+          bulk_load(ring, rt.cond + x0, bytes, &st.bar);
+          if (CFG) bulk_load(ring + slot_bytes, rt.uncond + x0, bytes, &st.bar);
+          if (ctx.mode == 0) {
+            bulk_load(ring + ARR * slot_bytes, rd.cond + x0, bytes, &st.bar);
+            if (CFG) bulk_load(ring + (ARR + 1) * slot_bytes, rd.uncond + x0, bytes, &st.bar);
+          }
+        }
+        if (!mbar_wait(&st.bar, phase)) status |= 8;
+        phase ^= 1u;
+        const int seg_tiles = (n + TILE - 1) / TILE;
+        // two tiles per warp and trip, so that their reductions overlap
+        for (int t0 = warp; t0 < seg_tiles; t0 += 2 * (NT / 32)) {
+          float acc2[2] = {0.0f, 0.0f};
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            const int xo = (t0 + r * (NT / 32)) * TILE + lane * VEC;   // offset inside the segment
+            if (xo < n) {
+              float zt[VEC], zd[VEC];
+              unpack_vec<T>(ring + xo * ES, zt);
+              if (CFG) {
+                float zu[VEC];
+                unpack_vec<T>(ring + slot_bytes + xo * ES, zu);
+#pragma unroll
+                for (int k = 0; k < VEC; ++k) zt[k] = cfg_mix(zt[k], zu[k], a.cfg_scale);
+              }
+              if (ctx.mode == 0) {
+                unpack_vec<T>(ring + ARR * slot_bytes + xo * ES, zd);
+                if (CFG) {
+                  float zu[VEC];
+                  unpack_vec<T>(ring + (ARR + 1) * slot_bytes + xo * ES, zu);
+#pragma unroll
+                  for (int k = 0; k < VEC; ++k) zd[k] = cfg_mix(zd[k], zu[k], a.cfg_scale);
+                }
+              }
+              float acc = 0.0f;
+#pragma unroll
+              for (int k = 0; k < VEC; ++k)
+                acc += weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
+              acc2[r] = acc;
+            }
+          }
+          double d0 = (double)acc2[0], d1 = (double)acc2[1];
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) {
+            d0 += __shfl_xor_sync(0xffffffffu, d0, off);
+            d1 += __shfl_xor_sync(0xffffffffu, d1, off);
+          }
+          if (lane == 0) {
+            tile_sums[x0 / TILE + t0] = d0;
+            if (t0 + NT / 32 < seg_tiles) tile_sums[x0 / TILE + t0 + NT / 32] = d1;
+          }
+        }
+      }
+      __syncthreads();
+      // ---- 5. locate the tile that holds the crossing C(x) > u Z ------------------
+      if (warp == 0) {
+        const int chunk = (ntiles + 31) / 32;
+        const int t0 = lane * chunk, t1 = min(ntiles, t0 + chunk);
+        double local = 0.0;
+        for (int t = t0; t < t1; ++t) local += tile_sums[t];
+        const double incl = warp_incl_scan_double(local, lane);
+        const double Z = __shfl_sync(0xffffffffu, incl, 31);
+        const double target = (double)u * Z;
+        const bool mine = incl > target && local > 0.0;
+        const unsigned ballot = __ballot_sync(0xffffffffu, mine);
+        if (lane == 0) { sm.Z = Z; sm.pick_tile = -1; }
+        __syncwarp();
+        if (ballot != 0 && lane == __ffs(ballot) - 1) {
+          double c = incl - local, c_pick = c;
+          int pick = t0;
+          for (int t = t0; t < t1; ++t) {
+            const double v = tile_sums[t];
+            if (v > 0.0) { pick = t; c_pick = c; }   // last tile with mass seen so far
+            if (c + v > target && v > 0.0) break;
+            c += v;
+          }
+          sm.pick_tile = pick;
+          sm.pick_prefix = c_pick;
+        }
+      }
+      __syncthreads();
+      const double Z = sm.Z;
+      if (!(Z > 0.0) || !(Z < (double)CSD_POS_INF)) {
+        if (attempt == 0 && ctx.mode == 0) {  // empty positive part: fall back to G := P_j
+          ctx.mode = 1;
+          status |= 4;
+          continue;
+        }
+        break;  // nothing to draw from
+      }
+      // ---- 6. scan inside that tile (its 32 vectors come from global memory again) -----------
+      if (warp == 0) {
+        const int tile = sm.pick_tile;
+        const double target = (double)u * Z;
+        const int x0 = tile * TILE + lane * VEC;
+        float zt[VEC], zd[VEC];
+        rt.load_tile(x0, V, 1, zt);
+        if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd);
+        double run[VEC];
+        double acc = 0.0;
+        int last_pos = -1;
+        unsigned posmask = 0;
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) {
+          const float g = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
+          if (g > 0.0f) { last_pos = k; posmask |= 1u << k; }
+          acc += (double)g;
+          run[k] = acc;
+        }
+        const double before = sm.pick_prefix + (warp_incl_scan_double(acc, lane) - acc);
+        int first = -1;
+#pragma unroll
+        for (int k = VEC - 1; k >= 0; --k)
+          if (before + run[k] > target && ((posmask >> k) & 1u)) first = k;
+        const unsigned hit = __ballot_sync(0xffffffffu, first >= 0);
+        const unsigned pos = __ballot_sync(0xffffffffu, last_pos >= 0);
+        if (hit != 0) {
+          if (lane == __ffs(hit) - 1) sm.token = x0 + first;
+        } else if (pos != 0) {  // rounding left no crossing: last token with positive weight
+          if (lane == 31 - __clz(pos)) sm.token = x0 + last_pos;
+        } else if (lane == 0) sm.token = -1;
+      }
+      __syncthreads();
+      token = sm.token;
+      // ---- 7. optional: write the distribution drawn from ------------------------------
+      if (G_out) {
+        const float invZ = (float)(1.0 / Z);
+        for (int tile = warp; tile < ntiles; tile += NT / 32) {
+          const int x0 = tile * TILE + lane * VEC;
+          float zt[VEC], zd[VEC];
+          rt.load_tile(x0, V, 1, zt);
+          if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd);
+#pragma unroll
+          for (int k = 0; k < VEC; ++k)
+            if (x0 + k < V)
+              G_out[x0 + k] = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx) * invZ;
+        }
+      }
+      break;
+    }
+  }
+  if (G_out && token < 0)
+    for (int x = tid; x < V; x += NT) G_out[x] = 0.0f;
+
+  // ---- 8. emit x_{1:tau+1} ---------------------------------------------------------
+  if (tid <= L) {
+    int v = -1;
+    if (tid < tau) v = st.tok[tid];
+    else if (tid == tau) v = token;
+    a.out_tokens[(int64_t)b * (L + 1) + tid] = v;
+  }
+  if (tid == 0) {
+    a.out_accept_len[b] = tau;
+    if (a.out_status) a.out_status[b] = status;
+  }
+  __syncthreads();  // the shared state may be reused for the next sequence
+}
+
+// Phase 2 tail shared by both kernels: run the finish of every sequence this block completed.
+template <typename T, bool CFG>
+__device__ __forceinline__ void finish_completed(const FusedArgs& a, int tid, const int* done, int n_done, bool aborted,
+                                                 unsigned char* ring, int ring_bytes, double* tile_sums,
+                                                 FinishSmem& fin, FinishStage& fst) {
+  if (n_done <= 0) return;
+  __threadfence();
+  const int extra = (aborted || __ldcg(a.error_flag)) ? 8 : 0;
+  uint32_t fin_phase = 0;
+  for (int d = 0; d < n_done; ++d) {
+    const int b = done[d];
+    finish_sequence_staged<T, CFG>(a, b, tid, ring, ring_bytes, tile_sums, fin, fst, fin_phase, extra);
+    if (tid == 0) a.counters[b] = 0;   // ready for the next call
+  }
+}
+
+// ======================= plain kernel: one pipeline per warp ============================
+// A warp owns a contiguous range of items (an item is a part of a row: chunks_per_part warp
+// stages), a private ring of kWStages stages of kWStageBytes, issues its own refills, and keeps
+// a running (m, s) per lane that it reduces once per item.  Eight such pipelines per block sit
+// at different points of their loops and hide each other's latencies; phase 1 has no block-wide
+// step at all.
+constexpr int kWStages = 3;
+constexpr int kWStageBytes = 2048;
+constexpr int kWarpStash = 96;
+constexpr int kPlainRingBytes = kFusedWarps * kWStages * kWStageBytes;
+
+struct PlainSmem {
+  alignas(128) unsigned char ring[kFusedWarps][kWStages][kWStageBytes];
+  alignas(8) uint64_t full[kFusedWarps][kWStages];
+  float2 stash[kFusedWarps][kWarpStash];
+  float stash_tokz[kFusedWarps][kWarpStash];   // logit of the row's drafted token, if this part holds it
+  unsigned char stash_has[kFusedWarps][kWarpStash];
+  int done[kFusedWarps * kWarpStash];
+  int n_done;
+  int abort;
+  FinishSmem fin;
+  FinishStage fst;
+  double tile_sums[kFinTiles];
+};
+
+template <typename T, bool CFG>
+__global__ void __launch_bounds__(kFusedThreads, 3) verify_plain_kernel(const FusedArgs a) {
+  constexpr int VEC = Elem<T>::kVec;
+  constexpr int ARR = CFG ? 2 : 1;
+  constexpr int EPS = kWStageBytes / ((int)sizeof(T) * ARR);   // elements of a row per warp stage
+  constexpr int VPL = EPS / 32;                                // values per lane per stage
+  constexpr int NVS = VPL / VEC;                               // 16-byte vectors per lane per stage
+  constexpr int GV = NVS > 2 ? 2 : NVS;                        // vectors reduced together (register budget)
+  extern __shared__ __align__(128) unsigned char fused_smem_raw[];
+  PlainSmem& sm = *reinterpret_cast<PlainSmem*>(fused_smem_raw);
+
+  pdl_launch_dependents();  // the next call on the stream may start its own phase 1
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const FinishArgs& f = a.fin;
+  const int V = f.V;
+  const int rows_per_seq = f.T + f.gamma;
+  const int part_elems = a.chunks_per_part * EPS;
+
+  if (tid == 0) { sm.n_done = 0; sm.abort = 0; mbar_init(&sm.fst.bar, 1); }
+  if (lane == 0) {
+    for (int s = 0; s < kWStages; ++s) mbar_init(&sm.full[warp][s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const long long gw = (long long)blockIdx.x * kFusedWarps + warp;
+  const long long GW = (long long)gridDim.x * kFusedWarps;
+  const int item_begin = (int)((long long)a.n_items * gw / GW);
+  const int item_end = (int)((long long)a.n_items * (gw + 1) / GW);
+
+  // producer cursor (meaningful in lane 0): the next chunk to copy
+  int p_item = item_begin, p_x = 0, p_xend = 0, p_s = 0;
+  const T *p_cond = nullptr, *p_uncond = nullptr;
+  auto producer_open_item = [&]() {   // sets the cursor to the first chunk of p_item
+    const int row_id = p_item / a.parts_per_row;
+    const int part = p_item - row_id * a.parts_per_row;
+    const int b = row_id / rows_per_seq;
+    const int r = row_id - b * rows_per_seq;
+    if (r < f.T) {
+      const int64_t off = (int64_t)b * f.tstride + (int64_t)r * V;
+      p_cond = reinterpret_cast<const T*>(f.target) + off;
+      p_uncond = CFG ? reinterpret_cast<const T*>(f.target_uncond) + off : nullptr;
+    } else {
+      const int64_t off = (int64_t)b * f.dstride + (int64_t)(r - f.T) * V;
+      p_cond = reinterpret_cast<const T*>(f.draft) + off;
+      p_uncond = CFG ? reinterpret_cast<const T*>(f.draft_uncond) + off : nullptr;
+    }
+    p_x = part * part_elems;
+    p_xend = min(V, p_x + part_elems);
+  };
+  auto producer_issue = [&]() {       // copies one chunk into the next stage of the ring, if any is left
+    if (p_item >= item_end) return;
+    const uint32_t bytes = (uint32_t)(min(EPS, p_xend - p_x) * (int)sizeof(T));
+    mbar_expect_tx(&sm.full[warp][p_s], bytes * ARR);
+    bulk_load(&sm.ring[warp][p_s][0], p_cond + p_x, bytes, &sm.full[warp][p_s]);
+    if (CFG) bulk_load(&sm.ring[warp][p_s][kWStageBytes / 2], p_uncond + p_x, bytes, &sm.full[warp][p_s]);
+    p_s = p_s + 1 == kWStages ? 0 : p_s + 1;
+    p_x += EPS;
+    if (p_x >= p_xend) {
+      ++p_item;
+      if (p_item < item_end) producer_open_item();
+    }
+  };
+  if (lane == 0 && item_begin < item_end) {
+    producer_open_item();
+    for (int s = 0; s < kWStages; ++s) producer_issue();
+  }
+
+  // drafted token of a row (-1 for the bonus row), loaded a row ahead of its use
+  auto token_of_row = [&](int row_id) -> int {
+    const int b = row_id / rows_per_seq;
+    const int r = row_id - b * rows_per_seq;
+    const int i = r < f.T ? r : r - f.T;
+    return i < f.gamma ? __ldg(f.tokens + (int64_t)b * f.gamma + i) : -1;
+  };
+
+  // ================================= phase 1 ===========================================
+  int n_my = 0;
+  {
+    int c_s = 0;          // stage the consumer reads next
+    uint32_t c_par = 0;   // its parity
+    int issued = 0;       // chunks consumed so far (for the bounded wait after a timeout)
+    bool ok = true;
+    int cur_row = -1, tok_cur = -1, tok_next = -1;
+    const int last_row = item_end > item_begin ? (item_end - 1) / a.parts_per_row : -1;
+    if (item_begin < item_end) tok_next = token_of_row(item_begin / a.parts_per_row);
+    for (int item = item_begin; item < item_end; ++item, ++n_my) {
+      const int row_id = item / a.parts_per_row;
+      const int part = item - row_id * a.parts_per_row;
+      const int x_begin = part * part_elems;
+      const int x_end = min(V, x_begin + part_elems);
+      if (row_id != cur_row) {
+        cur_row = row_id;
+        tok_cur = tok_next;
+        if (row_id < last_row) tok_next = token_of_row(row_id + 1);
+      }
+      float tokz = 0.0f;
+      bool has_tok = false;
+      float m = CSD_NEG_INF, s_acc = -1.0f;
+      for (int x0 = x_begin; x0 < x_end; x0 += EPS) {
+        if (ok && !mbar_wait(&sm.full[warp][c_s], c_par)) ok = false;
+        ++issued;
+        const int n = min(EPS, x_end - x0);
+        const unsigned char* stage = &sm.ring[warp][c_s][0];
+        float m_c = CSD_NEG_INF, s_c = -1.0f;
+#pragma unroll
+        for (int g0 = 0; g0 < NVS; g0 += GV) {
+          float vals[GV * VEC];
+#pragma unroll
+          for (int v = 0; v < GV; ++v) {
+            const int xo = ((g0 + v) * 32 + lane) * VEC;
+            float zc[VEC];
+            if (ok && xo < n) {
+              unpack_vec<T>(stage + xo * (int)sizeof(T), zc);
+              if (CFG) {
+                float zu[VEC];
+                unpack_vec<T>(stage + kWStageBytes / 2 + xo * (int)sizeof(T), zu);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) zc[e] = cfg_mix(zc[e], zu[e], f.cfg_scale);
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < VEC; ++e) zc[e] = ok ? CSD_NEG_INF : __int_as_float(0x7fc00000);
+            }
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) vals[v * VEC + e] = zc[e];
+          }
+          float m1, s1;
+          stat_of_values(vals, m1, s1);
+          if (g0 == 0) { m_c = m1; s_c = s1; }
+          else stat_merge(m_c, s_c, m1, s1);   // a group of padding only merges as the identity
+        }
+        const int tl = tok_cur - x0;
+        if (ok && tl >= 0 && tl < n) {   // the drafted token's logit passes by: keep it
+          float zc = load_scalar_smem<T>(stage + tl * (int)sizeof(T));
+          if (CFG) zc = cfg_mix(zc, load_scalar_smem<T>(stage + kWStageBytes / 2 + tl * (int)sizeof(T)), f.cfg_scale);
+          tokz = zc;
+          has_tok = true;
+        }
+        __syncwarp();
+        if (lane == 0) {   // the stage is free again: refill it with the chunk kWStages ahead
+          fence_before_bulk();
+          producer_issue();
+        }
+        if (lane * VEC < n || !ok) stat_merge(m, s_acc, m_c, s_c);
+        if (++c_s == kWStages) { c_s = 0; c_par ^= 1u; }
+      }
+      stat_warp_allreduce(m, s_acc);
+      if (lane == 0 && n_my < kWarpStash) {
+        sm.stash[warp][n_my] = make_float2(m, s_acc);
+        sm.stash_tokz[warp][n_my] = tokz;
+        sm.stash_has[warp][n_my] = has_tok ? 1 : 0;
+      }
+    }
+    if (!ok && lane == 0) {
+      sm.abort = 1;
+      atomicExch(a.error_flag, 1);
+      // copies this warp gave up on may still be in flight: wait for them, again bounded
+      for (int s = 0; s < kWStages; ++s)
+        if (issued > s) (void)mbar_wait(&sm.full[warp][s], ((issued - 1 - s) / kWStages) & 1);
+    }
+  }
+
+  // ================================= phase 2 ===========================================
+  pdl_wait();   // the previous call on the stream has finished with the workspace and the outputs
+  __syncwarp();
+  for (int idx = lane; idx < n_my; idx += 32) {
+    const_cast<float2*>(f.partials)[item_begin + idx] = sm.stash[warp][idx];
+    if (sm.stash_has[warp][idx]) a.tok_logit[(item_begin + idx) / a.parts_per_row] = sm.stash_tokz[warp][idx];
+  }
+  __threadfence();
+  __syncthreads();
+  for (int idx = lane; idx < n_my; idx += 32) {
+    const int row_id = (item_begin + idx) / a.parts_per_row;
+    const int b = row_id / rows_per_seq;
+    __threadfence();
+    const int old = atomicAdd(&a.counters[b], 1);
+    if (old + 1 == a.items_per_seq) {
+      const int slot = atomicAdd(&sm.n_done, 1);
+      sm.done[slot] = b;
+    }
+  }
+  __syncthreads();
+  finish_completed<T, CFG>(a, tid, sm.done, sm.n_done, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes, sm.tile_sums, sm.fin, sm.fst);
+}
+
+// ======================= top-k kernel: a block streams whole rows ========================
+constexpr int kTkStages = 2;
+constexpr int kTkStageBytes = 16384;
+constexpr int kTkRingBytes = kTkStages * kTkStageBytes;
+constexpr int kTkStash = 256;
+constexpr int kWarpList = 256;                // per-warp capacity of the list of values >= lo
+constexpr int kListCap = kFusedWarps * kWarpList;
+constexpr int kLinBins = 512;
+constexpr int kCandCap = 64;
+constexpr float kLinRangeSigmas = 4.75f;      // the histogram spans [lo, lo + this many deviations)
+
+// bin of v >= lo in the linear histogram; the same instructions wherever it is evaluated
+__device__ __forceinline__ int lin_bin(float v, float lo, float scale) {
+  return min(kLinBins - 1, (int)__fmul_rn(__fsub_rn(v, lo), scale));
+}
+
+struct TopkSmem {
+  alignas(128) unsigned char ring[kTkStages][kTkStageBytes];
+  alignas(8) uint64_t full[kTkStages];
+  int readers_done[kTkStages];      // warps that have finished reading the stage's current contents
+  alignas(16) int hist[kLinBins];   // linear histogram; first 256 bins double as the radix histogram
+  alignas(8) float list[kFusedWarps][kWarpList];   // per warp: the values >= lo it met (the finish keeps its tile sums here)
+  int wpos[kFusedWarps];            // per warp: next free slot of its list (may run past the capacity)
+  float cand[kCandCap];             // values in the bin of the k-th largest
+  int n_cand[2];                    // by row parity
+  float mom[kFusedWarps][4];        // per warp: sum, sum of squares, count of the sampled values
+  float wmax[kFusedWarps];
+  float part_acc[2][kFusedWarps];   // per warp, by row parity: sum of exp(z - max) over kept non-maximum values
+  int part_cmax[2][kFusedWarps];    //                          number of kept values equal to the maximum
+  float part_max[2];
+  float part_thr[2];
+  int bc_i[4];
+  float red_f[kFusedWarps][2];
+  float2 stash[kTkStash];
+  float stash_thr[kTkStash];
+  float stash_tokz[kTkStash];       // logit of the row's drafted token
+  int done[kTkStash];
+  int n_done;
+  int abort;
+  FinishSmem fin;
+  FinishStage fst;
+};
+
+// Bin (of kLinBins, counted in `hist`) that holds the k-th largest value, found by one warp:
+// 16 bins per lane from the top, a warp scan, then a second scan inside the owner's 16 bins.
+// *rank_in_bin gets the 1-based rank of the answer among the bin's values, from the top.
+__device__ __forceinline__ int warp_pick_bin(const int* hist, int k, int lane, int* rank_in_bin) {
+  constexpr int PER = kLinBins / 32;           // 16
+  const int hi = kLinBins - lane * PER;        // lane 0 owns the top bins [hi - PER, hi)
+  int local = 0;
+  {
+    const int4* v = reinterpret_cast<const int4*>(hist + hi - PER);
+#pragma unroll
+    for (int q4 = 0; q4 < PER / 4; ++q4) {
+      const int4 t = v[q4];
+      local += t.x + t.y + t.z + t.w;
+    }
+  }
+  int incl = local;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += t;
+  }
+  const unsigned ballot = __ballot_sync(0xffffffffu, incl >= k);
+  const int owner = ballot ? __ffs(ballot) - 1 : 31;
+  const int above_owner = __shfl_sync(0xffffffffu, incl - local, owner);
+  const int owner_hi = kLinBins - owner * PER;
+  // second level: lane l < PER looks at bin owner_hi - 1 - l
+  const int val = lane < PER ? hist[owner_hi - 1 - lane] : 0;
+  int incl2 = val;
+#pragma unroll
+  for (int off = 1; off < PER; off <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl2, off);
+    if (lane >= off) incl2 += t;
+  }
+  const unsigned b2 = __ballot_sync(0xffffffffu, lane < PER && above_owner + incl2 >= k);
+  const int pick = b2 ? __ffs(b2) - 1 : PER - 1;
+  const int before = __shfl_sync(0xffffffffu, above_owner + incl2 - val, pick);
+  *rank_in_bin = k - before;
+  return owner_hi - 1 - pick;
+}
+
+// Exact threshold and filtered statistics of one row read again from global memory: radix
+// select over order-preserving keys (four 8-bit digits), then one pass for (m, s).  All
+// threads of the block take part; the results are valid in thread 0.
+template <typename T, bool CFG>
+__device__ void exact_row_from_global(const Row<T, CFG>& row, int V, int k, TopkSmem& sm, int tid, float& out_m,
+                                      float& out_s, float& out_thr) {
+  constexpr int VEC = Elem<T>::kVec;
+  const int lane = tid & 31, warp = tid >> 5;
+  uint32_t prefix = 0, mask = 0;
+#pragma unroll 1
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    sm.hist[tid] = 0;   // 256 threads, 256 bins
+    __syncthreads();
+    for (int x0 = tid * VEC; x0 < V; x0 += kFusedThreads * VEC) {
+      float z[VEC];
+      row.load_vec(x0, z);
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) {
+        const uint32_t key = order_key(z[e]);
+        if ((key & mask) == prefix) atomicAdd(&sm.hist[(key >> shift) & 255], 1);
+      }
+    }
+    __syncthreads();
+    if (warp == 0) {
+      int above;
+      const int bin = select_bin_from_top(sm.hist, 256, k, lane, &above);
+      if (lane == 0) { sm.bc_i[0] = (int)(prefix | ((uint32_t)bin << shift)); sm.bc_i[1] = k - above; }
+    }
+    __syncthreads();
+    prefix = (uint32_t)sm.bc_i[0];
+    k = sm.bc_i[1];
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  const float thr = order_value(prefix);
+  float m = CSD_NEG_INF, s = -1.0f;
+  for (int x0 = tid * VEC; x0 < V; x0 += kFusedThreads * VEC) {
+    float z[VEC];
+    row.load_vec(x0, z);
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) z[e] = z[e] < thr ? CSD_NEG_INF : z[e];
+    float m1, s1;
+    stat_of_values(z, m1, s1);
+    stat_merge(m, s, m1, s1);
+  }
+  stat_warp_allreduce(m, s);
+  if (lane == 0) { sm.red_f[warp][0] = m; sm.red_f[warp][1] = s; }
+  __syncthreads();
+  if (tid == 0) {
+    float mm = sm.red_f[0][0], sv = sm.red_f[0][1];
+#pragma unroll
+    for (int w = 1; w < kFusedWarps; ++w) stat_merge(mm, sv, sm.red_f[w][0], sm.red_f[w][1]);
+    out_m = mm; out_s = sv; out_thr = thr;
+  }
+  __syncthreads();
+}
+
+template <typename T, bool CFG>
+__global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const FusedArgs a) {
+  constexpr int VEC = Elem<T>::kVec;
+  constexpr int ARR = CFG ? 2 : 1;
+  constexpr int EPS = kTkStageBytes / ((int)sizeof(T) * ARR);   // elements of a row per stage
+  constexpr int VPT = EPS / kFusedThreads;                      // values per thread per stage
+  constexpr int NVS = VPT / VEC;                                // 16-byte vectors per thread per stage
+  extern __shared__ __align__(128) unsigned char fused_smem_raw[];
+  TopkSmem& sm = *reinterpret_cast<TopkSmem*>(fused_smem_raw);
+
+  pdl_launch_dependents();  // the next call on the stream may start its own phase 1
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const FinishArgs& f = a.fin;
+  const int V = f.V;
+  const int rows_per_seq = f.T + f.gamma;
+  const int cpr = (V + EPS - 1) / EPS;   // stages per row
+  const int k_top = a.top_k;
+
+  if (tid == 0) {
+    for (int s = 0; s < kTkStages; ++s) { mbar_init(&sm.full[s], 1); sm.readers_done[s] = 0; }
+    mbar_init(&sm.fst.bar, 1);
+    sm.n_done = 0;
+    sm.abort = 0;
+    sm.n_cand[0] = 0;
+    sm.n_cand[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // this block's rows: a contiguous range, so that a sequence's rows sit in few blocks and
+  // the finishes spread over the grid
+  const int row_begin = (int)((long long)a.n_items * blockIdx.x / gridDim.x);
+  const int row_end = (int)((long long)a.n_items * (blockIdx.x + 1) / gridDim.x);
+
+  auto row_of = [&](int row_id) -> Row<T, CFG> {
+    const int b = row_id / rows_per_seq;
+    const int r = row_id - b * rows_per_seq;
+    Row<T, CFG> row;
+    row.scale = f.cfg_scale;
+    row.thr = CSD_NEG_INF;
+    if (r < f.T) {
+      const int64_t off = (int64_t)b * f.tstride + (int64_t)r * V;
+      row.cond = reinterpret_cast<const T*>(f.target) + off;
+      row.uncond = CFG ? reinterpret_cast<const T*>(f.target_uncond) + off : nullptr;
+    } else {
+      const int64_t off = (int64_t)b * f.dstride + (int64_t)(r - f.T) * V;
+      row.cond = reinterpret_cast<const T*>(f.draft) + off;
+      row.uncond = CFG ? reinterpret_cast<const T*>(f.draft_uncond) + off : nullptr;
+    }
+    return row;
+  };
+  auto token_of_row = [&](int row_id) -> int {
+    const int b = row_id / rows_per_seq;
+    const int r = row_id - b * rows_per_seq;
+    const int i = r < f.T ? r : r - f.T;
+    return i < f.gamma ? __ldg(f.tokens + (int64_t)b * f.gamma + i) : -1;
+  };
+  // Issues the copies of this block's q-th chunk (if there is one) into stage q % kTkStages.
+  auto issue_chunk = [&](int q) {
+    const int j = q / cpr;
+    const int c = q - j * cpr;
+    const int row_id = row_begin + j;
+    if (row_id >= row_end) return;
+    const Row<T, CFG> row = row_of(row_id);
+    const int s = q % kTkStages;
+    const int x0 = c * EPS;
+    const uint32_t bytes = (uint32_t)(min(EPS, V - x0) * (int)sizeof(T));
+    mbar_expect_tx(&sm.full[s], bytes * ARR);
+    bulk_load(&sm.ring[s][0], row.cond + x0, bytes, &sm.full[s]);
+    if (CFG) bulk_load(&sm.ring[s][kTkStageBytes / 2], row.uncond + x0, bytes, &sm.full[s]);
+  };
+  if (tid == 0) {
+    for (int q = 0; q < kTkStages; ++q) issue_chunk(q);
+  }
+
+  // Merges the per-warp partials of a finished row (parity par) into its stash entry.
+  auto stash_row = [&](int idx, int par) {
+    float tot = 0.0f;
+    int ctot = 0;
+#pragma unroll
+    for (int w = 0; w < kFusedWarps; ++w) { tot += sm.part_acc[par][w]; ctot += sm.part_cmax[par][w]; }
+    if (idx < kTkStash) {
+      sm.stash[idx] = make_float2(sm.part_max[par], tot + (float)(ctot - 1));
+      sm.stash_thr[idx] = sm.part_thr[par];
+    }
+  };
+
+  // ================================= phase 1 ===========================================
+  int n_my = 0;
+  {
+    int q = 0;
+    bool ok = true;
+    int tok_next = row_begin < row_end ? token_of_row(row_begin) : -1;
+    for (int row_id = row_begin; row_id < row_end; ++row_id, ++n_my) {
+      const int par = n_my & 1;
+      const int tok_cur = tok_next;
+      if (row_id + 1 < row_end) tok_next = token_of_row(row_id + 1);
+      float lo = 0.0f, scale = 0.0f;
+      float mx = CSD_NEG_INF;
+      if (lane == 0) sm.wpos[warp] = 0;
+      for (int d = tid; d < kLinBins; d += kFusedThreads) sm.hist[d] = 0;
+      for (int c = 0; c < cpr; ++c) {
+        const int s = q % kTkStages;
+        const uint32_t par_s = (uint32_t)(q / kTkStages) & 1u;
+        ++q;
+        if (ok && !mbar_wait(&sm.full[s], par_s)) ok = false;
+        const int x0 = c * EPS;
+        const int n = min(EPS, V - x0);
+        float z[VPT];
+#pragma unroll
+        for (int v = 0; v < NVS; ++v) {
+          const int xo = (v * kFusedThreads + tid) * VEC;
+          float zc[VEC];
+          if (ok && xo < n) {
+            unpack_vec<T>(&sm.ring[s][xo * (int)sizeof(T)], zc);
+            if (CFG) {
+              float zu[VEC];
+              unpack_vec<T>(&sm.ring[s][kTkStageBytes / 2 + xo * (int)sizeof(T)], zu);
+#pragma unroll
+              for (int e = 0; e < VEC; ++e) zc[e] = cfg_mix(zc[e], zu[e], f.cfg_scale);
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) zc[e] = ok ? CSD_NEG_INF : __int_as_float(0x7fc00000);
+          }
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) z[v * VEC + e] = zc[e];
+        }
+        const int tl = tok_cur - x0;
+        if (tid == 0 && ok && tl >= 0 && tl < n) {   // the drafted token's logit passes by: keep it
+          float zc = load_scalar_smem<T>(&sm.ring[s][tl * (int)sizeof(T)]);
+          if (CFG) zc = cfg_mix(zc, load_scalar_smem<T>(&sm.ring[s][kTkStageBytes / 2 + tl * (int)sizeof(T)]), f.cfg_scale);
+          if (n_my < kTkStash) sm.stash_tokz[n_my] = zc;
+        }
+        __syncwarp();
+        if (lane == 0) {   // this warp is done with the stage; the last one to say so refills it
+          __threadfence_block();
+          if (atomicAdd(&sm.readers_done[s], 1) == kFusedWarps - 1) {
+            sm.readers_done[s] = 0;
+            __threadfence_block();
+            fence_before_bulk();
+            issue_chunk(q - 1 + kTkStages);
+          }
+        }
+        // running maximum (NaN-propagating: a NaN must mark the row)
+        float m4[4] = {mx, CSD_NEG_INF, CSD_NEG_INF, CSD_NEG_INF};
+#pragma unroll
+        for (int e = 0; e < VPT; ++e) m4[e & 3] = max_nan(m4[e & 3], z[e]);
+        mx = max_nan(max_nan(m4[0], m4[1]), max_nan(m4[2], m4[3]));
+        if (c == 0) {
+          // the first stage is the sample for the threshold guess
+          float sum1 = 0.0f, sum2 = 0.0f, cnt = 0.0f;
+#pragma unroll
+          for (int v = 0; v < NVS; ++v) {
+            if ((v * kFusedThreads + tid) * VEC < n) {
+#pragma unroll
+              for (int e = 0; e < VEC; ++e) { sum1 += z[v * VEC + e]; sum2 = fmaf(z[v * VEC + e], z[v * VEC + e], sum2); }
+              cnt += (float)VEC;
+            }
+          }
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) {
+            sum1 += __shfl_xor_sync(0xffffffffu, sum1, off);
+            sum2 += __shfl_xor_sync(0xffffffffu, sum2, off);
+            cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
+          }
+          if (lane == 0) { sm.mom[warp][0] = sum1; sm.mom[warp][1] = sum2; sm.mom[warp][2] = cnt; }
+          __syncthreads();   // ---- S0: moments, cleared histogram and list cursors; the previous row is complete
+          if (tid == 0) {
+            sm.n_cand[par ^ 1] = 0;   // for the next row; nobody reads the previous row's count any more
+            if (n_my > 0) stash_row(n_my - 1, par ^ 1);
+          }
+          float s1 = 0.0f, s2 = 0.0f, nn = 0.0f;
+#pragma unroll
+          for (int w = 0; w < kFusedWarps; ++w) { s1 += sm.mom[w][0]; s2 += sm.mom[w][1]; nn += sm.mom[w][2]; }
+          const float mean = s1 / nn;
+          const float dev = sqrtf(fmaxf(s2 / nn - mean * mean, 0.0f));
+          lo = mean + a.lo_sigmas * dev;
+          scale = (float)kLinBins / (kLinRangeSigmas * dev);
+        }
+        // ---- gather this stage's values >= lo into the warp's list -------------------------
+        int cnt = 0;
+#pragma unroll
+        for (int e = 0; e < VPT; ++e) cnt += (z[e] >= lo) ? 1 : 0;
+        if (cnt > 0) {
+          int pos = atomicAdd(&sm.wpos[warp], cnt);
+#pragma unroll
+          for (int e = 0; e < VPT; ++e) {
+            if (z[e] >= lo) {
+              if (pos < kWarpList) sm.list[warp][pos] = z[e];
+              ++pos;
+            }
+          }
+        }
+      }
+      // ---- end of the row: this warp's maximum and its share of the histogram ---------------
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) mx = max_nan(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+      __syncwarp();
+      const int wc = sm.wpos[warp];
+      if (lane == 0) sm.wmax[warp] = mx;
+      if (wc <= kWarpList) {
+        for (int i = lane; i < wc; i += 32) atomicAdd(&sm.hist[lin_bin(sm.list[warp][i], lo, scale)], 1);
+      }
+      __syncthreads();   // ---- B: lists, maxima and histogram complete
+      int n_lo = 0;
+      bool fast = true;
+      mx = sm.wmax[0];
+#pragma unroll
+      for (int w = 0; w < kFusedWarps; ++w) {
+        const int cw = sm.wpos[w];
+        if (cw > kWarpList) fast = false;
+        n_lo += cw;
+        mx = max_nan(mx, sm.wmax[w]);
+      }
+      // NaN guesses, NaN / +inf rows and constant rows all fail one of these tests
+      fast = fast && n_lo >= k_top && (mx > lo) && (mx < CSD_POS_INF) && (scale > 0.0f) && (scale < CSD_POS_INF);
+      if (fast) {
+        int kk;
+        const int pick_bin = warp_pick_bin(sm.hist, k_top, lane, &kk);   // every warp computes it for itself
+        for (int i = lane; i < wc; i += 32) {
+          const float v = sm.list[warp][i];
+          if (lin_bin(v, lo, scale) == pick_bin) {
+            const int slot = atomicAdd(&sm.n_cand[par], 1);
+            if (slot < kCandCap) sm.cand[slot] = v;
+          }
+        }
+        __syncthreads();   // ---- D: candidates complete
+        const int n_cand = sm.n_cand[par];
+        if (n_cand <= kCandCap) {
+          // exact rank among the candidates, every warp for itself (two candidates per lane)
+          const float v0 = lane < n_cand ? sm.cand[lane] : CSD_NEG_INF;
+          const float v1 = lane + 32 < n_cand ? sm.cand[lane + 32] : CSD_NEG_INF;
+          int gt0 = 0, ge0 = 0, gt1 = 0, ge1 = 0;
+          for (int j2 = 0; j2 < n_cand; ++j2) {
+            const float w = sm.cand[j2];
+            gt0 += (w > v0) ? 1 : 0; ge0 += (w >= v0) ? 1 : 0;
+            gt1 += (w > v1) ? 1 : 0; ge1 += (w >= v1) ? 1 : 0;
+          }
+          const bool hit0 = lane < n_cand && gt0 < kk && kk <= ge0;
+          const bool hit1 = lane + 32 < n_cand && gt1 < kk && kk <= ge1;
+          const unsigned b0 = __ballot_sync(0xffffffffu, hit0);
+          const unsigned b1 = __ballot_sync(0xffffffffu, hit1);
+          const float thr = b0 ? __shfl_sync(0xffffffffu, v0, __ffs(b0) - 1)
+                               : __shfl_sync(0xffffffffu, v1, b1 ? __ffs(b1) - 1 : 0);
+          // ---- statistics of the kept values of this warp's list -------------------------
+          float acc = 0.0f;
+          int cmax = 0;
+          for (int i = lane; i < wc; i += 32) {
+            const float v = sm.list[warp][i];
+            if (v >= thr) {
+              if (v == mx) cmax += 1;
+              else acc += ex2f((v - mx) * kLog2e);
+            }
+          }
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) {
+            acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            cmax += __shfl_xor_sync(0xffffffffu, cmax, off);
+          }
+          if (lane == 0) { sm.part_acc[par][warp] = acc; sm.part_cmax[par][warp] = cmax; }
+          if (tid == 0) { sm.part_max[par] = mx; sm.part_thr[par] = thr; }
+          continue;   // the partials are merged after the next row's first barrier
+        }
+        // crowded bin: fall through (the same decision in every thread: n_cand is shared)
+      }
+      // ---- exact select and statistics from global memory (rare) ------------------------------
+      __syncthreads();
+      {
+        float m_e = 0.0f, s_e = 0.0f, thr_e = 0.0f;
+        exact_row_from_global<T, CFG>(row_of(row_id), V, k_top, sm, tid, m_e, s_e, thr_e);
+        if (tid == 0) {
+          // same form as the fast path's partials: one "maximum", the rest in warp 0's slot
+#pragma unroll
+          for (int w = 0; w < kFusedWarps; ++w) { sm.part_acc[par][w] = 0.0f; sm.part_cmax[par][w] = 0; }
+          sm.part_acc[par][0] = s_e;
+          sm.part_cmax[par][0] = 1;
+          sm.part_max[par] = m_e;
+          sm.part_thr[par] = thr_e;
+        }
+      }
+    }
+    __syncthreads();
+    if (tid == 0 && n_my > 0) stash_row(n_my - 1, (n_my - 1) & 1);
+    if (!ok && tid == 0) {
+      sm.abort = 1;
+      atomicExch(a.error_flag, 1);
+      // copies issued for stages this thread gave up on may still be in flight: wait for them, again bounded
+      for (int s = 0; s < kTkStages; ++s)
+        if (q > s) (void)mbar_wait(&sm.full[s], ((q - 1 - s) / kTkStages) & 1);
+    }
+  }
+
+  // ================================= phase 2 ===========================================
+  pdl_wait();   // the previous call on the stream has finished with the workspace and the outputs
+  __syncthreads();
+  for (int idx = tid; idx < n_my; idx += kFusedThreads) {
+    const int row_id = row_begin + idx;
+    const_cast<float2*>(f.partials)[row_id] = sm.stash[idx];
+    const_cast<float*>(f.thresholds)[row_id] = sm.stash_thr[idx];
+    a.tok_logit[row_id] = sm.stash_tokz[idx];
+  }
+  __threadfence();
+  __syncthreads();
+  for (int idx = tid; idx < n_my; idx += kFusedThreads) {
+    const int b = (row_begin + idx) / rows_per_seq;
+    __threadfence();
+    const int old = atomicAdd(&a.counters[b], 1);
+    if (old + 1 == a.items_per_seq) {
+      const int slot = atomicAdd(&sm.n_done, 1);
+      sm.done[slot] = b;
+    }
+  }
+  __syncthreads();
+  static_assert(sizeof(sm.list) >= kFinTiles * sizeof(double), "tile sums live in the list area");
+  finish_completed<T, CFG>(a, tid, sm.done, sm.n_done, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
+                           reinterpret_cast<double*>(&sm.list[0][0]), sm.fin, sm.fst);
+}
+
+}  // namespace csd
