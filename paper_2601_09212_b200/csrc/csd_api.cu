@@ -285,26 +285,34 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
     ua.tok_logit = reinterpret_cast<float*>((char*)p.workspace + lay.tok_logit_off);
     ua.counters = reinterpret_cast<int*>((char*)p.workspace + lay.counters_off);
     ua.error_flag = reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
-    long long grid, n_items;
+    // Blocks are aligned with sequences: either a sequence's items are split over ctas_per_seq
+    // blocks, or a block owns seqs_per_cta whole sequences.
+    const long long target_blocks = (topk ? 2LL : 3LL) * sms;
+    long long c = 1, spc = 1, grid;
+    if (p.B >= target_blocks) {
+      spc = (p.B + target_blocks - 1) / target_blocks;
+      grid = (p.B + spc - 1) / spc;
+    } else {
+      c = target_blocks / p.B;
+      grid = 0;   // set below
+    }
     if (topk) {
       // one block-wide item per row, streamed in stages
       ua.chunks_per_part = 0;
       ua.parts_per_row = 1;
       ua.fin.parts = 1;
-      n_items = rows;
+      ua.items_per_seq = rows_per_seq;
       const double k = p.top_k, v = p.V;
       const double tail = 1.25 * k / v + 4.0 * sqrt(k) / v + 16.0 / v;
       if (tail < 0.45 && tail * v < 0.8 * kListCap) ua.lo_sigmas = (float)normal_upper_quantile(tail);
-      grid = 2LL * sms;
-      if (grid > n_items) grid = n_items;
-      const long long need = (n_items + kTkStash - 1) / kTkStash;
-      if (grid < need) grid = need;
+      if (c > rows_per_seq) c = rows_per_seq;
+      // a block keeps one stash entry per row
+      while (spc * rows_per_seq > kTkStash) --spc;   // rows_per_seq <= 65 < kTkStash: spc stays >= 1
     } else {
       // warp-wide items: parts of rows, sized so that every warp of the grid gets several
       const int eps = kWStageBytes / (es * (cfg ? 2 : 1));
       const long long cpr = (p.V + eps - 1) / eps;
-      grid = 3LL * sms;
-      const long long warps = grid * kFusedWarps;
+      const long long warps = (c > 1 ? (long long)p.B * c : (p.B + spc - 1) / spc) * kFusedWarps;
       long long cpp = rows * cpr / (4 * warps);
       if (cpp < 1) cpp = 1;
       if (cpp > 8) cpp = 8;
@@ -313,17 +321,25 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
       const long long min_cpp = (cpr + max_parts - 1) / max_parts;
       if (cpp < min_cpp) cpp = min_cpp;
       if (cpp > cpr) cpp = cpr;
+      // a warp keeps one stash entry per item
+      for (;;) {
+        const long long parts = (cpr + cpp - 1) / cpp;
+        const long long per_block = (c > 1) ? (rows_per_seq * parts + c - 1) / c : spc * rows_per_seq * parts;
+        if ((per_block + kFusedWarps - 1) / kFusedWarps + 1 <= kWarpStash) break;
+        if (cpp < cpr) cpp = (cpp * 2 < cpr) ? cpp * 2 : cpr;
+        else if (spc > 1) --spc;
+        else break;   // one sequence per block, one part per row: at most 65 items per block
+      }
       ua.chunks_per_part = (int)cpp;
       ua.parts_per_row = (int)((cpr + cpp - 1) / cpp);
       ua.fin.parts = ua.parts_per_row;
-      n_items = rows * ua.parts_per_row;
-      if (n_items > 0x7fffffffLL) return CSD_ERR_SHAPE;
-      if (grid * kFusedWarps > n_items) grid = (n_items + kFusedWarps - 1) / kFusedWarps;
-      const long long need = (n_items + (long long)kFusedWarps * kWarpStash - 1) / ((long long)kFusedWarps * kWarpStash);
-      if (grid < need) grid = need;
+      ua.items_per_seq = rows_per_seq * ua.parts_per_row;
+      if (c > ua.items_per_seq) c = ua.items_per_seq;
     }
-    ua.n_items = (int)n_items;
-    ua.items_per_seq = (int)(n_items / p.B);
+    if (c > 1) grid = (long long)p.B * c;
+    else grid = (p.B + spc - 1) / spc;
+    ua.ctas_per_seq = (int)c;
+    ua.seqs_per_cta = (int)spc;
     cudaError_t fe;
     if (p.dtype == CSD_F32)
       fe = cfg ? launch_fused_t<float, true>(ua, topk, (int)grid, stream) : launch_fused_t<float, false>(ua, topk, (int)grid, stream);

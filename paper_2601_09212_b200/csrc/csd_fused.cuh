@@ -41,21 +41,24 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
+  // the last operand is a hint: the hardware may park the thread for up to that many ns
   asm volatile(
-      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(smem_addr(bar)), "r"(parity)
+      : "r"(smem_addr(bar)), "r"(parity), "r"(2000u)
       : "memory");
   return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within kWaitCycles.
+// Bounded wait: false if the phase did not complete within about kWaitCycles.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
     if (clock64() - t0 > kWaitCycles) return false;
   }
-  return true;
 }
 // global -> shared bulk copy of `bytes` (multiple of 16; both addresses 16-byte aligned),
 // completion counted in bytes on `bar`
@@ -105,10 +108,12 @@ __device__ __forceinline__ float load_scalar_smem<__nv_bfloat16>(const unsigned 
 
 struct FusedArgs {
   FinishArgs fin;       // inputs, outputs, partials [rows][fin.parts], thresholds [rows]
-  int n_items;          // plain: rows * parts_per_row; top-k: rows
   int chunks_per_part;  // plain kernel: warp stages per part
   int parts_per_row;    // plain kernel
-  int items_per_seq;
+  int items_per_seq;    // plain: rows per sequence * parts_per_row; top-k: rows per sequence
+  int ctas_per_seq;     // > 1: a sequence's items are split over this many blocks (its last block to
+                        //      arrive runs the finish); 1: a block owns seqs_per_cta whole sequences
+  int seqs_per_cta;
   int top_k;
   float lo_sigmas;      // top-k guess: lo = mean + lo_sigmas * deviation (NaN: always select exactly)
   float* tok_logit;     // [rows] (mixed, unfiltered) logit of the row's drafted token, written in phase 2
@@ -437,20 +442,52 @@ __device__ void finish_sequence_staged(const FusedArgs& ua, const int b, const i
   __syncthreads();  // the shared state may be reused for the next sequence
 }
 
-// Phase 2 tail shared by both kernels: run the finish of every sequence this block completed.
+// This block's share of the items (both kernels): either a slice of one sequence's items, or
+// all items of a few whole sequences.
+struct BlockShare {
+  int seq_begin, seq_end;     // sequences this block touches
+  int item_begin, item_end;   // global item indices
+};
+__device__ __forceinline__ BlockShare block_share(const FusedArgs& a) {
+  BlockShare sh;
+  const int ips = a.items_per_seq;
+  if (a.ctas_per_seq > 1) {
+    const int b = blockIdx.x / a.ctas_per_seq;
+    const int j = blockIdx.x - b * a.ctas_per_seq;
+    sh.seq_begin = b;
+    sh.seq_end = b + 1;
+    sh.item_begin = b * ips + (int)((long long)ips * j / a.ctas_per_seq);
+    sh.item_end = b * ips + (int)((long long)ips * (j + 1) / a.ctas_per_seq);
+  } else {
+    sh.seq_begin = min(a.fin.B, (int)blockIdx.x * a.seqs_per_cta);
+    sh.seq_end = min(a.fin.B, sh.seq_begin + a.seqs_per_cta);
+    sh.item_begin = sh.seq_begin * ips;
+    sh.item_end = sh.seq_end * ips;
+  }
+  return sh;
+}
+
+// Phase 2 tail shared by both kernels, entered after every thread's results are in global memory
+// (stores, __threadfence, __syncthreads): count this block's arrival and run the finishes it owes.
 template <typename T, bool CFG>
-__device__ __forceinline__ void finish_completed(const FusedArgs& a, int tid, const int* done, int n_done, bool aborted,
-                                                 unsigned char* ring, int ring_bytes, double* tile_sums,
-                                                 FinishSmem& fin, FinishStage& fst) {
-  if (n_done <= 0) return;
-  __threadfence();
+__device__ __forceinline__ void arrive_and_finish(const FusedArgs& a, const BlockShare& sh, int tid, int* flag_smem,
+                                                  bool aborted, unsigned char* ring, int ring_bytes,
+                                                  double* tile_sums, FinishSmem& fin, FinishStage& fst) {
+  if (a.ctas_per_seq > 1) {
+    if (tid == 0) {
+      __threadfence();
+      const int old = atomicAdd(&a.counters[sh.seq_begin], 1);
+      *flag_smem = (old + 1 == a.ctas_per_seq) ? 1 : 0;
+    }
+    __syncthreads();
+    if (*flag_smem == 0) return;   // another block of this sequence arrives later and finishes it
+    __threadfence();
+  }
   const int extra = (aborted || __ldcg(a.error_flag)) ? 8 : 0;
   uint32_t fin_phase = 0;
-  for (int d = 0; d < n_done; ++d) {
-    const int b = done[d];
+  for (int b = sh.seq_begin; b < sh.seq_end; ++b)
     finish_sequence_staged<T, CFG>(a, b, tid, ring, ring_bytes, tile_sums, fin, fst, fin_phase, extra);
-    if (tid == 0) a.counters[b] = 0;   // ready for the next call
-  }
+  if (a.ctas_per_seq > 1 && tid == 0) a.counters[sh.seq_begin] = 0;   // ready for the next call
 }
 
 // ======================= plain kernel: one pipeline per warp ============================
@@ -470,8 +507,7 @@ struct PlainSmem {
   float2 stash[kFusedWarps][kWarpStash];
   float stash_tokz[kFusedWarps][kWarpStash];   // logit of the row's drafted token, if this part holds it
   unsigned char stash_has[kFusedWarps][kWarpStash];
-  int done[kFusedWarps * kWarpStash];
-  int n_done;
+  int last_flag;
   int abort;
   FinishSmem fin;
   FinishStage fst;
@@ -497,17 +533,18 @@ __global__ void __launch_bounds__(kFusedThreads, 3) verify_plain_kernel(const Fu
   const int rows_per_seq = f.T + f.gamma;
   const int part_elems = a.chunks_per_part * EPS;
 
-  if (tid == 0) { sm.n_done = 0; sm.abort = 0; mbar_init(&sm.fst.bar, 1); }
+  if (tid == 0) { sm.last_flag = 0; sm.abort = 0; mbar_init(&sm.fst.bar, 1); }
   if (lane == 0) {
     for (int s = 0; s < kWStages; ++s) mbar_init(&sm.full[warp][s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
 
-  const long long gw = (long long)blockIdx.x * kFusedWarps + warp;
-  const long long GW = (long long)gridDim.x * kFusedWarps;
-  const int item_begin = (int)((long long)a.n_items * gw / GW);
-  const int item_end = (int)((long long)a.n_items * (gw + 1) / GW);
+  // the block's items (sequence-aligned, see block_share), split evenly over its warps
+  const BlockShare sh = block_share(a);
+  const int n_block = sh.item_end - sh.item_begin;
+  const int item_begin = sh.item_begin + (int)((long long)n_block * warp / kFusedWarps);
+  const int item_end = sh.item_begin + (int)((long long)n_block * (warp + 1) / kFusedWarps);
 
   // producer cursor (meaningful in lane 0): the next chunk to copy
   int p_item = item_begin, p_x = 0, p_xend = 0, p_s = 0;
@@ -651,18 +688,8 @@ __global__ void __launch_bounds__(kFusedThreads, 3) verify_plain_kernel(const Fu
   }
   __threadfence();
   __syncthreads();
-  for (int idx = lane; idx < n_my; idx += 32) {
-    const int row_id = (item_begin + idx) / a.parts_per_row;
-    const int b = row_id / rows_per_seq;
-    __threadfence();
-    const int old = atomicAdd(&a.counters[b], 1);
-    if (old + 1 == a.items_per_seq) {
-      const int slot = atomicAdd(&sm.n_done, 1);
-      sm.done[slot] = b;
-    }
-  }
-  __syncthreads();
-  finish_completed<T, CFG>(a, tid, sm.done, sm.n_done, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes, sm.tile_sums, sm.fin, sm.fst);
+  arrive_and_finish<T, CFG>(a, sh, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes, sm.tile_sums,
+                            sm.fin, sm.fst);
 }
 
 // ======================= top-k kernel: a block streams whole rows ========================
@@ -701,8 +728,7 @@ struct TopkSmem {
   float2 stash[kTkStash];
   float stash_thr[kTkStash];
   float stash_tokz[kTkStash];       // logit of the row's drafted token
-  int done[kTkStash];
-  int n_done;
+  int last_flag;
   int abort;
   FinishSmem fin;
   FinishStage fst;
@@ -828,7 +854,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
   if (tid == 0) {
     for (int s = 0; s < kTkStages; ++s) { mbar_init(&sm.full[s], 1); sm.readers_done[s] = 0; }
     mbar_init(&sm.fst.bar, 1);
-    sm.n_done = 0;
+    sm.last_flag = 0;
     sm.abort = 0;
     sm.n_cand[0] = 0;
     sm.n_cand[1] = 0;
@@ -836,10 +862,9 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
   }
   __syncthreads();
 
-  // this block's rows: a contiguous range, so that a sequence's rows sit in few blocks and
-  // the finishes spread over the grid
-  const int row_begin = (int)((long long)a.n_items * blockIdx.x / gridDim.x);
-  const int row_end = (int)((long long)a.n_items * (blockIdx.x + 1) / gridDim.x);
+  // this block's rows (sequence-aligned, see block_share)
+  const BlockShare sh = block_share(a);
+  const int row_begin = sh.item_begin, row_end = sh.item_end;
 
   auto row_of = [&](int row_id) -> Row<T, CFG> {
     const int b = row_id / rows_per_seq;
@@ -864,10 +889,8 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
     const int i = r < f.T ? r : r - f.T;
     return i < f.gamma ? __ldg(f.tokens + (int64_t)b * f.gamma + i) : -1;
   };
-  // Issues the copies of this block's q-th chunk (if there is one) into stage q % kTkStages.
-  auto issue_chunk = [&](int q) {
-    const int j = q / cpr;
-    const int c = q - j * cpr;
+  // Issues the copies of chunk c of this block's j-th row (if there is one) into stage q % kTkStages.
+  auto issue_chunk = [&](int q, int j, int c) {
     const int row_id = row_begin + j;
     if (row_id >= row_end) return;
     const Row<T, CFG> row = row_of(row_id);
@@ -879,8 +902,10 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
     if (CFG) bulk_load(&sm.ring[s][kTkStageBytes / 2], row.uncond + x0, bytes, &sm.full[s]);
   };
   if (tid == 0) {
-    for (int q = 0; q < kTkStages; ++q) issue_chunk(q);
+    for (int q = 0; q < kTkStages; ++q) issue_chunk(q, q / cpr, q % cpr);
   }
+  // (row, chunk) of the chunk kTkStages ahead of the one being read, kept incrementally
+  int ahead_j = kTkStages / cpr, ahead_c = kTkStages % cpr;
 
   // Merges the per-warp partials of a finished row (parity par) into its stash entry.
   auto stash_row = [&](int idx, int par) {
@@ -916,11 +941,11 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
         const int x0 = c * EPS;
         const int n = min(EPS, V - x0);
         float z[VPT];
+        if (ok && n == EPS) {   // the common case: a full stage, no bounds to check
 #pragma unroll
-        for (int v = 0; v < NVS; ++v) {
-          const int xo = (v * kFusedThreads + tid) * VEC;
-          float zc[VEC];
-          if (ok && xo < n) {
+          for (int v = 0; v < NVS; ++v) {
+            const int xo = (v * kFusedThreads + tid) * VEC;
+            float zc[VEC];
             unpack_vec<T>(&sm.ring[s][xo * (int)sizeof(T)], zc);
             if (CFG) {
               float zu[VEC];
@@ -928,12 +953,29 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
 #pragma unroll
               for (int e = 0; e < VEC; ++e) zc[e] = cfg_mix(zc[e], zu[e], f.cfg_scale);
             }
-          } else {
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) zc[e] = ok ? CSD_NEG_INF : __int_as_float(0x7fc00000);
+            for (int e = 0; e < VEC; ++e) z[v * VEC + e] = zc[e];
           }
+        } else {
 #pragma unroll
-          for (int e = 0; e < VEC; ++e) z[v * VEC + e] = zc[e];
+          for (int v = 0; v < NVS; ++v) {
+            const int xo = (v * kFusedThreads + tid) * VEC;
+            float zc[VEC];
+            if (ok && xo < n) {
+              unpack_vec<T>(&sm.ring[s][xo * (int)sizeof(T)], zc);
+              if (CFG) {
+                float zu[VEC];
+                unpack_vec<T>(&sm.ring[s][kTkStageBytes / 2 + xo * (int)sizeof(T)], zu);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) zc[e] = cfg_mix(zc[e], zu[e], f.cfg_scale);
+              }
+            } else {
+#pragma unroll
+              for (int e = 0; e < VEC; ++e) zc[e] = ok ? CSD_NEG_INF : __int_as_float(0x7fc00000);
+            }
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) z[v * VEC + e] = zc[e];
+          }
         }
         const int tl = tok_cur - x0;
         if (tid == 0 && ok && tl >= 0 && tl < n) {   // the drafted token's logit passes by: keep it
@@ -948,14 +990,10 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
             sm.readers_done[s] = 0;
             __threadfence_block();
             fence_before_bulk();
-            issue_chunk(q - 1 + kTkStages);
+            issue_chunk(q - 1 + kTkStages, ahead_j, ahead_c);
           }
         }
-        // running maximum (NaN-propagating: a NaN must mark the row)
-        float m4[4] = {mx, CSD_NEG_INF, CSD_NEG_INF, CSD_NEG_INF};
-#pragma unroll
-        for (int e = 0; e < VPT; ++e) m4[e & 3] = max_nan(m4[e & 3], z[e]);
-        mx = max_nan(max_nan(m4[0], m4[1]), max_nan(m4[2], m4[3]));
+        if (++ahead_c == cpr) { ahead_c = 0; ++ahead_j; }
         if (c == 0) {
           // the first stage is the sample for the threshold guess
           float sum1 = 0.0f, sum2 = 0.0f, cnt = 0.0f;
@@ -988,29 +1026,36 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
           scale = (float)kLinBins / (kLinRangeSigmas * dev);
         }
         // ---- gather this stage's values >= lo into the warp's list -------------------------
+        // (the test is "not below lo", so that a NaN lands in the list and marks the row through the maximum)
         int cnt = 0;
 #pragma unroll
-        for (int e = 0; e < VPT; ++e) cnt += (z[e] >= lo) ? 1 : 0;
+        for (int e = 0; e < VPT; ++e) cnt += !(z[e] < lo) ? 1 : 0;
         if (cnt > 0) {
           int pos = atomicAdd(&sm.wpos[warp], cnt);
+          if (pos + cnt <= kWarpList) {
 #pragma unroll
-          for (int e = 0; e < VPT; ++e) {
-            if (z[e] >= lo) {
-              if (pos < kWarpList) sm.list[warp][pos] = z[e];
-              ++pos;
+            for (int e = 0; e < VPT; ++e) {
+              const bool keep = !(z[e] < lo);
+              if (keep) sm.list[warp][pos] = z[e];
+              pos += keep ? 1 : 0;
             }
           }
         }
       }
       // ---- end of the row: this warp's maximum and its share of the histogram ---------------
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) mx = max_nan(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+      // the row maximum is among the gathered values whenever the fast path applies
       __syncwarp();
       const int wc = sm.wpos[warp];
-      if (lane == 0) sm.wmax[warp] = mx;
       if (wc <= kWarpList) {
-        for (int i = lane; i < wc; i += 32) atomicAdd(&sm.hist[lin_bin(sm.list[warp][i], lo, scale)], 1);
+        for (int i = lane; i < wc; i += 32) {
+          const float v = sm.list[warp][i];
+          mx = max_nan(mx, v);
+          atomicAdd(&sm.hist[lin_bin(v, lo, scale)], 1);
+        }
       }
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) mx = max_nan(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+      if (lane == 0) sm.wmax[warp] = mx;
       __syncthreads();   // ---- B: lists, maxima and histogram complete
       int n_lo = 0;
       bool fast = true;
@@ -1111,19 +1156,9 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
   }
   __threadfence();
   __syncthreads();
-  for (int idx = tid; idx < n_my; idx += kFusedThreads) {
-    const int b = (row_begin + idx) / rows_per_seq;
-    __threadfence();
-    const int old = atomicAdd(&a.counters[b], 1);
-    if (old + 1 == a.items_per_seq) {
-      const int slot = atomicAdd(&sm.n_done, 1);
-      sm.done[slot] = b;
-    }
-  }
-  __syncthreads();
   static_assert(sizeof(sm.list) >= kFinTiles * sizeof(double), "tile sums live in the list area");
-  finish_completed<T, CFG>(a, tid, sm.done, sm.n_done, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
-                           reinterpret_cast<double*>(&sm.list[0][0]), sm.fin, sm.fst);
+  arrive_and_finish<T, CFG>(a, sh, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
+                            reinterpret_cast<double*>(&sm.list[0][0]), sm.fin, sm.fst);
 }
 
 }  // namespace csd
