@@ -614,39 +614,90 @@ __global__ void __launch_bounds__(kFusedThreads, 3) verify_plain_kernel(const Fu
       }
       float tokz = 0.0f;
       bool has_tok = false;
-      float m = CSD_NEG_INF, s_acc = -1.0f;
+      // Running statistics of the item, relative to a maximum that is the same in every lane of
+      // the warp: Mw = largest value met so far by any lane, s = this lane's sum of
+      // exp(z - Mw) over its values below Mw, cnt = this lane's number of values equal to Mw.
+      // Because the reference is warp-uniform, a group of values below it is summed with no
+      // test per value, and the exact treatment of values equal to it is a uniform branch
+      // taken only where the maximum sits.
+      float Mw = CSD_NEG_INF, s_run = 0.0f;
+      int cnt_run = 0;
       for (int x0 = x_begin; x0 < x_end; x0 += EPS) {
         if (ok && !mbar_wait(&sm.full[warp][c_s], c_par)) ok = false;
         ++issued;
         const int n = min(EPS, x_end - x0);
         const unsigned char* stage = &sm.ring[warp][c_s][0];
-        float m_c = CSD_NEG_INF, s_c = -1.0f;
+        const bool full = ok && n == EPS;
 #pragma unroll
         for (int g0 = 0; g0 < NVS; g0 += GV) {
           float vals[GV * VEC];
+          float gm;   // this lane's largest value of the group
+          if (!CFG && sizeof(T) == 2 && full) {
+            // bf16, no mix: the maximum is taken on the packed pairs before unpacking
+            uint32_t w[GV * 4];
 #pragma unroll
-          for (int v = 0; v < GV; ++v) {
-            const int xo = ((g0 + v) * 32 + lane) * VEC;
-            float zc[VEC];
-            if (ok && xo < n) {
-              unpack_vec<T>(stage + xo * (int)sizeof(T), zc);
-              if (CFG) {
-                float zu[VEC];
-                unpack_vec<T>(stage + kWStageBytes / 2 + xo * (int)sizeof(T), zu);
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) zc[e] = cfg_mix(zc[e], zu[e], f.cfg_scale);
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < VEC; ++e) zc[e] = ok ? CSD_NEG_INF : __int_as_float(0x7fc00000);
+            for (int v = 0; v < GV; ++v) {
+              const uint4 q4 = *reinterpret_cast<const uint4*>(stage + ((g0 + v) * 32 + lane) * VEC * (int)sizeof(T));
+              w[v * 4 + 0] = q4.x; w[v * 4 + 1] = q4.y; w[v * 4 + 2] = q4.z; w[v * 4 + 3] = q4.w;
             }
+            uint32_t m2 = w[0];
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) vals[v * VEC + e] = zc[e];
+            for (int k = 1; k < GV * 4; ++k) asm("max.bf16x2 %0, %0, %1;" : "+r"(m2) : "r"(w[k]));
+            gm = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xffff0000u));
+#pragma unroll
+            for (int k = 0; k < GV * 4; ++k) {
+              vals[2 * k] = __uint_as_float(w[k] << 16);
+              vals[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+            }
+          } else {
+#pragma unroll
+            for (int v = 0; v < GV; ++v) {
+              const int xo = ((g0 + v) * 32 + lane) * VEC;
+              float zc[VEC];
+              if (full || (ok && xo < n)) {
+                unpack_vec<T>(stage + xo * (int)sizeof(T), zc);
+                if (CFG) {
+                  float zu[VEC];
+                  unpack_vec<T>(stage + kWStageBytes / 2 + xo * (int)sizeof(T), zu);
+#pragma unroll
+                  for (int e = 0; e < VEC; ++e) zc[e] = cfg_mix(zc[e], zu[e], f.cfg_scale);
+                }
+              } else {
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) zc[e] = ok ? CSD_NEG_INF : __int_as_float(0x7fc00000);
+              }
+#pragma unroll
+              for (int e = 0; e < VEC; ++e) vals[v * VEC + e] = zc[e];
+            }
+            float m4[4] = {CSD_NEG_INF, CSD_NEG_INF, CSD_NEG_INF, CSD_NEG_INF};
+#pragma unroll
+            for (int e = 0; e < GV * VEC; ++e) m4[e & 3] = fmaxf(m4[e & 3], vals[e]);
+            gm = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
           }
-          float m1, s1;
-          stat_of_values(vals, m1, s1);
-          if (g0 == 0) { m_c = m1; s_c = s1; }
-          else stat_merge(m_c, s_c, m1, s1);   // a group of padding only merges as the identity
+          // the group's largest value over the warp (one integer reduction on order-preserving keys)
+          int key = __float_as_int(gm);
+          key ^= (key >> 31) & 0x7fffffff;
+          key = __reduce_max_sync(0xffffffffu, key);
+          key ^= (key >> 31) & 0x7fffffff;
+          const float wm = __int_as_float(key);
+          if (wm > Mw) {   // a new maximum: what was counted as "equal to the maximum" becomes ordinary mass
+            s_run = (s_run + (float)cnt_run) * ex2f((Mw - wm) * kLog2e);
+            cnt_run = 0;
+            Mw = wm;
+          }
+          if (wm == Mw) {
+            // values equal to the reference may be present: they are counted, not summed
+#pragma unroll
+            for (int e = 0; e < GV * VEC; ++e) {
+              const float ex = ex2f((vals[e] - Mw) * kLog2e);
+              if (vals[e] == Mw) cnt_run += 1; else s_run += ex;   // NaN values poison s_run, which marks the row
+            }
+          } else {
+            float acc4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+            for (int e = 0; e < GV * VEC; ++e) acc4[e & 3] += ex2f((vals[e] - Mw) * kLog2e);
+            s_run += (acc4[0] + acc4[1]) + (acc4[2] + acc4[3]);
+          }
         }
         const int tl = tok_cur - x0;
         if (ok && tl >= 0 && tl < n) {   // the drafted token's logit passes by: keep it
@@ -660,12 +711,16 @@ __global__ void __launch_bounds__(kFusedThreads, 3) verify_plain_kernel(const Fu
           fence_before_bulk();
           producer_issue();
         }
-        if (lane * VEC < n || !ok) stat_merge(m, s_acc, m_c, s_c);
         if (++c_s == kWStages) { c_s = 0; c_par ^= 1u; }
       }
-      stat_warp_allreduce(m, s_acc);
+      // the item's pair: m = Mw, s = sum over everything except one entry at the maximum
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) {
+        s_run += __shfl_xor_sync(0xffffffffu, s_run, off);
+        cnt_run += __shfl_xor_sync(0xffffffffu, cnt_run, off);
+      }
       if (lane == 0 && n_my < kWarpStash) {
-        sm.stash[warp][n_my] = make_float2(m, s_acc);
+        sm.stash[warp][n_my] = make_float2(Mw, s_run + (float)(cnt_run - 1));
         sm.stash_tokz[warp][n_my] = tokz;
         sm.stash_has[warp][n_my] = has_tok ? 1 : 0;
       }
