@@ -17,7 +17,7 @@ namespace {
 using namespace csd;
 
 static_assert(sizeof(TopkSmem) <= 55 * 1024, "four blocks of the top-k kernel per SM must fit");
-static_assert(sizeof(PlainSmem) <= 74 * 1024, "three blocks of the plain kernel per SM must fit");
+static_assert(sizeof(PlainSmem) <= 112 * 1024, "two blocks of the plain kernel per SM must fit");
 
 constexpr int kMaxV = 1 << 20;
 constexpr int kMaxDevices = 64;
@@ -94,7 +94,7 @@ cudaError_t launch_fused(const FusedArgs& a, int grid, cudaStream_t stream) {
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(kFusedThreads);
+  cfg.blockDim = dim3(kTopkThreads);
   cfg.dynamicSmemBytes = sizeof(TopkSmem);
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -117,7 +117,7 @@ cudaError_t launch_plain(const FusedArgs& a, int grid, cudaStream_t stream) {
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(kFusedThreads);
+  cfg.blockDim = dim3(kPlainThreads);
   cfg.dynamicSmemBytes = sizeof(PlainSmem);
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -287,7 +287,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
     ua.error_flag = reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
     // Blocks are aligned with sequences: either a sequence's items are split over ctas_per_seq
     // blocks, or a block owns seqs_per_cta whole sequences.
-    const long long target_blocks = (topk ? 2LL : 3LL) * sms;
+    const long long target_blocks = 2LL * sms;
     long long c = 1, spc = 1, grid;
     if (p.B >= target_blocks) {
       spc = (p.B + target_blocks - 1) / target_blocks;
@@ -312,7 +312,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
       // warp-wide items: parts of rows, sized so that every warp of the grid gets several
       const int eps = kWStageBytes / (es * (cfg ? 2 : 1));
       const long long cpr = (p.V + eps - 1) / eps;
-      const long long warps = (c > 1 ? (long long)p.B * c : (p.B + spc - 1) / spc) * kFusedWarps;
+      const long long warps = (c > 1 ? (long long)p.B * c : (p.B + spc - 1) / spc) * kPlainWarps;
       long long cpp = rows * cpr / (4 * warps);
       if (cpp < 1) cpp = 1;
       if (cpp > 8) cpp = 8;
@@ -325,7 +325,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
       for (;;) {
         const long long parts = (cpr + cpp - 1) / cpp;
         const long long per_block = (c > 1) ? (rows_per_seq * parts + c - 1) / c : spc * rows_per_seq * parts;
-        if ((per_block + kFusedWarps - 1) / kFusedWarps + 1 <= kWarpStash) break;
+        if ((per_block + kPlainWarps - 1) / kPlainWarps + 1 <= kWarpStash) break;
         if (cpp < cpr) cpp = (cpp * 2 < cpr) ? cpp * 2 : cpr;
         else if (spc > 1) --spc;
         else break;   // one sequence per block, one part per row: at most 65 items per block

@@ -26,8 +26,10 @@
 
 namespace csd {
 
-constexpr int kFusedThreads = 256;
-constexpr int kFusedWarps = kFusedThreads / 32;
+constexpr int kPlainThreads = 384;   // plain kernel: 12 independent warp pipelines, two blocks per SM
+constexpr int kPlainWarps = kPlainThreads / 32;
+constexpr int kTopkThreads = 256;    // top-k kernel: 8 warps per row, four blocks per SM
+constexpr int kTopkWarps = kTopkThreads / 32;
 constexpr long long kWaitCycles = 1ll << 31;  // about a second: then give up and flag it
 constexpr int kFinTiles = 1024;               // tiles of 32 lanes x 16 bytes: V <= 131072 (fp32) / 262144 (bf16)
 
@@ -151,11 +153,10 @@ __device__ __forceinline__ void stat_warp_allreduce2(float& m0, float& s0, float
 
 // ring: `ring_bytes` of shared memory (multiple of 4 KB) that nothing else uses meanwhile;
 // tile_sums: kFinTiles doubles, likewise.
-template <typename T, bool CFG>
+template <typename T, bool CFG, int NT>
 __device__ void finish_sequence_staged(const FusedArgs& ua, const int b, const int tid, unsigned char* ring,
                                        const int ring_bytes, double* tile_sums, FinishSmem& sm, FinishStage& st,
                                        uint32_t& phase, const int extra_status) {
-  constexpr int NT = kFusedThreads;
   constexpr int VEC = Elem<T>::kVec;
   constexpr int TILE = 32 * VEC;
   constexpr int ARR = CFG ? 2 : 1;
@@ -469,7 +470,7 @@ __device__ __forceinline__ BlockShare block_share(const FusedArgs& a) {
 
 // Phase 2 tail shared by both kernels, entered after every thread's results are in global memory
 // (stores, __threadfence, __syncthreads): count this block's arrival and run the finishes it owes.
-template <typename T, bool CFG>
+template <typename T, bool CFG, int NT>
 __device__ __forceinline__ void arrive_and_finish(const FusedArgs& a, const BlockShare& sh, int tid, int* flag_smem,
                                                   bool aborted, unsigned char* ring, int ring_bytes,
                                                   double* tile_sums, FinishSmem& fin, FinishStage& fst) {
@@ -486,27 +487,27 @@ __device__ __forceinline__ void arrive_and_finish(const FusedArgs& a, const Bloc
   const int extra = (aborted || __ldcg(a.error_flag)) ? 8 : 0;
   uint32_t fin_phase = 0;
   for (int b = sh.seq_begin; b < sh.seq_end; ++b)
-    finish_sequence_staged<T, CFG>(a, b, tid, ring, ring_bytes, tile_sums, fin, fst, fin_phase, extra);
+    finish_sequence_staged<T, CFG, NT>(a, b, tid, ring, ring_bytes, tile_sums, fin, fst, fin_phase, extra);
   if (a.ctas_per_seq > 1 && tid == 0) a.counters[sh.seq_begin] = 0;   // ready for the next call
 }
 
 // ======================= plain kernel: one pipeline per warp ============================
 // A warp owns a contiguous range of items (an item is a part of a row: chunks_per_part warp
 // stages), a private ring of kWStages stages of kWStageBytes, issues its own refills, and keeps
-// a running (m, s) per lane that it reduces once per item.  Eight such pipelines per block sit
+// a running (m, s) per lane that it reduces once per item.  Twelve such pipelines per block sit
 // at different points of their loops and hide each other's latencies; phase 1 has no block-wide
 // step at all.
 constexpr int kWStages = 3;
 constexpr int kWStageBytes = 2048;
 constexpr int kWarpStash = 96;
-constexpr int kPlainRingBytes = kFusedWarps * kWStages * kWStageBytes;
+constexpr int kPlainRingBytes = kPlainWarps * kWStages * kWStageBytes;
 
 struct PlainSmem {
-  alignas(128) unsigned char ring[kFusedWarps][kWStages][kWStageBytes];
-  alignas(8) uint64_t full[kFusedWarps][kWStages];
-  float2 stash[kFusedWarps][kWarpStash];
-  float stash_tokz[kFusedWarps][kWarpStash];   // logit of the row's drafted token, if this part holds it
-  unsigned char stash_has[kFusedWarps][kWarpStash];
+  alignas(128) unsigned char ring[kPlainWarps][kWStages][kWStageBytes];
+  alignas(8) uint64_t full[kPlainWarps][kWStages];
+  float2 stash[kPlainWarps][kWarpStash];
+  float stash_tokz[kPlainWarps][kWarpStash];   // logit of the row's drafted token, if this part holds it
+  unsigned char stash_has[kPlainWarps][kWarpStash];
   int last_flag;
   int abort;
   FinishSmem fin;
@@ -515,7 +516,7 @@ struct PlainSmem {
 };
 
 template <typename T, bool CFG>
-__global__ void __launch_bounds__(kFusedThreads, 3) verify_plain_kernel(const FusedArgs a) {
+__global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const FusedArgs a) {
   constexpr int VEC = Elem<T>::kVec;
   constexpr int ARR = CFG ? 2 : 1;
   constexpr int EPS = kWStageBytes / ((int)sizeof(T) * ARR);   // elements of a row per warp stage
@@ -543,8 +544,8 @@ __global__ void __launch_bounds__(kFusedThreads, 3) verify_plain_kernel(const Fu
   // the block's items (sequence-aligned, see block_share), split evenly over its warps
   const BlockShare sh = block_share(a);
   const int n_block = sh.item_end - sh.item_begin;
-  const int item_begin = sh.item_begin + (int)((long long)n_block * warp / kFusedWarps);
-  const int item_end = sh.item_begin + (int)((long long)n_block * (warp + 1) / kFusedWarps);
+  const int item_begin = sh.item_begin + (int)((long long)n_block * warp / kPlainWarps);
+  const int item_end = sh.item_begin + (int)((long long)n_block * (warp + 1) / kPlainWarps);
 
   // producer cursor (meaningful in lane 0): the next chunk to copy
   int p_item = item_begin, p_x = 0, p_xend = 0, p_s = 0;
@@ -743,7 +744,7 @@ __global__ void __launch_bounds__(kFusedThreads, 3) verify_plain_kernel(const Fu
   }
   __threadfence();
   __syncthreads();
-  arrive_and_finish<T, CFG>(a, sh, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes, sm.tile_sums,
+  arrive_and_finish<T, CFG, kPlainThreads>(a, sh, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes, sm.tile_sums,
                             sm.fin, sm.fst);
 }
 
@@ -753,7 +754,7 @@ constexpr int kTkStageBytes = 16384;
 constexpr int kTkRingBytes = kTkStages * kTkStageBytes;
 constexpr int kTkStash = 256;
 constexpr int kWarpList = 256;                // per-warp capacity of the list of values >= lo
-constexpr int kListCap = kFusedWarps * kWarpList;
+constexpr int kListCap = kTopkWarps * kWarpList;
 constexpr int kLinBins = 512;
 constexpr int kCandCap = 64;
 constexpr float kLinRangeSigmas = 4.75f;      // the histogram spans [lo, lo + this many deviations)
@@ -768,18 +769,18 @@ struct TopkSmem {
   alignas(8) uint64_t full[kTkStages];
   int readers_done[kTkStages];      // warps that have finished reading the stage's current contents
   alignas(16) int hist[kLinBins];   // linear histogram; first 256 bins double as the radix histogram
-  alignas(8) float list[kFusedWarps][kWarpList];   // per warp: the values >= lo it met (the finish keeps its tile sums here)
-  int wpos[kFusedWarps];            // per warp: next free slot of its list (may run past the capacity)
+  alignas(8) float list[kTopkWarps][kWarpList];   // per warp: the values >= lo it met (the finish keeps its tile sums here)
+  int wpos[kTopkWarps];            // per warp: next free slot of its list (may run past the capacity)
   float cand[kCandCap];             // values in the bin of the k-th largest
   int n_cand[2];                    // by row parity
-  float mom[kFusedWarps][4];        // per warp: sum, sum of squares, count of the sampled values
-  float wmax[kFusedWarps];
-  float part_acc[2][kFusedWarps];   // per warp, by row parity: sum of exp(z - max) over kept non-maximum values
-  int part_cmax[2][kFusedWarps];    //                          number of kept values equal to the maximum
+  float mom[kTopkWarps][4];        // per warp: sum, sum of squares, count of the sampled values
+  float wmax[kTopkWarps];
+  float part_acc[2][kTopkWarps];   // per warp, by row parity: sum of exp(z - max) over kept non-maximum values
+  int part_cmax[2][kTopkWarps];    //                          number of kept values equal to the maximum
   float part_max[2];
   float part_thr[2];
   int bc_i[4];
-  float red_f[kFusedWarps][2];
+  float red_f[kTopkWarps][2];
   float2 stash[kTkStash];
   float stash_thr[kTkStash];
   float stash_tokz[kTkStash];       // logit of the row's drafted token
@@ -841,9 +842,9 @@ __device__ void exact_row_from_global(const Row<T, CFG>& row, int V, int k, Topk
 #pragma unroll 1
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
-    sm.hist[tid] = 0;   // 256 threads, 256 bins
+    if (tid < 256) sm.hist[tid] = 0;
     __syncthreads();
-    for (int x0 = tid * VEC; x0 < V; x0 += kFusedThreads * VEC) {
+    for (int x0 = tid * VEC; x0 < V; x0 += kTopkThreads * VEC) {
       float z[VEC];
       row.load_vec(x0, z);
 #pragma unroll
@@ -866,7 +867,7 @@ __device__ void exact_row_from_global(const Row<T, CFG>& row, int V, int k, Topk
   }
   const float thr = order_value(prefix);
   float m = CSD_NEG_INF, s = -1.0f;
-  for (int x0 = tid * VEC; x0 < V; x0 += kFusedThreads * VEC) {
+  for (int x0 = tid * VEC; x0 < V; x0 += kTopkThreads * VEC) {
     float z[VEC];
     row.load_vec(x0, z);
 #pragma unroll
@@ -881,18 +882,18 @@ __device__ void exact_row_from_global(const Row<T, CFG>& row, int V, int k, Topk
   if (tid == 0) {
     float mm = sm.red_f[0][0], sv = sm.red_f[0][1];
 #pragma unroll
-    for (int w = 1; w < kFusedWarps; ++w) stat_merge(mm, sv, sm.red_f[w][0], sm.red_f[w][1]);
+    for (int w = 1; w < kTopkWarps; ++w) stat_merge(mm, sv, sm.red_f[w][0], sm.red_f[w][1]);
     out_m = mm; out_s = sv; out_thr = thr;
   }
   __syncthreads();
 }
 
 template <typename T, bool CFG>
-__global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const FusedArgs a) {
+__global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const FusedArgs a) {
   constexpr int VEC = Elem<T>::kVec;
   constexpr int ARR = CFG ? 2 : 1;
   constexpr int EPS = kTkStageBytes / ((int)sizeof(T) * ARR);   // elements of a row per stage
-  constexpr int VPT = EPS / kFusedThreads;                      // values per thread per stage
+  constexpr int VPT = EPS / kTopkThreads;                      // values per thread per stage
   constexpr int NVS = VPT / VEC;                                // 16-byte vectors per thread per stage
   extern __shared__ __align__(128) unsigned char fused_smem_raw[];
   TopkSmem& sm = *reinterpret_cast<TopkSmem*>(fused_smem_raw);
@@ -967,7 +968,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
     float tot = 0.0f;
     int ctot = 0;
 #pragma unroll
-    for (int w = 0; w < kFusedWarps; ++w) { tot += sm.part_acc[par][w]; ctot += sm.part_cmax[par][w]; }
+    for (int w = 0; w < kTopkWarps; ++w) { tot += sm.part_acc[par][w]; ctot += sm.part_cmax[par][w]; }
     if (idx < kTkStash) {
       sm.stash[idx] = make_float2(sm.part_max[par], tot + (float)(ctot - 1));
       sm.stash_thr[idx] = sm.part_thr[par];
@@ -987,7 +988,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
       float lo = 0.0f, scale = 0.0f;
       float mx = CSD_NEG_INF;
       if (lane == 0) sm.wpos[warp] = 0;
-      for (int d = tid; d < kLinBins; d += kFusedThreads) sm.hist[d] = 0;
+      for (int d = tid; d < kLinBins; d += kTopkThreads) sm.hist[d] = 0;
       for (int c = 0; c < cpr; ++c) {
         const int s = q % kTkStages;
         const uint32_t par_s = (uint32_t)(q / kTkStages) & 1u;
@@ -999,7 +1000,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
         if (ok && n == EPS) {   // the common case: a full stage, no bounds to check
 #pragma unroll
           for (int v = 0; v < NVS; ++v) {
-            const int xo = (v * kFusedThreads + tid) * VEC;
+            const int xo = (v * kTopkThreads + tid) * VEC;
             float zc[VEC];
             unpack_vec<T>(&sm.ring[s][xo * (int)sizeof(T)], zc);
             if (CFG) {
@@ -1014,7 +1015,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
         } else {
 #pragma unroll
           for (int v = 0; v < NVS; ++v) {
-            const int xo = (v * kFusedThreads + tid) * VEC;
+            const int xo = (v * kTopkThreads + tid) * VEC;
             float zc[VEC];
             if (ok && xo < n) {
               unpack_vec<T>(&sm.ring[s][xo * (int)sizeof(T)], zc);
@@ -1041,7 +1042,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
         __syncwarp();
         if (lane == 0) {   // this warp is done with the stage; the last one to say so refills it
           __threadfence_block();
-          if (atomicAdd(&sm.readers_done[s], 1) == kFusedWarps - 1) {
+          if (atomicAdd(&sm.readers_done[s], 1) == kTopkWarps - 1) {
             sm.readers_done[s] = 0;
             __threadfence_block();
             fence_before_bulk();
@@ -1054,7 +1055,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
           float sum1 = 0.0f, sum2 = 0.0f, cnt = 0.0f;
 #pragma unroll
           for (int v = 0; v < NVS; ++v) {
-            if ((v * kFusedThreads + tid) * VEC < n) {
+            if ((v * kTopkThreads + tid) * VEC < n) {
 #pragma unroll
               for (int e = 0; e < VEC; ++e) { sum1 += z[v * VEC + e]; sum2 = fmaf(z[v * VEC + e], z[v * VEC + e], sum2); }
               cnt += (float)VEC;
@@ -1074,7 +1075,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
           }
           float s1 = 0.0f, s2 = 0.0f, nn = 0.0f;
 #pragma unroll
-          for (int w = 0; w < kFusedWarps; ++w) { s1 += sm.mom[w][0]; s2 += sm.mom[w][1]; nn += sm.mom[w][2]; }
+          for (int w = 0; w < kTopkWarps; ++w) { s1 += sm.mom[w][0]; s2 += sm.mom[w][1]; nn += sm.mom[w][2]; }
           const float mean = s1 / nn;
           const float dev = sqrtf(fmaxf(s2 / nn - mean * mean, 0.0f));
           lo = mean + a.lo_sigmas * dev;
@@ -1116,7 +1117,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
       bool fast = true;
       mx = sm.wmax[0];
 #pragma unroll
-      for (int w = 0; w < kFusedWarps; ++w) {
+      for (int w = 0; w < kTopkWarps; ++w) {
         const int cw = sm.wpos[w];
         if (cw > kWarpList) fast = false;
         n_lo += cw;
@@ -1181,7 +1182,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
         if (tid == 0) {
           // same form as the fast path's partials: one "maximum", the rest in warp 0's slot
 #pragma unroll
-          for (int w = 0; w < kFusedWarps; ++w) { sm.part_acc[par][w] = 0.0f; sm.part_cmax[par][w] = 0; }
+          for (int w = 0; w < kTopkWarps; ++w) { sm.part_acc[par][w] = 0.0f; sm.part_cmax[par][w] = 0; }
           sm.part_acc[par][0] = s_e;
           sm.part_cmax[par][0] = 1;
           sm.part_max[par] = m_e;
@@ -1203,7 +1204,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
   // ================================= phase 2 ===========================================
   pdl_wait();   // the previous call on the stream has finished with the workspace and the outputs
   __syncthreads();
-  for (int idx = tid; idx < n_my; idx += kFusedThreads) {
+  for (int idx = tid; idx < n_my; idx += kTopkThreads) {
     const int row_id = row_begin + idx;
     const_cast<float2*>(f.partials)[row_id] = sm.stash[idx];
     const_cast<float*>(f.thresholds)[row_id] = sm.stash_thr[idx];
@@ -1212,7 +1213,7 @@ __global__ void __launch_bounds__(kFusedThreads, 4) verify_topk_kernel(const Fus
   __threadfence();
   __syncthreads();
   static_assert(sizeof(sm.list) >= kFinTiles * sizeof(double), "tile sums live in the list area");
-  arrive_and_finish<T, CFG>(a, sh, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
+  arrive_and_finish<T, CFG, kTopkThreads>(a, sh, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
                             reinterpret_cast<double*>(&sm.list[0][0]), sm.fin, sm.fst);
 }
 
