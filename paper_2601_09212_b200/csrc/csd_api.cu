@@ -338,6 +338,8 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
     }
     if (c > 1) grid = (long long)p.B * c;
     else grid = (p.B + spc - 1) / spc;
+    // calls that move less than about 40 MB stream too briefly for their phase 1 to be worth overlapping
+    ua.early_trigger = ((double)rows * p.V * es * (cfg ? 2 : 1) >= 40e6) ? 1 : 0;
     ua.ctas_per_seq = (int)c;
     ua.seqs_per_cta = (int)spc;
     cudaError_t fe;

@@ -2,13 +2,25 @@
 //
 // Phase 1 streams this block's share of the logit rows through rings of
 // shared-memory stages filled by bulk asynchronous copies (mbarrier completion)
-// and keeps the per-item results in shared memory; nothing is written to global
-// memory yet, so phase 1 may overlap the previous call on the stream
-// (programmatic dependent launch).  After griddepcontrol.wait, phase 2 publishes
-// the results, counts arrivals per sequence, and the block that completes a
+// and keeps the per-item results in shared memory.  Phase 2 publishes them to the
+// workspace, counts arrivals per sequence, and the block that completes a
 // sequence runs its finish: accept tests, tau, Eq. opt_G at position tau+1 with
 // the two rows brought back through the ring, inverse-CDF draw, emit.  No block
 // ever waits for another block; every wait on a copy is bounded.
+//
+// Consecutive calls on a stream overlap (programmatic dependent launch) in one of
+// two ways, chosen by the host from the size of the call:
+//   early trigger (large calls): every block signals launch_dependents at once, so
+//     the next call's phase 1 streams alongside this call; a block then calls
+//     griddepcontrol.wait before phase 2, i.e. it publishes only when the previous
+//     call has completed and the workspace is free.
+//   late trigger (small calls, whose streaming is short anyway): a block signals
+//     launch_dependents when it has no further use for the workspace -- after its
+//     arrival, or for a finishing block after it has copied what it needs into
+//     shared memory -- so the next call starts, streams and publishes while this
+//     call's finishes still compute; a finishing block calls griddepcontrol.wait
+//     before it writes outputs, which keeps the outputs of consecutive calls in order
+//     and makes this call complete only after the previous one.
 //
 //   verify_plain_kernel  every warp streams its own parts of rows through its own
 //                        ring and keeps a running (m, s) per lane.
@@ -121,6 +133,7 @@ struct FusedArgs {
   float* tok_logit;     // [rows] (mixed, unfiltered) logit of the row's drafted token, written in phase 2
   int* counters;        // [B] arrivals per sequence; zero before the first call, left zero by every call
   int* error_flag;      // set when a bounded wait gave up
+  int early_trigger;    // how consecutive calls overlap, see the head of this file
 };
 
 // ---- finish with everything staged in shared memory ---------------------------------
@@ -156,7 +169,7 @@ __device__ __forceinline__ void stat_warp_allreduce2(float& m0, float& s0, float
 template <typename T, bool CFG, int NT>
 __device__ void finish_sequence_staged(const FusedArgs& ua, const int b, const int tid, unsigned char* ring,
                                        const int ring_bytes, double* tile_sums, FinishSmem& sm, FinishStage& st,
-                                       uint32_t& phase, const int extra_status) {
+                                       uint32_t& phase, const int extra_status, const bool last_use_of_workspace) {
   constexpr int VEC = Elem<T>::kVec;
   constexpr int TILE = 32 * VEC;
   constexpr int ARR = CFG ? 2 : 1;
@@ -188,6 +201,11 @@ __device__ void finish_sequence_staged(const FusedArgs& ua, const int b, const i
     }
   }
   __syncthreads();
+  // Everything this block needs from the workspace now sits in shared memory.
+  if (last_use_of_workspace && !ua.early_trigger) pdl_launch_dependents();
+  // Outputs are written only once the previous call on the stream has completed; with the
+  // diagnostic outputs that is from here on, otherwise just before the emit.
+  if (a.dbg_p || a.dbg_q || a.dbg_f) pdl_wait();
 
   // ---- 1. per position: merge parts, Eq. relax, accept test ------------------------------
   const int n_pos = a.T > L ? L + 1 : L;   // the bonus position only if its row exists
@@ -411,6 +429,7 @@ __device__ void finish_sequence_staged(const FusedArgs& ua, const int b, const i
       token = sm.token;
       // ---- 7. optional: write the distribution drawn from ------------------------------
       if (G_out) {
+        pdl_wait();
         const float invZ = (float)(1.0 / Z);
         for (int tile = warp; tile < ntiles; tile += NT / 32) {
           const int x0 = tile * TILE + lane * VEC;
@@ -426,6 +445,7 @@ __device__ void finish_sequence_staged(const FusedArgs& ua, const int b, const i
       break;
     }
   }
+  pdl_wait();   // the previous call on the stream has completed: outputs stay in order
   if (G_out && token < 0)
     for (int x = tid; x < V; x += NT) G_out[x] = 0.0f;
 
@@ -474,21 +494,33 @@ template <typename T, bool CFG, int NT>
 __device__ __forceinline__ void arrive_and_finish(const FusedArgs& a, const BlockShare& sh, int tid, int* flag_smem,
                                                   bool aborted, unsigned char* ring, int ring_bytes,
                                                   double* tile_sums, FinishSmem& fin, FinishStage& fst) {
+  if (sh.seq_begin >= sh.seq_end) {   // nothing to do in this block
+    if (!a.early_trigger) pdl_launch_dependents();
+    return;
+  }
   if (a.ctas_per_seq > 1) {
     if (tid == 0) {
       __threadfence();
       const int old = atomicAdd(&a.counters[sh.seq_begin], 1);
-      *flag_smem = (old + 1 == a.ctas_per_seq) ? 1 : 0;
+      const int last = (old + 1 == a.ctas_per_seq) ? 1 : 0;
+      if (last) {   // nobody else touches this counter any more: leave it ready for the next call
+        a.counters[sh.seq_begin] = 0;
+        __threadfence();
+      }
+      *flag_smem = last;
     }
     __syncthreads();
-    if (*flag_smem == 0) return;   // another block of this sequence arrives later and finishes it
+    if (*flag_smem == 0) {   // another block of this sequence arrives later and finishes it
+      if (!a.early_trigger) pdl_launch_dependents();
+      return;
+    }
     __threadfence();
   }
   const int extra = (aborted || __ldcg(a.error_flag)) ? 8 : 0;
   uint32_t fin_phase = 0;
   for (int b = sh.seq_begin; b < sh.seq_end; ++b)
-    finish_sequence_staged<T, CFG, NT>(a, b, tid, ring, ring_bytes, tile_sums, fin, fst, fin_phase, extra);
-  if (a.ctas_per_seq > 1 && tid == 0) a.counters[sh.seq_begin] = 0;   // ready for the next call
+    finish_sequence_staged<T, CFG, NT>(a, b, tid, ring, ring_bytes, tile_sums, fin, fst, fin_phase, extra,
+                                       b == sh.seq_end - 1);
 }
 
 // ======================= plain kernel: one pipeline per warp ============================
@@ -526,8 +558,7 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
   extern __shared__ __align__(128) unsigned char fused_smem_raw[];
   PlainSmem& sm = *reinterpret_cast<PlainSmem*>(fused_smem_raw);
 
-  pdl_launch_dependents();  // the next call on the stream may start its own phase 1
-
+  if (a.early_trigger) pdl_launch_dependents();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const FinishArgs& f = a.fin;
   const int V = f.V;
@@ -736,7 +767,7 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
   }
 
   // ================================= phase 2 ===========================================
-  pdl_wait();   // the previous call on the stream has finished with the workspace and the outputs
+  if (a.early_trigger) pdl_wait();   // the previous call has completed: the workspace is free
   __syncwarp();
   for (int idx = lane; idx < n_my; idx += 32) {
     const_cast<float2*>(f.partials)[item_begin + idx] = sm.stash[warp][idx];
@@ -898,8 +929,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   extern __shared__ __align__(128) unsigned char fused_smem_raw[];
   TopkSmem& sm = *reinterpret_cast<TopkSmem*>(fused_smem_raw);
 
-  pdl_launch_dependents();  // the next call on the stream may start its own phase 1
-
+  if (a.early_trigger) pdl_launch_dependents();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const FinishArgs& f = a.fin;
   const int V = f.V;
@@ -1202,7 +1232,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   }
 
   // ================================= phase 2 ===========================================
-  pdl_wait();   // the previous call on the stream has finished with the workspace and the outputs
+  if (a.early_trigger) pdl_wait();   // the previous call has completed: the workspace is free
   __syncthreads();
   for (int idx = tid; idx < n_my; idx += kTopkThreads) {
     const int row_id = row_begin + idx;
