@@ -257,7 +257,7 @@ def run_reference(args) -> None:
 def run_native(args) -> None:
     import torch
     import paper_2601_09212_b200 as csd
-    from paper_2601_09212_b200 import _build, workloads as W
+    from paper_2601_09212_b200 import _build, sharding, workloads as W
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -330,11 +330,7 @@ def run_native(args) -> None:
     sampler.sample_once()
     barrier()
     sampler.stop()
-    ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = sharding.max_over_ranks(e0.elapsed_time(e1), device=dev)
 
     # accepted lengths of the last lap (a property of the synthetic drafter, reported for context)
     mean_emit = float(np.mean([o["tau"].float().mean().item() + 1.0 for o in outs]))
@@ -368,11 +364,7 @@ def run_native(args) -> None:
         csd.csd_verify_host(hprm[i % host_n], staging[i % host_n])
     f1.record(stream)
     barrier()
-    e2e_ms = f0.elapsed_time(f1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = sharding.max_over_ranks(f0.elapsed_time(f1), device=dev)
     # the host arrays now hold the last step's results; they must equal the device-resident run's
     last = (e2e_steps - 1) % host_n
     same = bool(np.array_equal(hkeep[last]["ot"].numpy(), outs[last]["tok"].cpu().numpy()))
@@ -382,8 +374,7 @@ def run_native(args) -> None:
             dist.destroy_process_group()
         return
 
-    tokens = B * L * args.steps * world
-    value = tokens / (ms * 1e-3)
+    value = sharding.job_throughput(B * L * args.steps, world, ms * 1e-3)
     peak, peak_kind = measured_peak()
     step_s = ms * 1e-3 / args.steps
     achieved = step_bytes / step_s / 1e9

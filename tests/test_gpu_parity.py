@@ -155,6 +155,55 @@ def test_config_c3_guidance_and_topk():
         print("C3", rep.summary())
 
 
+@pytest.mark.parametrize("name,kw", [
+    ("late-trigger plain", dict(B=16, gamma=8, V=16384, dtype=W.F32)),
+    ("early-trigger plain", dict(B=64, gamma=8, V=16384, dtype=W.F32)),
+    ("top-k with guidance", dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000)),
+    ("several sequences per block", dict(B=600, gamma=2, V=2048, dtype=W.BF16)),
+])
+def test_back_to_back_calls_on_one_stream(name, kw):
+    """Consecutive calls overlap on the device (programmatic dependent launch) and share ONE
+    workspace and ONE set of output buffers per slot; every call's results must equal those of
+    the same call run alone, both when enqueued directly and when replayed as a CUDA graph."""
+    L = kw["gamma"]
+    n = 6
+    ws_shared = csd.new_workspace(kw["B"], L, kw["V"], kw["dtype"], DEV)
+    steps = [W.make("t", rho=0.9, schedule=sched(L), seed=100 + i, device=DEV, **kw) for i in range(n)]
+    alone = [run_gpu(w, want_dbg=False) for w in steps]
+    outs = [dict(tok=torch.full((w.B, L + 1), -7, dtype=torch.int32, device=DEV),
+                 tau=torch.full((w.B,), -7, dtype=torch.int32, device=DEV),
+                 st=torch.full((w.B,), -7, dtype=torch.int32, device=DEV)) for w in steps]
+    stream = torch.cuda.Stream()
+    prms = [csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
+                            o["tok"], o["tau"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
+                            cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=o["st"], workspace=ws_shared,
+                            stream=stream) for w, o in zip(steps, outs)]
+
+    def check_all(tag):
+        for i, (o, ref) in enumerate(zip(outs, alone)):
+            assert np.array_equal(o["tok"].cpu().numpy(), ref["tokens"]), (tag, name, i)
+            assert np.array_equal(o["tau"].cpu().numpy(), ref["accept_len"]), (tag, name, i)
+            assert np.array_equal(o["st"].cpu().numpy(), ref["status"]), (tag, name, i)
+            o["tok"].fill_(-7); o["tau"].fill_(-7); o["st"].fill_(-7)
+
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            for p in prms:
+                csd.csd_verify_ex(p)
+    stream.synchronize()
+    check_all("direct")
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        for p in prms:
+            csd.csd_verify_ex(p)
+    with torch.cuda.stream(stream):
+        for _ in range(5):
+            g.replay()
+    stream.synchronize()
+    check_all("graph")
+
+
 def test_batch_strides_and_unaligned_views():
     """Rows embedded in a larger buffer (batch stride > rows*V) and a base pointer that is
     only element-aligned (forces the scalar path)."""
