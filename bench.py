@@ -41,8 +41,9 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
-# one ncu capture, see profiles/).  Valid only for the kernel sources with this digest.
-NCU_TRAFFIC = {"sources_sha256": None, "workload": None, "bytes_per_launch": None}
+# one ncu capture, see profiles/verify_topk_kernel_C3.md).  Reported only while the kernel sources
+# still have the digest the capture was taken with; null otherwise.
+NCU_TRAFFIC = {"sources_sha256": "45b5c0f7d3192803", "workload": "C3", "bytes_per_launch": 68209664}
 
 
 def sources_digest() -> str:
@@ -399,7 +400,9 @@ def run_native(args) -> None:
                      "traffic": traffic, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                      "bytes_per_launch": step_bytes,
                      "duration_us": step_s * 1e6,
-                     "note": "duration = timed region / steps: all kernels of a step, an upper bound on the row-statistics kernel"},
+                     "kernel": "the single fused launch of a step" if kernels_per_step == 1 else "all launches of a step",
+                     "note": "duration = timed region / launches, CUDA events on the launching stream; calls overlap, so "
+                             "this is the sustained time per launch"},
         "emitted_tokens_per_step_mean": B * mean_emit,
     }
     if world == 1 and not args.no_cpu_baseline:
