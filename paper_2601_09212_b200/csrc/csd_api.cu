@@ -51,24 +51,24 @@ bool shape_ok(int B, int gamma, int V) {
 }
 
 // Workspace: [header: error flag][counters: B int][partials: rows * max_parts float2][thresholds: rows float]
-//            [token logits: rows float]
+//            [records: B * 32 SeqRecord (single-launch path)]
 // The header and the counters must be zero before the first call; every call leaves them zero.
 struct Layout {
-  size_t rows, max_parts, header_off, counters_off, partials_off, thresholds_off, tok_logit_off, zero_bytes, total;
+  size_t rows, max_parts, header_off, counters_off, partials_off, thresholds_off, records_off, zero_bytes, total;
 };
 Layout layout_for(int B, int gamma, int V, int dtype) {
   Layout l;
   l.rows = (size_t)B * (size_t)(2 * gamma + 1);
-  // finest split any path uses: one warp stage of the plain kernel with guidance (fp32: 256 elements)
-  const size_t min_part = (size_t)kWStageBytes / (2 * (size_t)elem_size(dtype));
+  // parts of the multi-launch path (the single-launch path keeps its partials in shared memory)
+  const size_t min_part = (size_t)kStatsThreads * vec_width(dtype);  // U = 1
   l.max_parts = ((size_t)V + min_part - 1) / min_part;
   l.header_off = 0;
   l.counters_off = kAlign;
   l.partials_off = l.counters_off + align_up((size_t)B * sizeof(int));
   l.zero_bytes = l.partials_off;
   l.thresholds_off = l.partials_off + align_up(l.rows * l.max_parts * sizeof(float2));
-  l.tok_logit_off = l.thresholds_off + align_up(l.rows * sizeof(float));
-  l.total = l.tok_logit_off + align_up(l.rows * sizeof(float));
+  l.records_off = l.thresholds_off + align_up(l.rows * sizeof(float));
+  l.total = l.records_off + align_up((size_t)B * kMaxGamma * sizeof(SeqRecord));
   return l;
 }
 
@@ -282,64 +282,47 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
     ua.fin = fa;
     ua.top_k = p.top_k;
     ua.lo_sigmas = nanf("");
-    ua.tok_logit = reinterpret_cast<float*>((char*)p.workspace + lay.tok_logit_off);
+    ua.records = reinterpret_cast<SeqRecord*>((char*)p.workspace + lay.records_off);
     ua.counters = reinterpret_cast<int*>((char*)p.workspace + lay.counters_off);
     ua.error_flag = reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
-    // Blocks are aligned with sequences: either a sequence's items are split over ctas_per_seq
-    // blocks, or a block owns seqs_per_cta whole sequences.
+    // Blocks are aligned with sequences and positions: either a sequence's draft positions are split
+    // over ctas_per_seq blocks (each with both rows of its positions), or a block owns seqs_per_cta
+    // whole sequences.
     const long long target_blocks = 2LL * sms;
-    long long c = 1, spc = 1, grid;
-    if (p.B >= target_blocks) {
-      spc = (p.B + target_blocks - 1) / target_blocks;
-      grid = (p.B + spc - 1) / spc;
-    } else {
-      c = target_blocks / p.B;
-      grid = 0;   // set below
-    }
+    long long c = 1, spc = 1;
+    if (p.B >= target_blocks) spc = (p.B + target_blocks - 1) / target_blocks;
+    else c = target_blocks / p.B;
+    if (c > p.gamma) c = p.gamma;
+    if (c < 1) c = 1;
+    while (spc > 1 && spc * rows_per_seq > kBlockRows) --spc;   // rows_per_seq <= 65 < kBlockRows
     if (topk) {
-      // one block-wide item per row, streamed in stages
       ua.chunks_per_part = 0;
       ua.parts_per_row = 1;
-      ua.fin.parts = 1;
-      ua.items_per_seq = rows_per_seq;
       const double k = p.top_k, v = p.V;
       const double tail = 1.25 * k / v + 4.0 * sqrt(k) / v + 16.0 / v;
       if (tail < 0.45 && tail * v < 0.8 * kListCap) ua.lo_sigmas = (float)normal_upper_quantile(tail);
-      if (c > rows_per_seq) c = rows_per_seq;
-      // a block keeps one stash entry per row
-      while (spc * rows_per_seq > kTkStash) --spc;   // rows_per_seq <= 65 < kTkStash: spc stays >= 1
     } else {
       // warp-wide items: parts of rows, sized so that every warp of the grid gets several
       const int eps = kWStageBytes / (es * (cfg ? 2 : 1));
       const long long cpr = (p.V + eps - 1) / eps;
-      const long long warps = (c > 1 ? (long long)p.B * c : (p.B + spc - 1) / spc) * kPlainWarps;
-      long long cpp = rows * cpr / (4 * warps);
+      const long long blocks = c > 1 ? (long long)p.B * c : (p.B + spc - 1) / spc;
+      long long cpp = rows * cpr / (4 * blocks * kPlainWarps);
       if (cpp < 1) cpp = 1;
       if (cpp > 8) cpp = 8;
-      // the finish stages a sequence's partials in the ring: 8 bytes each
-      const long long max_parts = (kPlainRingBytes / (long long)sizeof(float2)) / rows_per_seq;
-      const long long min_cpp = (cpr + max_parts - 1) / max_parts;
-      if (cpp < min_cpp) cpp = min_cpp;
       if (cpp > cpr) cpp = cpr;
-      // a warp keeps one stash entry per item
+      // a block keeps one stash entry per item
       for (;;) {
         const long long parts = (cpr + cpp - 1) / cpp;
-        const long long per_block = (c > 1) ? (rows_per_seq * parts + c - 1) / c : spc * rows_per_seq * parts;
-        if ((per_block + kPlainWarps - 1) / kPlainWarps + 1 <= kWarpStash) break;
+        const long long rows_block = (c > 1) ? (2LL * ((p.gamma + c - 1) / c) + 1) : spc * rows_per_seq;
+        if (rows_block * parts <= kBlockStash) break;
         if (cpp < cpr) cpp = (cpp * 2 < cpr) ? cpp * 2 : cpr;
         else if (spc > 1) --spc;
-        else break;   // one sequence per block, one part per row: at most 65 items per block
+        else break;   // one sequence per block, one part per row: at most 65 items
       }
       ua.chunks_per_part = (int)cpp;
       ua.parts_per_row = (int)((cpr + cpp - 1) / cpp);
-      ua.fin.parts = ua.parts_per_row;
-      ua.items_per_seq = rows_per_seq * ua.parts_per_row;
-      if (c > ua.items_per_seq) c = ua.items_per_seq;
     }
-    if (c > 1) grid = (long long)p.B * c;
-    else grid = (p.B + spc - 1) / spc;
-    // calls that move less than about 40 MB stream too briefly for their phase 1 to be worth overlapping
-    ua.early_trigger = ((double)rows * p.V * es * (cfg ? 2 : 1) >= 40e6) ? 1 : 0;
+    const long long grid = c > 1 ? (long long)p.B * c : (p.B + spc - 1) / spc;
     ua.ctas_per_seq = (int)c;
     ua.seqs_per_cta = (int)spc;
     cudaError_t fe;

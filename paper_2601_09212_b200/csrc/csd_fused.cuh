@@ -2,25 +2,21 @@
 //
 // Phase 1 streams this block's share of the logit rows through rings of
 // shared-memory stages filled by bulk asynchronous copies (mbarrier completion)
-// and keeps the per-item results in shared memory.  Phase 2 publishes them to the
-// workspace, counts arrivals per sequence, and the block that completes a
-// sequence runs its finish: accept tests, tau, Eq. opt_G at position tau+1 with
-// the two rows brought back through the ring, inverse-CDF draw, emit.  No block
-// ever waits for another block; every wait on a copy is bounded.
+// and keeps the per-row results in shared memory.  Phase 2 is the block's own
+// finish.  A block owns, for its sequence(s), a range of draft positions with both
+// rows of each, so it runs the accept tests of its positions itself and, at its first
+// rejection, draws the replacement token at once (Eq. opt_G with the two rows brought
+// back through the ring, inverse CDF) -- speculatively, since an earlier position of
+// another block may reject first.  Each block leaves a small record; the last block
+// of a sequence to arrive picks the first rejecting block's record and emits.  No
+// block ever waits for another block; every wait on a copy is bounded.
 //
-// Consecutive calls on a stream overlap (programmatic dependent launch) in one of
-// two ways, chosen by the host from the size of the call:
-//   early trigger (large calls): every block signals launch_dependents at once, so
-//     the next call's phase 1 streams alongside this call; a block then calls
-//     griddepcontrol.wait before phase 2, i.e. it publishes only when the previous
-//     call has completed and the workspace is free.
-//   late trigger (small calls, whose streaming is short anyway): a block signals
-//     launch_dependents when it has no further use for the workspace -- after its
-//     arrival, or for a finishing block after it has copied what it needs into
-//     shared memory -- so the next call starts, streams and publishes while this
-//     call's finishes still compute; a finishing block calls griddepcontrol.wait
-//     before it writes outputs, which keeps the outputs of consecutive calls in order
-//     and makes this call complete only after the previous one.
+// Consecutive calls on a stream overlap (programmatic dependent launch): every block
+// signals launch_dependents at once, and everything up to a block's first global write
+// -- streaming, accept tests, the draw -- reads only the call's inputs, so it runs beside
+// the previous call; griddepcontrol.wait comes just before that first write (the record,
+// or the outputs), which keeps the workspace and the outputs of consecutive calls in
+// order.  What is serialised between two calls is a 64-byte record, one atomic and the emit.
 //
 //   verify_plain_kernel  every warp streams its own parts of rows through its own
 //                        ring and keeps a running (m, s) per lane.
@@ -120,407 +116,505 @@ __device__ __forceinline__ float load_scalar_smem<__nv_bfloat16>(const unsigned 
   return __uint_as_float(((uint32_t) * reinterpret_cast<const unsigned short*>(p)) << 16);
 }
 
+// What a block reports about its positions of a sequence (workspace, one per block of the sequence).
+struct alignas(16) SeqRecord {
+  int first_rej;   // 0-based position of this block's first rejection, -1 if it accepted all of its positions
+  int token;       // token drawn at first_rej; for the block that owns the bonus row and accepted everything,
+                   // the bonus token; -1 if there was nothing to draw from
+  int status_at;   // status bits of that draw (bad row, bad token, Z fallback; for the bonus draw: bad row)
+  int status_any;  // status bits that hold whatever the other blocks say (a bounded wait gave up)
+  int mode;        // diagnostics: how the token was drawn (0: Eq. opt_G, 1: from P), and the statistics used
+  float Mt, St, Md, Sd, thr_t, thr_d, one_minus_omega;
+  double Z;
+  int pad[2];
+};
+static_assert(sizeof(SeqRecord) == 64, "records are copied as four 16-byte words");
+
 struct FusedArgs {
-  FinishArgs fin;       // inputs, outputs, partials [rows][fin.parts], thresholds [rows]
+  FinishArgs fin;       // inputs and outputs (the workspace arrays of the multi-launch path are unused)
   int chunks_per_part;  // plain kernel: warp stages per part
   int parts_per_row;    // plain kernel
-  int items_per_seq;    // plain: rows per sequence * parts_per_row; top-k: rows per sequence
-  int ctas_per_seq;     // > 1: a sequence's items are split over this many blocks (its last block to
-                        //      arrive runs the finish); 1: a block owns seqs_per_cta whole sequences
+  int ctas_per_seq;     // > 1: a sequence's positions are split over this many blocks (the last to
+                        //      arrive resolves the sequence); 1: a block owns seqs_per_cta whole sequences
   int seqs_per_cta;
   int top_k;
   float lo_sigmas;      // top-k guess: lo = mean + lo_sigmas * deviation (NaN: always select exactly)
-  float* tok_logit;     // [rows] (mixed, unfiltered) logit of the row's drafted token, written in phase 2
+  SeqRecord* records;   // [B][kMaxGamma], written and read only with ctas_per_seq > 1
   int* counters;        // [B] arrivals per sequence; zero before the first call, left zero by every call
   int* error_flag;      // set when a bounded wait gave up
-  int early_trigger;    // how consecutive calls overlap, see the head of this file
 };
 
-// ---- finish with everything staged in shared memory ---------------------------------
-// Few dependent round trips to global memory: one brings the sequence's partials,
-// thresholds, drafted tokens with their logits (found in phase 1 while the rows
-// streamed by), uniforms and multipliers into shared memory; after the accept tests,
-// bulk copies bring the two rows of position tau+1 into the ring, a segment at a
-// time, and Eq. opt_G is summed from there.
+// ---- a block's share of the work ------------------------------------------------------
+// Blocks are aligned with sequences AND with positions: a block owns, for each of its
+// sequences, a range of draft positions and BOTH rows (target, drafter) of each, so that it can
+// run the accept tests of its positions by itself and, where one of them rejects, draw the
+// replacement token right away -- speculatively, since an earlier position owned by another block
+// may have rejected first.  Local rows are ordered t_p0, d_p0, t_p0+1, d_p0+1, ..., [bonus row].
+struct BlockShare {
+  int seq_begin, seq_end;   // sequences this block works on
+  int pos_begin, pos_end;   // draft positions (0-based) it owns of each
+  int bonus;                // it also owns the bonus row (target row gamma)
+  int rows_per_seq;         // local rows per sequence
+  int n_rows;               // local rows in all
+  int slot;                 // its record slot within the sequence (ctas_per_seq > 1)
+};
+__device__ __forceinline__ BlockShare block_share(const FusedArgs& a) {
+  BlockShare sh;
+  const int L = a.fin.gamma;
+  const bool has_bonus_row = a.fin.T == L + 1;
+  if (a.ctas_per_seq > 1) {
+    const int b = blockIdx.x / a.ctas_per_seq;
+    const int j = blockIdx.x - b * a.ctas_per_seq;
+    sh.seq_begin = b;
+    sh.seq_end = b + 1;
+    sh.pos_begin = L * j / a.ctas_per_seq;
+    sh.pos_end = L * (j + 1) / a.ctas_per_seq;
+    sh.bonus = (has_bonus_row && j == a.ctas_per_seq - 1) ? 1 : 0;
+    sh.slot = j;
+  } else {
+    sh.seq_begin = min(a.fin.B, (int)blockIdx.x * a.seqs_per_cta);
+    sh.seq_end = min(a.fin.B, sh.seq_begin + a.seqs_per_cta);
+    sh.pos_begin = 0;
+    sh.pos_end = L;
+    sh.bonus = has_bonus_row ? 1 : 0;
+    sh.slot = 0;
+  }
+  sh.rows_per_seq = 2 * (sh.pos_end - sh.pos_begin) + sh.bonus;
+  sh.n_rows = (sh.seq_end - sh.seq_begin) * sh.rows_per_seq;
+  return sh;
+}
+// local row -> (sequence, 0 target / 1 drafter, position)
+__device__ __forceinline__ void local_row(const BlockShare& sh, int r_loc, int gamma, int& b, int& which, int& i) {
+  const int sl = r_loc / sh.rows_per_seq;
+  const int r = r_loc - sl * sh.rows_per_seq;
+  b = sh.seq_begin + sl;
+  if (r < 2 * (sh.pos_end - sh.pos_begin)) { i = sh.pos_begin + (r >> 1); which = r & 1; }
+  else { i = gamma; which = 0; }
+}
+template <typename T, bool CFG>
+__device__ __forceinline__ Row<T, CFG> row_at(const FinishArgs& f, int b, int which, int i) {
+  Row<T, CFG> row;
+  row.scale = f.cfg_scale;
+  row.thr = CSD_NEG_INF;
+  if (which == 0) {
+    const int64_t off = (int64_t)b * f.tstride + (int64_t)i * f.V;
+    row.cond = reinterpret_cast<const T*>(f.target) + off;
+    row.uncond = CFG ? reinterpret_cast<const T*>(f.target_uncond) + off : nullptr;
+  } else {
+    const int64_t off = (int64_t)b * f.dstride + (int64_t)i * f.V;
+    row.cond = reinterpret_cast<const T*>(f.draft) + off;
+    row.uncond = CFG ? reinterpret_cast<const T*>(f.draft_uncond) + off : nullptr;
+  }
+  return row;
+}
+constexpr int kBlockRows = 264;   // local rows a block may own (the host keeps it within this)
+
+// Per-row results of phase 1, in shared memory until the block's own finish consumes them.
+struct RowStats {
+  float2 ms[kBlockRows];     // (m, s) of the whole row
+  float thr[kBlockRows];     // top-k threshold (-inf without top-k)
+  float tokz[kBlockRows];    // logit of the row's drafted token (undefined if the token is out of range)
+};
+
+// ---- the block's finish on its own positions ----------------------------------------------
 struct FinishStage {
   int tok[kMaxGamma + 1];
   float uni[kMaxGamma + 1];
   float omega[kMaxGamma];
-  float tokz[2 * kMaxGamma + 1];
-  float thr_row[2 * kMaxGamma + 1];
+  float tokz[2][kMaxGamma + 1];
+  float p[kMaxGamma], q[kMaxGamma], f[kMaxGamma];
+  SeqRecord rec;
   alignas(8) uint64_t bar;
 };
 
-// both (m, s) pairs reduced over the warp in one interleaved loop
-__device__ __forceinline__ void stat_warp_allreduce2(float& m0, float& s0, float& m1, float& s1) {
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    const float a0 = __shfl_xor_sync(0xffffffffu, m0, off);
-    const float b0 = __shfl_xor_sync(0xffffffffu, s0, off);
-    const float a1 = __shfl_xor_sync(0xffffffffu, m1, off);
-    const float b1 = __shfl_xor_sync(0xffffffffu, s1, off);
-    stat_merge(m0, s0, a0, b0);
-    stat_merge(m1, s1, a1, b1);
-  }
-}
-
-// ring: `ring_bytes` of shared memory (multiple of 4 KB) that nothing else uses meanwhile;
-// tile_sums: kFinTiles doubles, likewise.
+// Eq. opt_G summed per tile over the whole row pair, rows brought through the ring by bulk copies;
+// then the tile of the crossing and the token inside it.  Returns the token (-1: nothing to draw
+// from); Z_out gets the normaliser, status gets bits 4 / 8 where they apply; ctx.mode may change to 1.
 template <typename T, bool CFG, int NT>
-__device__ void finish_sequence_staged(const FusedArgs& ua, const int b, const int tid, unsigned char* ring,
-                                       const int ring_bytes, double* tile_sums, FinishSmem& sm, FinishStage& st,
-                                       uint32_t& phase, const int extra_status, const bool last_use_of_workspace) {
+__device__ int draw_token(const FinishArgs& a, const Row<T, CFG>& rt, const Row<T, CFG>& rd, PairCtx& ctx, const float u,
+                          const int tid, unsigned char* ring, const int ring_bytes, double* tile_sums, FinishSmem& sm,
+                          FinishStage& st, uint32_t& phase, int& status, double& Z_out) {
   constexpr int VEC = Elem<T>::kVec;
   constexpr int TILE = 32 * VEC;
   constexpr int ARR = CFG ? 2 : 1;
   constexpr int ES = (int)sizeof(T);
-  const FinishArgs& a = ua.fin;
   const int lane = tid & 31, warp = tid >> 5;
-  const int L = a.gamma, V = a.V;
-  const int rows_per_seq = a.T + L;
-  const T* tgt = reinterpret_cast<const T*>(a.target) + (int64_t)b * a.tstride;
-  const T* dft = reinterpret_cast<const T*>(a.draft) + (int64_t)b * a.dstride;
-  const T* tgt_u = CFG ? reinterpret_cast<const T*>(a.target_uncond) + (int64_t)b * a.tstride : nullptr;
-  const T* dft_u = CFG ? reinterpret_cast<const T*>(a.draft_uncond) + (int64_t)b * a.dstride : nullptr;
-
-  // ---- 0. one round trip: everything the accept tests need ----------------------------
-  const int n_entries = rows_per_seq * a.parts;   // the host keeps this within the ring
-  float2* staged = reinterpret_cast<float2*>(ring);
-  {
-    const float2* src = a.partials + (int64_t)b * n_entries;
-    for (int idx = tid; idx < n_entries; idx += NT) staged[idx] = __ldcg(src + idx);
-    if (tid < L) {
-      st.tok[tid] = a.tokens[(int64_t)b * L + tid];
-      const float om = a.schedule[tid];
-      st.omega[tid] = om >= 0.0f ? om : 0.0f;
-    }
-    if (tid <= L) st.uni[tid] = a.uniforms[(int64_t)b * (L + 1) + tid];
-    if (tid < rows_per_seq) {
-      st.thr_row[tid] = a.use_topk ? __ldcg(a.thresholds + (int64_t)b * rows_per_seq + tid) : CSD_NEG_INF;
-      st.tokz[tid] = __ldcg(ua.tok_logit + (int64_t)b * rows_per_seq + tid);
-    }
-  }
-  __syncthreads();
-  // Everything this block needs from the workspace now sits in shared memory.
-  if (last_use_of_workspace && !ua.early_trigger) pdl_launch_dependents();
-  // Outputs are written only once the previous call on the stream has completed; with the
-  // diagnostic outputs that is from here on, otherwise just before the emit.
-  if (a.dbg_p || a.dbg_q || a.dbg_f) pdl_wait();
-
-  // ---- 1. per position: merge parts, Eq. relax, accept test ------------------------------
-  const int n_pos = a.T > L ? L + 1 : L;   // the bonus position only if its row exists
-  if (tid == 0 && n_pos == L) { sm.valid[0][L] = 0; sm.valid[1][L] = 0; sm.flag[L] = 0; }
-  for (int i = warp; i < n_pos; i += NT / 32) {
-    const bool has_d = i < L;   // has_t always holds here
-    float M[2] = {CSD_NEG_INF, CSD_NEG_INF}, S[2] = {-1.0f, -1.0f};
-    for (int p = lane; p < a.parts; p += 32) {
-      const float2 v = staged[i * a.parts + p];
-      stat_merge(M[0], S[0], v.x, v.y);
-      if (has_d) {
-        const float2 w = staged[(a.T + i) * a.parts + p];
-        stat_merge(M[1], S[1], w.x, w.y);
-      }
-    }
-    stat_warp_allreduce2(M[0], S[0], M[1], S[1]);
-    if (lane == 0) {
-      const float thr0 = st.thr_row[i], thr1 = has_d ? st.thr_row[a.T + i] : CSD_NEG_INF;
-      const bool t_ok = M[0] > CSD_NEG_INF && M[0] < CSD_POS_INF && S[0] >= 0.0f && S[0] < CSD_POS_INF;
-      const bool d_ok = has_d && M[1] > CSD_NEG_INF && M[1] < CSD_POS_INF && S[1] >= 0.0f && S[1] < CSD_POS_INF;
-      sm.M[0][i] = M[0]; sm.S[0][i] = S[0]; sm.thr[0][i] = thr0;
-      sm.M[1][i] = M[1]; sm.S[1][i] = S[1]; sm.thr[1][i] = thr1;
-      sm.valid[0][i] = t_ok; sm.valid[1][i] = d_ok;
-      int flag = 0;
-      if (i < L) {
-        const int tok = st.tok[i];
-        const bool tok_ok = tok >= 0 && tok < V;
-        const float omega = st.omega[i];
-        float f = 0.0f, p = __int_as_float(0x7fc00000), q = p;
-        if (!t_ok || !d_ok) flag = 1;
-        else if (!tok_ok) flag = 2;
-        else {
-          const float zt = st.tokz[i], zd = st.tokz[a.T + i];
-          const float dt = (zt < thr0 ? CSD_NEG_INF : zt) - M[0];
-          const float dd = (zd < thr1 ? CSD_NEG_INF : zd) - M[1];
-          p = ex2f(dt * kLog2e) / (1.0f + S[0]);
-          q = ex2f(dd * kLog2e) / (1.0f + S[1]);
-          if (dd == CSD_NEG_INF) f = 1.0f;         // q = 0: p/q = +inf, and 0/0 := 1
-          else if (dt == CSD_NEG_INF) f = 0.0f;    // p = 0 < q
-          else f = fminf(1.0f, omega * ex2f((dt - dd) * kLog2e) * ((1.0f + S[1]) / (1.0f + S[0])));
-        }
-        sm.acc[i] = (st.uni[i] <= f) ? 1 : 0;
-        if (a.dbg_p) a.dbg_p[(int64_t)b * L + i] = p;
-        if (a.dbg_q) a.dbg_q[(int64_t)b * L + i] = q;
-        if (a.dbg_f) a.dbg_f[(int64_t)b * L + i] = f;
-      }
-      sm.flag[i] = flag;
-    }
-  }
-  __syncthreads();
-
-  // ---- 2. tau = number of leading accepts (the for/break of Algorithm 1) --------
-  int tau = 0;
-  while (tau < L && sm.acc[tau]) ++tau;
-  int status = extra_status;
-  for (int i = 0; i <= min(tau, L - 1); ++i) status |= sm.flag[i];
-
-  // ---- 3. which row to draw from -------------------------------------------------
-  const int j = tau;  // 0-based row index of position tau+1 (j == L: bonus row)
-  PairCtx ctx;
-  bool draw = true;
-  if (j < L) {
-    if (!sm.valid[0][j]) draw = false;
-    ctx.mode = sm.valid[1][j] ? 0 : 1;
-  } else {
-    if (a.T == L + 1) {
-      ctx.mode = 1;
-      if (!sm.valid[0][L]) { draw = false; status |= 1; }
-    } else draw = false;
-  }
-  float* G_out = a.dbg_G ? a.dbg_G + (int64_t)b * V : nullptr;
+  const int V = a.V;
   const int ntiles = (V + TILE - 1) / TILE;
   int token = -1;
+  Z_out = 0.0;
+  for (int attempt = 0; attempt < 2; ++attempt) {
+    // ---- Eq. opt_G weights: one fp64 sum per tile ----------------------------------------
+    const int n_arr = (ctx.mode == 0 ? 2 : 1) * ARR;
+    const int seg_elems = (ring_bytes / n_arr / (TILE * ES)) * TILE;   // elements of each array per segment
+    const int slot_bytes = seg_elems * ES;
+    for (int x0 = 0; x0 < V; x0 += seg_elems) {
+      __syncthreads();   // everybody is done with what the ring held
+      const int n = min(seg_elems, V - x0);
+      if (tid == 0) {
+        fence_before_bulk();
+        const uint32_t bytes = (uint32_t)(n * ES);
+        mbar_expect_tx(&st.bar, bytes * n_arr);
+        bulk_load(ring, rt.cond + x0, bytes, &st.bar);
+        if (CFG) bulk_load(ring + slot_bytes, rt.uncond + x0, bytes, &st.bar);
+        if (ctx.mode == 0) {
+          bulk_load(ring + ARR * slot_bytes, rd.cond + x0, bytes, &st.bar);
+          if (CFG) bulk_load(ring + (ARR + 1) * slot_bytes, rd.uncond + x0, bytes, &st.bar);
+        }
+      }
+      if (!mbar_wait(&st.bar, phase)) status |= 8;
+      phase ^= 1u;
+      const int seg_tiles = (n + TILE - 1) / TILE;
+      // two tiles per warp and trip, so that their reductions overlap
+      for (int t0 = warp; t0 < seg_tiles; t0 += 2 * (NT / 32)) {
+        float acc2[2] = {0.0f, 0.0f};
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          const int xo = (t0 + r * (NT / 32)) * TILE + lane * VEC;   // offset inside the segment
+          if (xo < n) {
+            float zt[VEC], zd[VEC];
+            unpack_vec<T>(ring + xo * ES, zt);
+            if (CFG) {
+              float zu[VEC];
+              unpack_vec<T>(ring + slot_bytes + xo * ES, zu);
+#pragma unroll
+              for (int k = 0; k < VEC; ++k) zt[k] = cfg_mix(zt[k], zu[k], a.cfg_scale);
+            }
+            if (ctx.mode == 0) {
+              unpack_vec<T>(ring + ARR * slot_bytes + xo * ES, zd);
+              if (CFG) {
+                float zu[VEC];
+                unpack_vec<T>(ring + (ARR + 1) * slot_bytes + xo * ES, zu);
+#pragma unroll
+                for (int k = 0; k < VEC; ++k) zd[k] = cfg_mix(zd[k], zu[k], a.cfg_scale);
+              }
+            }
+            float acc = 0.0f;
+#pragma unroll
+            for (int k = 0; k < VEC; ++k)
+              acc += weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
+            acc2[r] = acc;
+          }
+        }
+        double d0 = (double)acc2[0], d1 = (double)acc2[1];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+          d0 += __shfl_xor_sync(0xffffffffu, d0, off);
+          d1 += __shfl_xor_sync(0xffffffffu, d1, off);
+        }
+        if (lane == 0) {
+          tile_sums[x0 / TILE + t0] = d0;
+          if (t0 + NT / 32 < seg_tiles) tile_sums[x0 / TILE + t0 + NT / 32] = d1;
+        }
+      }
+    }
+    __syncthreads();
+    // ---- locate the tile that holds the crossing C(x) > u Z ---------------------------------
+    if (warp == 0) {
+      const int chunk = (ntiles + 31) / 32;
+      const int t0 = lane * chunk, t1 = min(ntiles, t0 + chunk);
+      double local = 0.0;
+      for (int t = t0; t < t1; ++t) local += tile_sums[t];
+      const double incl = warp_incl_scan_double(local, lane);
+      const double Z = __shfl_sync(0xffffffffu, incl, 31);
+      const double target = (double)u * Z;
+      const bool mine = incl > target && local > 0.0;
+      const unsigned ballot = __ballot_sync(0xffffffffu, mine);
+      if (lane == 0) { sm.Z = Z; sm.pick_tile = -1; }
+      __syncwarp();
+      if (ballot != 0 && lane == __ffs(ballot) - 1) {
+        double c = incl - local, c_pick = c;
+        int pick = t0;
+        for (int t = t0; t < t1; ++t) {
+          const double v = tile_sums[t];
+          if (v > 0.0) { pick = t; c_pick = c; }   // last tile with mass seen so far
+          if (c + v > target && v > 0.0) break;
+          c += v;
+        }
+        sm.pick_tile = pick;
+        sm.pick_prefix = c_pick;
+      }
+    }
+    __syncthreads();
+    const double Z = sm.Z;
+    if (!(Z > 0.0) || !(Z < (double)CSD_POS_INF)) {
+      if (attempt == 0 && ctx.mode == 0) {  // empty positive part: fall back to G := P_j
+        ctx.mode = 1;
+        status |= 4;
+        continue;
+      }
+      break;  // nothing to draw from
+    }
+    Z_out = Z;
+    // ---- scan inside that tile (its 32 vectors come from global memory again) ------------------
+    if (warp == 0) {
+      const int tile = sm.pick_tile;
+      const double target = (double)u * Z;
+      const int x0 = tile * TILE + lane * VEC;
+      float zt[VEC], zd[VEC];
+      rt.load_tile(x0, V, 1, zt);
+      if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd);
+      double run[VEC];
+      double acc = 0.0;
+      int last_pos = -1;
+      unsigned posmask = 0;
+#pragma unroll
+      for (int k = 0; k < VEC; ++k) {
+        const float g = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
+        if (g > 0.0f) { last_pos = k; posmask |= 1u << k; }
+        acc += (double)g;
+        run[k] = acc;
+      }
+      const double before = sm.pick_prefix + (warp_incl_scan_double(acc, lane) - acc);
+      int first = -1;
+#pragma unroll
+      for (int k = VEC - 1; k >= 0; --k)
+        if (before + run[k] > target && ((posmask >> k) & 1u)) first = k;
+      const unsigned hit = __ballot_sync(0xffffffffu, first >= 0);
+      const unsigned pos = __ballot_sync(0xffffffffu, last_pos >= 0);
+      if (hit != 0) {
+        if (lane == __ffs(hit) - 1) sm.token = x0 + first;
+      } else if (pos != 0) {  // rounding left no crossing: last token with positive weight
+        if (lane == 31 - __clz(pos)) sm.token = x0 + last_pos;
+      } else if (lane == 0) sm.token = -1;
+    }
+    __syncthreads();
+    token = sm.token;
+    break;
+  }
+  return token;
+}
 
+// Writes the distribution a token was drawn from (diagnostic output), or zeros.
+template <typename T, bool CFG, int NT>
+__device__ void write_G(const FinishArgs& a, const int b, const int j, const SeqRecord& rec, const int tid) {
+  constexpr int VEC = Elem<T>::kVec;
+  constexpr int TILE = 32 * VEC;
+  const int lane = tid & 31, warp = tid >> 5;
+  const int V = a.V;
+  float* G_out = a.dbg_G + (int64_t)b * V;
+  if (rec.token < 0 || !(rec.Z > 0.0)) {
+    for (int x = tid; x < V; x += NT) G_out[x] = 0.0f;
+    return;
+  }
+  PairCtx ctx;
+  ctx.Mt = rec.Mt; ctx.St = rec.St; ctx.Md = rec.Md; ctx.Sd = rec.Sd;
+  ctx.inv_t = 1.0f / (1.0f + ctx.St);
+  ctx.inv_den = ctx.inv_t / (1.0f + ctx.Sd);
+  ctx.one_minus_omega = rec.one_minus_omega;
+  ctx.mode = rec.mode;
+  Row<T, CFG> rt = row_at<T, CFG>(a, b, 0, j);
+  rt.thr = rec.thr_t;
+  Row<T, CFG> rd = rt;
+  if (j < a.gamma) { rd = row_at<T, CFG>(a, b, 1, j); rd.thr = rec.thr_d; }
+  const float invZ = (float)(1.0 / rec.Z);
+  const int ntiles = (V + TILE - 1) / TILE;
+  for (int tile = warp; tile < ntiles; tile += NT / 32) {
+    const int x0 = tile * TILE + lane * VEC;
+    float zt[VEC], zd[VEC];
+    rt.load_tile(x0, V, 1, zt);
+    if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd);
+#pragma unroll
+    for (int k = 0; k < VEC; ++k)
+      if (x0 + k < V)
+        G_out[x0 + k] = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx) * invZ;
+  }
+}
+
+// The block's positions [pos_begin, pos_end) of sequence b: accept tests (Eq. relax), its first
+// rejection, and the draw there (Eq. opt_G) -- or the bonus draw if it owns the bonus row and accepted
+// everything.  Row statistics come from shared memory (rs, local rows of sequence slot sl).  Leaves
+// the record in st.rec and p, q, f of its positions in st; reads only the call's inputs.
+template <typename T, bool CFG, int NT>
+__device__ void finish_positions(const FusedArgs& ua, const BlockShare& sh, const int sl, const RowStats& rs,
+                                 const int tid, unsigned char* ring, const int ring_bytes, double* tile_sums,
+                                 FinishSmem& sm, FinishStage& st, uint32_t& phase, const int extra_status) {
+  const FinishArgs& a = ua.fin;
+  const int L = a.gamma, V = a.V;
+  const int b = sh.seq_begin + sl;
+  const int p0 = sh.pos_begin, p1 = sh.pos_end;
+  // ---- 0. inputs of these positions and the row statistics, into shared memory -------------------
+  if (tid >= p0 && tid < p1) {
+    st.tok[tid] = a.tokens[(int64_t)b * L + tid];
+    const float om = a.schedule[tid];
+    st.omega[tid] = om >= 0.0f ? om : 0.0f;
+    st.uni[tid] = a.uniforms[(int64_t)b * (L + 1) + tid];
+  }
+  if (tid == L) st.uni[L] = a.uniforms[(int64_t)b * (L + 1) + L];
+  if (tid < sh.rows_per_seq) {
+    int bb, which, i;
+    local_row(sh, sl * sh.rows_per_seq + tid, L, bb, which, i);
+    const int r_loc = sl * sh.rows_per_seq + tid;
+    sm.M[which][i] = rs.ms[r_loc].x;
+    sm.S[which][i] = rs.ms[r_loc].y;
+    sm.thr[which][i] = a.use_topk ? rs.thr[r_loc] : CSD_NEG_INF;
+    st.tokz[which][i] = rs.tokz[r_loc];
+  }
+  __syncthreads();
+  // ---- 1. Eq. relax and the accept test of every owned position ----------------------------------
+  if (tid >= p0 && tid < p1) {
+    const int i = tid;
+    const float M0 = sm.M[0][i], S0 = sm.S[0][i], M1 = sm.M[1][i], S1 = sm.S[1][i];
+    const float thr0 = sm.thr[0][i], thr1 = sm.thr[1][i];
+    const bool t_ok = M0 > CSD_NEG_INF && M0 < CSD_POS_INF && S0 >= 0.0f && S0 < CSD_POS_INF;
+    const bool d_ok = M1 > CSD_NEG_INF && M1 < CSD_POS_INF && S1 >= 0.0f && S1 < CSD_POS_INF;
+    sm.valid[0][i] = t_ok; sm.valid[1][i] = d_ok;
+    const int tok = st.tok[i];
+    const bool tok_ok = tok >= 0 && tok < V;
+    int flag = 0;
+    float f = 0.0f, p = __int_as_float(0x7fc00000), q = p;
+    if (!t_ok || !d_ok) flag = 1;
+    else if (!tok_ok) flag = 2;
+    else {
+      const float zt = st.tokz[0][i], zd = st.tokz[1][i];
+      const float dt = (zt < thr0 ? CSD_NEG_INF : zt) - M0;
+      const float dd = (zd < thr1 ? CSD_NEG_INF : zd) - M1;
+      p = ex2f(dt * kLog2e) / (1.0f + S0);
+      q = ex2f(dd * kLog2e) / (1.0f + S1);
+      if (dd == CSD_NEG_INF) f = 1.0f;         // q = 0: p/q = +inf, and 0/0 := 1
+      else if (dt == CSD_NEG_INF) f = 0.0f;    // p = 0 < q
+      else f = fminf(1.0f, st.omega[i] * ex2f((dt - dd) * kLog2e) * ((1.0f + S1) / (1.0f + S0)));
+    }
+    sm.acc[i] = (st.uni[i] <= f) ? 1 : 0;
+    sm.flag[i] = flag;
+    st.p[i] = p; st.q[i] = q; st.f[i] = f;
+  }
+  if (tid == L && sh.bonus) {
+    const float M0 = sm.M[0][L], S0 = sm.S[0][L];
+    sm.valid[0][L] = M0 > CSD_NEG_INF && M0 < CSD_POS_INF && S0 >= 0.0f && S0 < CSD_POS_INF;
+  }
+  __syncthreads();
+  // ---- 2. this block's first rejection (the for/break of Algorithm 1, on its positions) ----------
+  int j = p0;
+  while (j < p1 && sm.acc[j]) ++j;
+  const bool rejected = j < p1;
+  int status = extra_status & ~8;
+  PairCtx ctx;
+  bool draw = false;
+  if (rejected) {
+    status |= sm.flag[j];
+    draw = sm.valid[0][j] != 0;
+    ctx.mode = sm.valid[1][j] ? 0 : 1;
+  } else if (sh.bonus) {
+    j = L;
+    ctx.mode = 1;
+    draw = sm.valid[0][L] != 0;
+    if (!draw) status |= 1;
+  }
+  int token = -1;
+  double Z = 0.0;
+  Row<T, CFG> rt = row_at<T, CFG>(a, b, 0, min(j, a.T - 1));
+  Row<T, CFG> rd = rt;
   if (draw) {
     ctx.Mt = sm.M[0][j]; ctx.St = sm.S[0][j];
     ctx.Md = j < L ? sm.M[1][j] : 0.0f; ctx.Sd = j < L ? sm.S[1][j] : 0.0f;
     ctx.inv_t = 1.0f / (1.0f + ctx.St);
     ctx.inv_den = ctx.inv_t / (1.0f + ctx.Sd);
     ctx.one_minus_omega = 1.0f - (j < L ? st.omega[j] : 0.0f);
-    Row<T, CFG> rt{tgt + (int64_t)j * V, CFG ? tgt_u + (int64_t)j * V : nullptr, a.cfg_scale, sm.thr[0][j]};
-    Row<T, CFG> rd = rt;
-    if (j < L) rd = Row<T, CFG>{dft + (int64_t)j * V, CFG ? dft_u + (int64_t)j * V : nullptr, a.cfg_scale, sm.thr[1][j]};
-    const float u = st.uni[L];
-
-    for (int attempt = 0; attempt < 2; ++attempt) {
-      // ---- 4. Eq. opt_G weights: the rows come through the ring, one fp64 sum per tile ------
-      const int n_arr = (ctx.mode == 0 ? 2 : 1) * ARR;
-      const int seg_elems = (ring_bytes / n_arr / (TILE * ES)) * TILE;   // elements of each array per segment
-      const int slot_bytes = seg_elems * ES;
-      for (int x0 = 0; x0 < V; x0 += seg_elems) {
-        __syncthreads();   // everybody is done with what the ring held
-        const int n = min(seg_elems, V - x0);
-        if (tid == 0) {
-          fence_before_bulk();
-          const uint32_t bytes = (uint32_t)(n * ES);
-          mbar_expect_tx(&st.bar, bytes * n_arr);
-          bulk_load(ring, rt.cond + x0, bytes, &st.bar);
-          if (CFG) bulk_load(ring + slot_bytes, rt.uncond + x0, bytes, &st.bar);
-          if (ctx.mode == 0) {
-            bulk_load(ring + ARR * slot_bytes, rd.cond + x0, bytes, &st.bar);
-            if (CFG) bulk_load(ring + (ARR + 1) * slot_bytes, rd.uncond + x0, bytes, &st.bar);
-          }
-        }
-        if (!mbar_wait(&st.bar, phase)) status |= 8;
-        phase ^= 1u;
-        const int seg_tiles = (n + TILE - 1) / TILE;
-        // two tiles per warp and trip, so that their reductions overlap
-        for (int t0 = warp; t0 < seg_tiles; t0 += 2 * (NT / 32)) {
-          float acc2[2] = {0.0f, 0.0f};
-#pragma unroll
-          for (int r = 0; r < 2; ++r) {
-            const int xo = (t0 + r * (NT / 32)) * TILE + lane * VEC;   // offset inside the segment
-            if (xo < n) {
-              float zt[VEC], zd[VEC];
-              unpack_vec<T>(ring + xo * ES, zt);
-              if (CFG) {
-                float zu[VEC];
-                unpack_vec<T>(ring + slot_bytes + xo * ES, zu);
-#pragma unroll
-                for (int k = 0; k < VEC; ++k) zt[k] = cfg_mix(zt[k], zu[k], a.cfg_scale);
-              }
-              if (ctx.mode == 0) {
-                unpack_vec<T>(ring + ARR * slot_bytes + xo * ES, zd);
-                if (CFG) {
-                  float zu[VEC];
-                  unpack_vec<T>(ring + (ARR + 1) * slot_bytes + xo * ES, zu);
-#pragma unroll
-                  for (int k = 0; k < VEC; ++k) zd[k] = cfg_mix(zd[k], zu[k], a.cfg_scale);
-                }
-              }
-              float acc = 0.0f;
-#pragma unroll
-              for (int k = 0; k < VEC; ++k)
-                acc += weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
-              acc2[r] = acc;
-            }
-          }
-          double d0 = (double)acc2[0], d1 = (double)acc2[1];
-#pragma unroll
-          for (int off = 16; off > 0; off >>= 1) {
-            d0 += __shfl_xor_sync(0xffffffffu, d0, off);
-            d1 += __shfl_xor_sync(0xffffffffu, d1, off);
-          }
-          if (lane == 0) {
-            tile_sums[x0 / TILE + t0] = d0;
-            if (t0 + NT / 32 < seg_tiles) tile_sums[x0 / TILE + t0 + NT / 32] = d1;
-          }
-        }
-      }
-      __syncthreads();
-      // ---- 5. locate the tile that holds the crossing C(x) > u Z ------------------
-      if (warp == 0) {
-        const int chunk = (ntiles + 31) / 32;
-        const int t0 = lane * chunk, t1 = min(ntiles, t0 + chunk);
-        double local = 0.0;
-        for (int t = t0; t < t1; ++t) local += tile_sums[t];
-        const double incl = warp_incl_scan_double(local, lane);
-        const double Z = __shfl_sync(0xffffffffu, incl, 31);
-        const double target = (double)u * Z;
-        const bool mine = incl > target && local > 0.0;
-        const unsigned ballot = __ballot_sync(0xffffffffu, mine);
-        if (lane == 0) { sm.Z = Z; sm.pick_tile = -1; }
-        __syncwarp();
-        if (ballot != 0 && lane == __ffs(ballot) - 1) {
-          double c = incl - local, c_pick = c;
-          int pick = t0;
-          for (int t = t0; t < t1; ++t) {
-            const double v = tile_sums[t];
-            if (v > 0.0) { pick = t; c_pick = c; }   // last tile with mass seen so far
-            if (c + v > target && v > 0.0) break;
-            c += v;
-          }
-          sm.pick_tile = pick;
-          sm.pick_prefix = c_pick;
-        }
-      }
-      __syncthreads();
-      const double Z = sm.Z;
-      if (!(Z > 0.0) || !(Z < (double)CSD_POS_INF)) {
-        if (attempt == 0 && ctx.mode == 0) {  // empty positive part: fall back to G := P_j
-          ctx.mode = 1;
-          status |= 4;
-          continue;
-        }
-        break;  // nothing to draw from
-      }
-      // ---- 6. scan inside that tile (its 32 vectors come from global memory again) -----------
-      if (warp == 0) {
-        const int tile = sm.pick_tile;
-        const double target = (double)u * Z;
-        const int x0 = tile * TILE + lane * VEC;
-        float zt[VEC], zd[VEC];
-        rt.load_tile(x0, V, 1, zt);
-        if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd);
-        double run[VEC];
-        double acc = 0.0;
-        int last_pos = -1;
-        unsigned posmask = 0;
-#pragma unroll
-        for (int k = 0; k < VEC; ++k) {
-          const float g = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
-          if (g > 0.0f) { last_pos = k; posmask |= 1u << k; }
-          acc += (double)g;
-          run[k] = acc;
-        }
-        const double before = sm.pick_prefix + (warp_incl_scan_double(acc, lane) - acc);
-        int first = -1;
-#pragma unroll
-        for (int k = VEC - 1; k >= 0; --k)
-          if (before + run[k] > target && ((posmask >> k) & 1u)) first = k;
-        const unsigned hit = __ballot_sync(0xffffffffu, first >= 0);
-        const unsigned pos = __ballot_sync(0xffffffffu, last_pos >= 0);
-        if (hit != 0) {
-          if (lane == __ffs(hit) - 1) sm.token = x0 + first;
-        } else if (pos != 0) {  // rounding left no crossing: last token with positive weight
-          if (lane == 31 - __clz(pos)) sm.token = x0 + last_pos;
-        } else if (lane == 0) sm.token = -1;
-      }
-      __syncthreads();
-      token = sm.token;
-      // ---- 7. optional: write the distribution drawn from ------------------------------
-      if (G_out) {
-        pdl_wait();
-        const float invZ = (float)(1.0 / Z);
-        for (int tile = warp; tile < ntiles; tile += NT / 32) {
-          const int x0 = tile * TILE + lane * VEC;
-          float zt[VEC], zd[VEC];
-          rt.load_tile(x0, V, 1, zt);
-          if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd);
-#pragma unroll
-          for (int k = 0; k < VEC; ++k)
-            if (x0 + k < V)
-              G_out[x0 + k] = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx) * invZ;
-        }
-      }
-      break;
-    }
+    rt.thr = sm.thr[0][j];
+    if (j < L) { rd = row_at<T, CFG>(a, b, 1, j); rd.thr = sm.thr[1][j]; }
+    else rd = rt;
+    token = draw_token<T, CFG, NT>(a, rt, rd, ctx, st.uni[L], tid, ring, ring_bytes, tile_sums, sm, st, phase, status, Z);
   }
-  pdl_wait();   // the previous call on the stream has completed: outputs stay in order
-  if (G_out && token < 0)
-    for (int x = tid; x < V; x += NT) G_out[x] = 0.0f;
+  if (tid == 0) {
+    SeqRecord& rec = st.rec;
+    rec.first_rej = rejected ? j : -1;
+    rec.token = token;
+    rec.status_at = status;
+    rec.status_any = extra_status & 8;
+    rec.mode = draw ? ctx.mode : 1;
+    rec.Mt = draw ? ctx.Mt : 0.0f; rec.St = draw ? ctx.St : 0.0f;
+    rec.Md = draw ? ctx.Md : 0.0f; rec.Sd = draw ? ctx.Sd : 0.0f;
+    rec.thr_t = rt.thr; rec.thr_d = rd.thr;
+    rec.one_minus_omega = draw ? ctx.one_minus_omega : 1.0f;
+    rec.Z = Z;
+  }
+  __syncthreads();
+}
 
-  // ---- 8. emit x_{1:tau+1} ---------------------------------------------------------
+// Emits sequence b from the record of the block that decides it (winner): the accepted prefix, the
+// drawn token, padding; accepted length; status; optionally the distribution drawn from.
+template <typename T, bool CFG, int NT>
+__device__ void emit_sequence(const FusedArgs& ua, const int b, const SeqRecord& win, const int status_any,
+                              const int tid) {
+  const FinishArgs& a = ua.fin;
+  const int L = a.gamma;
+  const int tau = win.first_rej >= 0 ? win.first_rej : L;
   if (tid <= L) {
     int v = -1;
-    if (tid < tau) v = st.tok[tid];
-    else if (tid == tau) v = token;
+    if (tid < tau) v = a.tokens[(int64_t)b * L + tid];
+    else if (tid == tau) v = win.token;
     a.out_tokens[(int64_t)b * (L + 1) + tid] = v;
   }
   if (tid == 0) {
     a.out_accept_len[b] = tau;
-    if (a.out_status) a.out_status[b] = status;
+    if (a.out_status) a.out_status[b] = win.status_at | status_any;
   }
-  __syncthreads();  // the shared state may be reused for the next sequence
+  if (a.dbg_G) {
+    if (tau < a.T) write_G<T, CFG, NT>(a, b, tau, win, tid);
+    else for (int x = tid; x < a.V; x += NT) a.dbg_G[(int64_t)b * a.V + x] = 0.0f;
+  }
 }
 
-// This block's share of the items (both kernels): either a slice of one sequence's items, or
-// all items of a few whole sequences.
-struct BlockShare {
-  int seq_begin, seq_end;     // sequences this block touches
-  int item_begin, item_end;   // global item indices
-};
-__device__ __forceinline__ BlockShare block_share(const FusedArgs& a) {
-  BlockShare sh;
-  const int ips = a.items_per_seq;
-  if (a.ctas_per_seq > 1) {
-    const int b = blockIdx.x / a.ctas_per_seq;
-    const int j = blockIdx.x - b * a.ctas_per_seq;
-    sh.seq_begin = b;
-    sh.seq_end = b + 1;
-    sh.item_begin = b * ips + (int)((long long)ips * j / a.ctas_per_seq);
-    sh.item_end = b * ips + (int)((long long)ips * (j + 1) / a.ctas_per_seq);
-  } else {
-    sh.seq_begin = min(a.fin.B, (int)blockIdx.x * a.seqs_per_cta);
-    sh.seq_end = min(a.fin.B, sh.seq_begin + a.seqs_per_cta);
-    sh.item_begin = sh.seq_begin * ips;
-    sh.item_end = sh.seq_end * ips;
-  }
-  return sh;
-}
-
-// Phase 2 tail shared by both kernels, entered after every thread's results are in global memory
-// (stores, __threadfence, __syncthreads): count this block's arrival and run the finishes it owes.
+// Phase 2 of both kernels.  Entered by the whole block when its row statistics are complete in
+// shared memory.  Everything up to the griddepcontrol.wait reads only the call's inputs, so it runs
+// beside the previous call on the stream; after it come the few global writes.
 template <typename T, bool CFG, int NT>
-__device__ __forceinline__ void arrive_and_finish(const FusedArgs& a, const BlockShare& sh, int tid, int* flag_smem,
-                                                  bool aborted, unsigned char* ring, int ring_bytes,
-                                                  double* tile_sums, FinishSmem& fin, FinishStage& fst) {
-  if (sh.seq_begin >= sh.seq_end) {   // nothing to do in this block
-    if (!a.early_trigger) pdl_launch_dependents();
+__device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const RowStats& rs, const int tid,
+                             int* flag_smem, const bool aborted, unsigned char* ring, const int ring_bytes,
+                             double* tile_sums, FinishSmem& sm, FinishStage& st, SeqRecord* rec_smem /*[kMaxGamma]*/) {
+  const FinishArgs& a = ua.fin;
+  const int L = a.gamma;
+  const int extra = aborted ? 8 : 0;
+  uint32_t phase = 0;
+  auto write_pqf = [&](int b) {   // diagnostics of this block's positions
+    if (tid >= sh.pos_begin && tid < sh.pos_end) {
+      if (a.dbg_p) a.dbg_p[(int64_t)b * L + tid] = st.p[tid];
+      if (a.dbg_q) a.dbg_q[(int64_t)b * L + tid] = st.q[tid];
+      if (a.dbg_f) a.dbg_f[(int64_t)b * L + tid] = st.f[tid];
+    }
+  };
+  if (ua.ctas_per_seq == 1) {
+    // the block owns whole sequences: its records are final
+    pdl_wait();   // outputs of consecutive calls stay in order
+    const int sticky = __ldcg(ua.error_flag) ? 8 : 0;
+    for (int sl = 0; sl < sh.seq_end - sh.seq_begin; ++sl) {
+      const int b = sh.seq_begin + sl;
+      finish_positions<T, CFG, NT>(ua, sh, sl, rs, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
+      write_pqf(b);
+      emit_sequence<T, CFG, NT>(ua, b, st.rec, st.rec.status_any | sticky, tid);
+      __syncthreads();
+    }
     return;
   }
-  if (a.ctas_per_seq > 1) {
-    if (tid == 0) {
-      __threadfence();
-      const int old = atomicAdd(&a.counters[sh.seq_begin], 1);
-      const int last = (old + 1 == a.ctas_per_seq) ? 1 : 0;
-      if (last) {   // nobody else touches this counter any more: leave it ready for the next call
-        a.counters[sh.seq_begin] = 0;
-        __threadfence();
-      }
-      *flag_smem = last;
-    }
-    __syncthreads();
-    if (*flag_smem == 0) {   // another block of this sequence arrives later and finishes it
-      if (!a.early_trigger) pdl_launch_dependents();
-      return;
-    }
+  if (sh.seq_begin >= sh.seq_end) return;
+  const int b = sh.seq_begin;
+  finish_positions<T, CFG, NT>(ua, sh, 0, rs, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
+  pdl_wait();   // the previous call has completed: the records and the outputs are free
+  write_pqf(b);
+  if (tid == 0) {
+    ua.records[(int64_t)b * kMaxGamma + sh.slot] = st.rec;
     __threadfence();
+    const int old = atomicAdd(&ua.counters[b], 1);
+    const int last = (old + 1 == ua.ctas_per_seq) ? 1 : 0;
+    if (last) ua.counters[b] = 0;   // nobody else touches this counter any more: ready for the next call
+    *flag_smem = last;
   }
-  const int extra = (aborted || __ldcg(a.error_flag)) ? 8 : 0;
-  uint32_t fin_phase = 0;
-  for (int b = sh.seq_begin; b < sh.seq_end; ++b)
-    finish_sequence_staged<T, CFG, NT>(a, b, tid, ring, ring_bytes, tile_sums, fin, fst, fin_phase, extra,
-                                       b == sh.seq_end - 1);
+  __syncthreads();
+  if (*flag_smem == 0) return;   // another block of this sequence arrives later and resolves it
+  // ---- resolve: the first block, in position order, that rejected decides the sequence ------------
+  __threadfence();
+  if (tid < ua.ctas_per_seq) {
+    const int4* src = reinterpret_cast<const int4*>(&ua.records[(int64_t)b * kMaxGamma + tid]);
+    int4* dst = reinterpret_cast<int4*>(&rec_smem[tid]);
+#pragma unroll
+    for (int k = 0; k < (int)(sizeof(SeqRecord) / sizeof(int4)); ++k) dst[k] = __ldcg(src + k);
+  }
+  __syncthreads();
+  int w = 0, any = __ldcg(ua.error_flag) ? 8 : 0;
+  for (int k = 0; k < ua.ctas_per_seq; ++k) any |= rec_smem[k].status_any;
+  while (w < ua.ctas_per_seq - 1 && rec_smem[w].first_rej < 0) ++w;   // the last block also carries the bonus draw
+  emit_sequence<T, CFG, NT>(ua, b, rec_smem[w], any, tid);
 }
 
 // ======================= plain kernel: one pipeline per warp ============================
@@ -531,15 +625,15 @@ __device__ __forceinline__ void arrive_and_finish(const FusedArgs& a, const Bloc
 // step at all.
 constexpr int kWStages = 3;
 constexpr int kWStageBytes = 2048;
-constexpr int kWarpStash = 96;
+constexpr int kBlockStash = 1536;   // items (row parts) a block may own
 constexpr int kPlainRingBytes = kPlainWarps * kWStages * kWStageBytes;
 
 struct PlainSmem {
   alignas(128) unsigned char ring[kPlainWarps][kWStages][kWStageBytes];
   alignas(8) uint64_t full[kPlainWarps][kWStages];
-  float2 stash[kPlainWarps][kWarpStash];
-  float stash_tokz[kPlainWarps][kWarpStash];   // logit of the row's drafted token, if this part holds it
-  unsigned char stash_has[kPlainWarps][kWarpStash];
+  float2 stash[kBlockStash];   // (m, s) per item, by local item index
+  RowStats rs;
+  SeqRecord recs[kMaxGamma];
   int last_flag;
   int abort;
   FinishSmem fin;
@@ -558,12 +652,12 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
   extern __shared__ __align__(128) unsigned char fused_smem_raw[];
   PlainSmem& sm = *reinterpret_cast<PlainSmem*>(fused_smem_raw);
 
-  if (a.early_trigger) pdl_launch_dependents();
+  pdl_launch_dependents();   // the next call on the stream may start: see the head of this file
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const FinishArgs& f = a.fin;
   const int V = f.V;
-  const int rows_per_seq = f.T + f.gamma;
   const int part_elems = a.chunks_per_part * EPS;
+  const int parts = a.parts_per_row;
 
   if (tid == 0) { sm.last_flag = 0; sm.abort = 0; mbar_init(&sm.fst.bar, 1); }
   if (lane == 0) {
@@ -572,29 +666,23 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
   }
   __syncthreads();
 
-  // the block's items (sequence-aligned, see block_share), split evenly over its warps
+  // the block's items (parts of its local rows, see block_share), split evenly over its warps
   const BlockShare sh = block_share(a);
-  const int n_block = sh.item_end - sh.item_begin;
-  const int item_begin = sh.item_begin + (int)((long long)n_block * warp / kPlainWarps);
-  const int item_end = sh.item_begin + (int)((long long)n_block * (warp + 1) / kPlainWarps);
+  const int n_block = sh.n_rows * parts;
+  const int item_begin = (int)((long long)n_block * warp / kPlainWarps);
+  const int item_end = (int)((long long)n_block * (warp + 1) / kPlainWarps);
 
   // producer cursor (meaningful in lane 0): the next chunk to copy
   int p_item = item_begin, p_x = 0, p_xend = 0, p_s = 0;
   const T *p_cond = nullptr, *p_uncond = nullptr;
   auto producer_open_item = [&]() {   // sets the cursor to the first chunk of p_item
-    const int row_id = p_item / a.parts_per_row;
-    const int part = p_item - row_id * a.parts_per_row;
-    const int b = row_id / rows_per_seq;
-    const int r = row_id - b * rows_per_seq;
-    if (r < f.T) {
-      const int64_t off = (int64_t)b * f.tstride + (int64_t)r * V;
-      p_cond = reinterpret_cast<const T*>(f.target) + off;
-      p_uncond = CFG ? reinterpret_cast<const T*>(f.target_uncond) + off : nullptr;
-    } else {
-      const int64_t off = (int64_t)b * f.dstride + (int64_t)(r - f.T) * V;
-      p_cond = reinterpret_cast<const T*>(f.draft) + off;
-      p_uncond = CFG ? reinterpret_cast<const T*>(f.draft_uncond) + off : nullptr;
-    }
+    const int row_id = p_item / parts;
+    const int part = p_item - row_id * parts;
+    int b, which, i;
+    local_row(sh, row_id, f.gamma, b, which, i);
+    const Row<T, CFG> row = row_at<T, CFG>(f, b, which, i);
+    p_cond = row.cond;
+    p_uncond = row.uncond;
     p_x = part * part_elems;
     p_xend = min(V, p_x + part_elems);
   };
@@ -618,9 +706,8 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
 
   // drafted token of a row (-1 for the bonus row), loaded a row ahead of its use
   auto token_of_row = [&](int row_id) -> int {
-    const int b = row_id / rows_per_seq;
-    const int r = row_id - b * rows_per_seq;
-    const int i = r < f.T ? r : r - f.T;
+    int b, which, i;
+    local_row(sh, row_id, f.gamma, b, which, i);
     return i < f.gamma ? __ldg(f.tokens + (int64_t)b * f.gamma + i) : -1;
   };
 
@@ -632,11 +719,11 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
     int issued = 0;       // chunks consumed so far (for the bounded wait after a timeout)
     bool ok = true;
     int cur_row = -1, tok_cur = -1, tok_next = -1;
-    const int last_row = item_end > item_begin ? (item_end - 1) / a.parts_per_row : -1;
-    if (item_begin < item_end) tok_next = token_of_row(item_begin / a.parts_per_row);
+    const int last_row = item_end > item_begin ? (item_end - 1) / parts : -1;
+    if (item_begin < item_end) tok_next = token_of_row(item_begin / parts);
     for (int item = item_begin; item < item_end; ++item, ++n_my) {
-      const int row_id = item / a.parts_per_row;
-      const int part = item - row_id * a.parts_per_row;
+      const int row_id = item / parts;
+      const int part = item - row_id * parts;
       const int x_begin = part * part_elems;
       const int x_end = min(V, x_begin + part_elems);
       if (row_id != cur_row) {
@@ -751,10 +838,9 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
         s_run += __shfl_xor_sync(0xffffffffu, s_run, off);
         cnt_run += __shfl_xor_sync(0xffffffffu, cnt_run, off);
       }
-      if (lane == 0 && n_my < kWarpStash) {
-        sm.stash[warp][n_my] = make_float2(Mw, s_run + (float)(cnt_run - 1));
-        sm.stash_tokz[warp][n_my] = tokz;
-        sm.stash_has[warp][n_my] = has_tok ? 1 : 0;
+      if (lane == 0 && item < kBlockStash) {
+        sm.stash[item] = make_float2(Mw, s_run + (float)(cnt_run - 1));
+        if (has_tok && row_id < kBlockRows) sm.rs.tokz[row_id] = tokz;
       }
     }
     if (!ok && lane == 0) {
@@ -767,23 +853,26 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
   }
 
   // ================================= phase 2 ===========================================
-  if (a.early_trigger) pdl_wait();   // the previous call has completed: the workspace is free
-  __syncwarp();
-  for (int idx = lane; idx < n_my; idx += 32) {
-    const_cast<float2*>(f.partials)[item_begin + idx] = sm.stash[warp][idx];
-    if (sm.stash_has[warp][idx]) a.tok_logit[(item_begin + idx) / a.parts_per_row] = sm.stash_tokz[warp][idx];
-  }
-  __threadfence();
   __syncthreads();
-  arrive_and_finish<T, CFG, kPlainThreads>(a, sh, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes, sm.tile_sums,
-                            sm.fin, sm.fst);
+  // the statistics of each local row: its parts merged by one warp
+  for (int r = warp; r < sh.n_rows; r += kPlainWarps) {
+    float m = CSD_NEG_INF, s_acc = -1.0f;
+    for (int pp = lane; pp < parts; pp += 32) {
+      const float2 v = sm.stash[r * parts + pp];
+      stat_merge(m, s_acc, v.x, v.y);
+    }
+    stat_warp_allreduce(m, s_acc);
+    if (lane == 0) { sm.rs.ms[r] = make_float2(m, s_acc); sm.rs.thr[r] = CSD_NEG_INF; }
+  }
+  __syncthreads();
+  finish_block<T, CFG, kPlainThreads>(a, sh, sm.rs, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes,
+                                      sm.tile_sums, sm.fin, sm.fst, sm.recs);
 }
 
 // ======================= top-k kernel: a block streams whole rows ========================
 constexpr int kTkStages = 2;
 constexpr int kTkStageBytes = 16384;
 constexpr int kTkRingBytes = kTkStages * kTkStageBytes;
-constexpr int kTkStash = 256;
 constexpr int kWarpList = 256;                // per-warp capacity of the list of values >= lo
 constexpr int kListCap = kTopkWarps * kWarpList;
 constexpr int kLinBins = 512;
@@ -812,9 +901,8 @@ struct TopkSmem {
   float part_thr[2];
   int bc_i[4];
   float red_f[kTopkWarps][2];
-  float2 stash[kTkStash];
-  float stash_thr[kTkStash];
-  float stash_tokz[kTkStash];       // logit of the row's drafted token
+  RowStats rs;
+  SeqRecord recs[kMaxGamma];
   int last_flag;
   int abort;
   FinishSmem fin;
@@ -929,11 +1017,10 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   extern __shared__ __align__(128) unsigned char fused_smem_raw[];
   TopkSmem& sm = *reinterpret_cast<TopkSmem*>(fused_smem_raw);
 
-  if (a.early_trigger) pdl_launch_dependents();
+  pdl_launch_dependents();   // the next call on the stream may start: see the head of this file
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const FinishArgs& f = a.fin;
   const int V = f.V;
-  const int rows_per_seq = f.T + f.gamma;
   const int cpr = (V + EPS - 1) / EPS;   // stages per row
   const int k_top = a.top_k;
 
@@ -948,31 +1035,18 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   }
   __syncthreads();
 
-  // this block's rows (sequence-aligned, see block_share)
+  // this block's local rows (see block_share)
   const BlockShare sh = block_share(a);
-  const int row_begin = sh.item_begin, row_end = sh.item_end;
+  const int row_begin = 0, row_end = sh.n_rows;
 
   auto row_of = [&](int row_id) -> Row<T, CFG> {
-    const int b = row_id / rows_per_seq;
-    const int r = row_id - b * rows_per_seq;
-    Row<T, CFG> row;
-    row.scale = f.cfg_scale;
-    row.thr = CSD_NEG_INF;
-    if (r < f.T) {
-      const int64_t off = (int64_t)b * f.tstride + (int64_t)r * V;
-      row.cond = reinterpret_cast<const T*>(f.target) + off;
-      row.uncond = CFG ? reinterpret_cast<const T*>(f.target_uncond) + off : nullptr;
-    } else {
-      const int64_t off = (int64_t)b * f.dstride + (int64_t)(r - f.T) * V;
-      row.cond = reinterpret_cast<const T*>(f.draft) + off;
-      row.uncond = CFG ? reinterpret_cast<const T*>(f.draft_uncond) + off : nullptr;
-    }
-    return row;
+    int b, which, i;
+    local_row(sh, row_id, f.gamma, b, which, i);
+    return row_at<T, CFG>(f, b, which, i);
   };
   auto token_of_row = [&](int row_id) -> int {
-    const int b = row_id / rows_per_seq;
-    const int r = row_id - b * rows_per_seq;
-    const int i = r < f.T ? r : r - f.T;
+    int b, which, i;
+    local_row(sh, row_id, f.gamma, b, which, i);
     return i < f.gamma ? __ldg(f.tokens + (int64_t)b * f.gamma + i) : -1;
   };
   // Issues the copies of chunk c of this block's j-th row (if there is one) into stage q % kTkStages.
@@ -999,9 +1073,9 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
     int ctot = 0;
 #pragma unroll
     for (int w = 0; w < kTopkWarps; ++w) { tot += sm.part_acc[par][w]; ctot += sm.part_cmax[par][w]; }
-    if (idx < kTkStash) {
-      sm.stash[idx] = make_float2(sm.part_max[par], tot + (float)(ctot - 1));
-      sm.stash_thr[idx] = sm.part_thr[par];
+    if (idx < kBlockRows) {
+      sm.rs.ms[idx] = make_float2(sm.part_max[par], tot + (float)(ctot - 1));
+      sm.rs.thr[idx] = sm.part_thr[par];
     }
   };
 
@@ -1067,7 +1141,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         if (tid == 0 && ok && tl >= 0 && tl < n) {   // the drafted token's logit passes by: keep it
           float zc = load_scalar_smem<T>(&sm.ring[s][tl * (int)sizeof(T)]);
           if (CFG) zc = cfg_mix(zc, load_scalar_smem<T>(&sm.ring[s][kTkStageBytes / 2 + tl * (int)sizeof(T)]), f.cfg_scale);
-          if (n_my < kTkStash) sm.stash_tokz[n_my] = zc;
+          if (n_my < kBlockRows) sm.rs.tokz[n_my] = zc;
         }
         __syncwarp();
         if (lane == 0) {   // this warp is done with the stage; the last one to say so refills it
@@ -1232,19 +1306,10 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   }
 
   // ================================= phase 2 ===========================================
-  if (a.early_trigger) pdl_wait();   // the previous call has completed: the workspace is free
-  __syncthreads();
-  for (int idx = tid; idx < n_my; idx += kTopkThreads) {
-    const int row_id = row_begin + idx;
-    const_cast<float2*>(f.partials)[row_id] = sm.stash[idx];
-    const_cast<float*>(f.thresholds)[row_id] = sm.stash_thr[idx];
-    a.tok_logit[row_id] = sm.stash_tokz[idx];
-  }
-  __threadfence();
   __syncthreads();
   static_assert(sizeof(sm.list) >= kFinTiles * sizeof(double), "tile sums live in the list area");
-  arrive_and_finish<T, CFG, kTopkThreads>(a, sh, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
-                            reinterpret_cast<double*>(&sm.list[0][0]), sm.fin, sm.fst);
+  finish_block<T, CFG, kTopkThreads>(a, sh, sm.rs, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
+                                     reinterpret_cast<double*>(&sm.list[0][0]), sm.fin, sm.fst, sm.recs);
 }
 
 }  // namespace csd
