@@ -746,7 +746,7 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
         ++issued;
         const int n = min(EPS, x_end - x0);
         const unsigned char* stage = &sm.ring[warp][c_s][0];
-        const bool full = ok && n == EPS;
+        const bool full = n == EPS;   // (after a timeout the data is garbage anyway: the call is flagged)
 #pragma unroll
         for (int g0 = 0; g0 < NVS; g0 += GV) {
           float vals[GV * VEC];
@@ -773,7 +773,7 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
             for (int v = 0; v < GV; ++v) {
               const int xo = ((g0 + v) * 32 + lane) * VEC;
               float zc[VEC];
-              if (full || (ok && xo < n)) {
+              if (full || xo < n) {
                 unpack_vec<T>(stage + xo * (int)sizeof(T), zc);
                 if (CFG) {
                   float zu[VEC];
@@ -783,7 +783,7 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
                 }
               } else {
 #pragma unroll
-                for (int e = 0; e < VEC; ++e) zc[e] = ok ? CSD_NEG_INF : __int_as_float(0x7fc00000);
+                for (int e = 0; e < VEC; ++e) zc[e] = CSD_NEG_INF;
               }
 #pragma unroll
               for (int e = 0; e < VEC; ++e) vals[v * VEC + e] = zc[e];
@@ -819,7 +819,7 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
           }
         }
         const int tl = tok_cur - x0;
-        if (ok && tl >= 0 && tl < n) {   // the drafted token's logit passes by: keep it
+        if (tl >= 0 && tl < n) {   // the drafted token's logit passes by: keep it
           float zc = load_scalar_smem<T>(stage + tl * (int)sizeof(T));
           if (CFG) zc = cfg_mix(zc, load_scalar_smem<T>(stage + kWStageBytes / 2 + tl * (int)sizeof(T)), f.cfg_scale);
           tokz = zc;
@@ -900,6 +900,7 @@ struct TopkSmem {
   float part_max[2];
   float part_thr[2];
   int bc_i[4];
+  float bc_f;
   float red_f[kTopkWarps][2];
   RowStats rs;
   SeqRecord recs[kMaxGamma];
@@ -1101,7 +1102,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         const int x0 = c * EPS;
         const int n = min(EPS, V - x0);
         float z[VPT];
-        if (ok && n == EPS) {   // the common case: a full stage, no bounds to check
+        if (n == EPS) {   // the common case: a full stage, no bounds to check
 #pragma unroll
           for (int v = 0; v < NVS; ++v) {
             const int xo = (v * kTopkThreads + tid) * VEC;
@@ -1121,7 +1122,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
           for (int v = 0; v < NVS; ++v) {
             const int xo = (v * kTopkThreads + tid) * VEC;
             float zc[VEC];
-            if (ok && xo < n) {
+            if (xo < n) {
               unpack_vec<T>(&sm.ring[s][xo * (int)sizeof(T)], zc);
               if (CFG) {
                 float zu[VEC];
@@ -1131,14 +1132,14 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
               }
             } else {
 #pragma unroll
-              for (int e = 0; e < VEC; ++e) zc[e] = ok ? CSD_NEG_INF : __int_as_float(0x7fc00000);
+              for (int e = 0; e < VEC; ++e) zc[e] = CSD_NEG_INF;
             }
 #pragma unroll
             for (int e = 0; e < VEC; ++e) z[v * VEC + e] = zc[e];
           }
         }
         const int tl = tok_cur - x0;
-        if (tid == 0 && ok && tl >= 0 && tl < n) {   // the drafted token's logit passes by: keep it
+        if (tid == 0 && tl >= 0 && tl < n) {   // the drafted token's logit passes by: keep it
           float zc = load_scalar_smem<T>(&sm.ring[s][tl * (int)sizeof(T)]);
           if (CFG) zc = cfg_mix(zc, load_scalar_smem<T>(&sm.ring[s][kTkStageBytes / 2 + tl * (int)sizeof(T)]), f.cfg_scale);
           if (n_my < kBlockRows) sm.rs.tokz[n_my] = zc;
@@ -1186,23 +1187,27 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
           scale = (float)kLinBins / (kLinRangeSigmas * dev);
         }
         // ---- gather this stage's values >= lo into the warp's list -------------------------
-        // (the test is "not below lo", so that a NaN lands in the list and marks the row through the maximum)
-        int cnt = 0;
+        // (the test is "not below lo", so that a NaN lands in the list and marks the row through the
+        // maximum).  Two predicated passes, written out so that they stay free of branches: count,
+        // reserve the slots with one atomic, store.
+        uint32_t cnt = 0;
 #pragma unroll
-        for (int e = 0; e < VPT; ++e) cnt += !(z[e] < lo) ? 1 : 0;
+        for (int e = 0; e < VPT; ++e)
+          asm("{\n\t.reg .pred p;\n\tsetp.geu.f32 p, %1, %2;\n\t@p add.u32 %0, %0, 1;\n\t}" : "+r"(cnt) : "f"(z[e]), "f"(lo));
         if (cnt > 0) {
-          int pos = atomicAdd(&sm.wpos[warp], cnt);
-          if (pos + cnt <= kWarpList) {
+          const uint32_t pos = (uint32_t)atomicAdd(&sm.wpos[warp], (int)cnt);
+          if (pos + cnt <= (uint32_t)kWarpList) {
+            uint32_t addr = smem_addr(&sm.list[warp][pos]);
 #pragma unroll
-            for (int e = 0; e < VPT; ++e) {
-              const bool keep = !(z[e] < lo);
-              if (keep) sm.list[warp][pos] = z[e];
-              pos += keep ? 1 : 0;
-            }
+            for (int e = 0; e < VPT; ++e)
+              asm volatile(
+                  "{\n\t.reg .pred p;\n\tsetp.geu.f32 p, %1, %2;\n\t@p st.shared.f32 [%0], %1;\n\t@p add.u32 %0, %0, 4;\n\t}"
+                  : "+r"(addr)
+                  : "f"(z[e]), "f"(lo)
+                  : "memory");
           }
         }
       }
-      // ---- end of the row: this warp's maximum and its share of the histogram ---------------
       // the row maximum is among the gathered values whenever the fast path applies
       __syncwarp();
       const int wc = sm.wpos[warp];
@@ -1230,8 +1235,13 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
       // NaN guesses, NaN / +inf rows and constant rows all fail one of these tests
       fast = fast && n_lo >= k_top && (mx > lo) && (mx < CSD_POS_INF) && (scale > 0.0f) && (scale < CSD_POS_INF);
       if (fast) {
-        int kk;
-        const int pick_bin = warp_pick_bin(sm.hist, k_top, lane, &kk);   // every warp computes it for itself
+        if (warp == 0) {   // the bin of the k-th largest and the rank of the answer inside it
+          int kk;
+          const int bin = warp_pick_bin(sm.hist, k_top, lane, &kk);
+          if (lane == 0) { sm.bc_i[0] = bin; sm.bc_i[1] = kk; }
+        }
+        __syncthreads();   // ---- C: bin known
+        const int pick_bin = sm.bc_i[0];
         for (int i = lane; i < wc; i += 32) {
           const float v = sm.list[warp][i];
           if (lin_bin(v, lo, scale) == pick_bin) {
@@ -1242,21 +1252,27 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         __syncthreads();   // ---- D: candidates complete
         const int n_cand = sm.n_cand[par];
         if (n_cand <= kCandCap) {
-          // exact rank among the candidates, every warp for itself (two candidates per lane)
-          const float v0 = lane < n_cand ? sm.cand[lane] : CSD_NEG_INF;
-          const float v1 = lane + 32 < n_cand ? sm.cand[lane + 32] : CSD_NEG_INF;
-          int gt0 = 0, ge0 = 0, gt1 = 0, ge1 = 0;
-          for (int j2 = 0; j2 < n_cand; ++j2) {
-            const float w = sm.cand[j2];
-            gt0 += (w > v0) ? 1 : 0; ge0 += (w >= v0) ? 1 : 0;
-            gt1 += (w > v1) ? 1 : 0; ge1 += (w >= v1) ? 1 : 0;
-          }
-          const bool hit0 = lane < n_cand && gt0 < kk && kk <= ge0;
-          const bool hit1 = lane + 32 < n_cand && gt1 < kk && kk <= ge1;
-          const unsigned b0 = __ballot_sync(0xffffffffu, hit0);
-          const unsigned b1 = __ballot_sync(0xffffffffu, hit1);
-          const float thr = b0 ? __shfl_sync(0xffffffffu, v0, __ffs(b0) - 1)
+          if (warp == 0) {
+            // exact rank among the candidates (two per lane)
+            const int kk = sm.bc_i[1];
+            const float v0 = lane < n_cand ? sm.cand[lane] : CSD_NEG_INF;
+            const float v1 = lane + 32 < n_cand ? sm.cand[lane + 32] : CSD_NEG_INF;
+            int gt0 = 0, ge0 = 0, gt1 = 0, ge1 = 0;
+            for (int j2 = 0; j2 < n_cand; ++j2) {
+              const float w = sm.cand[j2];
+              gt0 += (w > v0) ? 1 : 0; ge0 += (w >= v0) ? 1 : 0;
+              gt1 += (w > v1) ? 1 : 0; ge1 += (w >= v1) ? 1 : 0;
+            }
+            const bool hit0 = lane < n_cand && gt0 < kk && kk <= ge0;
+            const bool hit1 = lane + 32 < n_cand && gt1 < kk && kk <= ge1;
+            const unsigned b0 = __ballot_sync(0xffffffffu, hit0);
+            const unsigned b1 = __ballot_sync(0xffffffffu, hit1);
+            const float t = b0 ? __shfl_sync(0xffffffffu, v0, __ffs(b0) - 1)
                                : __shfl_sync(0xffffffffu, v1, b1 ? __ffs(b1) - 1 : 0);
+            if (lane == 0) sm.bc_f = t;
+          }
+          __syncthreads();   // ---- E: threshold known
+          const float thr = sm.bc_f;
           // ---- statistics of the kept values of this warp's list -------------------------
           float acc = 0.0f;
           int cmax = 0;
