@@ -230,7 +230,7 @@ struct FinishStage {
 // Eq. opt_G summed per tile over the whole row pair, rows brought through the ring by bulk copies;
 // then the tile of the crossing and the token inside it.  Returns the token (-1: nothing to draw
 // from); Z_out gets the normaliser, status gets bits 4 / 8 where they apply; ctx.mode may change to 1.
-template <typename T, bool CFG, int NT>
+template <typename T, bool CFG, int NT, bool FILT>
 __device__ int draw_token(const FinishArgs& a, const Row<T, CFG>& rt, const Row<T, CFG>& rd, PairCtx& ctx, const float u,
                           const int tid, unsigned char* ring, const int ring_bytes, double* tile_sums, FinishSmem& sm,
                           FinishStage& st, uint32_t& phase, int& status, double& Z_out) {
@@ -292,7 +292,7 @@ __device__ int draw_token(const FinishArgs& a, const Row<T, CFG>& rt, const Row<
             float acc = 0.0f;
 #pragma unroll
             for (int k = 0; k < VEC; ++k)
-              acc += weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
+              acc += weight_of(FILT ? rt.filter(zt[k]) : zt[k], ctx.mode == 0 ? (FILT ? rd.filter(zd[k]) : zd[k]) : 0.0f, ctx);
             acc2[r] = acc;
           }
         }
@@ -360,7 +360,7 @@ __device__ int draw_token(const FinishArgs& a, const Row<T, CFG>& rt, const Row<
       unsigned posmask = 0;
 #pragma unroll
       for (int k = 0; k < VEC; ++k) {
-        const float g = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
+        const float g = weight_of(FILT ? rt.filter(zt[k]) : zt[k], ctx.mode == 0 ? (FILT ? rd.filter(zd[k]) : zd[k]) : 0.0f, ctx);
         if (g > 0.0f) { last_pos = k; posmask |= 1u << k; }
         acc += (double)g;
         run[k] = acc;
@@ -514,7 +514,10 @@ __device__ void finish_positions(const FusedArgs& ua, const BlockShare& sh, cons
     rt.thr = sm.thr[0][j];
     if (j < L) { rd = row_at<T, CFG>(a, b, 1, j); rd.thr = sm.thr[1][j]; }
     else rd = rt;
-    token = draw_token<T, CFG, NT>(a, rt, rd, ctx, st.uni[L], tid, ring, ring_bytes, tile_sums, sm, st, phase, status, Z);
+    token = a.use_topk ? draw_token<T, CFG, NT, true>(a, rt, rd, ctx, st.uni[L], tid, ring, ring_bytes, tile_sums, sm,
+                                                      st, phase, status, Z)
+                       : draw_token<T, CFG, NT, false>(a, rt, rd, ctx, st.uni[L], tid, ring, ring_bytes, tile_sums, sm,
+                                                       st, phase, status, Z);
   }
   if (tid == 0) {
     SeqRecord& rec = st.rec;
