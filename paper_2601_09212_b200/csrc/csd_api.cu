@@ -50,11 +50,10 @@ bool shape_ok(int B, int gamma, int V) {
   return B >= 1 && gamma >= 1 && gamma <= kMaxGamma && V >= 2 && V <= kMaxV;
 }
 
-// Workspace: [header: error flag][counters: B int][partials: rows * max_parts float2][thresholds: rows float]
-//            [records: B * 32 SeqRecord (single-launch path)]
-// The header and the counters must be zero before the first call; every call leaves them zero.
+// Workspace: [header: error flag][partials: rows * max_parts float2][thresholds: rows float]
+// (the last two: multi-launch path only).  The header must be zero before the first call.
 struct Layout {
-  size_t rows, max_parts, header_off, counters_off, partials_off, thresholds_off, records_off, zero_bytes, total;
+  size_t rows, max_parts, header_off, partials_off, thresholds_off, zero_bytes, total;
 };
 Layout layout_for(int B, int gamma, int V, int dtype) {
   Layout l;
@@ -63,12 +62,10 @@ Layout layout_for(int B, int gamma, int V, int dtype) {
   const size_t min_part = (size_t)kStatsThreads * vec_width(dtype);  // U = 1
   l.max_parts = ((size_t)V + min_part - 1) / min_part;
   l.header_off = 0;
-  l.counters_off = kAlign;
-  l.partials_off = l.counters_off + align_up((size_t)B * sizeof(int));
+  l.partials_off = kAlign;
   l.zero_bytes = l.partials_off;
   l.thresholds_off = l.partials_off + align_up(l.rows * l.max_parts * sizeof(float2));
-  l.records_off = l.thresholds_off + align_up(l.rows * sizeof(float));
-  l.total = l.records_off + align_up((size_t)B * kMaxGamma * sizeof(SeqRecord));
+  l.total = l.thresholds_off + align_up(l.rows * sizeof(float));
   return l;
 }
 
@@ -97,11 +94,18 @@ cudaError_t launch_fused(const FusedArgs& a, int grid, cudaStream_t stream) {
   cfg.blockDim = dim3(kTopkThreads);
   cfg.dynamicSmemBytes = sizeof(TopkSmem);
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (a.ctas_per_seq > 1) {   // the blocks of a sequence are one cluster
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)a.ctas_per_seq;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
   return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
@@ -120,11 +124,18 @@ cudaError_t launch_plain(const FusedArgs& a, int grid, cudaStream_t stream) {
   cfg.blockDim = dim3(kPlainThreads);
   cfg.dynamicSmemBytes = sizeof(PlainSmem);
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (a.ctas_per_seq > 1) {   // the blocks of a sequence are one cluster
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = (unsigned)a.ctas_per_seq;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+  }
   return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
@@ -282,18 +293,17 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
     ua.fin = fa;
     ua.top_k = p.top_k;
     ua.lo_sigmas = nanf("");
-    ua.records = reinterpret_cast<SeqRecord*>((char*)p.workspace + lay.records_off);
-    ua.counters = reinterpret_cast<int*>((char*)p.workspace + lay.counters_off);
     ua.error_flag = reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
     // Blocks are aligned with sequences and positions: either a sequence's draft positions are split
-    // over ctas_per_seq blocks (each with both rows of its positions), or a block owns seqs_per_cta
-    // whole sequences.
+    // over the ctas_per_seq blocks of one cluster (each with both rows of its positions; 2, 4 or 8
+    // blocks), or a block owns seqs_per_cta whole sequences.
     const long long target_blocks = 2LL * sms;
     long long c = 1, spc = 1;
     if (p.B >= target_blocks) spc = (p.B + target_blocks - 1) / target_blocks;
-    else c = target_blocks / p.B;
-    if (c > p.gamma) c = p.gamma;
-    if (c < 1) c = 1;
+    else {
+      const long long want = target_blocks / p.B;
+      while (2 * c <= want && 2 * c <= p.gamma && 2 * c <= kMaxCluster) c *= 2;
+    }
     while (spc > 1 && spc * rows_per_seq > kBlockRows) --spc;   // rows_per_seq <= 65 < kBlockRows
     if (topk) {
       ua.chunks_per_part = 0;

@@ -2,21 +2,20 @@
 //
 // Phase 1 streams this block's share of the logit rows through rings of
 // shared-memory stages filled by bulk asynchronous copies (mbarrier completion)
-// and keeps the per-row results in shared memory.  Phase 2 is the block's own
-// finish.  A block owns, for its sequence(s), a range of draft positions with both
-// rows of each, so it runs the accept tests of its positions itself and, at its first
-// rejection, draws the replacement token at once (Eq. opt_G with the two rows brought
-// back through the ring, inverse CDF) -- speculatively, since an earlier position of
-// another block may reject first.  Each block leaves a small record; the last block
-// of a sequence to arrive picks the first rejecting block's record and emits.  No
-// block ever waits for another block; every wait on a copy is bounded.
+// and keeps the per-row results in shared memory.  Phase 2 is the finish.  A block
+// owns, for its sequence(s), a range of draft positions with both rows of each, so
+// it runs the accept tests of its positions itself (Eq. relax).  Where a sequence is
+// split over several blocks, these form one thread-block cluster: each stores what it
+// found into its peers' shared memory, one cluster barrier later all of them know
+// which block holds the first rejection, and that block alone draws the replacement
+// token (Eq. opt_G with the two rows brought back through the ring, inverse CDF) and
+// emits the sequence.  Every wait on a copy is bounded.
 //
 // Consecutive calls on a stream overlap (programmatic dependent launch): every block
 // signals launch_dependents at once, and everything up to a block's first global write
-// -- streaming, accept tests, the draw -- reads only the call's inputs, so it runs beside
-// the previous call; griddepcontrol.wait comes just before that first write (the record,
-// or the outputs), which keeps the workspace and the outputs of consecutive calls in
-// order.  What is serialised between two calls is a 64-byte record, one atomic and the emit.
+// -- streaming, accept tests, the exchange, the draw -- reads only the call's inputs, so
+// it runs beside the previous call; griddepcontrol.wait comes just before that first
+// write, which keeps the outputs of consecutive calls in order.
 //
 //   verify_plain_kernel  every warp streams its own parts of rows through its own
 //                        ring and keeps a running (m, s) per lane.
@@ -88,6 +87,20 @@ __device__ __forceinline__ float max_nan(float x, float y) {
   return r;
 }
 
+// ---- thread-block cluster: the blocks of one sequence ---------------------------------------
+// Hardware barrier over all threads of all blocks of the cluster, split in two halves.  Every
+// thread of every block executes each half the same number of times, in the same order.
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// 32-bit store into the shared memory of block `rank` of this cluster, at the address that
+// `local` has in this block
+__device__ __forceinline__ void cluster_store(void* local, uint32_t rank, uint32_t v) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_addr(local)), "r"(rank));
+  asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"(v) : "memory");
+}
+constexpr int kMaxCluster = 8;   // portable cluster size
+
 template <typename T>
 __device__ __forceinline__ void unpack_vec(const unsigned char* p, float (&out)[Elem<T>::kVec]);
 template <>
@@ -116,47 +129,44 @@ __device__ __forceinline__ float load_scalar_smem<__nv_bfloat16>(const unsigned 
   return __uint_as_float(((uint32_t) * reinterpret_cast<const unsigned short*>(p)) << 16);
 }
 
-// What a block reports about its positions of a sequence (workspace, one per block of the sequence).
+// What a block found at the position it drew a token for.
 struct alignas(16) SeqRecord {
   int first_rej;   // 0-based position of this block's first rejection, -1 if it accepted all of its positions
   int token;       // token drawn at first_rej; for the block that owns the bonus row and accepted everything,
                    // the bonus token; -1 if there was nothing to draw from
   int status_at;   // status bits of that draw (bad row, bad token, Z fallback; for the bonus draw: bad row)
-  int status_any;  // status bits that hold whatever the other blocks say (a bounded wait gave up)
+  int status_any;  // status bits that hold wherever the sequence ends (a bounded wait gave up)
   int mode;        // diagnostics: how the token was drawn (0: Eq. opt_G, 1: from P), and the statistics used
   float Mt, St, Md, Sd, thr_t, thr_d, one_minus_omega;
   double Z;
   int pad[2];
 };
-static_assert(sizeof(SeqRecord) == 64, "records are copied as four 16-byte words");
 
 struct FusedArgs {
   FinishArgs fin;       // inputs and outputs (the workspace arrays of the multi-launch path are unused)
   int chunks_per_part;  // plain kernel: warp stages per part
   int parts_per_row;    // plain kernel
-  int ctas_per_seq;     // > 1: a sequence's positions are split over this many blocks (the last to
-                        //      arrive resolves the sequence); 1: a block owns seqs_per_cta whole sequences
+  int ctas_per_seq;     // > 1: a sequence's positions are split over the blocks of one cluster of this
+                        //      size; 1: a block owns seqs_per_cta whole sequences (no clusters)
   int seqs_per_cta;
   int top_k;
   float lo_sigmas;      // top-k guess: lo = mean + lo_sigmas * deviation (NaN: always select exactly)
-  SeqRecord* records;   // [B][kMaxGamma], written and read only with ctas_per_seq > 1
-  int* counters;        // [B] arrivals per sequence; zero before the first call, left zero by every call
   int* error_flag;      // set when a bounded wait gave up
 };
 
 // ---- a block's share of the work ------------------------------------------------------
 // Blocks are aligned with sequences AND with positions: a block owns, for each of its
 // sequences, a range of draft positions and BOTH rows (target, drafter) of each, so that it can
-// run the accept tests of its positions by itself and, where one of them rejects, draw the
-// replacement token right away -- speculatively, since an earlier position owned by another block
-// may have rejected first.  Local rows are ordered t_p0, d_p0, t_p0+1, d_p0+1, ..., [bonus row].
+// run the accept tests of its positions by itself and, if the sequence's first rejection turns out
+// to be among them, draw the replacement token.  Local rows are ordered t_p0, d_p0, t_p0+1, d_p0+1,
+// ..., [bonus row].
 struct BlockShare {
   int seq_begin, seq_end;   // sequences this block works on
   int pos_begin, pos_end;   // draft positions (0-based) it owns of each
   int bonus;                // it also owns the bonus row (target row gamma)
   int rows_per_seq;         // local rows per sequence
   int n_rows;               // local rows in all
-  int slot;                 // its record slot within the sequence (ctas_per_seq > 1)
+  int slot;                 // its rank among the blocks of the sequence (ctas_per_seq > 1)
 };
 __device__ __forceinline__ BlockShare block_share(const FusedArgs& a) {
   BlockShare sh;
@@ -224,6 +234,7 @@ struct FinishStage {
   float tokz[2][kMaxGamma + 1];
   float p[kMaxGamma], q[kMaxGamma], f[kMaxGamma];
   SeqRecord rec;
+  uint32_t xch[kMaxCluster];   // written by the blocks of the cluster: what each found (see finish_block)
   alignas(8) uint64_t bar;
 };
 
@@ -421,14 +432,13 @@ __device__ void write_G(const FinishArgs& a, const int b, const int j, const Seq
   }
 }
 
-// The block's positions [pos_begin, pos_end) of sequence b: accept tests (Eq. relax), its first
-// rejection, and the draw there (Eq. opt_G) -- or the bonus draw if it owns the bonus row and accepted
-// everything.  Row statistics come from shared memory (rs, local rows of sequence slot sl).  Leaves
-// the record in st.rec and p, q, f of its positions in st; reads only the call's inputs.
+// The block's positions [pos_begin, pos_end) of sequence b: accept tests (Eq. relax) and its first
+// rejection (the return value; pos_end if it accepted all of them).  Row statistics come from shared
+// memory (rs, local rows of sequence slot sl).  Leaves p, q, f of its positions in st; reads only the
+// call's inputs.
 template <typename T, bool CFG, int NT>
-__device__ void finish_positions(const FusedArgs& ua, const BlockShare& sh, const int sl, const RowStats& rs,
-                                 const int tid, unsigned char* ring, const int ring_bytes, double* tile_sums,
-                                 FinishSmem& sm, FinishStage& st, uint32_t& phase, const int extra_status) {
+__device__ int accept_positions(const FusedArgs& ua, const BlockShare& sh, const int sl, const RowStats& rs,
+                                const int tid, FinishSmem& sm, FinishStage& st) {
   const FinishArgs& a = ua.fin;
   const int L = a.gamma, V = a.V;
   const int b = sh.seq_begin + sl;
@@ -487,7 +497,20 @@ __device__ void finish_positions(const FusedArgs& ua, const BlockShare& sh, cons
   // ---- 2. this block's first rejection (the for/break of Algorithm 1, on its positions) ----------
   int j = p0;
   while (j < p1 && sm.acc[j]) ++j;
-  const bool rejected = j < p1;
+  return j;
+}
+
+// The draw at the block's first rejection j (Eq. opt_G) -- or, with j == pos_end in the block that
+// owns the bonus row, the bonus draw.  Follows accept_positions of the same sequence; leaves the
+// record in st.rec.
+template <typename T, bool CFG, int NT>
+__device__ void draw_position(const FusedArgs& ua, const BlockShare& sh, const int sl, int j, const int tid,
+                              unsigned char* ring, const int ring_bytes, double* tile_sums, FinishSmem& sm,
+                              FinishStage& st, uint32_t& phase, const int extra_status) {
+  const FinishArgs& a = ua.fin;
+  const int L = a.gamma;
+  const int b = sh.seq_begin + sl;
+  const bool rejected = j < sh.pos_end;
   int status = extra_status & ~8;
   PairCtx ctx;
   bool draw = false;
@@ -562,10 +585,17 @@ __device__ void emit_sequence(const FusedArgs& ua, const int b, const SeqRecord&
 // Phase 2 of both kernels.  Entered by the whole block when its row statistics are complete in
 // shared memory.  Everything up to the griddepcontrol.wait reads only the call's inputs, so it runs
 // beside the previous call on the stream; after it come the few global writes.
+//
+// With ctas_per_seq > 1 the blocks of a sequence form one cluster.  Each runs the accept tests of its
+// own positions and stores what it found -- its first rejection, if any -- into a word of every
+// peer's shared memory; after one cluster barrier every block knows which block holds the sequence's
+// first rejection (or that there is none: then the last block, which owns the bonus row).  That block
+// alone draws the token and emits the sequence; the others are done.  No block reads a peer's shared
+// memory, and none writes to it after the barrier, so blocks leave independently.
 template <typename T, bool CFG, int NT>
 __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const RowStats& rs, const int tid,
-                             int* flag_smem, const bool aborted, unsigned char* ring, const int ring_bytes,
-                             double* tile_sums, FinishSmem& sm, FinishStage& st, SeqRecord* rec_smem /*[kMaxGamma]*/) {
+                             const bool aborted, unsigned char* ring, const int ring_bytes, double* tile_sums,
+                             FinishSmem& sm, FinishStage& st) {
   const FinishArgs& a = ua.fin;
   const int L = a.gamma;
   const int extra = aborted ? 8 : 0;
@@ -578,46 +608,46 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
     }
   };
   if (ua.ctas_per_seq == 1) {
-    // the block owns whole sequences: its records are final
-    pdl_wait();   // outputs of consecutive calls stay in order
-    const int sticky = __ldcg(ua.error_flag) ? 8 : 0;
+    // the block owns whole sequences
+    int sticky = 0;
     for (int sl = 0; sl < sh.seq_end - sh.seq_begin; ++sl) {
       const int b = sh.seq_begin + sl;
-      finish_positions<T, CFG, NT>(ua, sh, sl, rs, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
+      const int j = accept_positions<T, CFG, NT>(ua, sh, sl, rs, tid, sm, st);
+      draw_position<T, CFG, NT>(ua, sh, sl, j, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
+      if (sl == 0) {   // before the block's first global write: outputs of consecutive calls stay in order
+        pdl_wait();
+        sticky = __ldcg(ua.error_flag) ? 8 : 0;
+      }
       write_pqf(b);
       emit_sequence<T, CFG, NT>(ua, b, st.rec, st.rec.status_any | sticky, tid);
       __syncthreads();
     }
     return;
   }
-  if (sh.seq_begin >= sh.seq_end) return;
   const int b = sh.seq_begin;
-  finish_positions<T, CFG, NT>(ua, sh, 0, rs, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
-  pdl_wait();   // the previous call has completed: the records and the outputs are free
+  const int c = ua.ctas_per_seq;
+  const int j = accept_positions<T, CFG, NT>(ua, sh, 0, rs, tid, sm, st);
+  // ---- tell every block of the sequence: bit 0 rejected, bit 1 a bounded wait gave up ------------
+  cluster_wait();   // second half of the barrier begun at kernel start: every peer is running
+  if (tid < c) cluster_store(&st.xch[sh.slot], (uint32_t)tid, (j < sh.pos_end ? 1u : 0u) | (aborted ? 2u : 0u));
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  int owner = c - 1, any = 0;
+  for (int k = c - 1; k >= 0; --k) {
+    const uint32_t w = st.xch[k];
+    if (w & 1u) owner = k;
+    if (w & 2u) any = 8;
+  }
+  if (owner != sh.slot) {   // another block decides the sequence
+    if (a.dbg_p || a.dbg_q || a.dbg_f) { pdl_wait(); write_pqf(b); }
+    return;
+  }
+  draw_position<T, CFG, NT>(ua, sh, 0, j, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
+  pdl_wait();   // the previous call has completed: outputs of consecutive calls stay in order
+  if (__ldcg(ua.error_flag)) any = 8;
   write_pqf(b);
-  if (tid == 0) {
-    ua.records[(int64_t)b * kMaxGamma + sh.slot] = st.rec;
-    __threadfence();
-    const int old = atomicAdd(&ua.counters[b], 1);
-    const int last = (old + 1 == ua.ctas_per_seq) ? 1 : 0;
-    if (last) ua.counters[b] = 0;   // nobody else touches this counter any more: ready for the next call
-    *flag_smem = last;
-  }
-  __syncthreads();
-  if (*flag_smem == 0) return;   // another block of this sequence arrives later and resolves it
-  // ---- resolve: the first block, in position order, that rejected decides the sequence ------------
-  __threadfence();
-  if (tid < ua.ctas_per_seq) {
-    const int4* src = reinterpret_cast<const int4*>(&ua.records[(int64_t)b * kMaxGamma + tid]);
-    int4* dst = reinterpret_cast<int4*>(&rec_smem[tid]);
-#pragma unroll
-    for (int k = 0; k < (int)(sizeof(SeqRecord) / sizeof(int4)); ++k) dst[k] = __ldcg(src + k);
-  }
-  __syncthreads();
-  int w = 0, any = __ldcg(ua.error_flag) ? 8 : 0;
-  for (int k = 0; k < ua.ctas_per_seq; ++k) any |= rec_smem[k].status_any;
-  while (w < ua.ctas_per_seq - 1 && rec_smem[w].first_rej < 0) ++w;   // the last block also carries the bonus draw
-  emit_sequence<T, CFG, NT>(ua, b, rec_smem[w], any, tid);
+  emit_sequence<T, CFG, NT>(ua, b, st.rec, any, tid);
 }
 
 // ======================= plain kernel: one pipeline per warp ============================
@@ -636,8 +666,6 @@ struct PlainSmem {
   alignas(8) uint64_t full[kPlainWarps][kWStages];
   float2 stash[kBlockStash];   // (m, s) per item, by local item index
   RowStats rs;
-  SeqRecord recs[kMaxGamma];
-  int last_flag;
   int abort;
   FinishSmem fin;
   FinishStage fst;
@@ -662,12 +690,13 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
   const int part_elems = a.chunks_per_part * EPS;
   const int parts = a.parts_per_row;
 
-  if (tid == 0) { sm.last_flag = 0; sm.abort = 0; mbar_init(&sm.fst.bar, 1); }
+  if (tid == 0) { sm.abort = 0; mbar_init(&sm.fst.bar, 1); }
   if (lane == 0) {
     for (int s = 0; s < kWStages; ++s) mbar_init(&sm.full[warp][s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  if (a.ctas_per_seq > 1) cluster_arrive();   // first half; finish_block waits before it writes to a peer
 
   // the block's items (parts of its local rows, see block_share), split evenly over its warps
   const BlockShare sh = block_share(a);
@@ -868,8 +897,8 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
     if (lane == 0) { sm.rs.ms[r] = make_float2(m, s_acc); sm.rs.thr[r] = CSD_NEG_INF; }
   }
   __syncthreads();
-  finish_block<T, CFG, kPlainThreads>(a, sh, sm.rs, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes,
-                                      sm.tile_sums, sm.fin, sm.fst, sm.recs);
+  finish_block<T, CFG, kPlainThreads>(a, sh, sm.rs, tid, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes,
+                                      sm.tile_sums, sm.fin, sm.fst);
 }
 
 // ======================= top-k kernel: a block streams whole rows ========================
@@ -906,8 +935,6 @@ struct TopkSmem {
   float bc_f;
   float red_f[kTopkWarps][2];
   RowStats rs;
-  SeqRecord recs[kMaxGamma];
-  int last_flag;
   int abort;
   FinishSmem fin;
   FinishStage fst;
@@ -1031,13 +1058,13 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   if (tid == 0) {
     for (int s = 0; s < kTkStages; ++s) { mbar_init(&sm.full[s], 1); sm.readers_done[s] = 0; }
     mbar_init(&sm.fst.bar, 1);
-    sm.last_flag = 0;
     sm.abort = 0;
     sm.n_cand[0] = 0;
     sm.n_cand[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  if (a.ctas_per_seq > 1) cluster_arrive();   // first half; finish_block waits before it writes to a peer
 
   // this block's local rows (see block_share)
   const BlockShare sh = block_share(a);
@@ -1327,8 +1354,8 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   // ================================= phase 2 ===========================================
   __syncthreads();
   static_assert(sizeof(sm.list) >= kFinTiles * sizeof(double), "tile sums live in the list area");
-  finish_block<T, CFG, kTopkThreads>(a, sh, sm.rs, tid, &sm.last_flag, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
-                                     reinterpret_cast<double*>(&sm.list[0][0]), sm.fin, sm.fst, sm.recs);
+  finish_block<T, CFG, kTopkThreads>(a, sh, sm.rs, tid, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
+                                     reinterpret_cast<double*>(&sm.list[0][0]), sm.fin, sm.fst);
 }
 
 }  // namespace csd
