@@ -296,20 +296,24 @@ def run_native(args) -> None:
     def enqueue(i):
         csd.csd_verify_ex(prms[i % ring_n])
 
-    # one lap of the ring as a CUDA graph: the launches inside are the library's own
+    # A few laps of the ring as one CUDA graph: the launches inside are the library's own.  Inside a
+    # graph consecutive calls keep their programmatic-launch edges and overlap as they do when enqueued
+    # directly; two replays do not overlap, so the graph is made long enough (>= 64 steps) for that
+    # boundary not to matter.
+    graph_steps = ring_n * max(1, -(-64 // ring_n))
     with torch.cuda.stream(stream):
         for i in range(ring_n):
             enqueue(i)
     stream.synchronize()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph, stream=stream):
-        for i in range(ring_n):
+        for i in range(graph_steps):
             enqueue(i)
 
     def run_steps(k):
-        laps, rest = divmod(k, ring_n)
+        replays, rest = divmod(k, graph_steps)
         with torch.cuda.stream(stream):
-            for _ in range(laps):
+            for _ in range(replays):
                 graph.replay()
             for i in range(rest):
                 enqueue(i)
@@ -390,7 +394,7 @@ def run_native(args) -> None:
         "config": dict(describe(name, kw, "exp delta=1.1 nu=0.7"),
                        parallelism=f"dp{world} (independent sequences, no exchange)",
                        l2=f"ring of {ring_n} distinct step inputs, {ring_n * step_bytes / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2",
-                       launch="CUDA graph of one ring lap, replayed"),
+                       launch=f"CUDA graph of {graph_steps} steps, replayed"),
         "clocks": sampler.summary(),
         "e2e": {"value": B * L * e2e_steps * world / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps, "entry": "csd_verify_host (pinned host buffers)",

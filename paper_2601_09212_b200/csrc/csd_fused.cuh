@@ -927,12 +927,17 @@ struct TopkSmem {
   int n_cand[2];                    // by row parity
   float mom[kTopkWarps][4];        // per warp: sum, sum of squares, count of the sampled values
   float wmax[kTopkWarps];
-  float part_acc[2][kTopkWarps];   // per warp, by row parity: sum of exp(z - max) over kept non-maximum values
-  int part_cmax[2][kTopkWarps];    //                          number of kept values equal to the maximum
+  // per warp, by row parity: sum of exp(z - max) over kept non-maximum values and number of kept values
+  // equal to the maximum; the extra slot takes the values of the bin that holds the threshold
+  float part_acc[2][kTopkWarps + 1];
+  int part_cmax[2][kTopkWarps + 1];
   float part_max[2];
   float part_thr[2];
   int bc_i[4];
-  float bc_f;
+  int arrive[2];                    // warps that have finished the first / the second pass over their lists
+  float row_mx;                     // set by the warp that picks the bin: the row maximum, and whether the
+  int row_fast;                     //   gathered lists can be used for this row
+  unsigned need_exact[(kBlockRows + 31) / 32];   // rows to be selected exactly from global memory, after the loop
   float red_f[kTopkWarps][2];
   RowStats rs;
   int abort;
@@ -1061,8 +1066,11 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
     sm.abort = 0;
     sm.n_cand[0] = 0;
     sm.n_cand[1] = 0;
+    sm.arrive[0] = 0;
+    sm.arrive[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (tid < (kBlockRows + 31) / 32) sm.need_exact[tid] = 0u;
   __syncthreads();
   if (a.ctas_per_seq > 1) cluster_arrive();   // first half; finish_block waits before it writes to a peer
 
@@ -1103,7 +1111,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
     float tot = 0.0f;
     int ctot = 0;
 #pragma unroll
-    for (int w = 0; w < kTopkWarps; ++w) { tot += sm.part_acc[par][w]; ctot += sm.part_cmax[par][w]; }
+    for (int w = 0; w <= kTopkWarps; ++w) { tot += sm.part_acc[par][w]; ctot += sm.part_cmax[par][w]; }
     if (idx < kBlockRows) {
       sm.rs.ms[idx] = make_float2(sm.part_max[par], tot + (float)(ctot - 1));
       sm.rs.thr[idx] = sm.part_thr[par];
@@ -1238,7 +1246,8 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
           }
         }
       }
-      // the row maximum is among the gathered values whenever the fast path applies
+      // ---- first pass over this warp's list: maximum and histogram -----------------------------
+      // (the row maximum is among the gathered values whenever the lists can be used)
       __syncwarp();
       const int wc = sm.wpos[warp];
       if (wc <= kWarpList) {
@@ -1250,40 +1259,83 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
       }
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) mx = max_nan(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-      if (lane == 0) sm.wmax[warp] = mx;
-      __syncthreads();   // ---- B: lists, maxima and histogram complete
-      int n_lo = 0;
-      bool fast = true;
-      mx = sm.wmax[0];
-#pragma unroll
-      for (int w = 0; w < kTopkWarps; ++w) {
-        const int cw = sm.wpos[w];
-        if (cw > kWarpList) fast = false;
-        n_lo += cw;
-        mx = max_nan(mx, sm.wmax[w]);
+      __syncwarp();
+      int last = 0;
+      if (lane == 0) {
+        sm.wmax[warp] = mx;
+        __threadfence_block();
+        last = atomicAdd(&sm.arrive[0], 1) == kTopkWarps - 1 ? 1 : 0;
       }
-      // NaN guesses, NaN / +inf rows and constant rows all fail one of these tests
-      fast = fast && n_lo >= k_top && (mx > lo) && (mx < CSD_POS_INF) && (scale > 0.0f) && (scale < CSD_POS_INF);
-      if (fast) {
-        if (warp == 0) {   // the bin of the k-th largest and the rank of the answer inside it
+      last = __shfl_sync(0xffffffffu, last, 0);
+      if (last) {
+        // The last warp to get here decides for the row: can the lists be used, and if so, which bin
+        // holds the k-th largest and which rank the answer has inside it.
+        if (lane == 0) sm.arrive[0] = 0;
+        __threadfence_block();
+        int n_lo = 0;
+        bool fast = true;
+        float m = sm.wmax[0];
+#pragma unroll
+        for (int w = 0; w < kTopkWarps; ++w) {
+          const int cw = sm.wpos[w];
+          if (cw > kWarpList) fast = false;
+          n_lo += cw;
+          m = max_nan(m, sm.wmax[w]);
+        }
+        // NaN guesses, NaN / +inf rows and constant rows all fail one of these tests
+        fast = fast && n_lo >= k_top && (m > lo) && (m < CSD_POS_INF) && (scale > 0.0f) && (scale < CSD_POS_INF);
+        if (fast) {
           int kk;
           const int bin = warp_pick_bin(sm.hist, k_top, lane, &kk);
           if (lane == 0) { sm.bc_i[0] = bin; sm.bc_i[1] = kk; }
         }
-        __syncthreads();   // ---- C: bin known
+        if (lane == 0) {
+          sm.row_mx = m;
+          sm.row_fast = fast ? 1 : 0;
+          if (!fast && n_my < kBlockRows) atomicOr(&sm.need_exact[n_my >> 5], 1u << (n_my & 31));
+        }
+      }
+      __syncthreads();   // ---- C: decision and bin known
+      if (!sm.row_fast) continue;   // selected exactly after the loop
+      mx = sm.row_mx;
+      {
+        // ---- second pass: statistics of the values above the bin; the bin's own values are set aside
         const int pick_bin = sm.bc_i[0];
+        float acc = 0.0f;
+        int cmax = 0;
         for (int i = lane; i < wc; i += 32) {
           const float v = sm.list[warp][i];
-          if (lin_bin(v, lo, scale) == pick_bin) {
+          const int bv = lin_bin(v, lo, scale);
+          if (bv > pick_bin) {
+            if (v == mx) cmax += 1;
+            else acc += ex2f((v - mx) * kLog2e);
+          } else if (bv == pick_bin) {
             const int slot = atomicAdd(&sm.n_cand[par], 1);
             if (slot < kCandCap) sm.cand[slot] = v;
           }
         }
-        __syncthreads();   // ---- D: candidates complete
-        const int n_cand = sm.n_cand[par];
-        if (n_cand <= kCandCap) {
-          if (warp == 0) {
-            // exact rank among the candidates (two per lane)
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+          acc += __shfl_xor_sync(0xffffffffu, acc, off);
+          cmax += __shfl_xor_sync(0xffffffffu, cmax, off);
+        }
+        __syncwarp();
+        last = 0;
+        if (lane == 0) {
+          sm.part_acc[par][warp] = acc;
+          sm.part_cmax[par][warp] = cmax;
+          __threadfence_block();
+          last = atomicAdd(&sm.arrive[1], 1) == kTopkWarps - 1 ? 1 : 0;
+        }
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+          // The last warp to get here ranks the bin's values exactly (two per lane): the threshold is
+          // the one of rank kk from the top; those not below it join the statistics.  The other warps
+          // have gone on to the next row; its first barrier orders these results before their use.
+          if (lane == 0) sm.arrive[1] = 0;
+          __threadfence_block();
+          const int n_cand = sm.n_cand[par];
+          if (n_cand <= kCandCap) {
             const int kk = sm.bc_i[1];
             const float v0 = lane < n_cand ? sm.cand[lane] : CSD_NEG_INF;
             const float v1 = lane + 32 < n_cand ? sm.cand[lane + 32] : CSD_NEG_INF;
@@ -1297,51 +1349,42 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
             const bool hit1 = lane + 32 < n_cand && gt1 < kk && kk <= ge1;
             const unsigned b0 = __ballot_sync(0xffffffffu, hit0);
             const unsigned b1 = __ballot_sync(0xffffffffu, hit1);
-            const float t = b0 ? __shfl_sync(0xffffffffu, v0, __ffs(b0) - 1)
-                               : __shfl_sync(0xffffffffu, v1, b1 ? __ffs(b1) - 1 : 0);
-            if (lane == 0) sm.bc_f = t;
-          }
-          __syncthreads();   // ---- E: threshold known
-          const float thr = sm.bc_f;
-          // ---- statistics of the kept values of this warp's list -------------------------
-          float acc = 0.0f;
-          int cmax = 0;
-          for (int i = lane; i < wc; i += 32) {
-            const float v = sm.list[warp][i];
-            if (v >= thr) {
-              if (v == mx) cmax += 1;
-              else acc += ex2f((v - mx) * kLog2e);
+            const float thr = b0 ? __shfl_sync(0xffffffffu, v0, __ffs(b0) - 1)
+                                 : __shfl_sync(0xffffffffu, v1, b1 ? __ffs(b1) - 1 : 0);
+            float acc2 = 0.0f;
+            int cmax2 = 0;
+            if (lane < n_cand && v0 >= thr) { if (v0 == mx) cmax2 += 1; else acc2 += ex2f((v0 - mx) * kLog2e); }
+            if (lane + 32 < n_cand && v1 >= thr) { if (v1 == mx) cmax2 += 1; else acc2 += ex2f((v1 - mx) * kLog2e); }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+              acc2 += __shfl_xor_sync(0xffffffffu, acc2, off);
+              cmax2 += __shfl_xor_sync(0xffffffffu, cmax2, off);
             }
+            if (lane == 0) {
+              sm.part_acc[par][kTopkWarps] = acc2;
+              sm.part_cmax[par][kTopkWarps] = cmax2;
+              sm.part_max[par] = mx;
+              sm.part_thr[par] = thr;
+            }
+          } else if (lane == 0 && n_my < kBlockRows) {   // crowded bin
+            atomicOr(&sm.need_exact[n_my >> 5], 1u << (n_my & 31));
           }
-#pragma unroll
-          for (int off = 16; off > 0; off >>= 1) {
-            acc += __shfl_xor_sync(0xffffffffu, acc, off);
-            cmax += __shfl_xor_sync(0xffffffffu, cmax, off);
-          }
-          if (lane == 0) { sm.part_acc[par][warp] = acc; sm.part_cmax[par][warp] = cmax; }
-          if (tid == 0) { sm.part_max[par] = mx; sm.part_thr[par] = thr; }
-          continue;   // the partials are merged after the next row's first barrier
-        }
-        // crowded bin: fall through (the same decision in every thread: n_cand is shared)
-      }
-      // ---- exact select and statistics from global memory (rare) ------------------------------
-      __syncthreads();
-      {
-        float m_e = 0.0f, s_e = 0.0f, thr_e = 0.0f;
-        exact_row_from_global<T, CFG>(row_of(row_id), V, k_top, sm, tid, m_e, s_e, thr_e);
-        if (tid == 0) {
-          // same form as the fast path's partials: one "maximum", the rest in warp 0's slot
-#pragma unroll
-          for (int w = 0; w < kTopkWarps; ++w) { sm.part_acc[par][w] = 0.0f; sm.part_cmax[par][w] = 0; }
-          sm.part_acc[par][0] = s_e;
-          sm.part_cmax[par][0] = 1;
-          sm.part_max[par] = m_e;
-          sm.part_thr[par] = thr_e;
         }
       }
     }
     __syncthreads();
     if (tid == 0 && n_my > 0) stash_row(n_my - 1, (n_my - 1) & 1);
+    // ---- rows whose lists could not be used: exact select and statistics from global memory (rare) ----
+    __syncthreads();
+    for (int r = 0; r < n_my && r < kBlockRows; ++r) {
+      if (((sm.need_exact[r >> 5] >> (r & 31)) & 1u) == 0u) continue;   // the same decision in every thread
+      float m_e = 0.0f, s_e = 0.0f, thr_e = 0.0f;
+      exact_row_from_global<T, CFG>(row_of(row_begin + r), V, k_top, sm, tid, m_e, s_e, thr_e);
+      if (tid == 0) {
+        sm.rs.ms[r] = make_float2(m_e, s_e);
+        sm.rs.thr[r] = thr_e;
+      }
+    }
     if (!ok && tid == 0) {
       sm.abort = 1;
       atomicExch(a.error_flag, 1);
