@@ -1228,19 +1228,30 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         // (the test is "not below lo", so that a NaN lands in the list and marks the row through the
         // maximum).  Two predicated passes, written out so that they stay free of branches: count,
         // reserve the slots with one atomic, store.
-        uint32_t cnt = 0;
+        // Four independent chains (every fourth value each), so that neither the counts nor the
+        // addresses form one long dependent sequence.
+        constexpr int NCH = (VPT % 4 == 0) ? 4 : 1;
+        uint32_t cn[NCH];
+#pragma unroll
+        for (int g = 0; g < NCH; ++g) cn[g] = 0;
 #pragma unroll
         for (int e = 0; e < VPT; ++e)
-          asm("{\n\t.reg .pred p;\n\tsetp.geu.f32 p, %1, %2;\n\t@p add.u32 %0, %0, 1;\n\t}" : "+r"(cnt) : "f"(z[e]), "f"(lo));
+          asm("{\n\t.reg .pred p;\n\tsetp.geu.f32 p, %1, %2;\n\t@p add.u32 %0, %0, 1;\n\t}" : "+r"(cn[e % NCH]) : "f"(z[e]), "f"(lo));
+        uint32_t cnt = cn[0];
+#pragma unroll
+        for (int g = 1; g < NCH; ++g) cnt += cn[g];
         if (cnt > 0) {
           const uint32_t pos = (uint32_t)atomicAdd(&sm.wpos[warp], (int)cnt);
           if (pos + cnt <= (uint32_t)kWarpList) {
-            uint32_t addr = smem_addr(&sm.list[warp][pos]);
+            uint32_t addr[NCH];
+            addr[0] = smem_addr(&sm.list[warp][pos]);
+#pragma unroll
+            for (int g = 1; g < NCH; ++g) addr[g] = addr[g - 1] + 4u * cn[g - 1];
 #pragma unroll
             for (int e = 0; e < VPT; ++e)
               asm volatile(
                   "{\n\t.reg .pred p;\n\tsetp.geu.f32 p, %1, %2;\n\t@p st.shared.f32 [%0], %1;\n\t@p add.u32 %0, %0, 4;\n\t}"
-                  : "+r"(addr)
+                  : "+r"(addr[e % NCH])
                   : "f"(z[e]), "f"(lo)
                   : "memory");
           }
@@ -1251,10 +1262,15 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
       __syncwarp();
       const int wc = sm.wpos[warp];
       if (wc <= kWarpList) {
-        for (int i = lane; i < wc; i += 32) {
-          const float v = sm.list[warp][i];
-          mx = max_nan(mx, v);
-          atomicAdd(&sm.hist[lin_bin(v, lo, scale)], 1);
+        // unrolled over the whole capacity, so that the loads and the bin arithmetic of all slots overlap
+#pragma unroll
+        for (int u = 0; u < kWarpList / 32; ++u) {
+          const int i = lane + 32 * u;
+          if (i < wc) {
+            const float v = sm.list[warp][i];
+            mx = max_nan(mx, v);
+            atomicAdd(&sm.hist[lin_bin(v, lo, scale)], 1);
+          }
         }
       }
 #pragma unroll
@@ -1303,13 +1319,16 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         const int pick_bin = sm.bc_i[0];
         float acc = 0.0f;
         int cmax = 0;
-        for (int i = lane; i < wc; i += 32) {
-          const float v = sm.list[warp][i];
-          const int bv = lin_bin(v, lo, scale);
-          if (bv > pick_bin) {
-            if (v == mx) cmax += 1;
-            else acc += ex2f((v - mx) * kLog2e);
-          } else if (bv == pick_bin) {
+#pragma unroll
+        for (int u = 0; u < kWarpList / 32; ++u) {   // unrolled and branch-free but for the rare bin member
+          const int i = lane + 32 * u;
+          const float v = i < wc ? sm.list[warp][i] : CSD_NEG_INF;   // -inf: below every bin
+          const int bv = i < wc ? lin_bin(v, lo, scale) : -1;
+          const float ev = ex2f((v - mx) * kLog2e);
+          const bool above = bv > pick_bin;
+          acc += (above && v != mx) ? ev : 0.0f;
+          cmax += (above && v == mx) ? 1 : 0;
+          if (bv == pick_bin) {
             const int slot = atomicAdd(&sm.n_cand[par], 1);
             if (slot < kCandCap) sm.cand[slot] = v;
           }
