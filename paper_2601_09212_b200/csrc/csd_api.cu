@@ -316,7 +316,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
       const int eps = kWStageBytes / (es * (cfg ? 2 : 1));
       const long long cpr = (p.V + eps - 1) / eps;
       const long long blocks = c > 1 ? (long long)p.B * c : (p.B + spc - 1) / spc;
-      long long cpp = rows * cpr / (4 * blocks * kPlainWarps);
+      long long cpp = 2 * rows * cpr / (5 * blocks * kPlainWarps);   // about 2.5 items per warp
       if (cpp < 1) cpp = 1;
       if (cpp > 8) cpp = 8;
       if (cpp > cpr) cpp = cpr;

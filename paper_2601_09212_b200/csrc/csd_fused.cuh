@@ -195,7 +195,7 @@ __device__ __forceinline__ BlockShare block_share(const FusedArgs& a) {
 }
 // local row -> (sequence, 0 target / 1 drafter, position)
 __device__ __forceinline__ void local_row(const BlockShare& sh, int r_loc, int gamma, int& b, int& which, int& i) {
-  const int sl = r_loc / sh.rows_per_seq;
+  const int sl = r_loc < sh.rows_per_seq ? 0 : r_loc / sh.rows_per_seq;   // (usually one sequence: no division)
   const int r = r_loc - sl * sh.rows_per_seq;
   b = sh.seq_begin + sl;
   if (r < 2 * (sh.pos_end - sh.pos_begin)) { i = sh.pos_begin + (r >> 1); which = r & 1; }
@@ -432,6 +432,24 @@ __device__ void write_G(const FinishArgs& a, const int b, const int j, const Seq
   }
 }
 
+// Tokens, multipliers and uniforms of the block's positions of its sl-th sequence, into shared memory.
+// Called for the first sequence when the kernel starts, so that these loads are long complete when
+// the accept tests need them.
+__device__ __forceinline__ void stage_inputs(const FusedArgs& ua, const BlockShare& sh, const int sl, const int tid,
+                                             FinishStage& st) {
+  const FinishArgs& a = ua.fin;
+  const int L = a.gamma;
+  const int b = sh.seq_begin + sl;
+  if (b >= sh.seq_end) return;
+  if (tid >= sh.pos_begin && tid < sh.pos_end) {
+    st.tok[tid] = a.tokens[(int64_t)b * L + tid];
+    const float om = a.schedule[tid];
+    st.omega[tid] = om >= 0.0f ? om : 0.0f;
+    st.uni[tid] = a.uniforms[(int64_t)b * (L + 1) + tid];
+  }
+  if (tid == L) st.uni[L] = a.uniforms[(int64_t)b * (L + 1) + L];
+}
+
 // The block's positions [pos_begin, pos_end) of sequence b: accept tests (Eq. relax) and its first
 // rejection (the return value; pos_end if it accepted all of them).  Row statistics come from shared
 // memory (rs, local rows of sequence slot sl).  Leaves p, q, f of its positions in st; reads only the
@@ -444,13 +462,7 @@ __device__ int accept_positions(const FusedArgs& ua, const BlockShare& sh, const
   const int b = sh.seq_begin + sl;
   const int p0 = sh.pos_begin, p1 = sh.pos_end;
   // ---- 0. inputs of these positions and the row statistics, into shared memory -------------------
-  if (tid >= p0 && tid < p1) {
-    st.tok[tid] = a.tokens[(int64_t)b * L + tid];
-    const float om = a.schedule[tid];
-    st.omega[tid] = om >= 0.0f ? om : 0.0f;
-    st.uni[tid] = a.uniforms[(int64_t)b * (L + 1) + tid];
-  }
-  if (tid == L) st.uni[L] = a.uniforms[(int64_t)b * (L + 1) + L];
+  if (sl > 0) stage_inputs(ua, sh, sl, tid, st);   // those of the block's first sequence are staged at kernel start
   if (tid < sh.rows_per_seq) {
     int bb, which, i;
     local_row(sh, sl * sh.rows_per_seq + tid, L, bb, which, i);
@@ -700,22 +712,24 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
 
   // the block's items (parts of its local rows, see block_share), split evenly over its warps
   const BlockShare sh = block_share(a);
+  stage_inputs(a, sh, 0, tid, sm.fst);
   const int n_block = sh.n_rows * parts;
   const int item_begin = (int)((long long)n_block * warp / kPlainWarps);
   const int item_end = (int)((long long)n_block * (warp + 1) / kPlainWarps);
 
   // producer cursor (meaningful in lane 0): the next chunk to copy
   int p_item = item_begin, p_x = 0, p_xend = 0, p_s = 0;
+  int p_row = item_begin / parts, p_part = item_begin - p_row * parts;   // kept incrementally from here on
   const T *p_cond = nullptr, *p_uncond = nullptr;
-  auto producer_open_item = [&]() {   // sets the cursor to the first chunk of p_item
-    const int row_id = p_item / parts;
-    const int part = p_item - row_id * parts;
+  auto producer_open_row = [&]() {    // pointers of row p_row
     int b, which, i;
-    local_row(sh, row_id, f.gamma, b, which, i);
+    local_row(sh, p_row, f.gamma, b, which, i);
     const Row<T, CFG> row = row_at<T, CFG>(f, b, which, i);
     p_cond = row.cond;
     p_uncond = row.uncond;
-    p_x = part * part_elems;
+  };
+  auto producer_open_item = [&]() {   // sets the cursor to the first chunk of part p_part of the open row
+    p_x = p_part * part_elems;
     p_xend = min(V, p_x + part_elems);
   };
   auto producer_issue = [&]() {       // copies one chunk into the next stage of the ring, if any is left
@@ -728,10 +742,12 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
     p_x += EPS;
     if (p_x >= p_xend) {
       ++p_item;
+      if (++p_part == parts) { p_part = 0; ++p_row; if (p_item < item_end) producer_open_row(); }
       if (p_item < item_end) producer_open_item();
     }
   };
   if (lane == 0 && item_begin < item_end) {
+    producer_open_row();
     producer_open_item();
     for (int s = 0; s < kWStages; ++s) producer_issue();
   }
@@ -752,10 +768,10 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
     bool ok = true;
     int cur_row = -1, tok_cur = -1, tok_next = -1;
     const int last_row = item_end > item_begin ? (item_end - 1) / parts : -1;
-    if (item_begin < item_end) tok_next = token_of_row(item_begin / parts);
-    for (int item = item_begin; item < item_end; ++item, ++n_my) {
-      const int row_id = item / parts;
-      const int part = item - row_id * parts;
+    int row_id = item_begin / parts, part = item_begin - row_id * parts;   // kept incrementally
+    if (item_begin < item_end) tok_next = token_of_row(row_id);
+    for (int item = item_begin; item < item_end; ++item, ++n_my, ++part) {
+      if (part == parts) { part = 0; ++row_id; }
       const int x_begin = part * part_elems;
       const int x_end = min(V, x_begin + part_elems);
       if (row_id != cur_row) {
@@ -1076,6 +1092,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
 
   // this block's local rows (see block_share)
   const BlockShare sh = block_share(a);
+  stage_inputs(a, sh, 0, tid, sm.fst);
   const int row_begin = 0, row_end = sh.n_rows;
 
   auto row_of = [&](int row_id) -> Row<T, CFG> {
