@@ -43,7 +43,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
 # one ncu capture, see profiles/verify_topk_kernel_C3.md).  Reported only while the kernel sources
 # still have the digest the capture was taken with; null otherwise.
-NCU_TRAFFIC = {"sources_sha256": "45b5c0f7d3192803", "workload": "C3", "bytes_per_launch": 68209664}
+NCU_TRAFFIC = {"sources_sha256": "c7103d0b4c29dc9b", "workload": "C3", "bytes_per_launch": 68064768}
 
 
 def sources_digest() -> str:
