@@ -127,7 +127,7 @@ int csd_verify(const float* target_logits, const float* draft_logits, const int3
  *   - Problems whose csd_workspace_size(B, gamma, V, CSD_F32) exceeds
  *     CSD_STATIC_SCRATCH_BYTES are refused with CSD_ERR_STATIC_LIMIT before
  *     anything is enqueued (for scale: B=256, gamma=16, V=16384 needs about
- *     1.6 MB and fits; B=512, gamma=8, V=16384 needs 2.2 MB and does not).
+ *     1.1 MB and fits; B=512, gamma=16, V=16384 needs 2.2 MB and does not).
  *   - The first call on each device looks up the device address of the array
  *     (a cudaGetSymbolAddress call, made with that device current) and keeps
  *     it; make that first call outside any stream capture.
