@@ -185,6 +185,15 @@ typedef struct csd_params {
                                   overlap on the GPU need different workspaces.             */
   size_t workspace_bytes;
   void* stream;
+  int single_call_latency;     /* How the work of one call is spread over the GPU.
+                                  0 (default): for the throughput of calls enqueued back to back on
+                                  a stream -- one thread block per sequence once B >= 16, so that
+                                  the blocks of many consecutive calls share the GPU (a call's
+                                  streaming overlaps its predecessors' through programmatic
+                                  dependent launch; outputs still appear in call order).
+                                  1: for the latency of a call that runs alone -- each sequence is
+                                  split over up to 8 blocks until the GPU is full.  Results are
+                                  identical either way.                                          */
 } csd_params;
 
 int csd_verify_ex(const csd_params* p);

@@ -294,14 +294,19 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
     ua.top_k = p.top_k;
     ua.lo_sigmas = nanf("");
     ua.error_flag = reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
-    // Blocks are aligned with sequences and positions: either a sequence's draft positions are split
-    // over the ctas_per_seq blocks of one cluster (each with both rows of its positions; 2, 4 or 8
-    // blocks), or a block owns seqs_per_cta whole sequences.
-    const long long target_blocks = 2LL * sms;
+    // Blocks are aligned with sequences and positions: a block owns a whole sequence; or, for very
+    // large batches, seqs_per_cta whole sequences; or a sequence's draft positions are split over the
+    // ctas_per_seq blocks of one cluster (each with both rows of its positions; 2, 4 or 8 blocks).
+    // Consecutive calls overlap on the GPU as deeply as their grids allow (a call may start once every
+    // block of its predecessor has started), so for throughput few long-lived blocks per call are
+    // best: one per sequence, split only when the batch is too small to give 16 blocks.  For the
+    // latency of a single call the sequences are split until the GPU is full.
+    const long long fill_blocks = 2LL * sms;
+    const long long split_below = p.single_call_latency ? fill_blocks : 16;
     long long c = 1, spc = 1;
-    if (p.B >= target_blocks) spc = (p.B + target_blocks - 1) / target_blocks;
-    else {
-      const long long want = target_blocks / p.B;
+    if (p.B > fill_blocks) spc = (p.B + fill_blocks - 1) / fill_blocks;
+    else if (p.B < split_below) {
+      const long long want = split_below / p.B;
       while (2 * c <= want && 2 * c <= p.gamma && 2 * c <= kMaxCluster) c *= 2;
     }
     while (spc > 1 && spc * rows_per_seq > kBlockRows) --spc;   // rows_per_seq <= 65 < kBlockRows

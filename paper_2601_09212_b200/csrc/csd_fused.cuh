@@ -459,7 +459,6 @@ __device__ int accept_positions(const FusedArgs& ua, const BlockShare& sh, const
                                 const int tid, FinishSmem& sm, FinishStage& st) {
   const FinishArgs& a = ua.fin;
   const int L = a.gamma, V = a.V;
-  const int b = sh.seq_begin + sl;
   const int p0 = sh.pos_begin, p1 = sh.pos_end;
   // ---- 0. inputs of these positions and the row statistics, into shared memory -------------------
   if (sl > 0) stage_inputs(ua, sh, sl, tid, st);   // those of the block's first sequence are staged at kernel start
@@ -515,7 +514,7 @@ __device__ int accept_positions(const FusedArgs& ua, const BlockShare& sh, const
 // The draw at the block's first rejection j (Eq. opt_G) -- or, with j == pos_end in the block that
 // owns the bonus row, the bonus draw.  Follows accept_positions of the same sequence; leaves the
 // record in st.rec.
-template <typename T, bool CFG, int NT>
+template <typename T, bool CFG, int NT, bool FILT>
 __device__ void draw_position(const FusedArgs& ua, const BlockShare& sh, const int sl, int j, const int tid,
                               unsigned char* ring, const int ring_bytes, double* tile_sums, FinishSmem& sm,
                               FinishStage& st, uint32_t& phase, const int extra_status) {
@@ -549,10 +548,8 @@ __device__ void draw_position(const FusedArgs& ua, const BlockShare& sh, const i
     rt.thr = sm.thr[0][j];
     if (j < L) { rd = row_at<T, CFG>(a, b, 1, j); rd.thr = sm.thr[1][j]; }
     else rd = rt;
-    token = a.use_topk ? draw_token<T, CFG, NT, true>(a, rt, rd, ctx, st.uni[L], tid, ring, ring_bytes, tile_sums, sm,
-                                                      st, phase, status, Z)
-                       : draw_token<T, CFG, NT, false>(a, rt, rd, ctx, st.uni[L], tid, ring, ring_bytes, tile_sums, sm,
-                                                       st, phase, status, Z);
+    token = draw_token<T, CFG, NT, FILT>(a, rt, rd, ctx, st.uni[L], tid, ring, ring_bytes, tile_sums, sm, st, phase,
+                                         status, Z);
   }
   if (tid == 0) {
     SeqRecord& rec = st.rec;
@@ -604,7 +601,7 @@ __device__ void emit_sequence(const FusedArgs& ua, const int b, const SeqRecord&
 // first rejection (or that there is none: then the last block, which owns the bonus row).  That block
 // alone draws the token and emits the sequence; the others are done.  No block reads a peer's shared
 // memory, and none writes to it after the barrier, so blocks leave independently.
-template <typename T, bool CFG, int NT>
+template <typename T, bool CFG, int NT, bool FILT>
 __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const RowStats& rs, const int tid,
                              const bool aborted, unsigned char* ring, const int ring_bytes, double* tile_sums,
                              FinishSmem& sm, FinishStage& st) {
@@ -625,7 +622,7 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
     for (int sl = 0; sl < sh.seq_end - sh.seq_begin; ++sl) {
       const int b = sh.seq_begin + sl;
       const int j = accept_positions<T, CFG, NT>(ua, sh, sl, rs, tid, sm, st);
-      draw_position<T, CFG, NT>(ua, sh, sl, j, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
+      draw_position<T, CFG, NT, FILT>(ua, sh, sl, j, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
       if (sl == 0) {   // before the block's first global write: outputs of consecutive calls stay in order
         pdl_wait();
         sticky = __ldcg(ua.error_flag) ? 8 : 0;
@@ -655,7 +652,7 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
     if (a.dbg_p || a.dbg_q || a.dbg_f) { pdl_wait(); write_pqf(b); }
     return;
   }
-  draw_position<T, CFG, NT>(ua, sh, 0, j, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
+  draw_position<T, CFG, NT, FILT>(ua, sh, 0, j, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
   pdl_wait();   // the previous call has completed: outputs of consecutive calls stay in order
   if (__ldcg(ua.error_flag)) any = 8;
   write_pqf(b);
@@ -913,7 +910,7 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
     if (lane == 0) { sm.rs.ms[r] = make_float2(m, s_acc); sm.rs.thr[r] = CSD_NEG_INF; }
   }
   __syncthreads();
-  finish_block<T, CFG, kPlainThreads>(a, sh, sm.rs, tid, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes,
+  finish_block<T, CFG, kPlainThreads, false>(a, sh, sm.rs, tid, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes,
                                       sm.tile_sums, sm.fin, sm.fst);
 }
 
@@ -1433,7 +1430,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   // ================================= phase 2 ===========================================
   __syncthreads();
   static_assert(sizeof(sm.list) >= kFinTiles * sizeof(double), "tile sums live in the list area");
-  finish_block<T, CFG, kTopkThreads>(a, sh, sm.rs, tid, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
+  finish_block<T, CFG, kTopkThreads, true>(a, sh, sm.rs, tid, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
                                      reinterpret_cast<double*>(&sm.list[0][0]), sm.fin, sm.fst);
 }
 

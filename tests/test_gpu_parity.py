@@ -145,6 +145,26 @@ def test_topk_with_masked_and_tied_rows():
     assert_ok(rep)
 
 
+@pytest.mark.parametrize("kw", [
+    dict(B=64, gamma=8, V=16384, dtype=W.F32),
+    dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000),
+    dict(B=40, gamma=16, V=8192, dtype=W.BF16, bonus_row=True),
+    dict(B=3, gamma=7, V=32768, dtype=W.F32, bonus_row=True, top_k=50),
+    dict(B=24, gamma=5, V=4100, dtype=W.BF16),
+])
+def test_single_call_latency_partition(kw):
+    """The partition for the latency of one call (sequences split over the blocks of a cluster)
+    against the oracle, and against the default partition: identical integer outputs."""
+    L = kw["gamma"]
+    w = W.make("t", rho=0.9, schedule=sched(L), seed=77, device=DEV, **kw)
+    rep, got, ref = check(w, single_call_latency=True)
+    assert_ok(rep)
+    base = run_gpu(w, want_dbg=False)
+    assert np.array_equal(got["tokens"], base["tokens"])
+    assert np.array_equal(got["accept_len"], base["accept_len"])
+    assert np.array_equal(got["status"], base["status"])
+
+
 def test_config_c3_guidance_and_topk():
     """B=64, gamma=8, V=16384, bf16, guidance mix s=4 fused into the load, top-k 1000."""
     L = W.CONFIGS["C3"]["gamma"]
@@ -155,13 +175,16 @@ def test_config_c3_guidance_and_topk():
         print("C3", rep.summary())
 
 
-@pytest.mark.parametrize("name,kw", [
-    ("late-trigger plain", dict(B=16, gamma=8, V=16384, dtype=W.F32)),
-    ("early-trigger plain", dict(B=64, gamma=8, V=16384, dtype=W.F32)),
-    ("top-k with guidance", dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000)),
-    ("several sequences per block", dict(B=600, gamma=2, V=2048, dtype=W.BF16)),
+@pytest.mark.parametrize("name,kw,lat", [
+    ("plain, one block per sequence", dict(B=16, gamma=8, V=16384, dtype=W.F32), False),
+    ("plain, clusters of 8", dict(B=16, gamma=8, V=16384, dtype=W.F32), True),
+    ("plain, clusters of 4", dict(B=64, gamma=8, V=16384, dtype=W.F32), True),
+    ("plain, clusters of 2, small batch", dict(B=8, gamma=8, V=16384, dtype=W.BF16), False),
+    ("top-k with guidance, one block per sequence", dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000), False),
+    ("top-k with guidance, clusters of 4", dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000), True),
+    ("several sequences per block", dict(B=600, gamma=2, V=2048, dtype=W.BF16), False),
 ])
-def test_back_to_back_calls_on_one_stream(name, kw):
+def test_back_to_back_calls_on_one_stream(name, kw, lat):
     """Consecutive calls overlap on the device (programmatic dependent launch) and share ONE
     workspace and ONE set of output buffers per slot; every call's results must equal those of
     the same call run alone, both when enqueued directly and when replayed as a CUDA graph."""
@@ -177,7 +200,7 @@ def test_back_to_back_calls_on_one_stream(name, kw):
     prms = [csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
                             o["tok"], o["tau"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
                             cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=o["st"], workspace=ws_shared,
-                            stream=stream) for w, o in zip(steps, outs)]
+                            stream=stream, single_call_latency=lat) for w, o in zip(steps, outs)]
 
     def check_all(tag):
         for i, (o, ref) in enumerate(zip(outs, alone)):
