@@ -29,6 +29,8 @@
 //                        and selected exactly by radix, so the result never
 //                        depends on the guess.
 #pragma once
+#include <type_traits>
+
 #include "csd_kernels.cuh"
 
 namespace csd {
@@ -1248,9 +1250,17 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         uint32_t cn[NCH];
 #pragma unroll
         for (int g = 0; g < NCH; ++g) cn[g] = 0;
+        // (count: two comparisons that give all-ones or zero, subtracted by one three-input add)
 #pragma unroll
-        for (int e = 0; e < VPT; ++e)
-          asm("{\n\t.reg .pred p;\n\tsetp.geu.f32 p, %1, %2;\n\t@p add.u32 %0, %0, 1;\n\t}" : "+r"(cn[e % NCH]) : "f"(z[e]), "f"(lo));
+        for (int e = 0; e + 2 * NCH <= VPT; e += 2 * NCH) {
+#pragma unroll
+          for (int g = 0; g < NCH; ++g)
+            asm("{\n\t.reg .u32 a, b;\n\tset.geu.u32.f32 a, %1, %3;\n\tset.geu.u32.f32 b, %2, %3;\n\t"
+                "sub.u32 %0, %0, a;\n\tsub.u32 %0, %0, b;\n\t}"
+                : "+r"(cn[g])
+                : "f"(z[e + g]), "f"(z[e + NCH + g]), "f"(lo));
+        }
+        static_assert(VPT % (2 * NCH) == 0, "the count takes the values in pairs per chain");
         uint32_t cnt = cn[0];
 #pragma unroll
         for (int g = 1; g < NCH; ++g) cnt += cn[g];
@@ -1275,10 +1285,12 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
       // (the row maximum is among the gathered values whenever the lists can be used)
       __syncwarp();
       const int wc = sm.wpos[warp];
-      if (wc <= kWarpList) {
-        // unrolled over the whole capacity, so that the loads and the bin arithmetic of all slots overlap
+      // Both passes over the list are unrolled over its slots (so that the loads and the bin
+      // arithmetic of all slots overlap), in two versions: three quarters of the capacity, which is
+      // what a list normally holds, and all of it.
+      auto first_pass = [&](auto nslots) {
 #pragma unroll
-        for (int u = 0; u < kWarpList / 32; ++u) {
+        for (int u = 0; u < decltype(nslots)::value; ++u) {
           const int i = lane + 32 * u;
           if (i < wc) {
             const float v = sm.list[warp][i];
@@ -1286,7 +1298,10 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
             atomicAdd(&sm.hist[lin_bin(v, lo, scale)], 1);
           }
         }
-      }
+      };
+      constexpr int kSlotsAll = kWarpList / 32, kSlotsUsual = (3 * kSlotsAll) / 4;
+      if (wc <= 32 * kSlotsUsual) first_pass(std::integral_constant<int, kSlotsUsual>());
+      else if (wc <= kWarpList) first_pass(std::integral_constant<int, kSlotsAll>());
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) mx = max_nan(mx, __shfl_xor_sync(0xffffffffu, mx, off));
       __syncwarp();
@@ -1333,20 +1348,24 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         const int pick_bin = sm.bc_i[0];
         float acc = 0.0f;
         int cmax = 0;
+        auto second_pass = [&](auto nslots) {   // branch-free but for the rare bin member
 #pragma unroll
-        for (int u = 0; u < kWarpList / 32; ++u) {   // unrolled and branch-free but for the rare bin member
-          const int i = lane + 32 * u;
-          const float v = i < wc ? sm.list[warp][i] : CSD_NEG_INF;   // -inf: below every bin
-          const int bv = i < wc ? lin_bin(v, lo, scale) : -1;
-          const float ev = ex2f((v - mx) * kLog2e);
-          const bool above = bv > pick_bin;
-          acc += (above && v != mx) ? ev : 0.0f;
-          cmax += (above && v == mx) ? 1 : 0;
-          if (bv == pick_bin) {
-            const int slot = atomicAdd(&sm.n_cand[par], 1);
-            if (slot < kCandCap) sm.cand[slot] = v;
+          for (int u = 0; u < decltype(nslots)::value; ++u) {
+            const int i = lane + 32 * u;
+            const float v = i < wc ? sm.list[warp][i] : CSD_NEG_INF;   // -inf: below every bin
+            const int bv = i < wc ? lin_bin(v, lo, scale) : -1;
+            const float ev = ex2f((v - mx) * kLog2e);
+            const bool above = bv > pick_bin;
+            acc += (above && v != mx) ? ev : 0.0f;
+            cmax += (above && v == mx) ? 1 : 0;
+            if (bv == pick_bin) {
+              const int slot = atomicAdd(&sm.n_cand[par], 1);
+              if (slot < kCandCap) sm.cand[slot] = v;
+            }
           }
-        }
+        };
+        if (wc <= 32 * kSlotsUsual) second_pass(std::integral_constant<int, kSlotsUsual>());
+        else second_pass(std::integral_constant<int, kSlotsAll>());
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
           acc += __shfl_xor_sync(0xffffffffu, acc, off);
