@@ -69,6 +69,7 @@ typedef enum {
 
 /* Bits of out_status[b]; they refer only to positions the algorithm looked at
  * (1..tau+1 and the bonus row), like the sequential loop of Algorithm 1. */
+/* Finite logits are expected within +-1e37: the exponent arithmetic multiplies them by log2(e). */
 typedef enum {
   CSD_STATUS_BADROW = 1,   /* a row held NaN or +inf, or no finite entry: that position
                               rejects (f := 0).  An unusable drafter row resamples from

@@ -786,7 +786,11 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
       // Because the reference is warp-uniform, a group of values below it is summed with no
       // test per value, and the exact treatment of values equal to it is a uniform branch
       // taken only where the maximum sits.
+      // The exponent (z - Mw) log2(e) is formed by one fused multiply-add, z * log2(e) - MwL with MwL
+      // the ROUNDED product Mw * log2(e); its rounding error dlt = Mw * log2(e) - MwL (exact, again by
+      // a fused multiply-add) is a common factor 2^dlt of the sum and is divided out once per item.
       float Mw = CSD_NEG_INF, s_run = 0.0f;
+      float nMwL = CSD_POS_INF, dlt = 0.0f;   // -MwL and dlt of the current reference
       int cnt_run = 0;
       for (int x0 = x_begin; x0 < x_end; x0 += EPS) {
         if (ok && !mbar_wait(&sm.full[warp][c_s], c_par)) ok = false;
@@ -847,21 +851,25 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
           key ^= (key >> 31) & 0x7fffffff;
           const float wm = __int_as_float(key);
           if (wm > Mw) {   // a new maximum: what was counted as "equal to the maximum" becomes ordinary mass
-            s_run = (s_run + (float)cnt_run) * ex2f((Mw - wm) * kLog2e);
+            const float MwL = wm * kLog2e;
+            const float dlt_new = fmaf(wm, kLog2e, -MwL);
+            s_run = (s_run * ex2f(-dlt) + (float)cnt_run) * ex2f((Mw - wm) * kLog2e) * ex2f(dlt_new);
             cnt_run = 0;
             Mw = wm;
+            nMwL = -MwL;
+            dlt = dlt_new;
           }
           if (wm == Mw) {
             // values equal to the reference may be present: they are counted, not summed
 #pragma unroll
             for (int e = 0; e < GV * VEC; ++e) {
-              const float ex = ex2f((vals[e] - Mw) * kLog2e);
+              const float ex = ex2f(fmaf(vals[e], kLog2e, nMwL));
               if (vals[e] == Mw) cnt_run += 1; else s_run += ex;   // NaN values poison s_run, which marks the row
             }
           } else {
             float acc4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-            for (int e = 0; e < GV * VEC; ++e) acc4[e & 3] += ex2f((vals[e] - Mw) * kLog2e);
+            for (int e = 0; e < GV * VEC; ++e) acc4[e & 3] += ex2f(fmaf(vals[e], kLog2e, nMwL));
             s_run += (acc4[0] + acc4[1]) + (acc4[2] + acc4[3]);
           }
         }
@@ -886,7 +894,7 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
         cnt_run += __shfl_xor_sync(0xffffffffu, cnt_run, off);
       }
       if (lane == 0 && item < kBlockStash) {
-        sm.stash[item] = make_float2(Mw, s_run + (float)(cnt_run - 1));
+        sm.stash[item] = make_float2(Mw, s_run * ex2f(-dlt) + (float)(cnt_run - 1));
         if (has_tok && row_id < kBlockRows) sm.rs.tokz[row_id] = tokz;
       }
     }
