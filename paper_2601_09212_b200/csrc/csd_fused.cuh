@@ -290,16 +290,14 @@ __device__ int draw_token(const FinishArgs& a, const Row<T, CFG>& rt, const Row<
             if (CFG) {
               float zu[VEC];
               unpack_vec<T>(ring + slot_bytes + xo * ES, zu);
-#pragma unroll
-              for (int k = 0; k < VEC; ++k) zt[k] = cfg_mix(zt[k], zu[k], a.cfg_scale);
+              cfg_mix_vec<VEC>(zt, zu, a.cfg_scale);
             }
             if (ctx.mode == 0) {
               unpack_vec<T>(ring + ARR * slot_bytes + xo * ES, zd);
               if (CFG) {
                 float zu[VEC];
                 unpack_vec<T>(ring + (ARR + 1) * slot_bytes + xo * ES, zu);
-#pragma unroll
-                for (int k = 0; k < VEC; ++k) zd[k] = cfg_mix(zd[k], zu[k], a.cfg_scale);
+                cfg_mix_vec<VEC>(zd, zu, a.cfg_scale);
               }
             }
             float acc = 0.0f;
@@ -829,8 +827,7 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
                 if (CFG) {
                   float zu[VEC];
                   unpack_vec<T>(stage + kWStageBytes / 2 + xo * (int)sizeof(T), zu);
-#pragma unroll
-                  for (int e = 0; e < VEC; ++e) zc[e] = cfg_mix(zc[e], zu[e], f.cfg_scale);
+                  cfg_mix_vec<VEC>(zc, zu, f.cfg_scale);
                 }
               } else {
 #pragma unroll
@@ -1173,8 +1170,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
             if (CFG) {
               float zu[VEC];
               unpack_vec<T>(&sm.ring[s][kTkStageBytes / 2 + xo * (int)sizeof(T)], zu);
-#pragma unroll
-              for (int e = 0; e < VEC; ++e) zc[e] = cfg_mix(zc[e], zu[e], f.cfg_scale);
+              cfg_mix_vec<VEC>(zc, zu, f.cfg_scale);
             }
 #pragma unroll
             for (int e = 0; e < VEC; ++e) z[v * VEC + e] = zc[e];
@@ -1189,8 +1185,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
               if (CFG) {
                 float zu[VEC];
                 unpack_vec<T>(&sm.ring[s][kTkStageBytes / 2 + xo * (int)sizeof(T)], zu);
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) zc[e] = cfg_mix(zc[e], zu[e], f.cfg_scale);
+                cfg_mix_vec<VEC>(zc, zu, f.cfg_scale);
               }
             } else {
 #pragma unroll

@@ -110,6 +110,38 @@ __device__ __forceinline__ float cfg_mix(float c, float u, float s) {
   return __fmaf_rn(s, __fsub_rn(c, u), u);
 }
 
+// ---- two fp32 operations per instruction (packed fp32 pairs in 64-bit registers) -----------------
+// Each half is the IEEE operation, so results are bit-identical to the scalar forms.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// cfg_mix of VEC values in pairs: c - u as fma(u, -1, c) (one rounding, like the subtraction)
+template <int VEC>
+__device__ __forceinline__ void cfg_mix_vec(float (&c)[VEC], const float (&u)[VEC], float s) {
+  const uint64_t s2 = pack2(s, s), m1 = pack2(-1.0f, -1.0f);
+#pragma unroll
+  for (int k = 0; k < VEC; k += 2) {
+    const uint64_t u2 = pack2(u[k], u[k + 1]);
+    const uint64_t d2 = fma2(u2, m1, pack2(c[k], c[k + 1]));
+    unpack2(fma2(s2, d2, u2), c[k], c[k + 1]);
+  }
+}
+
 // One logical row: conditional array, optional unconditional array, optional
 // top-k threshold.  Loads VEC consecutive logits starting at element x0.
 template <typename T, bool CFG>
@@ -125,8 +157,7 @@ struct Row {
     if (CFG) {
       float u[kVec];
       Elem<T>::load_vec(uncond + x0, u);
-#pragma unroll
-      for (int k = 0; k < kVec; ++k) z[k] = cfg_mix(z[k], u[k], scale);
+      cfg_mix_vec<kVec>(z, u, scale);
     }
   }
   __device__ __forceinline__ float load_one(int x) const {
