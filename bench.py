@@ -43,7 +43,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
 # one ncu capture, see profiles/verify_topk_kernel_C3.md).  Reported only while the kernel sources
 # still have the digest the capture was taken with; null otherwise.
-NCU_TRAFFIC = {"sources_sha256": "c7103d0b4c29dc9b", "workload": "C3", "bytes_per_launch": 68064768}
+NCU_TRAFFIC = {"sources_sha256": "0b78236a6d63017b", "workload": "C3", "bytes_per_launch": 68067840}
 
 
 def sources_digest() -> str:
@@ -290,7 +290,8 @@ def run_native(args) -> None:
     prms = [csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
                             o["tok"], o["tau"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
                             cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=o["st"], workspace=o["ws"],
-                            stream=stream) for w, o in zip(ring, outs)]
+                            stream=stream, single_call_latency=args.single_call_latency)
+            for w, o in zip(ring, outs)]
     kernels_per_step = csd.csd_launch_count(prms[0])
 
     def enqueue(i):
@@ -385,7 +386,7 @@ def run_native(args) -> None:
     achieved = step_bytes / step_s / 1e9
     digest = sources_digest()
     traffic = None
-    if NCU_TRAFFIC["sources_sha256"] == digest and NCU_TRAFFIC["workload"] == name:
+    if NCU_TRAFFIC["sources_sha256"] == digest and NCU_TRAFFIC["workload"] == name and not args.single_call_latency:
         traffic = NCU_TRAFFIC["bytes_per_launch"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -394,7 +395,8 @@ def run_native(args) -> None:
         "config": dict(describe(name, kw, "exp delta=1.1 nu=0.7"),
                        parallelism=f"dp{world} (independent sequences, no exchange)",
                        l2=f"ring of {ring_n} distinct step inputs, {ring_n * step_bytes / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2",
-                       launch=f"CUDA graph of {graph_steps} steps, replayed"),
+                       launch=f"CUDA graph of {graph_steps} steps, replayed",
+                       partition="per-call latency" if args.single_call_latency else "throughput (default)"),
         "clocks": sampler.summary(),
         "e2e": {"value": B * L * e2e_steps * world / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps, "entry": "csd_verify_host (pinned host buffers)",
@@ -424,6 +426,8 @@ def run_native(args) -> None:
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--single-call-latency", action="store_true",
+                    help="spread each call over the whole GPU (csd_params.single_call_latency = 1)")
     ap.add_argument("--steps", type=int, default=5760)
     ap.add_argument("--warmup", type=int, default=64)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
