@@ -17,7 +17,7 @@ namespace {
 using namespace csd;
 
 static_assert(sizeof(TopkSmem) <= 55 * 1024, "four blocks of the top-k kernel per SM must fit");
-static_assert(sizeof(PlainSmem) <= 112 * 1024, "two blocks of the plain kernel per SM must fit");
+static_assert(sizeof(PlainSmem) <= 75 * 1024, "three blocks of the plain kernel per SM must fit");
 
 constexpr int kMaxV = 1 << 20;
 constexpr int kMaxDevices = 64;

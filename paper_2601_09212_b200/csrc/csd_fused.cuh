@@ -35,7 +35,7 @@
 
 namespace csd {
 
-constexpr int kPlainThreads = 384;   // plain kernel: 12 independent warp pipelines, two blocks per SM
+constexpr int kPlainThreads = 256;   // plain kernel: 8 independent warp pipelines, three blocks per SM
 constexpr int kPlainWarps = kPlainThreads / 32;
 constexpr int kTopkThreads = 256;    // top-k kernel: 8 warps per row, four blocks per SM
 constexpr int kTopkWarps = kTopkThreads / 32;
@@ -662,7 +662,7 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
 // ======================= plain kernel: one pipeline per warp ============================
 // A warp owns a contiguous range of items (an item is a part of a row: chunks_per_part warp
 // stages), a private ring of kWStages stages of kWStageBytes, issues its own refills, and keeps
-// a running (m, s) per lane that it reduces once per item.  Twelve such pipelines per block sit
+// a running (m, s) per lane that it reduces once per item.  Eight such pipelines per block sit
 // at different points of their loops and hide each other's latencies; phase 1 has no block-wide
 // step at all.
 constexpr int kWStages = 3;
@@ -673,16 +673,17 @@ constexpr int kPlainRingBytes = kPlainWarps * kWStages * kWStageBytes;
 struct PlainSmem {
   alignas(128) unsigned char ring[kPlainWarps][kWStages][kWStageBytes];
   alignas(8) uint64_t full[kPlainWarps][kWStages];
-  float2 stash[kBlockStash];   // (m, s) per item, by local item index
+  alignas(8) float2 stash[kBlockStash];   // (m, s) per item, by local item index; after the rows' parts have
+                                          // been merged, the draw keeps its tile sums here
   RowStats rs;
   int abort;
   FinishSmem fin;
   FinishStage fst;
-  double tile_sums[kFinTiles];
 };
+static_assert(sizeof(float2) * kBlockStash >= sizeof(double) * kFinTiles, "tile sums live in the stash");
 
 template <typename T, bool CFG>
-__global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const FusedArgs a) {
+__global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const FusedArgs a) {
   constexpr int VEC = Elem<T>::kVec;
   constexpr int ARR = CFG ? 2 : 1;
   constexpr int EPS = kWStageBytes / ((int)sizeof(T) * ARR);   // elements of a row per warp stage
@@ -918,7 +919,7 @@ __global__ void __launch_bounds__(kPlainThreads, 2) verify_plain_kernel(const Fu
   }
   __syncthreads();
   finish_block<T, CFG, kPlainThreads, false>(a, sh, sm.rs, tid, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes,
-                                      sm.tile_sums, sm.fin, sm.fst);
+                                      reinterpret_cast<double*>(&sm.stash[0]), sm.fin, sm.fst);
 }
 
 // ======================= top-k kernel: a block streams whole rows ========================
