@@ -165,6 +165,23 @@ def test_single_call_latency_partition(kw):
     assert np.array_equal(got["status"], base["status"])
 
 
+@pytest.mark.parametrize("kw", [
+    dict(B=4, gamma=3, V=65536, dtype=W.BF16, bonus_row=True),
+    dict(B=2, gamma=2, V=131072, dtype=W.F32),                      # the last size of the single-launch path (fp32)
+    dict(B=2, gamma=2, V=131076, dtype=W.F32),                      # one tile more: multi-launch path
+    dict(B=2, gamma=3, V=262144, dtype=W.BF16, top_k=1000),
+    dict(B=1, gamma=2, V=2 ** 20, dtype=W.F32, bonus_row=True),     # the largest vocabulary accepted
+    dict(B=1, gamma=2, V=2 ** 20, dtype=W.BF16, top_k=50),
+    dict(B=1, gamma=16, V=8192, dtype=W.F32, bonus_row=True),       # clusters of 8 with single_call_latency
+])
+def test_large_vocabularies_and_limits(kw):
+    L = kw["gamma"]
+    w = W.make("t", rho=0.9, schedule=sched(L), seed=5, device=DEV, **kw)
+    for lat in (False, True):
+        rep, got, ref = check(w, single_call_latency=lat)
+        assert_ok(rep)
+
+
 def test_config_c3_guidance_and_topk():
     """B=64, gamma=8, V=16384, bf16, guidance mix s=4 fused into the load, top-k 1000."""
     L = W.CONFIGS["C3"]["gamma"]
