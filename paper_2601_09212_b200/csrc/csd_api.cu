@@ -653,6 +653,6 @@ const char* csd_error_string(int code) {
   }
 }
 
-int csd_version(void) { return 200; }
+int csd_version(void) { return 300; }
 
 }  // extern "C"
