@@ -216,7 +216,9 @@ int csd_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  * Host-buffer form: the same round for a caller whose logits, tokens, uniforms
  * and schedule sit in HOST memory (pinned memory makes the copies asynchronous).
  * Every data pointer of `host` (inputs, outputs, optional diagnostics) is a
- * HOST pointer; host->workspace / workspace_bytes are ignored.  `staging` is a
+ * HOST pointer; host->workspace / workspace_bytes and single_call_latency are
+ * ignored (between its copies the kernel runs alone, so it is always spread over
+ * the whole GPU).  `staging` is a
  * DEVICE buffer of at least csd_host_staging_size(host) bytes, 256-byte
  * aligned, that the library uses for the device copies of inputs and outputs
  * and for its workspace.  The call enqueues host->device copies, the kernels and

@@ -592,6 +592,7 @@ int csd_verify_host(const csd_params* host, void* staging, size_t staging_bytes)
   d.dbg_G = h.dbg_G ? (float*)(base + pl.off_G) : nullptr;
   d.workspace = base + pl.off_ws;
   d.workspace_bytes = pl.ws_bytes;
+  d.single_call_latency = 1;   // between the copies over the bus the kernel runs alone
   if (cudaMemsetAsync(d.workspace, 0, layout_for(h.B, h.gamma, h.V, h.dtype).zero_bytes, stream) != cudaSuccess)
     return CSD_ERR_LAUNCH;
   const int rc = verify_impl(d);
