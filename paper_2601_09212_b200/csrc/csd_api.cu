@@ -301,10 +301,10 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
     // block of its predecessor has started), so for throughput few long-lived blocks per call are
     // best: one per sequence, split only when the batch is too small to give 16 blocks.  For the
     // latency of a single call the sequences are split until the GPU is full.
-    const long long fill_blocks = 2LL * sms;
-    const long long split_below = p.single_call_latency ? fill_blocks : 16;
+    const long long merge_above = 8LL * sms;   // beyond this many sequences a block takes several
+    const long long split_below = p.single_call_latency ? 2LL * sms : 16;
     long long c = 1, spc = 1;
-    if (p.B > fill_blocks) spc = (p.B + fill_blocks - 1) / fill_blocks;
+    if (p.B > merge_above) spc = (p.B + merge_above - 1) / merge_above;
     else if (p.B < split_below) {
       const long long want = split_below / p.B;
       while (2 * c <= want && 2 * c <= p.gamma && 2 * c <= kMaxCluster) c *= 2;

@@ -199,7 +199,7 @@ def test_config_c3_guidance_and_topk():
     ("plain, clusters of 2, small batch", dict(B=8, gamma=8, V=16384, dtype=W.BF16), False),
     ("top-k with guidance, one block per sequence", dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000), False),
     ("top-k with guidance, clusters of 4", dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000), True),
-    ("several sequences per block", dict(B=600, gamma=2, V=2048, dtype=W.BF16), False),
+    ("several sequences per block", dict(B=1500, gamma=2, V=2048, dtype=W.BF16), False),
 ])
 def test_back_to_back_calls_on_one_stream(name, kw, lat):
     """Consecutive calls overlap on the device (programmatic dependent launch) and share ONE
