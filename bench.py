@@ -43,7 +43,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
 # one ncu capture, see profiles/verify_topk_kernel_C3.md).  Reported only while the kernel sources
 # still have the digest the capture was taken with; null otherwise.
-NCU_TRAFFIC = {"sources_sha256": "704bf0286787ae7d", "workload": "C3", "bytes_per_launch": 68067840}
+NCU_TRAFFIC = {"sources_sha256": "1eeba23edc60426c", "workload": "C3", "bytes_per_launch": 68067840}
 
 
 def sources_digest() -> str:
@@ -290,7 +290,7 @@ def run_native(args) -> None:
     prms = [csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
                             o["tok"], o["tau"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
                             cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=o["st"], workspace=o["ws"],
-                            stream=stream, single_call_latency=args.single_call_latency)
+                            stream=stream, back_to_back=not args.single_call_latency)
             for w, o in zip(ring, outs)]
     kernels_per_step = csd.csd_launch_count(prms[0])
 
@@ -396,7 +396,8 @@ def run_native(args) -> None:
                        parallelism=f"dp{world} (independent sequences, no exchange)",
                        l2=f"ring of {ring_n} distinct step inputs, {ring_n * step_bytes / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2",
                        launch=f"CUDA graph of {graph_steps} steps, replayed",
-                       partition="per-call latency" if args.single_call_latency else "throughput (default)"),
+                       partition=("one call at a time: ordinary stream order, sequences split over clusters" if args.single_call_latency
+                                  else "back_to_back: one block per sequence, consecutive calls overlap")),
         "clocks": sampler.summary(),
         "e2e": {"value": B * L * e2e_steps * world / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps, "entry": "csd_verify_host (pinned host buffers)",
@@ -427,7 +428,7 @@ def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--single-call-latency", action="store_true",
-                    help="spread each call over the whole GPU (csd_params.single_call_latency = 1)")
+                    help="csd_params.back_to_back = 0: ordinary stream order, each call spread over the whole GPU")
     ap.add_argument("--steps", type=int, default=5760)
     ap.add_argument("--warmup", type=int, default=64)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])

@@ -186,15 +186,21 @@ typedef struct csd_params {
                                   overlap on the GPU need different workspaces.             */
   size_t workspace_bytes;
   void* stream;
-  int single_call_latency;     /* How the work of one call is spread over the GPU.
-                                  0 (default): for the throughput of calls enqueued back to back on
-                                  a stream -- one thread block per sequence once B >= 16, so that
-                                  the blocks of many consecutive calls share the GPU (a call's
-                                  streaming overlaps its predecessors' through programmatic
-                                  dependent launch; outputs still appear in call order).
-                                  1: for the latency of a call that runs alone -- each sequence is
-                                  split over up to 8 blocks until the GPU is full.  Results are
-                                  identical either way.                                          */
+  int back_to_back;            /* 0 (default): ordinary stream order.  The call starts when everything
+                                  enqueued before it on the stream has completed, and its work is
+                                  spread over the whole GPU (each sequence over up to 8 thread
+                                  blocks): the shortest time for one call, and safe after any
+                                  producer of its inputs.
+                                  1: for many calls enqueued back to back.  The call may START while
+                                  the operation before it on the stream is still running
+                                  (programmatic dependent launch) and uses one thread block per
+                                  sequence once B >= 16, so that the blocks of several consecutive
+                                  calls share the GPU; its outputs still become visible in call
+                                  order.  The caller guarantees that the inputs of such a call are
+                                  NOT produced by the operation that immediately precedes it on
+                                  the stream (another call of this library is fine: it writes only
+                                  its outputs and its workspace).  Results are identical either
+                                  way.                                                           */
 } csd_params;
 
 int csd_verify_ex(const csd_params* p);
@@ -216,9 +222,8 @@ int csd_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  * Host-buffer form: the same round for a caller whose logits, tokens, uniforms
  * and schedule sit in HOST memory (pinned memory makes the copies asynchronous).
  * Every data pointer of `host` (inputs, outputs, optional diagnostics) is a
- * HOST pointer; host->workspace / workspace_bytes and single_call_latency are
- * ignored (between its copies the kernel runs alone, so it is always spread over
- * the whole GPU).  `staging` is a
+ * HOST pointer; host->workspace / workspace_bytes and back_to_back are ignored
+ * (the kernel follows its own input copies in ordinary stream order).  `staging` is a
  * DEVICE buffer of at least csd_host_staging_size(host) bytes, 256-byte
  * aligned, that the library uses for the device copies of inputs and outputs
  * and for its workspace.  The call enqueues host->device copies, the kernels and

@@ -80,7 +80,7 @@ double normal_upper_quantile(double tail) {
 }
 
 template <typename T, bool CFG>
-cudaError_t launch_fused(const FusedArgs& a, int grid, cudaStream_t stream) {
+cudaError_t launch_fused(const FusedArgs& a, int grid, bool overlap, cudaStream_t stream) {
   auto kern = verify_topk_kernel<T, CFG>;
   static bool configured = false;
   if (!configured) {
@@ -95,22 +95,26 @@ cudaError_t launch_fused(const FusedArgs& a, int grid, cudaStream_t stream) {
   cfg.dynamicSmemBytes = sizeof(TopkSmem);
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  if (a.ctas_per_seq > 1) {   // the blocks of a sequence are one cluster
-    attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = (unsigned)a.ctas_per_seq;
-    attr[1].val.clusterDim.y = 1;
-    attr[1].val.clusterDim.z = 1;
-    cfg.numAttrs = 2;
+  int n_attr = 0;
+  if (overlap) {   // the call may start while the operation before it on the stream is still running
+    attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+    ++n_attr;
   }
+  if (a.ctas_per_seq > 1) {   // the blocks of a sequence are one cluster
+    attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+    attr[n_attr].val.clusterDim.x = (unsigned)a.ctas_per_seq;
+    attr[n_attr].val.clusterDim.y = 1;
+    attr[n_attr].val.clusterDim.z = 1;
+    ++n_attr;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n_attr;
   return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
 template <typename T, bool CFG>
-cudaError_t launch_plain(const FusedArgs& a, int grid, cudaStream_t stream) {
+cudaError_t launch_plain(const FusedArgs& a, int grid, bool overlap, cudaStream_t stream) {
   auto kern = verify_plain_kernel<T, CFG>;
   static bool configured = false;
   if (!configured) {
@@ -125,23 +129,27 @@ cudaError_t launch_plain(const FusedArgs& a, int grid, cudaStream_t stream) {
   cfg.dynamicSmemBytes = sizeof(PlainSmem);
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  if (a.ctas_per_seq > 1) {   // the blocks of a sequence are one cluster
-    attr[1].id = cudaLaunchAttributeClusterDimension;
-    attr[1].val.clusterDim.x = (unsigned)a.ctas_per_seq;
-    attr[1].val.clusterDim.y = 1;
-    attr[1].val.clusterDim.z = 1;
-    cfg.numAttrs = 2;
+  int n_attr = 0;
+  if (overlap) {   // the call may start while the operation before it on the stream is still running
+    attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+    ++n_attr;
   }
+  if (a.ctas_per_seq > 1) {   // the blocks of a sequence are one cluster
+    attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+    attr[n_attr].val.clusterDim.x = (unsigned)a.ctas_per_seq;
+    attr[n_attr].val.clusterDim.y = 1;
+    attr[n_attr].val.clusterDim.z = 1;
+    ++n_attr;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = n_attr;
   return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
 template <typename T, bool CFG>
-cudaError_t launch_fused_t(const FusedArgs& a, bool topk, int grid, cudaStream_t stream) {
-  return topk ? launch_fused<T, CFG>(a, grid, stream) : launch_plain<T, CFG>(a, grid, stream);
+cudaError_t launch_fused_t(const FusedArgs& a, bool topk, int grid, bool overlap, cudaStream_t stream) {
+  return topk ? launch_fused<T, CFG>(a, grid, overlap, stream) : launch_plain<T, CFG>(a, grid, overlap, stream);
 }
 
 template <typename T, bool CFG, int U, bool TOPK>
@@ -294,15 +302,15 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
     ua.top_k = p.top_k;
     ua.lo_sigmas = nanf("");
     ua.error_flag = reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
-    // Blocks are aligned with sequences and positions: a block owns a whole sequence; or, for very
-    // large batches, seqs_per_cta whole sequences; or a sequence's draft positions are split over the
-    // ctas_per_seq blocks of one cluster (each with both rows of its positions; 2, 4 or 8 blocks).
-    // Consecutive calls overlap on the GPU as deeply as their grids allow (a call may start once every
-    // block of its predecessor has started), so for throughput few long-lived blocks per call are
-    // best: one per sequence, split only when the batch is too small to give 16 blocks.  For the
-    // latency of a single call the sequences are split until the GPU is full.
+    // Blocks are aligned with sequences and positions.  For calls enqueued back to back a block owns a
+    // whole sequence (for very large batches seqs_per_cta of them): such calls overlap on the GPU as
+    // deeply as their grids allow (a call may start once every block of its predecessor has started),
+    // so few long-lived blocks per call are best, split only when the batch is too small to give 16
+    // blocks.  Otherwise the call runs alone, and a sequence's draft positions are split over the
+    // ctas_per_seq blocks of one cluster (each with both rows of its positions; 2, 4 or 8 blocks)
+    // until the GPU is full.
     const long long merge_above = 8LL * sms;   // beyond this many sequences a block takes several
-    const long long split_below = p.single_call_latency ? 2LL * sms : 16;
+    const long long split_below = p.back_to_back ? 16 : 2LL * sms;
     long long c = 1, spc = 1;
     if (p.B > merge_above) spc = (p.B + merge_above - 1) / merge_above;
     else if (p.B < split_below) {
@@ -341,11 +349,13 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
     ua.ctas_per_seq = (int)c;
     ua.seqs_per_cta = (int)spc;
     cudaError_t fe;
+    const bool overlap = p.back_to_back != 0;
     if (p.dtype == CSD_F32)
-      fe = cfg ? launch_fused_t<float, true>(ua, topk, (int)grid, stream) : launch_fused_t<float, false>(ua, topk, (int)grid, stream);
+      fe = cfg ? launch_fused_t<float, true>(ua, topk, (int)grid, overlap, stream)
+               : launch_fused_t<float, false>(ua, topk, (int)grid, overlap, stream);
     else
-      fe = cfg ? launch_fused_t<__nv_bfloat16, true>(ua, topk, (int)grid, stream)
-               : launch_fused_t<__nv_bfloat16, false>(ua, topk, (int)grid, stream);
+      fe = cfg ? launch_fused_t<__nv_bfloat16, true>(ua, topk, (int)grid, overlap, stream)
+               : launch_fused_t<__nv_bfloat16, false>(ua, topk, (int)grid, overlap, stream);
     return fe == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
   }
 
@@ -592,7 +602,7 @@ int csd_verify_host(const csd_params* host, void* staging, size_t staging_bytes)
   d.dbg_G = h.dbg_G ? (float*)(base + pl.off_G) : nullptr;
   d.workspace = base + pl.off_ws;
   d.workspace_bytes = pl.ws_bytes;
-  d.single_call_latency = 1;   // between the copies over the bus the kernel runs alone
+  d.back_to_back = 0;   // the kernel follows its own input copies: ordinary stream order
   if (cudaMemsetAsync(d.workspace, 0, layout_for(h.B, h.gamma, h.V, h.dtype).zero_bytes, stream) != cudaSuccess)
     return CSD_ERR_LAUNCH;
   const int rc = verify_impl(d);

@@ -9,7 +9,7 @@ import paper_2601_09212_b200 as csd
 TOL = {csd.CSD_F32: 1e-5, csd.CSD_BF16: 2e-3}   # absolute, on p, q, f and on the distribution drawn from
 
 
-def run_gpu(w, *, want_dbg=True, stream=None, workspace=None, single_call_latency=False):
+def run_gpu(w, *, want_dbg=True, stream=None, workspace=None, back_to_back=False):
     dev = w.target_logits.device
     B, L, V = w.B, w.gamma, w.V
     out = dict(
@@ -25,7 +25,7 @@ def run_gpu(w, *, want_dbg=True, stream=None, workspace=None, single_call_latenc
         out["tokens"], out["accept_len"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
         cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=out["status"],
         dbg_p=out.get("p"), dbg_q=out.get("q"), dbg_f=out.get("f"), dbg_G=out.get("G"),
-        workspace=ws, stream=stream, single_call_latency=single_call_latency)
+        workspace=ws, stream=stream, back_to_back=back_to_back)
     csd.csd_verify_ex(prm)
     torch.cuda.synchronize()
     return {k: v.cpu().numpy() for k, v in out.items()}

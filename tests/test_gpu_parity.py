@@ -152,12 +152,13 @@ def test_topk_with_masked_and_tied_rows():
     dict(B=3, gamma=7, V=32768, dtype=W.F32, bonus_row=True, top_k=50),
     dict(B=24, gamma=5, V=4100, dtype=W.BF16),
 ])
-def test_single_call_latency_partition(kw):
-    """The partition for the latency of one call (sequences split over the blocks of a cluster)
-    against the oracle, and against the default partition: identical integer outputs."""
+def test_back_to_back_partition(kw):
+    """The partition for calls enqueued back to back (one block per sequence, programmatic launch)
+    against the oracle, and against the default partition (sequences split over the blocks of a
+    cluster): identical integer outputs."""
     L = kw["gamma"]
     w = W.make("t", rho=0.9, schedule=sched(L), seed=77, device=DEV, **kw)
-    rep, got, ref = check(w, single_call_latency=True)
+    rep, got, ref = check(w, back_to_back=True)
     assert_ok(rep)
     base = run_gpu(w, want_dbg=False)
     assert np.array_equal(got["tokens"], base["tokens"])
@@ -172,13 +173,13 @@ def test_single_call_latency_partition(kw):
     dict(B=2, gamma=3, V=262144, dtype=W.BF16, top_k=1000),
     dict(B=1, gamma=2, V=2 ** 20, dtype=W.F32, bonus_row=True),     # the largest vocabulary accepted
     dict(B=1, gamma=2, V=2 ** 20, dtype=W.BF16, top_k=50),
-    dict(B=1, gamma=16, V=8192, dtype=W.F32, bonus_row=True),       # clusters of 8 with single_call_latency
+    dict(B=1, gamma=16, V=8192, dtype=W.F32, bonus_row=True),       # clusters of 8 by default
 ])
 def test_large_vocabularies_and_limits(kw):
     L = kw["gamma"]
     w = W.make("t", rho=0.9, schedule=sched(L), seed=5, device=DEV, **kw)
-    for lat in (False, True):
-        rep, got, ref = check(w, single_call_latency=lat)
+    for b2b in (False, True):
+        rep, got, ref = check(w, back_to_back=b2b)
         assert_ok(rep)
 
 
@@ -192,18 +193,22 @@ def test_config_c3_guidance_and_topk():
         print("C3", rep.summary())
 
 
-@pytest.mark.parametrize("name,kw,lat", [
-    ("plain, one block per sequence", dict(B=16, gamma=8, V=16384, dtype=W.F32), False),
-    ("plain, clusters of 8", dict(B=16, gamma=8, V=16384, dtype=W.F32), True),
-    ("plain, clusters of 4", dict(B=64, gamma=8, V=16384, dtype=W.F32), True),
-    ("plain, clusters of 2, small batch", dict(B=8, gamma=8, V=16384, dtype=W.BF16), False),
-    ("top-k with guidance, one block per sequence", dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000), False),
-    ("top-k with guidance, clusters of 4", dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000), True),
-    ("several sequences per block", dict(B=1500, gamma=2, V=2048, dtype=W.BF16), False),
+@pytest.mark.parametrize("name,kw,b2b", [
+    ("plain, one block per sequence, overlapping", dict(B=16, gamma=8, V=16384, dtype=W.F32), True),
+    ("plain, clusters of 8, stream order", dict(B=16, gamma=8, V=16384, dtype=W.F32), False),
+    ("plain, clusters of 4, stream order", dict(B=64, gamma=8, V=16384, dtype=W.F32), False),
+    ("plain, clusters of 2, overlapping", dict(B=8, gamma=8, V=16384, dtype=W.BF16), True),
+    ("top-k with guidance, one block per sequence, overlapping",
+     dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000), True),
+    ("top-k with guidance, clusters of 4, stream order",
+     dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000), False),
+    ("top-k with guidance, clusters of 4, overlapping",
+     dict(B=4, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000), True),
+    ("several sequences per block, overlapping", dict(B=1500, gamma=2, V=2048, dtype=W.BF16), True),
 ])
-def test_back_to_back_calls_on_one_stream(name, kw, lat):
-    """Consecutive calls overlap on the device (programmatic dependent launch) and share ONE
-    workspace and ONE set of output buffers per slot; every call's results must equal those of
+def test_back_to_back_calls_on_one_stream(name, kw, b2b):
+    """Consecutive calls (with back_to_back they overlap on the device through programmatic dependent
+    launch) share ONE workspace and ONE set of output buffers per slot; every call's results must equal those of
     the same call run alone, both when enqueued directly and when replayed as a CUDA graph."""
     L = kw["gamma"]
     n = 6
@@ -217,7 +222,7 @@ def test_back_to_back_calls_on_one_stream(name, kw, lat):
     prms = [csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
                             o["tok"], o["tau"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
                             cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=o["st"], workspace=ws_shared,
-                            stream=stream, single_call_latency=lat) for w, o in zip(steps, outs)]
+                            stream=stream, back_to_back=b2b) for w, o in zip(steps, outs)]
 
     def check_all(tag):
         for i, (o, ref) in enumerate(zip(outs, alone)):
