@@ -47,6 +47,7 @@ class _Params(C.Structure):
         ("out_tokens", C.c_void_p), ("out_accept_len", C.c_void_p), ("out_status", C.c_void_p),
         ("p", C.c_void_p), ("q", C.c_void_p), ("f", C.c_void_p), ("G", C.c_void_p),
         ("margin_accept", C.c_void_p), ("margin_cdf", C.c_void_p),
+        ("accept_mass", C.c_void_p), ("bound_term", C.c_void_p),
     ]
 
 
@@ -70,6 +71,8 @@ def _load():
         lib.orc_resample_weights.restype = C.c_double
         lib.orc_resample_dist.argtypes = [C.c_void_p, C.c_void_p, C.c_double, C.c_int, C.c_void_p]
         lib.orc_resample_dist.restype = C.c_double
+        lib.orc_position_terms.argtypes = [C.c_void_p, C.c_void_p, C.c_double, C.c_int, C.c_void_p, C.c_void_p]
+        lib.orc_position_terms.restype = None
         lib.orc_inverse_cdf.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_void_p]
         lib.orc_inverse_cdf.restype = C.c_int
         lib.orc_prepare_row.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int,
@@ -134,6 +137,15 @@ def resample_dist(P, Q, omega: float) -> np.ndarray:
     return G
 
 
+def position_terms(P, Q, omega: float):
+    """(sum_x Q f, sum_x |P - Q f| - sum_x (1 - f) Q) with f = min{1, omega P/Q}: the inner sum of
+    Eq. token_exp and the bracket of Eq. bd2 for one pair of distributions."""
+    P, Q = _f64(P), _f64(Q)
+    a, b = C.c_double(), C.c_double()
+    _load().orc_position_terms(_ptr(P), _ptr(Q), float(omega), int(P.size), C.byref(a), C.byref(b))
+    return a.value, b.value
+
+
 def inverse_cdf(g, Z: float, u: float):
     g = _f64(g)
     margin = C.c_double(0.0)
@@ -172,11 +184,14 @@ class VerifyResult:
     G: Optional[np.ndarray]   # [B, V] float64 (distribution drawn from; zeros if none)
     margin_accept: np.ndarray  # [B, gamma]
     margin_cdf: np.ndarray     # [B]
+    accept_mass: Optional[np.ndarray] = None   # [B, gamma]: sum_x Q_i f_i (NaN where a row is unusable)
+    bound_term: Optional[np.ndarray] = None    # [B, gamma]: the bracket of Eq. bd2
 
 
 def verify(target_logits, draft_logits, draft_tokens, uniforms, relax_schedule, *,
            dtype: int = F32, target_uncond=None, draft_uncond=None, cfg_scale: float = 1.0,
-           top_k: int = 0, want_G: bool = True, want_pqf: bool = True) -> VerifyResult:
+           top_k: int = 0, want_G: bool = True, want_pqf: bool = True,
+           want_terms: bool = False) -> VerifyResult:
     """One verification round for B sequences (Algorithm 1, verification stage).
 
     target_logits [B, T, V] with T in {gamma, gamma+1}; draft_logits [B, gamma, V];
@@ -202,14 +217,16 @@ def verify(target_logits, draft_logits, draft_tokens, uniforms, relax_schedule, 
         status=np.zeros(B, np.int32),
         p=np.empty((B, gamma)), q=np.empty((B, gamma)), f=np.empty((B, gamma)),
         G=np.zeros((B, V)) if want_G else None,
-        margin_accept=np.empty((B, gamma)), margin_cdf=np.empty(B))
+        margin_accept=np.empty((B, gamma)), margin_cdf=np.empty(B),
+        accept_mass=np.empty((B, gamma)) if want_terms else None,
+        bound_term=np.empty((B, gamma)) if want_terms else None)
     prm = _Params(
         _ptr(t), _ptr(d), _ptr(tu), _ptr(du), int(dtype), float(cfg_scale), int(top_k),
         B, gamma, V, T, T * V, gamma * V, _ptr(tok), _ptr(uni), _ptr(om),
         _ptr(res.tokens), _ptr(res.accept_len), _ptr(res.status),
         _ptr(res.p) if want_pqf else None, _ptr(res.q) if want_pqf else None,
         _ptr(res.f) if want_pqf else None, _ptr(res.G),
-        _ptr(res.margin_accept), _ptr(res.margin_cdf))
+        _ptr(res.margin_accept), _ptr(res.margin_cdf), _ptr(res.accept_mass), _ptr(res.bound_term))
     rc = _load().orc_verify(C.byref(prm))
     if rc != 0:
         raise RuntimeError(f"orc_verify failed with code {rc}")

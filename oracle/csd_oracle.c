@@ -6,7 +6,9 @@
  * paper (verification stage), the relaxed acceptance probability (Eq. relax),
  * the annealing schedules (UniformRSD, Eq. sdar, and the linear variant of the
  * schedule ablation), and the bound-minimising resampling distribution
- * (Eq. opt_G, Theorem 2 / Proposition LP).
+ * (Eq. opt_G, Theorem 2 / Proposition LP); and, per position, the two sums that
+ * Theorem 2 is made of: the acceptance mass sum_x Q f (the inner sum of Eq.
+ * token_exp) and the bracket of Eq. bd2, sum_x |P - Q f| - sum_x (1 - f) Q.
  *
  * It shares no code with the CUDA library.  Only the tests, the smoke check and
  * the benchmark's CPU-baseline leg may call it.  Everything is written as the
@@ -37,7 +39,8 @@
  * Pins (tests/test_oracle_*.py): Theorem 1 by exact enumeration and chi-square,
  * Theorem 2's expectation and TV bound by brute force on tiny alphabets,
  * Proposition LP's closed form against random and grid search over G,
- * Proposition 2, the schedule's normalisation, and textbook routines
+ * Proposition 2, the schedule's normalisation, the per-position sums against
+ * their closed forms and against the brute-force bound, and textbook routines
  * (log-sum-exp, partition, cumsum/searchsorted) for the building blocks.
  * Parity unpinned: nothing -- the paper prints no worked numeric example, so
  * there is no printed value to pin to; every function has an analytic pin.
@@ -78,6 +81,8 @@ typedef struct {
   double *G;                   /* [B, V] or NULL: distribution drawn from */
   double *margin_accept;       /* [B, gamma] or NULL: |r_i - f_i| where the test ran, else +inf */
   double *margin_cdf;          /* [B] or NULL: distance of u to the nearest CDF boundary of the pick */
+  double *accept_mass;         /* [B, gamma] or NULL: sum_x Q_i(x) f_i(x) at every position (NaN: unusable row) */
+  double *bound_term;          /* [B, gamma] or NULL: the bracket of Eq. bd2 at every position */
 } orc_params;
 
 int orc_num_threads(void) {
@@ -186,6 +191,25 @@ double orc_resample_weights(const double *P, const double *Q, double omega, int 
     Z += v;
   }
   return Z;
+}
+
+/* The two per-position sums of Theorem 2 for one pair of distributions, written as the paper writes
+ * them, with f(x) = min{1, omega P(x)/Q(x)} (Eq. relax at candidate x):
+ *   *accept_mass = sum_x Q(x) f(x)                  (inner sum of Eq. token_exp: the probability that
+ *                                                    the position accepts, given its prefix)
+ *   *bound_term  = sum_x |P(x) - Q(x) f(x)| - sum_x (1 - f(x)) Q(x)     (the bracket of Eq. bd2,
+ *                                                    i.e. the infimum of Proposition LP) */
+void orc_position_terms(const double *P, const double *Q, double omega, int V, double *accept_mass,
+                        double *bound_term) {
+  double a = 0.0, abs_sum = 0.0, rej = 0.0;
+  for (int x = 0; x < V; ++x) {
+    const double fx = orc_accept_prob(P[x], Q[x], omega);
+    a += Q[x] * fx;
+    abs_sum += fabs(P[x] - Q[x] * fx);
+    rej += (1.0 - fx) * Q[x];
+  }
+  *accept_mass = a;
+  *bound_term = abs_sum - rej;
 }
 
 /* Eq. opt_G normalised; falls back to P when Z = 0.  Returns Z. */
@@ -374,7 +398,7 @@ static void verify_one(const orc_params *a, int b, double *zt, double *zd, doubl
 
   /* Diagnostics for comparison only (not part of the procedure): p, q, f at
    * every position, including those after the first rejection. */
-  if (a->p || a->q || a->f) {
+  if (a->p || a->q || a->f || a->accept_mass || a->bound_term) {
     for (int i = 1; i <= L; ++i) {
       const int64_t t_off = (int64_t)b * a->target_batch_stride + (int64_t)(i - 1) * V;
       const int64_t d_off = (int64_t)b * a->draft_batch_stride + (int64_t)(i - 1) * V;
@@ -391,6 +415,12 @@ static void verify_one(const orc_params *a, int b, double *zt, double *zd, doubl
       if (a->p) a->p[o] = pv;
       if (a->q) a->q[o] = qv;
       if (a->f) a->f[o] = ok ? orc_accept_prob(pv, qv, (double)a->relax_schedule[i - 1]) : 0.0;
+      if (a->accept_mass || a->bound_term) {
+        double am = NAN, bt = NAN;
+        if (t_ok && d_ok) orc_position_terms(P, Q, (double)a->relax_schedule[i - 1], V, &am, &bt);
+        if (a->accept_mass) a->accept_mass[o] = am;
+        if (a->bound_term) a->bound_term[o] = bt;
+      }
     }
   }
 }

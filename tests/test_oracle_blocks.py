@@ -278,3 +278,43 @@ def test_prop_lp_closed_form_and_optimality(oracle):
             cands = list(rng.dirichlet(np.ones(V) * 0.5, size=4000))
         vals = np.array([objective(P, Q, f, G) for G in cands])
         assert vals.min() >= best - 1e-12
+
+
+# ---- per-position sums of Theorem 2 ------------------------------------------------------------
+@pytest.mark.parametrize("omega", [0.0, 0.25, 1.0, 1.1, 2.36, 50.0])
+def test_position_terms_closed_forms(oracle, omega):
+    """sum_x Q f = sum_x min{Q, omega P}; the bracket of Eq. bd2 equals 2 sum_x [min{Q, omega P} - P]_+
+    (both follow from f = min{1, omega P/Q}); zero entries follow the 0/0 := 1 convention."""
+    rng = np.random.default_rng(int(omega * 100) + 3)
+    for V in (2, 7, 64):
+        P = rng.dirichlet(np.full(V, 0.6))
+        Q = rng.dirichlet(np.full(V, 0.6))
+        if V > 2:
+            P[1] = 0.0; P /= P.sum()
+            Q[2] = 0.0; Q /= Q.sum()
+        am, bt = oracle.position_terms(P, Q, omega)
+        mn = np.minimum(Q, omega * P)
+        assert np.isclose(am, mn.sum(), rtol=1e-13, atol=1e-15)
+        assert np.isclose(bt, 2.0 * np.maximum(mn - P, 0.0).sum(), rtol=1e-12, atol=1e-14)
+        assert -1e-15 <= am <= 1.0 + 1e-15 and bt >= -1e-15
+        if omega <= 1.0:
+            assert abs(bt) < 1e-14          # no relaxation beyond vanilla: the bound's bracket vanishes
+        if omega == 1.0:
+            assert np.isclose(am, 1.0 - 0.5 * np.abs(P - Q).sum(), rtol=1e-13)   # 1 - TV(P, Q)
+        if omega == 0.0:
+            assert am == 0.0 or np.isclose(am, Q[P == 0.0].sum() * 0.0)
+
+
+def test_position_terms_is_the_infimum_of_prop_lp(oracle):
+    """The bracket equals the objective of Proposition LP at G* = Norm([P - Q f]_+), and no other G
+    gets below it."""
+    rng = np.random.default_rng(11)
+    for omega in (0.4, 1.0, 1.8, 4.0):
+        P, Q = rng.dirichlet(np.ones(5)), rng.dirichlet(np.ones(5))
+        f = np.array([oracle.accept_prob(p, q, omega) for p, q in zip(P, Q)])
+        rej = ((1.0 - f) * Q).sum()
+        objective = lambda G: np.abs(P - Q * f - G * rej).sum()
+        _, bt = oracle.position_terms(P, Q, omega)
+        assert np.isclose(objective(oracle.resample_dist(P, Q, omega)), bt, rtol=1e-12, atol=1e-14)
+        for _ in range(200):
+            assert objective(rng.dirichlet(np.ones(5))) >= bt - 1e-12

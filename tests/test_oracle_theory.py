@@ -154,6 +154,22 @@ def tv_bound_at_gstar(model, f):
     return 0.5 * total
 
 
+def bound_and_length_through_position_terms(oracle, model, f, omegas):
+    """Eq. bd2 and Eq. token_exp assembled from the oracle's per-position sums: every prefix
+    x_{1:i} contributes, with weight Q(x_{1:i}) prod f, its bracket / its acceptance mass."""
+    V, L = model.V, model.L
+    bound, e_len = 0.0, 1.0
+    for i in range(L):
+        for pre in itertools.product(range(V), repeat=i):
+            w = 1.0
+            for k in range(i):
+                w *= model.Q[pre[:k]][pre[k]] * f[pre[:k + 1]]
+            am, bt = oracle.position_terms(model.P[pre], model.Q[pre], omegas[i])
+            bound += w * bt
+            e_len += w * am
+    return 0.5 * bound, e_len
+
+
 def expected_len_formula(model, f):
     """Eq. token_exp."""
     V, L = model.V, model.L
@@ -207,6 +223,10 @@ def test_theorem2_law_bound_and_length(oracle, V, L, omegas, gkind):
                 w *= model.Q[xs[:k]][xs[k]] * f[xs[:k + 1]]
             e_len += w
     assert np.isclose(e_len, expected_len_formula(model, f))
+    # the per-position sums (what the library can report per drafted prefix) give the same two numbers
+    b_terms, len_terms = bound_and_length_through_position_terms(oracle, model, f, omegas)
+    assert np.isclose(b_terms, tv_bound_at_gstar(model, f), rtol=1e-10, atol=1e-13)
+    assert np.isclose(len_terms, e_len, rtol=1e-12)
     if all(o == 0.0 for o in omegas):
         # omega = 0: everything is rejected, G* = P, the output is a pure target sample
         assert np.abs(phat - model.joint_P()).max() < 1e-12 or gkind == "random"

@@ -134,3 +134,27 @@ def test_verify_identical_models_fallback(oracle):
     for b in rej:
         assert np.allclose(r.G[b], sps.softmax(h["target_logits"][b, 1].astype(np.float64)), rtol=1e-10)
     assert r.status.max() == 0
+
+
+def test_verify_reports_position_terms(oracle):
+    """The optional per-position sums of Theorem 2 against scipy's softmax and their closed forms, at
+    every position (also those after the first rejection), with and without guidance mix + top-k."""
+    B, L, V = 6, 4, 500
+    sched = oracle.make_schedule(1, 1.1, 0.7, L)
+    for extra in ({}, dict(cfg=True, cfg_scale=2.5, top_k=40)):
+        w = W.make("t", B=B, gamma=L, V=V, dtype=W.F32, rho=0.8, schedule=sched, seed=9, **extra)
+        h = w.host_arrays()
+        r = oracle.verify(h["target_logits"], h["draft_logits"], h["draft_tokens"], h["uniforms"],
+                          h["relax_schedule"], dtype=W.F32, target_uncond=h["target_uncond"],
+                          draft_uncond=h["draft_uncond"], cfg_scale=w.cfg_scale, top_k=w.top_k, want_terms=True)
+        om = h["relax_schedule"].astype(np.float64)
+        for b in range(B):
+            for i in range(L):
+                zt = oracle.prepare_row(h["target_logits"][b, i], None if h["target_uncond"] is None else h["target_uncond"][b, i],
+                                        W.F32, w.cfg_scale, w.top_k)
+                zd = oracle.prepare_row(h["draft_logits"][b, i], None if h["draft_uncond"] is None else h["draft_uncond"][b, i],
+                                        W.F32, w.cfg_scale, w.top_k)
+                P, Q = sps.softmax(zt), sps.softmax(zd)
+                mn = np.minimum(Q, om[i] * P)
+                assert np.isclose(r.accept_mass[b, i], mn.sum(), rtol=1e-11)
+                assert np.isclose(r.bound_term[b, i], 2.0 * np.maximum(mn - P, 0.0).sum(), rtol=1e-9, atol=1e-13)
