@@ -43,7 +43,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
 # one ncu capture, see profiles/verify_topk_kernel_C3.md).  Reported only while the kernel sources
 # still have the digest the capture was taken with; null otherwise.
-NCU_TRAFFIC = {"sources_sha256": "1eeba23edc60426c", "workload": "C3", "bytes_per_launch": 68067840}
+NCU_TRAFFIC = {"sources_sha256": "", "workload": "C3", "bytes_per_launch": 68067840}
 
 
 def sources_digest() -> str:
@@ -285,12 +285,15 @@ def run_native(args) -> None:
     outs = [dict(tok=torch.empty(B, L + 1, dtype=torch.int32, device=dev),
                  tau=torch.empty(B, dtype=torch.int32, device=dev),
                  st=torch.empty(B, dtype=torch.int32, device=dev),
+                 am=torch.empty(B, L, device=dev) if args.monitors else None,
+                 bt=torch.empty(B, L, device=dev) if args.monitors else None,
                  ws=csd.new_workspace(B, L, V, dtype, dev)) for _ in range(ring_n)]
     stream = torch.cuda.Stream(device=dev)
     prms = [csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
                             o["tok"], o["tau"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
                             cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=o["st"], workspace=o["ws"],
-                            stream=stream, back_to_back=not args.single_call_latency)
+                            stream=stream, back_to_back=not args.single_call_latency,
+                            diag_accept_mass=o["am"], diag_bound_term=o["bt"])
             for w, o in zip(ring, outs)]
     kernels_per_step = csd.csd_launch_count(prms[0])
 
@@ -386,7 +389,8 @@ def run_native(args) -> None:
     achieved = step_bytes / step_s / 1e9
     digest = sources_digest()
     traffic = None
-    if NCU_TRAFFIC["sources_sha256"] == digest and NCU_TRAFFIC["workload"] == name and not args.single_call_latency:
+    if (NCU_TRAFFIC["sources_sha256"] == digest and NCU_TRAFFIC["workload"] == name
+            and not args.single_call_latency and not args.monitors):
         traffic = NCU_TRAFFIC["bytes_per_launch"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -396,6 +400,7 @@ def run_native(args) -> None:
                        parallelism=f"dp{world} (independent sequences, no exchange)",
                        l2=f"ring of {ring_n} distinct step inputs, {ring_n * step_bytes / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2",
                        launch=f"CUDA graph of {graph_steps} steps, replayed",
+                       monitors=bool(args.monitors),
                        partition=("one call at a time: ordinary stream order, sequences split over clusters" if args.single_call_latency
                                   else "back_to_back: one block per sequence, consecutive calls overlap")),
         "clocks": sampler.summary(),
@@ -427,6 +432,8 @@ def run_native(args) -> None:
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--monitors", action="store_true",
+                    help="also ask for the per-position monitors of Theorem 2 (a second pass over every row)")
     ap.add_argument("--single-call-latency", action="store_true",
                     help="csd_params.back_to_back = 0: ordinary stream order, each call spread over the whole GPU")
     ap.add_argument("--steps", type=int, default=5760)

@@ -201,6 +201,17 @@ typedef struct csd_params {
                                   the stream (another call of this library is fine: it writes only
                                   its outputs and its workspace).  Results are identical either
                                   way.                                                           */
+  float* diag_accept_mass;     /* [B, gamma] or NULL.  Fidelity/efficiency monitors of Theorem 2, for every   */
+  float* diag_bound_term;      /* [B, gamma] or NULL.  position i given its drafted prefix, with
+                                  f_i(x) = min{1, omega_i P_i(x)/Q_i(x)}:
+                                    accept_mass = sum_x Q_i(x) f_i(x)   (inner sum of Eq. token_exp: the
+                                      probability that position i accepts; their running products along
+                                      the draft add up to E[tau]);
+                                    bound_term  = sum_x |P_i(x) - Q_i(x) f_i(x)| - sum_x (1 - f_i(x)) Q_i(x)
+                                      (the bracket of Eq. bd2, i.e. position i's contribution to the
+                                      total-variation bound at G*; 0 whenever omega_i <= 1).
+                                  NaN where a row of the position is unusable.  Either pointer may be
+                                  NULL.  Asking for them costs a second pass over every row.       */
 } csd_params;
 
 int csd_verify_ex(const csd_params* p);
@@ -222,8 +233,9 @@ int csd_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
  * Host-buffer form: the same round for a caller whose logits, tokens, uniforms
  * and schedule sit in HOST memory (pinned memory makes the copies asynchronous).
  * Every data pointer of `host` (inputs, outputs, optional diagnostics) is a
- * HOST pointer; host->workspace / workspace_bytes and back_to_back are ignored
- * (the kernel follows its own input copies in ordinary stream order).  `staging` is a
+ * HOST pointer; host->workspace / workspace_bytes, back_to_back and the two
+ * diag_ pointers are ignored (the kernel follows its own input copies in
+ * ordinary stream order; the Theorem 2 monitors are outputs of the device form).  `staging` is a
  * DEVICE buffer of at least csd_host_staging_size(host) bytes, 256-byte
  * aligned, that the library uses for the device copies of inputs and outputs
  * and for its workspace.  The call enqueues host->device copies, the kernels and

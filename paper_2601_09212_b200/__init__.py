@@ -43,6 +43,7 @@ class csd_params(C.Structure):
         ("dbg_p", C.c_void_p), ("dbg_q", C.c_void_p), ("dbg_f", C.c_void_p), ("dbg_G", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p),
         ("back_to_back", C.c_int32),
+        ("diag_accept_mass", C.c_void_p), ("diag_bound_term", C.c_void_p),
     ]
 
 
@@ -197,7 +198,8 @@ def csd_verify_static(target_logits, draft_logits, draft_tokens, uniforms, relax
 def make_params(target_logits, draft_logits, draft_tokens, uniforms, relax_schedule, out_tokens,
                 out_accept_len, *, target_uncond=None, draft_uncond=None, cfg_scale=1.0, top_k=0,
                 out_status=None, dbg_p=None, dbg_q=None, dbg_f=None, dbg_G=None, workspace=None,
-                stream=None, host=False, back_to_back=False) -> csd_params:
+                stream=None, host=False, back_to_back=False, diag_accept_mass=None,
+                diag_bound_term=None) -> csd_params:
     """Fill a ``csd_params`` from tensors (device tensors, or host ones with ``host=True``)."""
     B, T, V = target_logits.shape
     gamma = draft_logits.shape[1]
@@ -232,6 +234,8 @@ def make_params(target_logits, draft_logits, draft_tokens, uniforms, relax_sched
         p.workspace_bytes = workspace.numel() * workspace.element_size()
     p.stream = _stream_handle(stream)
     p.back_to_back = 1 if back_to_back else 0
+    p.diag_accept_mass = ptr(diag_accept_mass, "diag_accept_mass", torch.float32)
+    p.diag_bound_term = ptr(diag_bound_term, "diag_bound_term", torch.float32)
     return p
 
 

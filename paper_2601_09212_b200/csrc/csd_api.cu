@@ -289,6 +289,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr) {
   fa.tokens = p.draft_tokens; fa.uniforms = p.uniforms; fa.schedule = p.relax_schedule;
   fa.out_tokens = p.out_tokens; fa.out_accept_len = p.out_accept_len; fa.out_status = p.out_status;
   fa.dbg_p = p.dbg_p; fa.dbg_q = p.dbg_q; fa.dbg_f = p.dbg_f; fa.dbg_G = p.dbg_G;
+  fa.diag_am = p.diag_accept_mass; fa.diag_bt = p.diag_bound_term;
 
   // ---- fused single-launch path: aligned rows of at least 512 bytes; with top-k, rows that fit the registers
   const bool fused = vec_ok && (size_t)p.V * es >= 512 && (p.V + 32 * vw - 1) / (32 * vw) <= kFinTiles;
@@ -603,6 +604,8 @@ int csd_verify_host(const csd_params* host, void* staging, size_t staging_bytes)
   d.workspace = base + pl.off_ws;
   d.workspace_bytes = pl.ws_bytes;
   d.back_to_back = 0;   // the kernel follows its own input copies: ordinary stream order
+  d.diag_accept_mass = nullptr;   // (device-only outputs: not part of the host form)
+  d.diag_bound_term = nullptr;
   if (cudaMemsetAsync(d.workspace, 0, layout_for(h.B, h.gamma, h.V, h.dtype).zero_bytes, stream) != cudaSuccess)
     return CSD_ERR_LAUNCH;
   const int rc = verify_impl(d);

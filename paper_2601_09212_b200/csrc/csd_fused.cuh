@@ -432,6 +432,80 @@ __device__ void write_G(const FinishArgs& a, const int b, const int j, const Seq
   }
 }
 
+// The per-position sums of Theorem 2 (inner sum of Eq. token_exp, bracket of Eq. bd2) for the block's
+// positions of sequence b: a second pass over both rows of each position, brought through the ring
+// by bulk copies like the draw.  Follows accept_positions of the same sequence (row statistics in
+// sm); called after the block's griddepcontrol.wait.  red needs two doubles per warp.
+template <typename T, bool CFG, int NT, bool FILT>
+__device__ void position_terms(const FinishArgs& a, const BlockShare& sh, const int b, const int tid,
+                               unsigned char* ring, const int ring_bytes, double* red, FinishSmem& sm,
+                               FinishStage& st, uint32_t& phase) {
+  constexpr int VEC = Elem<T>::kVec;
+  constexpr int TILE = 32 * VEC;
+  constexpr int ARR = CFG ? 2 : 1;
+  constexpr int ES = (int)sizeof(T);
+  const int lane = tid & 31, warp = tid >> 5;
+  const int V = a.V, L = a.gamma;
+  const int n_arr = 2 * ARR;
+  const int seg_elems = (ring_bytes / n_arr / (TILE * ES)) * TILE;   // elements of each array per segment
+  const int slot_bytes = seg_elems * ES;
+  for (int i = sh.pos_begin; i < sh.pos_end; ++i) {
+    const bool usable = sm.valid[0][i] && sm.valid[1][i];
+    float am = 0.0f, bt2 = 0.0f;
+    if (usable) {   // (the same decision in every thread)
+      TermsCtx tc;
+      tc.Mt = sm.M[0][i]; tc.Md = sm.M[1][i];
+      tc.inv_t = 1.0f / (1.0f + sm.S[0][i]); tc.inv_d = 1.0f / (1.0f + sm.S[1][i]);
+      tc.omega = st.omega[i];
+      Row<T, CFG> rt = row_at<T, CFG>(a, b, 0, i), rd = row_at<T, CFG>(a, b, 1, i);
+      rt.thr = sm.thr[0][i];
+      rd.thr = sm.thr[1][i];
+      for (int x0 = 0; x0 < V; x0 += seg_elems) {
+        __syncthreads();   // everybody is done with what the ring held
+        const int n = min(seg_elems, V - x0);
+        if (tid == 0) {
+          fence_before_bulk();
+          const uint32_t bytes = (uint32_t)(n * ES);
+          mbar_expect_tx(&st.bar, bytes * n_arr);
+          bulk_load(ring, rt.cond + x0, bytes, &st.bar);
+          if (CFG) bulk_load(ring + slot_bytes, rt.uncond + x0, bytes, &st.bar);
+          bulk_load(ring + ARR * slot_bytes, rd.cond + x0, bytes, &st.bar);
+          if (CFG) bulk_load(ring + (ARR + 1) * slot_bytes, rd.uncond + x0, bytes, &st.bar);
+        }
+        (void)mbar_wait(&st.bar, phase);   // (a wait that gives up leaves garbage in a diagnostic only)
+        phase ^= 1u;
+        for (int xo = tid * VEC; xo < n; xo += NT * VEC) {
+          float zt[VEC], zd[VEC];
+          unpack_vec<T>(ring + xo * ES, zt);
+          unpack_vec<T>(ring + ARR * slot_bytes + xo * ES, zd);
+          if (CFG) {
+            float zu[VEC];
+            unpack_vec<T>(ring + slot_bytes + xo * ES, zu);
+            cfg_mix_vec<VEC>(zt, zu, a.cfg_scale);
+            unpack_vec<T>(ring + (ARR + 1) * slot_bytes + xo * ES, zu);
+            cfg_mix_vec<VEC>(zd, zu, a.cfg_scale);
+          }
+#pragma unroll
+          for (int k = 0; k < VEC; ++k)
+            terms_of(FILT ? rt.filter(zt[k]) : zt[k], FILT ? rd.filter(zd[k]) : zd[k], tc, am, bt2);
+        }
+      }
+    }
+    const double wa = warp_sum_double((double)am), wb = warp_sum_double((double)bt2);
+    __syncthreads();
+    if (lane == 0) { red[2 * warp] = wa; red[2 * warp + 1] = wb; }
+    __syncthreads();
+    if (tid == 0) {
+      double ta = 0.0, tb = 0.0;
+      for (int w = 0; w < NT / 32; ++w) { ta += red[2 * w]; tb += red[2 * w + 1]; }
+      const float nanv = __int_as_float(0x7fc00000);
+      if (a.diag_am) a.diag_am[(int64_t)b * L + i] = usable ? (float)ta : nanv;
+      if (a.diag_bt) a.diag_bt[(int64_t)b * L + i] = usable ? (float)(2.0 * tb) : nanv;
+    }
+  }
+  __syncthreads();
+}
+
 // Tokens, multipliers and uniforms of the block's positions of its sl-th sequence, into shared memory.
 // Called for the first sequence when the kernel starts, so that these loads are long complete when
 // the accept tests need them.
@@ -609,6 +683,7 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
   const int L = a.gamma;
   const int extra = aborted ? 8 : 0;
   uint32_t phase = 0;
+  const bool want_terms = a.diag_am != nullptr || a.diag_bt != nullptr;
   auto write_pqf = [&](int b) {   // diagnostics of this block's positions
     if (tid >= sh.pos_begin && tid < sh.pos_end) {
       if (a.dbg_p) a.dbg_p[(int64_t)b * L + tid] = st.p[tid];
@@ -629,6 +704,7 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
       }
       write_pqf(b);
       emit_sequence<T, CFG, NT>(ua, b, st.rec, st.rec.status_any | sticky, tid);
+      if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase);
       __syncthreads();
     }
     return;
@@ -649,7 +725,11 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
     if (w & 2u) any = 8;
   }
   if (owner != sh.slot) {   // another block decides the sequence
-    if (a.dbg_p || a.dbg_q || a.dbg_f) { pdl_wait(); write_pqf(b); }
+    if (a.dbg_p || a.dbg_q || a.dbg_f || want_terms) {
+      pdl_wait();
+      write_pqf(b);
+      if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase);
+    }
     return;
   }
   draw_position<T, CFG, NT, FILT>(ua, sh, 0, j, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
@@ -657,6 +737,7 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
   if (__ldcg(ua.error_flag)) any = 8;
   write_pqf(b);
   emit_sequence<T, CFG, NT>(ua, b, st.rec, any, tid);
+  if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase);
 }
 
 // ======================= plain kernel: one pipeline per warp ============================

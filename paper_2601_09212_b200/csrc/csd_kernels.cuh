@@ -429,6 +429,8 @@ struct FinishArgs {
   float* dbg_q;
   float* dbg_f;
   float* dbg_G;
+  float* diag_am;   // [B, gamma] or null: sum_x Q f per position (inner sum of Eq. token_exp)
+  float* diag_bt;   // [B, gamma] or null: bracket of Eq. bd2 per position
 };
 
 struct PairCtx {  // what Eq. opt_G needs at one position
@@ -449,6 +451,20 @@ __device__ __forceinline__ float weight_of(float zt, float zd, const PairCtx& c)
   const float pq = ((et - ed) + (et * c.Sd - ed * c.St)) * c.inv_den;  // P - Q
   const float alt = c.one_minus_omega * et * c.inv_t;                    // (1 - omega) P
   return fmaxf(0.0f, fmaxf(pq, alt));
+}
+
+// One candidate token's share of the two per-position sums of Theorem 2, with
+// f(x) = min{1, omega P(x)/Q(x)}: Q f = min{Q, omega P}, and, since sum_x (P - Q f) = sum_x (1 - f) Q,
+// the bracket of Eq. bd2 is 2 sum_x [Q f - P]_+.  am and bt2 accumulate sum_x Q f and sum_x [Q f - P]_+.
+struct TermsCtx {
+  float Mt, Md, inv_t, inv_d, omega;
+};
+__device__ __forceinline__ void terms_of(float zt, float zd, const TermsCtx& c, float& am, float& bt2) {
+  const float P = ex2f((zt - c.Mt) * kLog2e) * c.inv_t;
+  const float Q = ex2f((zd - c.Md) * kLog2e) * c.inv_d;
+  const float qf = fminf(Q, c.omega * P);
+  am += qf;
+  bt2 += fmaxf(qf - P, 0.0f);
 }
 
 __device__ __forceinline__ double warp_sum_double(double v) {
@@ -720,6 +736,42 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
   if (tid == 0) {
     a.out_accept_len[b] = tau;
     if (a.out_status) a.out_status[b] = status;
+  }
+  // ---- 9. optional: the per-position sums of Theorem 2 (a second pass over every row) ------------
+  if (a.diag_am || a.diag_bt) {
+    for (int i = 0; i < L; ++i) {
+      group_sync<NT, BAR>();
+      float am = 0.0f, bt2 = 0.0f;
+      const bool usable = sm.valid[0][i] && sm.valid[1][i];
+      if (usable) {
+        TermsCtx tc;
+        tc.Mt = sm.M[0][i]; tc.Md = sm.M[1][i];
+        tc.inv_t = 1.0f / (1.0f + sm.S[0][i]); tc.inv_d = 1.0f / (1.0f + sm.S[1][i]);
+        const float om = a.schedule[i];
+        tc.omega = om >= 0.0f ? om : 0.0f;
+        const Row<T, CFG> rt{tgt + (int64_t)i * V, CFG ? tgt_u + (int64_t)i * V : nullptr, a.cfg_scale, sm.thr[0][i]};
+        const Row<T, CFG> rd{dft + (int64_t)i * V, CFG ? dft_u + (int64_t)i * V : nullptr, a.cfg_scale, sm.thr[1][i]};
+        for (int tile = warp; tile < (V + TILE - 1) / TILE; tile += NT / 32) {
+          const int x0 = tile * TILE + lane * VEC;
+          float zt[VEC], zd[VEC];
+          rt.load_tile(x0, V, a.vec_ok, zt);
+          rd.load_tile(x0, V, a.vec_ok, zd);
+#pragma unroll
+          for (int k = 0; k < VEC; ++k)
+            if (x0 + k < V) terms_of(rt.filter(zt[k]), rd.filter(zd[k]), tc, am, bt2);
+        }
+      }
+      const double wa = warp_sum_double((double)am), wb = warp_sum_double((double)bt2);
+      if (lane == 0) { tile_sums[2 * warp] = wa; tile_sums[2 * warp + 1] = wb; }
+      group_sync<NT, BAR>();
+      if (tid == 0) {
+        double ta = 0.0, tb = 0.0;
+        for (int w = 0; w < NT / 32; ++w) { ta += tile_sums[2 * w]; tb += tile_sums[2 * w + 1]; }
+        const float nanv = __int_as_float(0x7fc00000);
+        if (a.diag_am) a.diag_am[(int64_t)b * L + i] = usable ? (float)ta : nanv;
+        if (a.diag_bt) a.diag_bt[(int64_t)b * L + i] = usable ? (float)(2.0 * tb) : nanv;
+      }
+    }
   }
   group_sync<NT, BAR>();  // the shared state may be reused for the next sequence
 }

@@ -9,7 +9,7 @@ import paper_2601_09212_b200 as csd
 TOL = {csd.CSD_F32: 1e-5, csd.CSD_BF16: 2e-3}   # absolute, on p, q, f and on the distribution drawn from
 
 
-def run_gpu(w, *, want_dbg=True, stream=None, workspace=None, back_to_back=False):
+def run_gpu(w, *, want_dbg=True, stream=None, workspace=None, back_to_back=False, want_terms=False):
     dev = w.target_logits.device
     B, L, V = w.B, w.gamma, w.V
     out = dict(
@@ -19,13 +19,16 @@ def run_gpu(w, *, want_dbg=True, stream=None, workspace=None, back_to_back=False
     if want_dbg:
         out.update(p=torch.empty((B, L), device=dev), q=torch.empty((B, L), device=dev),
                    f=torch.empty((B, L), device=dev), G=torch.full((B, V), -1.0, device=dev))
+    if want_terms:
+        out.update(accept_mass=torch.full((B, L), -7.0, device=dev), bound_term=torch.full((B, L), -7.0, device=dev))
     ws = workspace if workspace is not None else csd.new_workspace(B, L, V, w.dtype, dev)
     prm = csd.make_params(
         w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
         out["tokens"], out["accept_len"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
         cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=out["status"],
         dbg_p=out.get("p"), dbg_q=out.get("q"), dbg_f=out.get("f"), dbg_G=out.get("G"),
-        workspace=ws, stream=stream, back_to_back=back_to_back)
+        workspace=ws, stream=stream, back_to_back=back_to_back,
+        diag_accept_mass=out.get("accept_mass"), diag_bound_term=out.get("bound_term"))
     csd.csd_verify_ex(prm)
     torch.cuda.synchronize()
     return {k: v.cpu().numpy() for k, v in out.items()}

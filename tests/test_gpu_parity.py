@@ -183,6 +183,47 @@ def test_large_vocabularies_and_limits(kw):
         assert_ok(rep)
 
 
+@pytest.mark.parametrize("b2b", [False, True])
+@pytest.mark.parametrize("kw", [
+    dict(B=20, gamma=8, V=16384, dtype=W.F32),
+    dict(B=20, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000),
+    dict(B=3, gamma=6, V=8192, dtype=W.BF16, bonus_row=True),
+    dict(B=5, gamma=4, V=4100, dtype=W.F32, top_k=37),           # multi-launch path
+    dict(B=40, gamma=3, V=2048, dtype=W.F32),
+])
+def test_theorem2_position_terms(kw, b2b):
+    """The optional per-position monitors (inner sum of Eq. token_exp, bracket of Eq. bd2) against the
+    oracle's, at every position of every sequence; asking for them must not change the round itself."""
+    L = kw["gamma"]
+    for schedule in (sched(L), csd.csd_make_schedule(0, 1.7, 0.0, L), np.ones(L, np.float32)):
+        w = W.make("t", rho=0.85, schedule=schedule, seed=31, device=DEV, **kw)
+        got = run_gpu(w, want_dbg=False, want_terms=True, back_to_back=b2b)
+        base = run_gpu(w, want_dbg=False, back_to_back=b2b)
+        assert np.array_equal(got["tokens"], base["tokens"]) and np.array_equal(got["accept_len"], base["accept_len"])
+        h = w.host_arrays()
+        ref = oracle.verify(h["target_logits"], h["draft_logits"], h["draft_tokens"], h["uniforms"],
+                            h["relax_schedule"], dtype=w.dtype, target_uncond=h["target_uncond"],
+                            draft_uncond=h["draft_uncond"], cfg_scale=w.cfg_scale, top_k=w.top_k,
+                            want_G=False, want_terms=True)
+        tol = 1e-5 if w.dtype == W.F32 else 2e-3
+        assert np.abs(got["accept_mass"] - ref.accept_mass).max() < tol
+        assert np.abs(got["bound_term"] - ref.bound_term).max() < 2 * tol
+        if np.all(np.asarray(schedule) <= 1.0):
+            assert np.abs(got["bound_term"]).max() < 2 * tol     # vanilla: the bound's bracket vanishes
+
+
+def test_position_terms_on_unusable_rows():
+    L = 4
+    w = W.make("t", B=6, gamma=L, V=4096, dtype=W.F32, rho=0.9, schedule=sched(L), seed=8, device=DEV)
+    w.target_logits[1, 2, 17] = float("nan")
+    w.draft_logits[3, 0, :] = float("-inf")
+    got = run_gpu(w, want_dbg=False, want_terms=True)
+    assert np.isnan(got["accept_mass"][1, 2]) and np.isnan(got["bound_term"][1, 2])
+    assert np.isnan(got["accept_mass"][3, 0]) and np.isnan(got["bound_term"][3, 0])
+    ok = np.ones((6, L), bool); ok[1, 2] = ok[3, 0] = False
+    assert np.all(np.isfinite(got["accept_mass"][ok])) and np.all(got["accept_mass"][ok] <= 1.0 + 1e-5)
+
+
 def test_config_c3_guidance_and_topk():
     """B=64, gamma=8, V=16384, bf16, guidance mix s=4 fused into the load, top-k 1000."""
     L = W.CONFIGS["C3"]["gamma"]
