@@ -235,9 +235,11 @@ struct FinishStage {
   float omega[kMaxGamma];
   float tokz[2][kMaxGamma + 1];
   float p[kMaxGamma], q[kMaxGamma], f[kMaxGamma];
+  float mon_am[kMaxGamma], mon_bt[kMaxGamma];   // per-position monitors of Theorem 2, until they are written out
   SeqRecord rec;
   uint32_t xch[kMaxCluster];   // written by the blocks of the cluster: what each found (see finish_block)
   alignas(8) uint64_t bar;
+  alignas(8) uint64_t bar2;    // second copy barrier of the per-position monitors
 };
 
 // Eq. opt_G summed per tile over the whole row pair, rows brought through the ring by bulk copies;
@@ -433,74 +435,94 @@ __device__ void write_G(const FinishArgs& a, const int b, const int j, const Seq
 }
 
 // The per-position sums of Theorem 2 (inner sum of Eq. token_exp, bracket of Eq. bd2) for the block's
-// positions of sequence b: a second pass over both rows of each position, brought through the ring
-// by bulk copies like the draw.  Follows accept_positions of the same sequence (row statistics in
-// sm); called after the block's griddepcontrol.wait.  red needs two doubles per warp.
+// positions of sequence b: a second pass over both rows of each position, brought through the two
+// halves of the ring by bulk copies (the copies of the next segment run while this one is summed).
+// Follows accept_positions of the same sequence (row statistics in sm); reads only the call's inputs
+// and leaves the results in st.mon_am / st.mon_bt, so it runs before the block's griddepcontrol.wait.
+// red needs two doubles per warp; phase and phase2 are the parities of st.bar and st.bar2.
 template <typename T, bool CFG, int NT, bool FILT>
 __device__ void position_terms(const FinishArgs& a, const BlockShare& sh, const int b, const int tid,
                                unsigned char* ring, const int ring_bytes, double* red, FinishSmem& sm,
-                               FinishStage& st, uint32_t& phase) {
+                               FinishStage& st, uint32_t& phase, uint32_t& phase2) {
   constexpr int VEC = Elem<T>::kVec;
   constexpr int TILE = 32 * VEC;
   constexpr int ARR = CFG ? 2 : 1;
   constexpr int ES = (int)sizeof(T);
   const int lane = tid & 31, warp = tid >> 5;
-  const int V = a.V, L = a.gamma;
+  const int V = a.V;
   const int n_arr = 2 * ARR;
-  const int seg_elems = (ring_bytes / n_arr / (TILE * ES)) * TILE;   // elements of each array per segment
+  const int buf_bytes = ring_bytes / 2;
+  const int seg_elems = (buf_bytes / n_arr / (TILE * ES)) * TILE;   // elements of each array per segment
   const int slot_bytes = seg_elems * ES;
-  for (int i = sh.pos_begin; i < sh.pos_end; ++i) {
-    const bool usable = sm.valid[0][i] && sm.valid[1][i];
-    float am = 0.0f, bt2 = 0.0f;
-    if (usable) {   // (the same decision in every thread)
+  const int nseg = (V + seg_elems - 1) / seg_elems;
+  const int npos = sh.pos_end - sh.pos_begin;
+  const int njobs = npos * nseg;   // job j: segment j % nseg of position pos_begin + j / nseg
+  auto issue = [&](int j) {        // thread 0; the buffer's last reader is behind a barrier
+    const int i = sh.pos_begin + j / nseg;
+    if (!(sm.valid[0][i] && sm.valid[1][i])) return;   // nothing is read for an unusable position
+    const int x0 = (j % nseg) * seg_elems;
+    const uint32_t bytes = (uint32_t)(min(seg_elems, V - x0) * ES);
+    unsigned char* buf = ring + (j & 1) * buf_bytes;
+    uint64_t* bar = (j & 1) ? &st.bar2 : &st.bar;
+    const Row<T, CFG> rt = row_at<T, CFG>(a, b, 0, i), rd = row_at<T, CFG>(a, b, 1, i);
+    fence_before_bulk();
+    mbar_expect_tx(bar, bytes * n_arr);
+    bulk_load(buf, rt.cond + x0, bytes, bar);
+    if (CFG) bulk_load(buf + slot_bytes, rt.uncond + x0, bytes, bar);
+    bulk_load(buf + ARR * slot_bytes, rd.cond + x0, bytes, bar);
+    if (CFG) bulk_load(buf + (ARR + 1) * slot_bytes, rd.uncond + x0, bytes, bar);
+  };
+  __syncthreads();   // everybody is done with what the ring held
+  if (tid == 0 && njobs > 0) issue(0);
+  float am = 0.0f, bt2 = 0.0f;
+  for (int j = 0; j < njobs; ++j) {
+    const int i = sh.pos_begin + j / nseg;
+    const int sg = j % nseg;
+    const bool usable = sm.valid[0][i] && sm.valid[1][i];   // (the same decision in every thread)
+    if (j > 0) __syncthreads();   // job j-1 has been summed: its buffer takes job j+1
+    if (tid == 0 && j + 1 < njobs) issue(j + 1);
+    if (usable) {
+      if (j & 1) { (void)mbar_wait(&st.bar2, phase2); phase2 ^= 1u; }
+      else { (void)mbar_wait(&st.bar, phase); phase ^= 1u; }
+      // (a wait that gives up leaves garbage in a diagnostic only)
       TermsCtx tc;
       tc.Mt = sm.M[0][i]; tc.Md = sm.M[1][i];
       tc.inv_t = 1.0f / (1.0f + sm.S[0][i]); tc.inv_d = 1.0f / (1.0f + sm.S[1][i]);
       tc.omega = st.omega[i];
-      Row<T, CFG> rt = row_at<T, CFG>(a, b, 0, i), rd = row_at<T, CFG>(a, b, 1, i);
+      Row<T, CFG> rt, rd;   // only the thresholds are used here
       rt.thr = sm.thr[0][i];
       rd.thr = sm.thr[1][i];
-      for (int x0 = 0; x0 < V; x0 += seg_elems) {
-        __syncthreads();   // everybody is done with what the ring held
-        const int n = min(seg_elems, V - x0);
-        if (tid == 0) {
-          fence_before_bulk();
-          const uint32_t bytes = (uint32_t)(n * ES);
-          mbar_expect_tx(&st.bar, bytes * n_arr);
-          bulk_load(ring, rt.cond + x0, bytes, &st.bar);
-          if (CFG) bulk_load(ring + slot_bytes, rt.uncond + x0, bytes, &st.bar);
-          bulk_load(ring + ARR * slot_bytes, rd.cond + x0, bytes, &st.bar);
-          if (CFG) bulk_load(ring + (ARR + 1) * slot_bytes, rd.uncond + x0, bytes, &st.bar);
+      const unsigned char* buf = ring + (j & 1) * buf_bytes;
+      const int n = min(seg_elems, V - sg * seg_elems);
+      for (int xo = tid * VEC; xo < n; xo += NT * VEC) {
+        float zt[VEC], zd[VEC];
+        unpack_vec<T>(buf + xo * ES, zt);
+        unpack_vec<T>(buf + ARR * slot_bytes + xo * ES, zd);
+        if (CFG) {
+          float zu[VEC];
+          unpack_vec<T>(buf + slot_bytes + xo * ES, zu);
+          cfg_mix_vec<VEC>(zt, zu, a.cfg_scale);
+          unpack_vec<T>(buf + (ARR + 1) * slot_bytes + xo * ES, zu);
+          cfg_mix_vec<VEC>(zd, zu, a.cfg_scale);
         }
-        (void)mbar_wait(&st.bar, phase);   // (a wait that gives up leaves garbage in a diagnostic only)
-        phase ^= 1u;
-        for (int xo = tid * VEC; xo < n; xo += NT * VEC) {
-          float zt[VEC], zd[VEC];
-          unpack_vec<T>(ring + xo * ES, zt);
-          unpack_vec<T>(ring + ARR * slot_bytes + xo * ES, zd);
-          if (CFG) {
-            float zu[VEC];
-            unpack_vec<T>(ring + slot_bytes + xo * ES, zu);
-            cfg_mix_vec<VEC>(zt, zu, a.cfg_scale);
-            unpack_vec<T>(ring + (ARR + 1) * slot_bytes + xo * ES, zu);
-            cfg_mix_vec<VEC>(zd, zu, a.cfg_scale);
-          }
 #pragma unroll
-          for (int k = 0; k < VEC; ++k)
-            terms_of(FILT ? rt.filter(zt[k]) : zt[k], FILT ? rd.filter(zd[k]) : zd[k], tc, am, bt2);
-        }
+        for (int k = 0; k < VEC; ++k)
+          terms_of(FILT ? rt.filter(zt[k]) : zt[k], FILT ? rd.filter(zd[k]) : zd[k], tc, am, bt2);
       }
     }
-    const double wa = warp_sum_double((double)am), wb = warp_sum_double((double)bt2);
-    __syncthreads();
-    if (lane == 0) { red[2 * warp] = wa; red[2 * warp + 1] = wb; }
-    __syncthreads();
-    if (tid == 0) {
-      double ta = 0.0, tb = 0.0;
-      for (int w = 0; w < NT / 32; ++w) { ta += red[2 * w]; tb += red[2 * w + 1]; }
-      const float nanv = __int_as_float(0x7fc00000);
-      if (a.diag_am) a.diag_am[(int64_t)b * L + i] = usable ? (float)ta : nanv;
-      if (a.diag_bt) a.diag_bt[(int64_t)b * L + i] = usable ? (float)(2.0 * tb) : nanv;
+    if (sg == nseg - 1) {   // the position is complete
+      const double wa = warp_sum_double((double)am), wb = warp_sum_double((double)bt2);
+      if (lane == 0) { red[2 * warp] = wa; red[2 * warp + 1] = wb; }
+      __syncthreads();
+      if (tid == 0) {
+        double ta = 0.0, tb = 0.0;
+        for (int w = 0; w < NT / 32; ++w) { ta += red[2 * w]; tb += red[2 * w + 1]; }
+        const float nanv = __int_as_float(0x7fc00000);
+        st.mon_am[i] = usable ? (float)ta : nanv;
+        st.mon_bt[i] = usable ? (float)(2.0 * tb) : nanv;
+      }
+      am = 0.0f;
+      bt2 = 0.0f;
     }
   }
   __syncthreads();
@@ -682,13 +704,15 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
   const FinishArgs& a = ua.fin;
   const int L = a.gamma;
   const int extra = aborted ? 8 : 0;
-  uint32_t phase = 0;
+  uint32_t phase = 0, phase2 = 0;
   const bool want_terms = a.diag_am != nullptr || a.diag_bt != nullptr;
-  auto write_pqf = [&](int b) {   // diagnostics of this block's positions
+  auto write_pqf = [&](int b) {   // diagnostics and monitors of this block's positions
     if (tid >= sh.pos_begin && tid < sh.pos_end) {
       if (a.dbg_p) a.dbg_p[(int64_t)b * L + tid] = st.p[tid];
       if (a.dbg_q) a.dbg_q[(int64_t)b * L + tid] = st.q[tid];
       if (a.dbg_f) a.dbg_f[(int64_t)b * L + tid] = st.f[tid];
+      if (a.diag_am) a.diag_am[(int64_t)b * L + tid] = st.mon_am[tid];
+      if (a.diag_bt) a.diag_bt[(int64_t)b * L + tid] = st.mon_bt[tid];
     }
   };
   if (ua.ctas_per_seq == 1) {
@@ -698,13 +722,13 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
       const int b = sh.seq_begin + sl;
       const int j = accept_positions<T, CFG, NT>(ua, sh, sl, rs, tid, sm, st);
       draw_position<T, CFG, NT, FILT>(ua, sh, sl, j, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
+      if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase, phase2);
       if (sl == 0) {   // before the block's first global write: outputs of consecutive calls stay in order
         pdl_wait();
         sticky = __ldcg(ua.error_flag) ? 8 : 0;
       }
       write_pqf(b);
       emit_sequence<T, CFG, NT>(ua, b, st.rec, st.rec.status_any | sticky, tid);
-      if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase);
       __syncthreads();
     }
     return;
@@ -726,18 +750,18 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
   }
   if (owner != sh.slot) {   // another block decides the sequence
     if (a.dbg_p || a.dbg_q || a.dbg_f || want_terms) {
+      if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase, phase2);
       pdl_wait();
       write_pqf(b);
-      if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase);
     }
     return;
   }
   draw_position<T, CFG, NT, FILT>(ua, sh, 0, j, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
+  if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase, phase2);
   pdl_wait();   // the previous call has completed: outputs of consecutive calls stay in order
   if (__ldcg(ua.error_flag)) any = 8;
   write_pqf(b);
   emit_sequence<T, CFG, NT>(ua, b, st.rec, any, tid);
-  if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase);
 }
 
 // ======================= plain kernel: one pipeline per warp ============================
@@ -781,7 +805,7 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
   const int part_elems = a.chunks_per_part * EPS;
   const int parts = a.parts_per_row;
 
-  if (tid == 0) { sm.abort = 0; mbar_init(&sm.fst.bar, 1); }
+  if (tid == 0) { sm.abort = 0; mbar_init(&sm.fst.bar, 1); mbar_init(&sm.fst.bar2, 1); }
   if (lane == 0) {
     for (int s = 0; s < kWStages; ++s) mbar_init(&sm.full[warp][s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1164,7 +1188,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
 
   if (tid == 0) {
     for (int s = 0; s < kTkStages; ++s) { mbar_init(&sm.full[s], 1); sm.readers_done[s] = 0; }
-    mbar_init(&sm.fst.bar, 1);
+    mbar_init(&sm.fst.bar, 1); mbar_init(&sm.fst.bar2, 1);
     sm.abort = 0;
     sm.n_cand[0] = 0;
     sm.n_cand[1] = 0;
