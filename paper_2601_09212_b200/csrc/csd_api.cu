@@ -82,11 +82,14 @@ double normal_upper_quantile(double tail) {
 template <typename T, bool CFG>
 cudaError_t launch_fused(const FusedArgs& a, int grid, bool overlap, cudaStream_t stream) {
   auto kern = verify_topk_kernel<T, CFG>;
-  static bool configured = false;
-  if (!configured) {
+  // the attribute belongs to (function, device): set it once per device (setting it twice is harmless)
+  static bool configured[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TopkSmem));
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured[dev] = true;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
@@ -116,11 +119,14 @@ cudaError_t launch_fused(const FusedArgs& a, int grid, bool overlap, cudaStream_
 template <typename T, bool CFG>
 cudaError_t launch_plain(const FusedArgs& a, int grid, bool overlap, cudaStream_t stream) {
   auto kern = verify_plain_kernel<T, CFG>;
-  static bool configured = false;
-  if (!configured) {
+  // the attribute belongs to (function, device): set it once per device (setting it twice is harmless)
+  static bool configured[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PlainSmem));
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured[dev] = true;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
