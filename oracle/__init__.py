@@ -78,6 +78,9 @@ def _load():
         lib.orc_prepare_row.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int,
                                         C.c_float, C.c_int, C.c_void_p, C.c_void_p]
         lib.orc_prepare_row.restype = None
+        lib.orc_sample_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_float, C.c_int, C.c_int, C.c_int,
+                                        C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.orc_sample_rows.restype = C.c_int
         lib.orc_verify.argtypes = [C.POINTER(_Params)]
         lib.orc_verify.restype = C.c_int
         _lib = lib
@@ -171,6 +174,22 @@ def prepare_row(cond, uncond, dtype: int, cfg_scale: float, top_k: int) -> np.nd
     _load().orc_prepare_row(_ptr(cond), _ptr(un), int(dtype), 0, V, float(cfg_scale), int(top_k),
                             _ptr(z), _ptr(scratch))
     return z
+
+
+def sample_rows(logits, uniforms, *, dtype: int = F32, uncond=None, cfg_scale: float = 1.0, top_k: int = 0):
+    """Algorithm 1, drafting stage: one inverse-CDF draw per row of ``logits`` [R, V] with ``uniforms`` [R].
+    Returns (tokens int32 [R], status int32 [R], margin float64 [R])."""
+    z = _raw(logits, dtype)
+    R, V = z.shape
+    zu = None if uncond is None else _raw(uncond, dtype)
+    uni = np.ascontiguousarray(uniforms, dtype=np.float32)
+    assert uni.shape == (R,)
+    tok, st, mg = np.empty(R, np.int32), np.zeros(R, np.int32), np.empty(R)
+    rc = _load().orc_sample_rows(_ptr(z), _ptr(zu), int(dtype), float(cfg_scale), int(top_k), R, V, V,
+                                 _ptr(uni), _ptr(tok), _ptr(st), _ptr(mg))
+    if rc != 0:
+        raise RuntimeError(f"orc_sample_rows failed with code {rc}")
+    return tok, st, mg
 
 
 @dataclass

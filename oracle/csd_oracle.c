@@ -6,7 +6,8 @@
  * paper (verification stage), the relaxed acceptance probability (Eq. relax),
  * the annealing schedules (UniformRSD, Eq. sdar, and the linear variant of the
  * schedule ablation), and the bound-minimising resampling distribution
- * (Eq. opt_G, Theorem 2 / Proposition LP); and, per position, the two sums that
+ * (Eq. opt_G, Theorem 2 / Proposition LP); the drafting stage's token draws
+ * x~_i ~ Q(. | prefix) (Algorithm 1, drafting stage); and, per position, the two sums that
  * Theorem 2 is made of: the acceptance mass sum_x Q f (the inner sum of Eq.
  * token_exp) and the bracket of Eq. bd2, sum_x |P - Q f| - sum_x (1 - f) Q.
  *
@@ -423,6 +424,38 @@ static void verify_one(const orc_params *a, int b, double *zt, double *zd, doubl
       }
     }
   }
+}
+
+/* ---- Algorithm 1, drafting stage: one token per row -------------------------------------------
+ * x~ ~ Q(. | prefix): for each of R rows of logits (prepared like the verification's rows: optional
+ * guidance mix in fp32, optional top-k), the softmax and one inverse-CDF draw with the row's supplied
+ * uniform (same convention as the verification's draws).  out_tokens[r] = -1 and status bit BADROW for
+ * an unusable row.  margin[r] (optional) is the distance of u to the nearest CDF boundary of the pick.
+ * Returns 0, or -1 on bad shapes, -2 if memory could not be had. */
+int orc_sample_rows(const void *logits, const void *uncond, int dtype, float cfg_scale, int top_k, int R,
+                    int V, int64_t row_stride, const float *uniforms, int32_t *out_tokens,
+                    int32_t *out_status, double *margin) {
+  if (!logits || !uniforms || !out_tokens || R < 1 || V < 2 || row_stride < V) return -1;
+  double *buf = (double *)malloc(3 * (size_t)V * sizeof(double));
+  if (!buf) return -2;
+  double *z = buf, *P = buf + V, *scratch = buf + 2 * (size_t)V;
+  for (int r = 0; r < R; ++r) {
+    orc_prepare_row(logits, uncond, dtype, (int64_t)r * row_stride, V, cfg_scale, top_k, z, scratch);
+    int status = 0;
+    double mg = INFINITY;
+    if (orc_softmax(z, V, P)) {
+      double Z = 0.0;
+      for (int x = 0; x < V; ++x) Z += P[x];
+      out_tokens[r] = orc_inverse_cdf(P, V, Z, (double)uniforms[r], &mg);
+    } else {
+      out_tokens[r] = -1;
+      status = ORC_STATUS_BADROW;
+    }
+    if (out_status) out_status[r] = status;
+    if (margin) margin[r] = mg;
+  }
+  free(buf);
+  return 0;
 }
 
 /* Batched driver: sequences are independent.  Returns 0, or -1 on bad shapes,

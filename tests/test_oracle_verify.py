@@ -158,3 +158,40 @@ def test_verify_reports_position_terms(oracle):
                 mn = np.minimum(Q, om[i] * P)
                 assert np.isclose(r.accept_mass[b, i], mn.sum(), rtol=1e-11)
                 assert np.isclose(r.bound_term[b, i], 2.0 * np.maximum(mn - P, 0.0).sum(), rtol=1e-9, atol=1e-13)
+
+
+@pytest.mark.parametrize("dtype", [W.F32, W.BF16])
+def test_sample_rows_against_library_routines(oracle, dtype):
+    """Drafting-stage draws: scipy softmax + cumsum/searchsorted on the prepared rows; chi-square of the
+    drawn tokens against the row's distribution; an unusable row gives -1 and the status bit."""
+    rng = np.random.default_rng(4)
+    R, V = 40, 300
+    w = W.make("t", B=R, gamma=1, V=V, dtype=dtype, rho=0.8, schedule=np.ones(1, np.float32), seed=12,
+               cfg=True, cfg_scale=3.0, top_k=25)
+    h = w.host_arrays()
+    logits, unc = h["draft_logits"][:, 0], h["draft_uncond"][:, 0]
+    uni = ((rng.integers(0, 2 ** 23, size=R) * 2 + 1) * 2.0 ** -24).astype(np.float32)
+    tok, st, mg = oracle.sample_rows(logits, uni, dtype=dtype, uncond=unc, cfg_scale=3.0, top_k=25)
+    for r in range(R):
+        z = oracle.prepare_row(logits[r], unc[r], dtype, 3.0, 25)
+        P = sps.softmax(z)
+        cum = np.cumsum(P)
+        assert tok[r] == int(np.searchsorted(cum, float(uni[r]) * cum[-1], side="right")) and P[tok[r]] > 0
+        assert (np.isfinite(z)).sum() >= 25 and st[r] == 0
+    # the law of the draw: many uniforms on one row
+    n = 20000
+    row = np.repeat(logits[:1], n, axis=0)
+    us = ((rng.integers(0, 2 ** 23, size=n) * 2 + 1) * 2.0 ** -24).astype(np.float32)
+    toks, _, _ = oracle.sample_rows(row, us, dtype=dtype, uncond=np.repeat(unc[:1], n, axis=0), cfg_scale=3.0, top_k=25)
+    P = sps.softmax(oracle.prepare_row(logits[0], unc[0], dtype, 3.0, 25))
+    keep = P > 0
+    obs = np.bincount(toks, minlength=V)[keep]
+    assert obs.sum() == n
+    chi2 = ((obs - n * P[keep]) ** 2 / (n * P[keep])).sum()
+    assert chi2 < 25 + 6 * np.sqrt(2 * 25)          # about 6 sigma for keep.sum() - 1 degrees of freedom
+    bad = np.array(logits[:2], copy=True)
+    bad_f = _decode(bad, dtype)
+    if dtype == W.F32:
+        bad[1, 3] = np.nan
+        tok2, st2, _ = oracle.sample_rows(bad, uni[:2], dtype=dtype, uncond=unc[:2], cfg_scale=3.0, top_k=25)
+        assert tok2[1] == -1 and st2[1] == oracle.STATUS_BADROW and tok2[0] == tok[0]
