@@ -43,7 +43,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
 # one ncu capture, see profiles/verify_topk_kernel_C3.md).  Reported only while the kernel sources
 # still have the digest the capture was taken with; null otherwise.
-NCU_TRAFFIC = {"sources_sha256": "9ececc5a050525b5", "workload": "C3", "bytes_per_launch": 68067840}
+NCU_TRAFFIC = {"sources_sha256": "47cd41dbc14a77a7", "workload": "C3", "bytes_per_launch": 68067840}
 
 
 def sources_digest() -> str:
@@ -429,6 +429,74 @@ def run_native(args) -> None:
         dist.destroy_process_group()
 
 
+def run_drafting_stage(args) -> None:
+    """Side measurement (not the headline): csd_sample_rows on the drafter rows of the workload --
+    R = B * gamma rows, one token each -- timed like the round: resident inputs larger than L2, a CUDA
+    graph of 64 calls replayed, CUDA events on the launching stream.  One GPU."""
+    import torch
+    from paper_2601_09212_b200 import _build, workloads as W
+    import paper_2601_09212_b200 as csd
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    _build.build_library()
+    name = args.workload
+    kw = workload_kwargs(name)
+    B, L, V, dtype = kw["B"], kw["gamma"], kw["V"], kw.get("dtype", W.F32)
+    R = B * L
+    arrays = 2 if kw.get("cfg") else 1
+    step_bytes = R * V * (2 if dtype == W.BF16 else 4) * arrays + 8 * R
+    ring_n = min(64, max(4, -(-4 * L2_BYTES // step_bytes)))
+    sched = csd.csd_make_schedule(1, 1.1, 0.7, L)
+    ring = [W.make(name, seed=1, step=s, schedule=sched, device=dev, **kw) for s in range(ring_n)]
+    stream = torch.cuda.Stream(device=dev)
+    calls = []
+    for w in ring:
+        calls.append(dict(
+            logits=w.draft_logits.reshape(R, V), unc=None if w.draft_uncond is None else w.draft_uncond.reshape(R, V),
+            uni=torch.rand(R, device=dev) * 0.999 + 0.0005, tok=torch.empty(R, dtype=torch.int32, device=dev),
+            ws=torch.zeros(csd.csd_sample_workspace_size(R, V, dtype), dtype=torch.uint8, device=dev),
+            scale=w.cfg_scale, k=w.top_k))
+
+    def enqueue(i):
+        c = calls[i % ring_n]
+        csd.csd_sample_rows(c["logits"], c["uni"], c["tok"], uncond=c["unc"], cfg_scale=c["scale"], top_k=c["k"],
+                            workspace=c["ws"], back_to_back=not args.single_call_latency, stream=stream)
+
+    graph_steps = ring_n * max(1, -(-64 // ring_n))
+    with torch.cuda.stream(stream):
+        for i in range(ring_n):
+            enqueue(i)
+    stream.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        for i in range(graph_steps):
+            enqueue(i)
+    replays = max(1, args.steps // graph_steps)
+    with torch.cuda.stream(stream):
+        for _ in range(max(1, args.warmup // graph_steps)):
+            graph.replay()
+    stream.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        e0.record(stream)
+        for _ in range(replays):
+            graph.replay()
+        e1.record(stream)
+    stream.synchronize()
+    steps = replays * graph_steps
+    ms = e0.elapsed_time(e1)
+    peak, peak_kind = measured_peak()
+    achieved = step_bytes / (ms * 1e-3 / steps) / 1e9
+    print(json.dumps({
+        "metric": "sampled_draft_tokens_per_sec", "value": R * steps / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+        "steps": steps, "ms_per_step": ms / steps, "higher_is_better": True, "data": "synthetic",
+        "config": dict(describe(name, kw, "-"), rows=R, op="csd_sample_rows (Algorithm 1, drafting stage)",
+                       launch=f"CUDA graph of {graph_steps} calls, replayed"),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": peak_kind, "bytes_per_launch": step_bytes, "traffic": None},
+    }))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -441,9 +509,13 @@ def main() -> None:
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="C3")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--drafting-stage", action="store_true",
+                    help="side measurement: time csd_sample_rows on the workload's drafter rows instead of the round")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.drafting_stage:
+        run_drafting_stage(args)
     else:
         run_native(args)
 

@@ -247,6 +247,27 @@ int csd_verify_host(const csd_params* host, void* staging, size_t staging_bytes)
 size_t csd_host_staging_size(const csd_params* host);
 
 /*
+ * Drafting stage (Algorithm 1, "x~_i ~ Q(. | prefix)"): one token per row of logits, drawn from the
+ * row's softmax with the same input preparation as the verification (guidance mix fused into the
+ * load -- the paper runs the drafter under classifier-free guidance, Additional Implementation
+ * Details -- and top-k) and the same inverse-CDF convention.
+ *   logits      DEVICE, R rows of V elements (fp32 or bf16), row r at element r*row_stride
+ *               (row_stride 0 means V); 16-byte alignment as for csd_verify_ex's fast path
+ *   uncond      DEVICE, same layout, or NULL (no guidance mix)
+ *   uniforms    DEVICE [R] in (0, 1): token r = smallest x with C_r(x) > uniforms[r] * Z_r
+ *   out_tokens  DEVICE [R]; -1 for a row that holds NaN or +inf or no finite entry
+ *   out_status  DEVICE [R] or NULL: CSD_STATUS_BADROW / CSD_STATUS_TIMEOUT
+ *   workspace   DEVICE, >= csd_sample_workspace_size(R, V, dtype) bytes, 256-byte aligned, zero-filled
+ *               once before its first use
+ *   back_to_back  as in csd_params
+ * Returns CSD_OK or a negative csd_error; nothing is enqueued on an error.
+ */
+size_t csd_sample_workspace_size(int R, int V, int dtype);
+int csd_sample_rows(const void* logits, const void* uncond, float cfg_scale, int top_k, int dtype, int R, int V,
+                    int64_t row_stride, const float* uniforms, int32_t* out_tokens, int32_t* out_status,
+                    void* workspace, size_t workspace_bytes, int back_to_back, void* stream);
+
+/*
  * Relaxation schedules, written to HOST memory out_host[0..L-1] = omega_1..omega_L.
  *   kind 0  UniformRSD: omega_i = delta.
  *   kind 1  Cool-SD, Eq. sdar: omega_i = delta * exp(-nu*i - mu) with mu fixed by

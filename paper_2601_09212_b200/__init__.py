@@ -21,7 +21,8 @@ CSD_F32, CSD_BF16 = 0, 1
 CSD_STATUS_BADROW, CSD_STATUS_BADTOKEN, CSD_STATUS_ZFALLBACK, CSD_STATUS_TIMEOUT = 1, 2, 4, 8
 CSD_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
 EXPORTS = ("csd_verify", "csd_verify_static", "csd_verify_ex", "csd_workspace_size", "csd_workspace_init", "csd_launch_count", "csd_verify_host",
-           "csd_host_staging_size", "csd_make_schedule", "csd_error_string", "csd_version")
+           "csd_host_staging_size", "csd_make_schedule", "csd_error_string", "csd_version",
+           "csd_sample_rows", "csd_sample_workspace_size")
 
 
 class CsdError(RuntimeError):
@@ -80,6 +81,12 @@ def library() -> C.CDLL:
         lib.csd_error_string.argtypes = [C.c_int]
         lib.csd_error_string.restype = C.c_char_p
         lib.csd_version.restype = C.c_int
+        lib.csd_sample_workspace_size.argtypes = [C.c_int] * 3
+        lib.csd_sample_workspace_size.restype = C.c_size_t
+        lib.csd_sample_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_int, C.c_int, C.c_int, C.c_int,
+                                        C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                        C.c_int, C.c_void_p]
+        lib.csd_sample_rows.restype = C.c_int
         _lib = lib
     return _lib
 
@@ -270,6 +277,27 @@ def new_workspace(B: int, gamma: int, V: int, dtype: int, device="cuda") -> torc
     if n == 0:
         raise CsdError(-2, "csd_workspace_size")
     return torch.zeros(n, dtype=torch.uint8, device=device)
+
+
+def csd_sample_workspace_size(R: int, V: int, dtype: int) -> int:
+    return int(library().csd_sample_workspace_size(int(R), int(V), int(dtype)))
+
+
+def csd_sample_rows(logits, uniforms, out_tokens, *, uncond=None, cfg_scale=1.0, top_k=0, out_status=None,
+                    workspace=None, back_to_back=False, stream=None) -> None:
+    """Drafting stage: one inverse-CDF draw per row of ``logits`` [R, V] (device tensors)."""
+    R, V = logits.shape
+    dt = _logit_dtype(logits)
+    ldt = logits.dtype
+    if workspace is None:
+        workspace = torch.zeros(csd_sample_workspace_size(R, V, dt), dtype=torch.uint8, device=logits.device)
+    rc = library().csd_sample_rows(
+        _dev_ptr(logits, "logits", ldt), _dev_ptr(uncond, "uncond", ldt), float(cfg_scale), int(top_k), dt, R, V,
+        V, _dev_ptr(uniforms, "uniforms", torch.float32), _dev_ptr(out_tokens, "out_tokens", torch.int32),
+        _dev_ptr(out_status, "out_status", torch.int32), _dev_ptr(workspace, "workspace"),
+        workspace.numel() * workspace.element_size(), 1 if back_to_back else 0, _stream_handle(stream))
+    if rc != 0:
+        raise CsdError(rc, "csd_sample_rows")
 
 
 def csd_workspace_init(workspace: torch.Tensor, stream=None) -> None:

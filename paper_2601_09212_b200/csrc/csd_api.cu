@@ -220,12 +220,21 @@ cudaError_t launch_finish(const FinishArgs& a, cudaStream_t stream) {
   return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
-int verify_impl(const csd_params& p, int* plan_only = nullptr) {
-  if (!p.target_logits || !p.draft_logits || !p.draft_tokens || !p.uniforms || !p.relax_schedule ||
-      !p.out_tokens || !p.out_accept_len)
+// sampling: the degenerate round used by csd_sample_rows -- no draft positions (gamma = 0), one
+// "target" row per sequence, whose bonus draw is the wanted token; the drafter-side pointers are unused.
+int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = false) {
+  if (sampling) {
+    if (!p.target_logits || !p.uniforms || !p.out_tokens) return CSD_ERR_NULL;
+  } else if (!p.target_logits || !p.draft_logits || !p.draft_tokens || !p.uniforms || !p.relax_schedule ||
+             !p.out_tokens || !p.out_accept_len) {
     return CSD_ERR_NULL;
+  }
   if (p.dtype != CSD_F32 && p.dtype != CSD_BF16) return CSD_ERR_DTYPE;
-  if (!shape_ok(p.B, p.gamma, p.V)) return CSD_ERR_SHAPE;
+  if (sampling) {
+    if (p.B < 1 || p.gamma != 0 || p.target_rows != 1 || p.V < 2 || p.V > kMaxV) return CSD_ERR_SHAPE;
+  } else if (!shape_ok(p.B, p.gamma, p.V)) {
+    return CSD_ERR_SHAPE;
+  }
   if (p.target_rows != p.gamma && p.target_rows != p.gamma + 1) return CSD_ERR_SHAPE;
   const int64_t tstride = p.target_batch_stride ? p.target_batch_stride : (int64_t)p.target_rows * p.V;
   const int64_t dstride = p.draft_batch_stride ? p.draft_batch_stride : (int64_t)p.gamma * p.V;
@@ -416,6 +425,35 @@ int csd_launch_count(const csd_params* p) {
 int csd_verify_ex(const csd_params* p) {
   if (!p) return CSD_ERR_NULL;
   return verify_impl(*p);
+}
+
+size_t csd_sample_workspace_size(int R, int V, int dtype) {
+  if (R < 1 || V < 2 || V > kMaxV || (dtype != CSD_F32 && dtype != CSD_BF16)) return 0;
+  return layout_for(R, 0, V, dtype).total;
+}
+
+int csd_sample_rows(const void* logits, const void* uncond, float cfg_scale, int top_k, int dtype, int R, int V,
+                    int64_t row_stride, const float* uniforms, int32_t* out_tokens, int32_t* out_status,
+                    void* workspace, size_t workspace_bytes, int back_to_back, void* stream) {
+  csd_params p;
+  memset(&p, 0, sizeof p);
+  p.target_logits = logits;
+  p.draft_logits = logits;       // unused: there are no draft positions
+  p.target_uncond = uncond;
+  p.draft_uncond = uncond;
+  p.cfg_scale = cfg_scale;
+  p.top_k = top_k;
+  p.dtype = dtype;
+  p.B = R; p.gamma = 0; p.V = V; p.target_rows = 1;
+  p.target_batch_stride = row_stride;
+  p.uniforms = uniforms;         // [R]: the round's layout [B, gamma + 1] with gamma = 0
+  p.out_tokens = out_tokens;     // [R]: the round's layout [B, gamma + 1]
+  p.out_status = out_status;
+  p.workspace = workspace;
+  p.workspace_bytes = workspace_bytes;
+  p.back_to_back = back_to_back;
+  p.stream = stream;
+  return verify_impl(p, nullptr, true);
 }
 
 int csd_verify(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,

@@ -678,7 +678,7 @@ __device__ void emit_sequence(const FusedArgs& ua, const int b, const SeqRecord&
     a.out_tokens[(int64_t)b * (L + 1) + tid] = v;
   }
   if (tid == 0) {
-    a.out_accept_len[b] = tau;
+    if (a.out_accept_len) a.out_accept_len[b] = tau;
     if (a.out_status) a.out_status[b] = win.status_at | status_any;
   }
   if (a.dbg_G) {

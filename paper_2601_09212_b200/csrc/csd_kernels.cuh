@@ -734,7 +734,7 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
     a.out_tokens[(int64_t)b * (L + 1) + tid] = v;
   }
   if (tid == 0) {
-    a.out_accept_len[b] = tau;
+    if (a.out_accept_len) a.out_accept_len[b] = tau;
     if (a.out_status) a.out_status[b] = status;
   }
   // ---- 9. optional: the per-position sums of Theorem 2 (a second pass over every row) ------------

@@ -224,6 +224,58 @@ def test_position_terms_on_unusable_rows():
     assert np.all(np.isfinite(got["accept_mass"][ok])) and np.all(got["accept_mass"][ok] <= 1.0 + 1e-5)
 
 
+@pytest.mark.parametrize("b2b", [False, True])
+@pytest.mark.parametrize("kw", [
+    dict(R=64, V=16384, dtype=W.F32),
+    dict(R=300, V=16384, dtype=W.BF16, cfg=True, top_k=1000),
+    dict(R=5, V=65536, dtype=W.BF16),
+    dict(R=33, V=4100, dtype=W.F32, top_k=50),            # multi-launch path
+    dict(R=1, V=2048, dtype=W.F32, cfg=True),
+])
+def test_drafting_stage_sampling(kw, b2b):
+    """csd_sample_rows (Algorithm 1, drafting stage) against the oracle's draws on the same rows and
+    uniforms: identical tokens except where the oracle reports the uniform within 1e-6 of a CDF boundary."""
+    kw = dict(kw)
+    R = kw.pop("R")
+    w = W.make("t", B=R, gamma=1, rho=0.9, schedule=np.ones(1, np.float32), seed=41, device=DEV, **kw)
+    logits = w.draft_logits[:, 0].contiguous()
+    unc = None if w.draft_uncond is None else w.draft_uncond[:, 0].contiguous()
+    uni = w.uniforms[:, 0].contiguous()
+    tok = torch.full((R,), -7, dtype=torch.int32, device=DEV)
+    st = torch.full((R,), -7, dtype=torch.int32, device=DEV)
+    csd.csd_sample_rows(logits, uni, tok, uncond=unc, cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=st,
+                        back_to_back=b2b)
+    torch.cuda.synchronize()
+    h = w.host_arrays()
+    ref_tok, ref_st, margin = oracle.sample_rows(
+        h["draft_logits"][:, 0], h["uniforms"][:, 0], dtype=w.dtype,
+        uncond=None if h["draft_uncond"] is None else h["draft_uncond"][:, 0], cfg_scale=w.cfg_scale, top_k=w.top_k)
+    got = tok.cpu().numpy()
+    differ = got != ref_tok
+    assert np.all(margin[differ] < 1e-6), (np.flatnonzero(differ)[:5], margin[differ][:5])
+    assert differ.sum() <= max(1, R // 50)
+    assert np.array_equal(st.cpu().numpy(), ref_st)
+    assert got.min() >= 0 and got.max() < w.V
+
+
+def test_drafting_stage_sampling_bad_row_and_errors():
+    R, V = 6, 4096
+    logits = torch.randn(R, V, device=DEV)
+    logits[2, 7] = float("nan")
+    logits[4, :] = float("-inf")
+    uni = torch.full((R,), 0.37, device=DEV)
+    tok = torch.full((R,), -7, dtype=torch.int32, device=DEV)
+    st = torch.full((R,), -7, dtype=torch.int32, device=DEV)
+    csd.csd_sample_rows(logits, uni, tok, out_status=st)
+    torch.cuda.synchronize()
+    t, s_ = tok.cpu().numpy(), st.cpu().numpy()
+    assert t[2] == -1 and t[4] == -1 and s_[2] == 1 and s_[4] == 1
+    assert np.all(t[[0, 1, 3, 5]] >= 0) and np.all(s_[[0, 1, 3, 5]] == 0)
+    lib = csd.library()
+    assert lib.csd_sample_rows(None, None, 1.0, 0, 0, R, V, 0, None, None, None, None, 0, 0, None) == -1
+    assert csd.csd_sample_workspace_size(0, V, 0) == 0
+
+
 def test_config_c3_guidance_and_topk():
     """B=64, gamma=8, V=16384, bf16, guidance mix s=4 fused into the load, top-k 1000."""
     L = W.CONFIGS["C3"]["gamma"]
