@@ -231,6 +231,7 @@ def test_position_terms_on_unusable_rows():
     dict(R=5, V=65536, dtype=W.BF16),
     dict(R=33, V=4100, dtype=W.F32, top_k=50),            # multi-launch path
     dict(R=1, V=2048, dtype=W.F32, cfg=True),
+    dict(R=1500, V=2048, dtype=W.BF16),                   # several rows per block
 ])
 def test_drafting_stage_sampling(kw, b2b):
     """csd_sample_rows (Algorithm 1, drafting stage) against the oracle's draws on the same rows and
