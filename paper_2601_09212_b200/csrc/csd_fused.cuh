@@ -770,8 +770,8 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
 // a running (m, s) per lane that it reduces once per item.  Eight such pipelines per block sit
 // at different points of their loops and hide each other's latencies; phase 1 has no block-wide
 // step at all.
-constexpr int kWStages = 3;
-constexpr int kWStageBytes = 2048;
+constexpr int kWStages = 2;
+constexpr int kWStageBytes = 3072;
 constexpr int kBlockStash = 1536;   // items (row parts) a block may own
 constexpr int kPlainRingBytes = kPlainWarps * kWStages * kWStageBytes;
 
@@ -794,7 +794,8 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
   constexpr int EPS = kWStageBytes / ((int)sizeof(T) * ARR);   // elements of a row per warp stage
   constexpr int VPL = EPS / 32;                                // values per lane per stage
   constexpr int NVS = VPL / VEC;                               // 16-byte vectors per lane per stage
-  constexpr int GV = NVS > 2 ? 2 : NVS;                        // vectors reduced together (register budget)
+  constexpr int GV = (NVS % 2 == 0) ? 2 : 1;                   // vectors reduced together (register budget)
+  static_assert(NVS % GV == 0 && NVS >= 1, "a stage is a whole number of groups");
   extern __shared__ __align__(128) unsigned char fused_smem_raw[];
   PlainSmem& sm = *reinterpret_cast<PlainSmem*>(fused_smem_raw);
 
