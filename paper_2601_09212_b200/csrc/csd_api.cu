@@ -317,6 +317,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
     ua.fin = fa;
     ua.top_k = p.top_k;
     ua.lo_sigmas = nanf("");
+    ua.lo_delta = 0.0f;
     ua.error_flag = reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
     // Blocks are aligned with sequences and positions.  For calls enqueued back to back a block owns a
     // whole sequence (for very large batches seqs_per_cta of them): such calls overlap on the GPU as
@@ -339,7 +340,10 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
       ua.parts_per_row = 1;
       const double k = p.top_k, v = p.V;
       const double tail = 1.25 * k / v + 4.0 * sqrt(k) / v + 16.0 / v;
-      if (tail < 0.45 && tail * v < 0.8 * kListCap) ua.lo_sigmas = (float)normal_upper_quantile(tail);
+      if (tail < 0.45 && tail * v < 0.8 * kListCap) {
+        ua.lo_sigmas = (float)normal_upper_quantile(tail);
+        ua.lo_delta = ua.lo_sigmas - (float)normal_upper_quantile(k / v);
+      }
     } else {
       // warp-wide items: parts of rows, sized so that every warp of the grid gets several
       const int eps = kWStageBytes / (es * (cfg ? 2 : 1));

@@ -153,6 +153,7 @@ struct FusedArgs {
   int seqs_per_cta;
   int top_k;
   float lo_sigmas;      // top-k guess: lo = mean + lo_sigmas * deviation (NaN: always select exactly)
+  float lo_delta;       // how many deviations below a row's exact threshold the next guess should sit (< 0)
   int* error_flag;      // set when a bounded wait gave up
 };
 
@@ -1070,6 +1071,10 @@ struct TopkSmem {
   int abort;
   FinishSmem fin;
   FinishStage fst;
+  float c_kind[2];                  // by row parity (target / drafter rows alternate): the multiplier of the
+                                    //   deviation in the guess, adapted from the rows already done
+  float row_mean[2], row_dev[2];    // by row parity: the sample's moments (for that adaptation)
+  int adapt_on;                     // set once a guess has missed: from then on every row adapts the multiplier
 };
 
 // Bin (of kLinBins, counted in `hist`) that holds the k-th largest value, found by one warp:
@@ -1195,6 +1200,9 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
     sm.n_cand[1] = 0;
     sm.arrive[0] = 0;
     sm.arrive[1] = 0;
+    sm.c_kind[0] = a.lo_sigmas;
+    sm.c_kind[1] = a.lo_sigmas;
+    sm.adapt_on = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < (kBlockRows + 31) / 32) sm.need_exact[tid] = 0u;
@@ -1347,8 +1355,9 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
           for (int w = 0; w < kTopkWarps; ++w) { s1 += sm.mom[w][0]; s2 += sm.mom[w][1]; nn += sm.mom[w][2]; }
           const float mean = s1 / nn;
           const float dev = sqrtf(fmaxf(s2 / nn - mean * mean, 0.0f));
-          lo = mean + a.lo_sigmas * dev;
+          lo = mean + sm.c_kind[par] * dev;
           scale = (float)kLinBins / (kLinRangeSigmas * dev);
+          if (tid == 0) { sm.row_mean[par] = mean; sm.row_dev[par] = dev; }
         }
         // ---- gather this stage's values >= lo into the warp's list -------------------------
         // (the test is "not below lo", so that a NaN lands in the list and marks the row through the
@@ -1445,6 +1454,10 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
           if (lane == 0) { sm.bc_i[0] = bin; sm.bc_i[1] = kk; }
         }
         if (lane == 0) {
+          // a guess that missed moves the next one of this kind of row: down if too few values were
+          // gathered, up if a list overflowed (a NaN multiplier -- no guess at all -- stays NaN)
+          if (!fast && n_lo < k_top) { sm.c_kind[par] -= 0.5f; sm.adapt_on = 1; }
+          else if (!fast && n_lo > kListCap / 2) { sm.c_kind[par] += 0.35f; sm.adapt_on = 1; }
           sm.row_mx = m;
           sm.row_fast = fast ? 1 : 0;
           if (!fast && n_my < kBlockRows) atomicOr(&sm.need_exact[n_my >> 5], 1u << (n_my & 31));
@@ -1527,6 +1540,13 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
               sm.part_cmax[par][kTopkWarps] = cmax2;
               sm.part_max[par] = mx;
               sm.part_thr[par] = thr;
+              // where the threshold really sat, in deviations from the mean: the next row of this kind
+              // guesses a little below that (half-way from the current multiplier)
+              // (only once the plain guess has missed in this block: data it fits is left alone)
+              if (sm.adapt_on) {
+                const float c_seen = (thr - sm.row_mean[par]) / sm.row_dev[par] + a.lo_delta;
+                if (c_seen == c_seen && fabsf(c_seen) < 64.0f) sm.c_kind[par] = 0.5f * (sm.c_kind[par] + c_seen);
+              }
             }
           } else if (lane == 0 && n_my < kBlockRows) {   // crowded bin
             atomicOr(&sm.need_exact[n_my >> 5], 1u << (n_my & 31));
