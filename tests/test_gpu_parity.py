@@ -277,6 +277,21 @@ def test_drafting_stage_sampling_bad_row_and_errors():
     assert csd.csd_sample_workspace_size(0, V, 0) == 0
 
 
+@pytest.mark.parametrize("b2b", [False, True])
+def test_topk_on_heavy_tailed_rows(b2b):
+    """Student-t logits: the normal-quantile guess of the streaming selection misses, rows are selected
+    exactly or with the adapted guess; the results must not depend on which."""
+    L = 8
+    w = W.make("t", B=20, gamma=L, V=16384, dtype=W.BF16, rho=0.85, law="student3", top_k=1000,
+               schedule=sched(L), seed=13, device=DEV)
+    rep, got, ref = check(w, back_to_back=b2b)
+    assert_ok(rep)
+    w = W.make("t", B=6, gamma=4, V=16384, dtype=W.F32, rho=0.85, law="student3", cfg=True, top_k=300,
+               schedule=sched(4), seed=14, device=DEV)
+    rep, got, ref = check(w, back_to_back=b2b)
+    assert_ok(rep)
+
+
 def test_config_c3_guidance_and_topk():
     """B=64, gamma=8, V=16384, bf16, guidance mix s=4 fused into the load, top-k 1000."""
     L = W.CONFIGS["C3"]["gamma"]
