@@ -30,9 +30,15 @@ STATUS_BADROW, STATUS_BADTOKEN, STATUS_ZFALLBACK = 1, 2, 4
 def build(force: bool = False) -> str:
     """Compile the C oracle with gcc (OpenMP on, no fast-math, no contraction)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = f"{_LIB}.{os.getpid()}.tmp"   # moved into place when complete: no process sees half a library
         cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
-               "-fno-fast-math", "-Wall", "-Wextra", "-o", _LIB, _SRC, "-lm"]
-        subprocess.run(cmd, check=True)
+               "-fno-fast-math", "-Wall", "-Wextra", "-o", tmp, _SRC, "-lm"]
+        try:
+            subprocess.run(cmd, check=True)
+            os.replace(tmp, _LIB)
+        finally:
+            if os.path.exists(tmp):
+                os.remove(tmp)
     return _LIB
 
 

@@ -23,11 +23,28 @@ def is_stale() -> bool:
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
-    if force or is_stale():
-        os.makedirs(LIB_DIR, exist_ok=True)
-        nvcc = os.environ.get("NVCC", "nvcc")
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB_PATH] + SOURCES
-        subprocess.run(cmd, check=True)
+    """Compiles the library if it is missing or older than its sources.  Safe when several processes
+    (one per GPU) start at once: one of them builds, under a file lock, into a temporary file that is
+    then moved into place; the others wait and find it fresh."""
+    if not (force or is_stale()):
+        return LIB_PATH
+    import fcntl
+    os.makedirs(LIB_DIR, exist_ok=True)
+    with open(os.path.join(LIB_DIR, ".build.lock"), "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            if force or is_stale():
+                nvcc = os.environ.get("NVCC", "nvcc")
+                tmp = f"{LIB_PATH}.{os.getpid()}.tmp"
+                cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
+                try:
+                    subprocess.run(cmd, check=True)
+                    os.replace(tmp, LIB_PATH)
+                finally:
+                    if os.path.exists(tmp):
+                        os.remove(tmp)
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
     return LIB_PATH
 
 
