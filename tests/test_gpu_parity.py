@@ -183,6 +183,38 @@ def test_large_vocabularies_and_limits(kw):
         assert_ok(rep)
 
 
+def _random_case(i):
+    """Case i of a seeded sweep over the launch partition's inputs: batch sizes on both sides of the
+    points where sequences are split over a cluster, kept one per block or merged several per block;
+    every draft length class; vocabularies with ragged tails; dtype, guidance mix, top-k, bonus row."""
+    r = np.random.default_rng(1000 + i)
+    B = int(r.choice([1, 2, 3, 5, 9, 15, 16, 17, 33, 70, 149, 297, 600, 1300]))
+    L = int(r.choice([1, 2, 3, 4, 7, 8, 12, 16, 32]))
+    V = int(r.choice([16, 250, 1000, 2048, 3001, 4096, 8200, 16384, 40000]))
+    while B * L * V > 2.2e7:                       # keep the oracle to a few seconds per case
+        if V > 1000: V //= 2
+        else: B = max(1, B // 2)
+    kw = dict(B=B, gamma=L, V=V, dtype=[W.F32, W.BF16][int(r.integers(2))], bonus_row=bool(r.integers(2)),
+              rho=float(r.choice([0.5, 0.9, 0.99])))
+    if r.integers(3) == 0:
+        kw["cfg"] = True
+    if r.integers(3) == 0:
+        kw["top_k"] = int(min(V - 1, r.choice([1, 7, 100, 1000])))
+    return kw, bool(r.integers(2))
+
+
+@pytest.mark.parametrize("i", range(96))
+def test_seeded_sweep_of_partitions(i):
+    kw, b2b = _random_case(i)
+    L = kw["gamma"]
+    w = W.make("t", schedule=sched(L, "exp" if i % 3 else "vanilla"), seed=300 + i, device=DEV, **kw)
+    rep, got, ref = check(w, back_to_back=b2b, want_dbg=kw["B"] * kw["V"] <= 4e6)
+    assert_ok(rep)
+    other = run_gpu(w, want_dbg=False, back_to_back=not b2b)
+    for key in ("tokens", "accept_len", "status"):
+        assert np.array_equal(got[key], other[key]), (key, kw, b2b)
+
+
 @pytest.mark.parametrize("b2b", [False, True])
 @pytest.mark.parametrize("kw", [
     dict(B=20, gamma=8, V=16384, dtype=W.F32),
