@@ -201,7 +201,9 @@ template <typename T, bool CFG>
 cudaError_t launch_finish(const FinishArgs& a, cudaStream_t stream) {
   auto kern = finish_kernel<T, CFG>;
   constexpr int TILE = 32 * Elem<T>::kVec;
-  const size_t smem = (size_t)((a.V + TILE - 1) / TILE) * sizeof(double);
+  size_t slots = (size_t)((a.V + TILE - 1) / TILE);
+  if (slots < 2 * (kFinishThreads / 32)) slots = 2 * (kFinishThreads / 32);   // the monitors' two sums per warp
+  const size_t smem = slots * sizeof(double);
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

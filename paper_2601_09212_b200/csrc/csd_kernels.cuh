@@ -501,7 +501,7 @@ __device__ __forceinline__ void group_sync() {
 // Everything after the row statistics for sequence b, run by NT threads (tid in
 // [0, NT)): merge the parts, Eq. relax and the accept tests, tau, Eq. opt_G at
 // position tau+1, the inverse-CDF draw, the emitted block.  tile_sums needs one
-// double per tile of 32 * (16 bytes / element size) tokens.
+// double per tile of 32 * (16 bytes / element size) tokens, and at least two per warp.
 template <typename T, bool CFG, int NT, int BAR>
 __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid, double* tile_sums,
                                 FinishSmem& sm, const int extra_status) {

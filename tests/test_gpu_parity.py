@@ -200,6 +200,8 @@ def _random_case(i):
         kw["cfg"] = True
     if r.integers(3) == 0:
         kw["top_k"] = int(min(V - 1, r.choice([1, 7, 100, 1000])))
+    if r.integers(4) == 0:
+        kw["law"] = "student3"                     # heavy tails: the selection's guess misses and adapts
     return kw, bool(r.integers(2))
 
 
@@ -213,6 +215,27 @@ def test_seeded_sweep_of_partitions(i):
     other = run_gpu(w, want_dbg=False, back_to_back=not b2b)
     for key in ("tokens", "accept_len", "status"):
         assert np.array_equal(got[key], other[key]), (key, kw, b2b)
+    if i % 4 == 0:                                  # the per-position monitors on the same inputs
+        mon = run_gpu(w, want_dbg=False, want_terms=True, back_to_back=b2b)
+        assert np.array_equal(mon["tokens"], got["tokens"])
+        _, ref_t = run_oracle(w, want_G=False, want_terms=True)
+        tol = 1e-5 if w.dtype == W.F32 else 2e-3
+        assert np.abs(mon["accept_mass"] - ref_t.accept_mass).max() < tol
+        assert np.abs(mon["bound_term"] - ref_t.bound_term).max() < 2 * tol
+    if i % 4 == 1:                                  # the drafting stage's draw on the first draft rows
+        logits = w.draft_logits[:, 0].contiguous()
+        unc = None if w.draft_uncond is None else w.draft_uncond[:, 0].contiguous()
+        uni = w.uniforms[:, 0].contiguous()
+        tok = torch.full((w.B,), -7, dtype=torch.int32, device=DEV)
+        csd.csd_sample_rows(logits, uni, tok, uncond=unc, cfg_scale=w.cfg_scale, top_k=w.top_k, back_to_back=b2b)
+        torch.cuda.synchronize()
+        h = w.host_arrays()
+        ref_tok, _, margin = oracle.sample_rows(
+            h["draft_logits"][:, 0], h["uniforms"][:, 0], dtype=w.dtype,
+            uncond=None if h["draft_uncond"] is None else h["draft_uncond"][:, 0], cfg_scale=w.cfg_scale,
+            top_k=w.top_k)
+        differ = tok.cpu().numpy() != ref_tok
+        assert np.all(margin[differ] < 1e-6) and differ.sum() <= max(1, w.B // 50)
 
 
 @pytest.mark.parametrize("b2b", [False, True])
