@@ -52,6 +52,7 @@ __device__ __forceinline__ void stat_merge(float& m, float& s, float m2, float s
     t = s; s = s2; s2 = t;
   }
   if (m2 != CSD_NEG_INF) s += (1.0f + s2) * ex2f((m2 - m) * kLog2e);
+  else s += s2 - s2;   // nothing to add, but a NaN sum (a NaN beside nothing but masked values) must survive
 }
 
 __device__ __forceinline__ void stat_warp_allreduce(float& m, float& s) {
