@@ -37,6 +37,13 @@
  *     value of Eq. opt_G at f = 0); an invalid target row emits -1.
  *   - a draft token outside [0, V) rejects (f := 0) and is flagged.
  *
+ * Resolution: the weights of Eq. opt_G are formed from fp64 probabilities, as
+ * the equation is written, so each carries an absolute rounding of about 1e-16.
+ * Where both models put all but that much of their mass on one token, the
+ * difference of two probabilities next to 1 at that token is lost; a draw at a
+ * position whose normaliser Z is below about 1e-10 is therefore outside what
+ * this oracle resolves (a valid draft token is rejected there with probability Z).
+ *
  * Pins (tests/test_oracle_*.py): Theorem 1 by exact enumeration and chi-square,
  * Theorem 2's expectation and TV bound by brute force on tiny alphabets,
  * Proposition LP's closed form against random and grid search over G,
