@@ -413,6 +413,75 @@ def test_back_to_back_calls_on_one_stream(name, kw, b2b):
     check_all("graph")
 
 
+@pytest.mark.parametrize("b2b", [False, True])
+def test_mixed_calls_share_one_stream_and_workspace(b2b):
+    """Calls of different shapes and kinds -- both single-launch kernels in every partition, the
+    multi-launch path, the drafting-stage draw -- enqueued one after the other on one stream with ONE
+    workspace, directly and as a replayed CUDA graph: each must give what it gives alone."""
+    kinds = [
+        dict(B=16, gamma=8, V=16384, dtype=W.F32),
+        dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000),
+        dict(B=5, gamma=4, V=3001, dtype=W.F32, top_k=20),                 # multi-launch path
+        dict(B=3, gamma=16, V=8192, dtype=W.BF16, bonus_row=True),         # clusters
+        dict(B=9, gamma=3, V=250, dtype=W.BF16, cfg=True),                 # multi-launch path
+        dict(B=700, gamma=2, V=2048, dtype=W.BF16, bonus_row=True),
+        dict(B=1500, gamma=2, V=1024, dtype=W.F32, top_k=5),               # several sequences per block
+    ]
+    steps = [W.make("t", rho=0.9, schedule=sched(kw["gamma"]), seed=200 + i, device=DEV, **kw)
+             for i, kw in enumerate(kinds)]
+    alone = [run_gpu(w, want_dbg=False) for w in steps]
+    size = max(csd.csd_workspace_size(w.B, w.gamma, w.V, w.dtype) for w in steps)
+    size = max(size, csd.csd_sample_workspace_size(64, 16384, W.BF16))
+    ws = torch.zeros(size, dtype=torch.uint8, device=DEV)
+    outs = [dict(tok=torch.full((w.B, w.gamma + 1), -7, dtype=torch.int32, device=DEV),
+                 tau=torch.full((w.B,), -7, dtype=torch.int32, device=DEV),
+                 st=torch.full((w.B,), -7, dtype=torch.int32, device=DEV)) for w in steps]
+    stream = torch.cuda.Stream()
+    prms = [csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
+                            o["tok"], o["tau"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
+                            cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=o["st"], workspace=ws,
+                            stream=stream, back_to_back=b2b) for w, o in zip(steps, outs)]
+    # the drafting-stage draw between them, on the guided rows of the second workload
+    d = steps[1]
+    d_logits, d_unc = d.draft_logits[:, 0].contiguous(), d.draft_uncond[:, 0].contiguous()
+    d_uni = d.uniforms[:, 0].contiguous()
+    d_tok = torch.full((d.B,), -7, dtype=torch.int32, device=DEV)
+    csd.csd_sample_rows(d_logits, d_uni, d_tok, uncond=d_unc, cfg_scale=d.cfg_scale, top_k=d.top_k)
+    torch.cuda.synchronize()
+    d_alone = d_tok.cpu().numpy().copy()
+
+    def enqueue():
+        for i, p in enumerate(prms):
+            csd.csd_verify_ex(p)
+            if i % 3 == 1:
+                csd.csd_sample_rows(d_logits, d_uni, d_tok, uncond=d_unc, cfg_scale=d.cfg_scale, top_k=d.top_k,
+                                    workspace=ws, back_to_back=b2b, stream=stream)
+
+    def check_all(tag):
+        for i, (o, ref) in enumerate(zip(outs, alone)):
+            assert np.array_equal(o["tok"].cpu().numpy(), ref["tokens"]), (tag, i)
+            assert np.array_equal(o["tau"].cpu().numpy(), ref["accept_len"]), (tag, i)
+            assert np.array_equal(o["st"].cpu().numpy(), ref["status"]), (tag, i)
+            o["tok"].fill_(-7); o["tau"].fill_(-7); o["st"].fill_(-7)
+        assert np.array_equal(d_tok.cpu().numpy(), d_alone), tag
+        d_tok.fill_(-7)
+
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            enqueue()
+    stream.synchronize()
+    check_all("direct")
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        enqueue()
+    with torch.cuda.stream(stream):
+        for _ in range(4):
+            g.replay()
+    stream.synchronize()
+    check_all("graph")
+
+
 def test_batch_strides_and_unaligned_views():
     """Rows embedded in a larger buffer (batch stride > rows*V) and a base pointer that is
     only element-aligned (forces the scalar path)."""
