@@ -670,6 +670,39 @@ def test_host_buffer_form():
     assert np.array_equal(out_s.numpy(), got["status"])
 
 
+@pytest.mark.parametrize("i", range(10))
+def test_seeded_sweep_of_host_form_and_static_scratch(i):
+    """The entry points that wrap the device call -- host buffers with copies enqueued by the library,
+    and (fp32, plain inputs) the form whose scratch is a fixed array inside the library -- on random
+    shapes: the same integers as csd_verify_ex on device buffers."""
+    kw, _ = _random_case(800 + i)
+    kw["B"] = min(kw["B"], 300)
+    L = kw["gamma"]
+    w = W.make("t", schedule=sched(L), seed=1300 + i, device=DEV, **kw)
+    got = run_gpu(w, want_dbg=False)
+    pin = lambda t: None if t is None else t.cpu().pin_memory()
+    out_t = torch.full((w.B, L + 1), -7, dtype=torch.int32).pin_memory()
+    out_l = torch.full((w.B,), -7, dtype=torch.int32).pin_memory()
+    out_s = torch.full((w.B,), -7, dtype=torch.int32).pin_memory()
+    prm = csd.make_params(pin(w.target_logits), pin(w.draft_logits), pin(w.draft_tokens), pin(w.uniforms),
+                          pin(w.relax_schedule), out_t, out_l, target_uncond=pin(w.target_uncond),
+                          draft_uncond=pin(w.draft_uncond), cfg_scale=w.cfg_scale, top_k=w.top_k,
+                          out_status=out_s, host=True)
+    staging = torch.empty(csd.csd_host_staging_size(prm), dtype=torch.uint8, device=DEV)
+    csd.csd_verify_host(prm, staging)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_t.numpy(), got["tokens"])
+    assert np.array_equal(out_l.numpy(), got["accept_len"])
+    assert np.array_equal(out_s.numpy(), got["status"])
+    plain = w.dtype == W.F32 and w.target_uncond is None and not w.top_k and w.target_logits.shape[1] == L
+    if plain and csd.csd_workspace_size(w.B, L, w.V, W.F32) <= csd.CSD_STATIC_SCRATCH_BYTES:
+        tok = torch.full((w.B, L + 1), -9, dtype=torch.int32, device=DEV)
+        tau = torch.full((w.B,), -9, dtype=torch.int32, device=DEV)
+        csd.csd_verify_static(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule, tok, tau)
+        torch.cuda.synchronize()
+        assert np.array_equal(tok.cpu().numpy(), got["tokens"]) and np.array_equal(tau.cpu().numpy(), got["accept_len"])
+
+
 def test_argument_errors():
     w = W.make("t", B=2, gamma=2, V=64, schedule=sched(2), device=DEV)
     out_t = torch.empty(2, 3, dtype=torch.int32, device=DEV)
