@@ -579,6 +579,22 @@ def test_seeded_sweep_of_unusable_inputs(i):
     other = run_gpu(w, want_dbg=False, back_to_back=not b2b)
     for key in ("tokens", "accept_len", "status"):
         assert np.array_equal(got[key], other[key]), (key, kw, b2b)
+    # the drafting-stage draw on the same damaged rows (the drafter's first and the target's last)
+    h = w.host_arrays()   # bf16 as bit patterns, like every oracle input
+    for key_l, key_u, col, dev_l, dev_u in (("draft_logits", "draft_uncond", 0, w.draft_logits, w.draft_uncond),
+                                            ("target_logits", "target_uncond", T - 1, w.target_logits, w.target_uncond)):
+        tok = torch.full((B,), -7, dtype=torch.int32, device=DEV)
+        st = torch.full((B,), -7, dtype=torch.int32, device=DEV)
+        csd.csd_sample_rows(dev_l[:, col].contiguous(), w.uniforms[:, L].contiguous(), tok,
+                            uncond=None if dev_u is None else dev_u[:, col].contiguous(), cfg_scale=w.cfg_scale,
+                            top_k=w.top_k, out_status=st, back_to_back=b2b)
+        torch.cuda.synchronize()
+        ref_tok, ref_st, margin = oracle.sample_rows(
+            h[key_l][:, col], h["uniforms"][:, L], dtype=w.dtype,
+            uncond=None if h[key_u] is None else h[key_u][:, col], cfg_scale=w.cfg_scale, top_k=w.top_k)
+        differ = tok.cpu().numpy() != ref_tok
+        assert np.all(margin[differ] < 1e-6) and differ.sum() <= max(1, B // 50), (key_l, np.flatnonzero(differ)[:5])
+        assert np.array_equal(st.cpu().numpy(), ref_st), key_l
 
 
 def _below_resolution(w, got, ref, b):
