@@ -579,6 +579,16 @@ def test_seeded_sweep_of_unusable_inputs(i):
     other = run_gpu(w, want_dbg=False, back_to_back=not b2b)
     for key in ("tokens", "accept_len", "status"):
         assert np.array_equal(got[key], other[key]), (key, kw, b2b)
+    # the per-position monitors: NaN exactly where a row is unusable, the oracle's values elsewhere
+    mon = run_gpu(w, want_dbg=False, want_terms=True, back_to_back=b2b)
+    assert np.array_equal(mon["tokens"], got["tokens"]) and np.array_equal(mon["status"], got["status"])
+    _, ref_t = run_oracle(w, want_G=False, want_terms=True)
+    usable = np.isfinite(ref_t.accept_mass)
+    assert np.array_equal(np.isfinite(mon["accept_mass"]), usable) and np.array_equal(np.isfinite(mon["bound_term"]), usable)
+    tol = 1e-5 if w.dtype == W.F32 else 2e-3
+    if usable.any():
+        assert np.abs(mon["accept_mass"][usable] - ref_t.accept_mass[usable]).max() < tol
+        assert np.abs(mon["bound_term"][usable] - ref_t.bound_term[usable]).max() < 2 * tol * max(1.0, float(schedule.max()))
     # the drafting-stage draw on the same damaged rows (the drafter's first and the target's last)
     h = w.host_arrays()   # bf16 as bit patterns, like every oracle input
     for key_l, key_u, col, dev_l, dev_u in (("draft_logits", "draft_uncond", 0, w.draft_logits, w.draft_uncond),
