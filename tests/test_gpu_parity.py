@@ -183,6 +183,21 @@ def test_large_vocabularies_and_limits(kw):
         assert_ok(rep)
 
 
+@pytest.mark.parametrize("B", [147, 148, 149, 295, 296, 297, 1183, 1184, 1185, 2368, 2369])
+def test_partition_boundaries(B):
+    """Batch sizes on both sides of every point where the launch partition changes (multiples of the 148
+    SMs: clusters -> one block per sequence -> several sequences per block), both stream modes."""
+    L = 3
+    for dtype, V, top_k in ((W.BF16, 1024, 0), (W.F32, 512, 40)):
+        w = W.make("t", B=B, gamma=L, V=V, dtype=dtype, rho=0.9, bonus_row=True, top_k=top_k, schedule=sched(L),
+                   seed=B, device=DEV)
+        rep, got, ref = check(w, want_dbg=False)
+        assert_ok(rep)
+        other = run_gpu(w, want_dbg=False, back_to_back=True)
+        for key in ("tokens", "accept_len", "status"):
+            assert np.array_equal(got[key], other[key]), (key, B)
+
+
 def _random_case(i):
     """Case i of a seeded sweep over the launch partition's inputs: batch sizes on both sides of the
     points where sequences are split over a cluster, kept one per block or merged several per block;
