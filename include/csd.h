@@ -75,7 +75,10 @@ typedef enum {
                               rejects (f := 0).  An unusable drafter row resamples from
                               P_j (Eq. opt_G at f = 0); an unusable target row emits -1. */
   CSD_STATUS_BADTOKEN = 2, /* draft token outside [0, V): that position rejects */
-  CSD_STATUS_ZFALLBACK = 4, /* empty positive part: drew from P_j instead */
+  CSD_STATUS_ZFALLBACK = 4, /* empty positive part of Eq. opt_G (its sum is zero, or below the 1e-38
+                               that the fp32 weights can hold): drew from P_j instead.  A valid
+                               draft token is rejected at such a position with that probability,
+                               so in practice only a CSD_STATUS_BADTOKEN rejection gets here. */
   CSD_STATUS_TIMEOUT = 8    /* a bounded wait inside the kernel gave up (a copy into shared memory did
                                not arrive within about a second): results of this call are unreliable.
                                The condition stays set in the workspace until csd_workspace_init. */
