@@ -100,6 +100,32 @@ def test_bf16_large_batch_c4_sampled():
             assert got["G"][b, got["tokens"][b, tau[b]]] > 0
 
 
+@pytest.mark.parametrize("kw", [
+    dict(B=256, gamma=16, V=65536, dtype=W.BF16),
+    dict(B=256, gamma=4, V=65536, dtype=W.F32),
+    dict(B=64, gamma=16, V=32768, dtype=W.F32),
+    dict(B=16, gamma=8, V=4096, dtype=W.BF16),
+    dict(B=1, gamma=16, V=65536, dtype=W.F32),
+])
+def test_sweep_grid_corners_sampled(kw):
+    """Corners of the V x gamma x B x dtype sweep at full size, in the partition used for timing
+    (calls enqueued back to back): the oracle on a sample of sequences, structure on all of them."""
+    L, B = kw["gamma"], kw["B"]
+    w = W.make("t", rho=0.9, schedule=sched(L), seed=55, device=DEV, **kw)
+    rows = np.unique(np.linspace(0, B - 1, 8).astype(int))
+    rep, got, ref = check(w, rows=rows, want_dbg=True, back_to_back=True)
+    assert_ok(rep)
+    tau, tok = got["accept_len"], w.draft_tokens.cpu().numpy()
+    assert tau.min() >= 0 and tau.max() <= L and np.all(got["status"] == 0)
+    for b in range(B):
+        assert np.array_equal(got["tokens"][b, :tau[b]], tok[b, :tau[b]])
+        assert np.all(got["tokens"][b, tau[b] + 1:] == -1)
+        if tau[b] < L:
+            assert 0 <= got["tokens"][b, tau[b]] < w.V and got["G"][b, got["tokens"][b, tau[b]]] > 0
+    base = run_gpu(w, want_dbg=False)
+    assert np.array_equal(base["tokens"], got["tokens"]) and np.array_equal(base["accept_len"], got["accept_len"])
+
+
 def test_cfg_mix_fused():
     L = 6
     for dtype in (W.F32, W.BF16):
