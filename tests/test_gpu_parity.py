@@ -126,6 +126,30 @@ def test_sweep_grid_corners_sampled(kw):
     assert np.array_equal(base["tokens"], got["tokens"]) and np.array_equal(base["accept_len"], got["accept_len"])
 
 
+@pytest.mark.parametrize("i", range(16))
+def test_seeded_sweep_of_tied_topk_rows(i):
+    """Logits rounded to a coarse grid: the k-th largest value is shared by many tokens (all of them are
+    kept), histogram bins are crowded, candidate lists overflow -- the streaming selection has to hand
+    such rows to the exact one, and both must agree with the oracle's threshold rule."""
+    r = np.random.default_rng(4000 + i)
+    V = int(r.choice([1000, 4096, 16384, 20000]))
+    kw = dict(B=int(r.choice([2, 9, 40])), gamma=int(r.choice([2, 5, 8])), V=V,
+              dtype=[W.F32, W.BF16][int(r.integers(2))], bonus_row=bool(r.integers(2)), cfg=bool(r.integers(2)),
+              top_k=int(r.integers(1, max(2, V // 4))), rho=0.9)
+    L = kw["gamma"]
+    w = W.make("t", schedule=sched(L), seed=4100 + i, device=DEV, **kw)
+    q = float(r.choice([0.125, 0.5, 2.0]))
+    for t in (w.target_logits, w.draft_logits, w.target_uncond, w.draft_uncond):
+        if t is not None:
+            t.copy_((t.float() / q).round() * q)
+    b2b = bool(r.integers(2))
+    rep, got, ref = check(w, back_to_back=b2b, want_dbg=kw["B"] * V <= 4e6)
+    assert_ok(rep)
+    other = run_gpu(w, want_dbg=False, back_to_back=not b2b)
+    for key in ("tokens", "accept_len", "status"):
+        assert np.array_equal(got[key], other[key]), (key, kw, b2b)
+
+
 def test_cfg_mix_fused():
     L = 6
     for dtype in (W.F32, W.BF16):
