@@ -586,6 +586,43 @@ def test_batch_strides_and_unaligned_views():
     assert np.array_equal(out_l.cpu().numpy(), got_plain["accept_len"])
 
 
+@pytest.mark.parametrize("i", range(12))
+def test_seeded_sweep_of_batch_strides(i):
+    """Sequences embedded in larger buffers (batch stride > rows x V) on random shapes: with a padding that
+    keeps rows 16-byte aligned (single-launch kernels) and one that does not (multi-launch path), the
+    same integers as from contiguous inputs."""
+    kw, b2b = _random_case(1500 + i)
+    kw["B"] = min(kw["B"], 200)
+    L = kw["gamma"]
+    w = W.make("t", schedule=sched(L), seed=1600 + i, device=DEV, **kw)
+    base = run_gpu(w, want_dbg=False, back_to_back=b2b)
+    B, V, T = w.B, w.V, w.target_logits.shape[1]
+    for pad in (64, 3):
+        def embed(t, rows):
+            if t is None:
+                return None
+            big = torch.zeros(B, rows * V + pad, dtype=t.dtype, device=DEV)
+            big[:, :rows * V] = t.reshape(B, -1)
+            return big
+        bt, bd, btu, bdu = embed(w.target_logits, T), embed(w.draft_logits, L), embed(w.target_uncond, T), embed(w.draft_uncond, L)
+        out_t = torch.full((B, L + 1), -7, dtype=torch.int32, device=DEV)
+        out_l = torch.full((B,), -7, dtype=torch.int32, device=DEV)
+        out_s = torch.full((B,), -7, dtype=torch.int32, device=DEV)
+        prm = csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
+                              out_t, out_l, target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
+                              cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=out_s,
+                              workspace=csd.new_workspace(B, L, V, w.dtype), back_to_back=b2b)
+        prm.target_logits, prm.draft_logits = bt.data_ptr(), bd.data_ptr()
+        if btu is not None:
+            prm.target_uncond, prm.draft_uncond = btu.data_ptr(), bdu.data_ptr()
+        prm.target_batch_stride, prm.draft_batch_stride = bt.shape[1], bd.shape[1]
+        csd.csd_verify_ex(prm)
+        torch.cuda.synchronize()
+        assert np.array_equal(out_t.cpu().numpy(), base["tokens"]), (pad, kw)
+        assert np.array_equal(out_l.cpu().numpy(), base["accept_len"]), (pad, kw)
+        assert np.array_equal(out_s.cpu().numpy(), base["status"]), (pad, kw)
+
+
 def test_bad_data_is_reported_not_trapped():
     B, L, V = 5, 3, 64
     w = W.make("t", B=B, gamma=L, V=V, rho=0.9, bonus_row=True, schedule=np.full(L, 1e6, np.float32),
