@@ -285,15 +285,27 @@ def csd_sample_workspace_size(R: int, V: int, dtype: int) -> int:
 
 def csd_sample_rows(logits, uniforms, out_tokens, *, uncond=None, cfg_scale=1.0, top_k=0, out_status=None,
                     workspace=None, back_to_back=False, stream=None) -> None:
-    """Drafting stage: one inverse-CDF draw per row of ``logits`` [R, V] (device tensors)."""
+    """Drafting stage: one inverse-CDF draw per row of ``logits`` [R, V] (device tensors).
+
+    ``logits`` (and ``uncond``, with the same strides) may be a view whose rows are contiguous but
+    spaced apart, such as ``all_logits[:, -1]`` of a ``[B, T, V]`` tensor: the row stride is passed on."""
     R, V = logits.shape
     dt = _logit_dtype(logits)
     ldt = logits.dtype
+
+    def rows_ptr(t, name):
+        if t is None:
+            return None
+        if (not t.is_cuda or t.dtype != ldt or t.dim() != 2 or t.shape != logits.shape or t.stride(1) != 1
+                or t.stride(0) != logits.stride(0) or t.stride(0) < V):
+            raise ValueError(f"{name} must be a CUDA tensor [R, V] of {ldt} with contiguous rows and the row stride of logits")
+        return t.data_ptr()
+
     if workspace is None:
         workspace = torch.zeros(csd_sample_workspace_size(R, V, dt), dtype=torch.uint8, device=logits.device)
     rc = library().csd_sample_rows(
-        _dev_ptr(logits, "logits", ldt), _dev_ptr(uncond, "uncond", ldt), float(cfg_scale), int(top_k), dt, R, V,
-        V, _dev_ptr(uniforms, "uniforms", torch.float32), _dev_ptr(out_tokens, "out_tokens", torch.int32),
+        rows_ptr(logits, "logits"), rows_ptr(uncond, "uncond"), float(cfg_scale), int(top_k), dt, R, V,
+        int(logits.stride(0)) if R > 1 else V, _dev_ptr(uniforms, "uniforms", torch.float32), _dev_ptr(out_tokens, "out_tokens", torch.int32),
         _dev_ptr(out_status, "out_status", torch.int32), _dev_ptr(workspace, "workspace"),
         workspace.numel() * workspace.element_size(), 1 if back_to_back else 0, _stream_handle(stream))
     if rc != 0:

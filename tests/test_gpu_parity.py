@@ -379,6 +379,35 @@ def test_drafting_stage_sampling(kw, b2b):
     assert got.min() >= 0 and got.max() < w.V
 
 
+@pytest.mark.parametrize("kw", [
+    dict(B=40, gamma=3, V=4096, dtype=W.BF16, cfg=True, top_k=200),
+    dict(B=7, gamma=2, V=16384, dtype=W.F32),
+    dict(B=300, gamma=1, V=1000, dtype=W.BF16, bonus_row=True),
+])
+def test_drafting_stage_sampling_of_spaced_rows(kw):
+    """Rows taken out of a [B, T, V] tensor (the last position of every sequence): the row stride reaches
+    the library, and the draws equal those from a packed copy of the same rows."""
+    w = W.make("t", rho=0.9, schedule=sched(kw["gamma"]), seed=61, device=DEV, **kw)
+    last = w.target_logits.shape[1] - 1
+    view = w.target_logits[:, last]
+    unc = None if w.target_uncond is None else w.target_uncond[:, last]
+    assert not view.is_contiguous() or last == 0
+    uni = w.uniforms[:, 0].contiguous()
+    toks = []
+    for lg, un in ((view, unc), (view.contiguous(), None if unc is None else unc.contiguous())):
+        tok = torch.full((w.B,), -7, dtype=torch.int32, device=DEV)
+        csd.csd_sample_rows(lg, uni, tok, uncond=un, cfg_scale=w.cfg_scale, top_k=w.top_k)
+        torch.cuda.synchronize()
+        toks.append(tok.cpu().numpy())
+    assert np.array_equal(toks[0], toks[1]) and toks[0].min() >= 0
+    h = w.host_arrays()
+    ref_tok, _, margin = oracle.sample_rows(
+        h["target_logits"][:, last], h["uniforms"][:, 0], dtype=w.dtype,
+        uncond=None if h["target_uncond"] is None else h["target_uncond"][:, last], cfg_scale=w.cfg_scale, top_k=w.top_k)
+    differ = toks[0] != ref_tok
+    assert np.all(margin[differ] < 1e-6) and differ.sum() <= max(1, w.B // 50)
+
+
 def test_drafting_stage_sampling_bad_row_and_errors():
     R, V = 6, 4096
     logits = torch.randn(R, V, device=DEV)
