@@ -36,6 +36,8 @@
  *     position rejects (f := 0); an invalid drafter row resamples from P (the
  *     value of Eq. opt_G at f = 0); an invalid target row emits -1.
  *   - a draft token outside [0, V) rejects (f := 0) and is flagged.
+ *   - a multiplier omega_i that is negative or NaN counts as 0 (Eq. relax is
+ *     stated for omega >= 0).
  *
  * Resolution: the weights of Eq. opt_G are formed from fp64 probabilities, as
  * the equation is written, so each carries an absolute rounding of about 1e-16.
@@ -164,10 +166,13 @@ int orc_make_schedule(int kind, double delta, double nu_or_ell, int L, double *o
 
 /* ---- building blocks -------------------------------------------------------*/
 
-/* Relaxed acceptance probability, Eq. relax: min{1, omega p / q}, 0/0 := 1. */
+/* Relaxed acceptance probability, Eq. relax: min{1, omega p / q}, 0/0 := 1.
+ * Eq. relax is stated for omega >= 0; a multiplier that is negative or NaN is
+ * read as 0 (no relaxation can make f negative), so f = 0 wherever q > 0. */
 double orc_accept_prob(double p, double q, double omega) {
   if (q == 0.0) return 1.0; /* p/q = +inf for p > 0, and 0/0 := 1 */
   if (p == 0.0) return 0.0;
+  if (!(omega >= 0.0)) omega = 0.0;
   double ratio = omega * p / q;
   return ratio < 1.0 ? ratio : 1.0;
 }

@@ -75,6 +75,14 @@ def test_accept_prob_cases(oracle):
     assert oracle.accept_prob(0.0, 0.0, 0.5) == 1.0
     assert oracle.accept_prob(0.3, 0.0, 1.0) == 1.0          # p/0 = +inf
     assert oracle.accept_prob(0.0, 0.3, 2.0) == 0.0
+    # Eq. relax is stated for omega >= 0: a negative or NaN multiplier is read as 0
+    assert oracle.accept_prob(0.25, 0.5, float("nan")) == 0.0
+    assert oracle.accept_prob(0.25, 0.5, -3.0) == 0.0
+    assert oracle.accept_prob(0.0, 0.0, float("nan")) == 1.0  # 0/0 := 1 is kept
+    # ... and Eq. opt_G then gives the target distribution itself (f = 0 everywhere)
+    P, Q = np.array([0.5, 0.3, 0.2]), np.array([0.2, 0.2, 0.6])
+    for om in (float("nan"), -1.0, 0.0):
+        assert np.allclose(oracle.resample_dist(P, Q, om), P, atol=1e-15)
 
 
 def test_accept_rate_is_overlap(oracle):
