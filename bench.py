@@ -10,7 +10,10 @@ image tokens, bf16 logits, conditional/unconditional rows mixed on load (scale 4
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl native|reference] [--workload C3]
 
 One JSON line on stdout (rank 0).  `value` is verified draft tokens per second with the inputs
-resident in HBM (a ring of distinct step inputs larger than L2, replayed as a CUDA graph);
+resident in HBM (a ring of distinct step inputs larger than L2, replayed as a CUDA graph; the timed
+region is always whole replays -- at least max(K, 2048) calls per repetition, 7 repetitions, the
+median reported -- so the figure does not depend on K); `stream_order` is the same call in
+ordinary stream order, one call at a time, as a decoding loop issues it;
 `e2e` is the same metric through the host-buffer entry point, host->device and device->host
 copies inside the timed region; `roofline` compares the step's algorithmic bytes with the
 measured HBM copy bandwidth; `cpu_baseline` is the fp64 CPU oracle timed on a bounded sample.
@@ -34,6 +37,8 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+MIN_TIMED_CALLS = 2048   # calls per timed repetition, at least (whole graph replays)
+REPS = 7                 # timed repetitions; the median is reported
 METRIC = "verified_draft_tokens_per_sec"
 UNIT = "tokens/s"
 L2_BYTES = 126 * 1024 * 1024
@@ -41,8 +46,8 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum,
-# one ncu capture, see profiles/verify_topk_kernel_C3.md).  Reported only while the kernel sources
-# still have the digest the capture was taken with; null otherwise.
+# one ncu capture of this workload).  Reported only while the kernel sources still have the digest
+# the capture was taken with; null otherwise.
 NCU_TRAFFIC = {"sources_sha256": "7d64f1757e59a585", "workload": "C3", "bytes_per_launch": 67848448}
 
 
@@ -297,49 +302,79 @@ def run_native(args) -> None:
             for w, o in zip(ring, outs)]
     kernels_per_step = csd.csd_launch_count(prms[0])
 
-    def enqueue(i):
-        csd.csd_verify_ex(prms[i % ring_n])
+    # The same calls in ordinary stream order (back_to_back = 0): what a decoding loop sees, whose logits
+    # come from the forward pass just before the call.  Timed beside the headline, reported beside it.
+    prms_so = [csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
+                               o["tok"], o["tau"], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
+                               cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=o["st"], workspace=o["ws"],
+                               stream=stream, back_to_back=False,
+                               diag_accept_mass=o["am"], diag_bound_term=o["bt"])
+               for w, o in zip(ring, outs)]
 
     # A few laps of the ring as one CUDA graph: the launches inside are the library's own.  Inside a
     # graph consecutive calls keep their programmatic-launch edges and overlap as they do when enqueued
-    # directly; two replays do not overlap, so the graph is made long enough (>= 64 steps) for that
-    # boundary not to matter.
+    # directly; two replays do not overlap, so the graph is made long enough (>= 64 calls) for that
+    # boundary not to matter.  Whatever --steps is, the timed region is whole replays of that graph:
+    # REPS repetitions of at least max(steps, MIN_TIMED_CALLS) calls each, each repetition between its
+    # own pair of events; the reported time per step is the median repetition.
     graph_steps = ring_n * max(1, -(-64 // ring_n))
-    with torch.cuda.stream(stream):
-        for i in range(ring_n):
-            enqueue(i)
-    stream.synchronize()
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph, stream=stream):
-        for i in range(graph_steps):
-            enqueue(i)
 
-    def run_steps(k):
-        replays, rest = divmod(k, graph_steps)
+    def capture(params):
         with torch.cuda.stream(stream):
-            for _ in range(replays):
-                graph.replay()
-            for i in range(rest):
-                enqueue(i)
+            for i in range(ring_n):
+                csd.csd_verify_ex(params[i])
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(graph_steps):
+                csd.csd_verify_ex(params[i % ring_n])
+        return g
+
+    graph = capture(prms)
+    graph_so = capture(prms_so)
+    replays = max(1, -(-max(args.steps, MIN_TIMED_CALLS) // graph_steps))
+    replays_so = max(1, replays // 4)
+    timed_calls = replays * graph_steps
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    run_steps(max(args.warmup, 3))
+    def timed_reps(g, n_replays, reps):
+        """ms of each of `reps` repetitions of n_replays replays (max over ranks each)."""
+        out = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            barrier()
+            with torch.cuda.stream(stream):
+                a.record(stream)
+                for _ in range(n_replays):
+                    g.replay()
+                b.record(stream)
+            barrier()
+            out.append(sharding.max_over_ranks(a.elapsed_time(b), device=dev))
+        return out
+
+    warm_replays = max(1, -(-max(args.warmup, 3) // graph_steps))
+    with torch.cuda.stream(stream):
+        for _ in range(warm_replays):
+            graph.replay()
+            graph_so.replay()
     barrier()
     props = torch.cuda.get_device_properties(dev)
     sampler = ClockSampler(f"{props.pci_domain_id:08x}:{props.pci_bus_id:02x}:{props.pci_device_id:02x}.0")
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler.start()
-    e0.record(stream)
-    run_steps(args.steps)
-    e1.record(stream)
+    rep_ms = timed_reps(graph, replays, REPS)
     sampler.sample_once()
-    barrier()
     sampler.stop()
-    ms = sharding.max_over_ranks(e0.elapsed_time(e1), device=dev)
+    so_ms = timed_reps(graph_so, replays_so, 3)
+    step_ms_reps = sorted(m / timed_calls for m in rep_ms)
+    step_ms = float(np.median(step_ms_reps))
+    so_step_ms = float(np.median(so_ms)) / (replays_so * graph_steps)
+    with torch.cuda.stream(stream):   # leave the outputs of the headline mode in place for the checks below
+        graph.replay()
+    barrier()
 
     # accepted lengths of the last lap (a property of the synthetic drafter, reported for context)
     mean_emit = float(np.mean([o["tau"].float().mean().item() + 1.0 for o in outs]))
@@ -383,10 +418,11 @@ def run_native(args) -> None:
             dist.destroy_process_group()
         return
 
-    value = sharding.job_throughput(B * L * args.steps, world, ms * 1e-3)
+    value = sharding.job_throughput(B * L, world, step_ms * 1e-3)
     peak, peak_kind = measured_peak()
-    step_s = ms * 1e-3 / args.steps
+    step_s = step_ms * 1e-3
     achieved = step_bytes / step_s / 1e9
+    so_achieved = step_bytes / (so_step_ms * 1e-3) / 1e9
     digest = sources_digest()
     traffic = None
     if (NCU_TRAFFIC["sources_sha256"] == digest and NCU_TRAFFIC["workload"] == name
@@ -394,36 +430,52 @@ def run_native(args) -> None:
         traffic = NCU_TRAFFIC["bytes_per_launch"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": dict(describe(name, kw, "exp delta=1.1 nu=0.7"),
-                       parallelism=f"dp{world} (independent sequences, no exchange)",
-                       l2=f"ring of {ring_n} distinct step inputs, {ring_n * step_bytes / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2",
-                       launch=f"CUDA graph of {graph_steps} steps, replayed",
-                       monitors=bool(args.monitors),
-                       partition=("one call at a time: ordinary stream order, sequences split over clusters" if args.single_call_latency
-                                  else "back_to_back: one block per sequence, consecutive calls overlap")),
+        "config": describe(name, kw, "exp delta=1.1 nu=0.7"),
+        "timed_calls": timed_calls, "reps": REPS,
+        "ms_per_step_reps": {"min": step_ms_reps[0], "median": step_ms, "max": step_ms_reps[-1]},
+        "run": {"parallelism": f"dp{world} (independent sequences, no exchange)",
+                "l2": f"ring of {ring_n} distinct step inputs, {ring_n * step_bytes / 1e6:.0f} MB > {L2_BYTES / 1e6:.0f} MB L2",
+                "launch": f"CUDA graph of {graph_steps} calls, {replays} replays per repetition, {REPS} repetitions "
+                          f"(median reported); warm-up {warm_replays} replays",
+                "monitors": bool(args.monitors),
+                "partition": ("one call at a time: ordinary stream order, sequences split over clusters" if args.single_call_latency
+                              else "back_to_back: consecutive calls overlap (programmatic dependent launch)"),
+                "arithmetic": "fp32 exponentials and sums, fp64 running sums in the draw; logits stored as "
+                              + ("bf16" if dtype == W.BF16 else "fp32")},
         "clocks": sampler.summary(),
         "e2e": {"value": B * L * e2e_steps * world / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": e2e_steps, "entry": "csd_verify_host (pinned host buffers)",
                 "matches_device_run": same},
-        "gpu_launches": kernels_per_step * args.steps,
+        "gpu_launches": kernels_per_step * timed_calls * REPS,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
                      "bytes_per_launch": step_bytes,
                      "duration_us": step_s * 1e6,
                      "kernel": "the single fused launch of a step" if kernels_per_step == 1 else "all launches of a step",
-                     "note": "duration = timed region / launches, CUDA events on the launching stream; calls overlap, so "
-                             "this is the sustained time per launch"},
+                     "note": "duration = median repetition / its launches, CUDA events on the launching stream; calls "
+                             "overlap, so this is the sustained time per launch"},
+        "stream_order": {"us_per_call": so_step_ms * 1e3, "achieved": so_achieved, "unit": "GB/s", "frac": so_achieved / peak,
+                         "calls": replays_so * graph_steps, "reps": 3,
+                         "note": "back_to_back = 0: each call starts when the one before it has completed, as in a "
+                                 "decoding loop whose logits come from the forward pass just before the call"},
         "emitted_tokens_per_step_mean": B * mean_emit,
     }
     if world == 1 and not args.no_cpu_baseline:
         t1, n1, threads = time_oracle(name, kw, 1, B, device=dev)
         n = int(min(64, max(1, round(12.0 / max(t1, 1e-3)))))
         t, nseq, threads = time_oracle(name, kw, n, B, seed=7, device=dev)
+        import oracle
+        oracle.set_num_threads(1)
+        n_one = int(min(B, 8))   # one thread: a few sequences are a few seconds
+        ts, ns, _ = time_oracle(name, kw, 1, n_one, seed=11, device=dev)
+        oracle.set_num_threads(threads)
         line["cpu_baseline"] = {"value": nseq * L / t, "unit": UNIT, "cores": threads, "kind": "oracle",
                                 "sample": f"{n} full steps ({nseq} sequences, ring of 4 seeded batches) of the "
-                                          f"same workload, {t:.1f} s wall"}
+                                          f"same workload, {t:.1f} s wall",
+                                "single_thread": {"value": ns * L / ts, "unit": UNIT, "cores": 1,
+                                                  "sample": f"{ns} sequences of one step, {ts:.1f} s wall"}}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
@@ -504,7 +556,7 @@ def main() -> None:
                     help="also ask for the per-position monitors of Theorem 2 (a second pass over every row)")
     ap.add_argument("--single-call-latency", action="store_true",
                     help="csd_params.back_to_back = 0: ordinary stream order, each call spread over the whole GPU")
-    ap.add_argument("--steps", type=int, default=5760)
+    ap.add_argument("--steps", type=int, default=2048)
     ap.add_argument("--warmup", type=int, default=64)
     ap.add_argument("--impl", default="native", choices=["native", "reference"])
     ap.add_argument("--workload", default="C3")

@@ -62,7 +62,8 @@ typedef enum {
   CSD_ERR_WORKSPACE = -4, /* workspace NULL, misaligned (256 B) or smaller than csd_workspace_size */
   CSD_ERR_ARG = -5,       /* inconsistent options (one unconditional array without the other, top_k < 0, ...) */
   CSD_ERR_LAUNCH = -6,    /* the CUDA runtime refused a launch or copy; see cudaGetLastError */
-  CSD_ERR_ALLOC = -7,     /* csd_verify only: its internal workspace could not be allocated */
+  CSD_ERR_ALIGN = -7,     /* csd_verify only: the inputs need the scalar path, which needs a workspace
+                             (logits not 16-byte aligned, V not a multiple of 4, or V < 128) */
   CSD_ERR_STATIC_LIMIT = -8 /* csd_verify_static only: the problem needs more scratch than the
                                built-in CSD_STATIC_SCRATCH_BYTES */
 } csd_error;
@@ -99,11 +100,12 @@ typedef enum {
  *   out_tokens     [B, gamma+1]   device, written; x_{1:tau+1}, then -1
  *   out_accept_len [B]            device, written; tau in [0, gamma]
  *
- * Scratch: this form keeps one workspace per device inside the library,
- * allocated with cudaMalloc on first use and grown when a larger problem
- * arrives (so the first call of a given size must not be inside a stream
- * capture, and concurrent calls on different streams of one device must use
- * csd_verify_ex with their own workspaces instead).
+ * Scratch: none.  This form never allocates, frees or synchronises and keeps no
+ * state between calls, so it may be called from any number of streams at once.
+ * It serves only inputs the single-launch path can take -- 16-byte aligned logit
+ * pointers, V a multiple of 4, V >= 128 -- and returns CSD_ERR_ALIGN otherwise
+ * (csd_verify_ex with a workspace takes any layout).  It has no status output:
+ * unusable rows or tokens still give the defined results, silently.
  */
 int csd_verify(const float* target_logits, const float* draft_logits, const int32_t* draft_tokens,
                const float* uniforms, const float* relax_schedule, int B, int gamma, int V,
@@ -137,9 +139,13 @@ int csd_verify(const float* target_logits, const float* draft_logits, const int3
  *     it; make that first call outside any stream capture.
  *   - All calls on one device share the one array.  Nothing in it has to start
  *     at a value the caller provides -- each call overwrites what it later reads -- so no
- *     clearing is needed between calls (the few words that must be zero are zero
- *     when the library is loaded and every call puts them back), and what a call
- *     leaves behind is otherwise meaningless.  Two calls that may run on the GPU at the same time (different
+ *     clearing is needed between calls, and what a call leaves behind is otherwise
+ *     meaningless.  One word is an exception: if a bounded wait inside a kernel ever
+ *     gives up (CSD_STATUS_TIMEOUT), that is recorded in the array and stays there
+ *     for the life of the process -- the caller cannot run csd_workspace_init on it.
+ *     This form has no status output, so nothing reads that word and later calls
+ *     are unaffected; a caller that must learn of timeouts uses csd_verify_ex.
+ *     Two calls that may run on the GPU at the same time (different
  *     streams, no ordering between them) would overwrite each other's scratch:
  *     keep calls on one device ordered, or use csd_verify_ex with separate
  *     workspaces for the concurrent ones.
@@ -280,6 +286,19 @@ int csd_sample_rows(const void* logits, const void* uncond, float cfg_scale, int
  * Returns CSD_OK, CSD_ERR_NULL or CSD_ERR_ARG.
  */
 int csd_make_schedule(int kind, double delta, double nu_or_ell, int L, float* out_host);
+
+/*
+ * Testing aid for the bounded waits (every wait of a kernel on a copy into shared memory gives up
+ * after a limit and reports CSD_STATUS_TIMEOUT instead of hanging).  Process-wide, applies to calls
+ * made afterwards:
+ *   wait_limit_log2_cycles  0: the normal limit (2^31 SM cycles, about a second); 10..40: 2^n cycles
+ *   drop_first_copy         non-zero: in every following call, the first copy of thread block 0 is
+ *                           announced to its barrier but never issued, so the wait on it runs out
+ *                           (nothing is left in flight; the block finishes and the call reports
+ *                           CSD_STATUS_TIMEOUT for every sequence)
+ * csd_test_hooks(0, 0) restores normal operation.  Returns CSD_OK or CSD_ERR_ARG.  Not for production use.
+ */
+int csd_test_hooks(int wait_limit_log2_cycles, int drop_first_copy);
 
 /* Static, NUL-terminated description of a csd_error value. */
 const char* csd_error_string(int code);

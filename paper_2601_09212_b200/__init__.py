@@ -22,7 +22,7 @@ CSD_STATUS_BADROW, CSD_STATUS_BADTOKEN, CSD_STATUS_ZFALLBACK, CSD_STATUS_TIMEOUT
 CSD_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
 EXPORTS = ("csd_verify", "csd_verify_static", "csd_verify_ex", "csd_workspace_size", "csd_workspace_init", "csd_launch_count", "csd_verify_host",
            "csd_host_staging_size", "csd_make_schedule", "csd_error_string", "csd_version",
-           "csd_sample_rows", "csd_sample_workspace_size")
+           "csd_sample_rows", "csd_sample_workspace_size", "csd_test_hooks")
 
 
 class CsdError(RuntimeError):
@@ -81,6 +81,8 @@ def library() -> C.CDLL:
         lib.csd_error_string.argtypes = [C.c_int]
         lib.csd_error_string.restype = C.c_char_p
         lib.csd_version.restype = C.c_int
+        lib.csd_test_hooks.argtypes = [C.c_int, C.c_int]
+        lib.csd_test_hooks.restype = C.c_int
         lib.csd_sample_workspace_size.argtypes = [C.c_int] * 3
         lib.csd_sample_workspace_size.restype = C.c_size_t
         lib.csd_sample_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_int, C.c_int, C.c_int, C.c_int,
@@ -100,6 +102,13 @@ csd_error_string = error_string
 
 def csd_version() -> int:
     return int(library().csd_version())
+
+
+def csd_test_hooks(wait_limit_log2_cycles: int = 0, drop_first_copy: bool = False) -> None:
+    """Testing aid for the bounded waits (see csd.h); ``csd_test_hooks()`` restores normal operation."""
+    rc = library().csd_test_hooks(int(wait_limit_log2_cycles), int(bool(drop_first_copy)))
+    if rc != 0:
+        raise CsdError(rc, "csd_test_hooks")
 
 
 def csd_make_schedule(kind: int, delta: float, nu_or_ell: float, L: int) -> np.ndarray:

@@ -79,60 +79,27 @@ double normal_upper_quantile(double tail) {
   return 0.5 * (lo + hi);
 }
 
-template <typename T, bool CFG>
+// Launches one of the two single-launch kernels (KERNEL: 0 plain, 1 top-k) with its shared-memory
+// size, optionally with programmatic stream serialisation and as clusters of ctas_per_seq blocks.
+template <typename T, bool CFG, int KERNEL>
 cudaError_t launch_fused(const FusedArgs& a, int grid, bool overlap, cudaStream_t stream) {
-  auto kern = verify_topk_kernel<T, CFG>;
+  auto kern = KERNEL ? verify_topk_kernel<T, CFG> : verify_plain_kernel<T, CFG>;
+  constexpr size_t kSmem = KERNEL ? sizeof(TopkSmem) : sizeof(PlainSmem);
+  constexpr int kThreads = KERNEL ? kTopkThreads : kPlainThreads;
   // the attribute belongs to (function, device): set it once per device (setting it twice is harmless)
   static bool configured[kMaxDevices] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
   if (!configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(TopkSmem));
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(kTopkThreads);
-  cfg.dynamicSmemBytes = sizeof(TopkSmem);
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[2];
-  int n_attr = 0;
-  if (overlap) {   // the call may start while the operation before it on the stream is still running
-    attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
-    ++n_attr;
-  }
-  if (a.ctas_per_seq > 1) {   // the blocks of a sequence are one cluster
-    attr[n_attr].id = cudaLaunchAttributeClusterDimension;
-    attr[n_attr].val.clusterDim.x = (unsigned)a.ctas_per_seq;
-    attr[n_attr].val.clusterDim.y = 1;
-    attr[n_attr].val.clusterDim.z = 1;
-    ++n_attr;
-  }
-  cfg.attrs = attr;
-  cfg.numAttrs = n_attr;
-  return cudaLaunchKernelEx(&cfg, kern, a);
-}
-
-template <typename T, bool CFG>
-cudaError_t launch_plain(const FusedArgs& a, int grid, bool overlap, cudaStream_t stream) {
-  auto kern = verify_plain_kernel<T, CFG>;
-  // the attribute belongs to (function, device): set it once per device (setting it twice is harmless)
-  static bool configured[kMaxDevices] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  if (!configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(PlainSmem));
-    if (e != cudaSuccess) return e;
-    configured[dev] = true;
-  }
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof cfg);
-  cfg.gridDim = dim3((unsigned)grid);
-  cfg.blockDim = dim3(kPlainThreads);
-  cfg.dynamicSmemBytes = sizeof(PlainSmem);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmem;
   cfg.stream = stream;
   cudaLaunchAttribute attr[2];
   int n_attr = 0;
@@ -155,7 +122,7 @@ cudaError_t launch_plain(const FusedArgs& a, int grid, bool overlap, cudaStream_
 
 template <typename T, bool CFG>
 cudaError_t launch_fused_t(const FusedArgs& a, bool topk, int grid, bool overlap, cudaStream_t stream) {
-  return topk ? launch_fused<T, CFG>(a, grid, overlap, stream) : launch_plain<T, CFG>(a, grid, overlap, stream);
+  return topk ? launch_fused<T, CFG, 1>(a, grid, overlap, stream) : launch_fused<T, CFG, 0>(a, grid, overlap, stream);
 }
 
 template <typename T, bool CFG, int U, bool TOPK>
@@ -222,9 +189,15 @@ cudaError_t launch_finish(const FinishArgs& a, cudaStream_t stream) {
   return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
+// Test aids (csd_test_hooks): process-wide, read at every launch of the single-launch path.
+long long g_wait_limit = kWaitCycles;
+int g_drop_first_copy = 0;
+
 // sampling: the degenerate round used by csd_sample_rows -- no draft positions (gamma = 0), one
 // "target" row per sequence, whose bonus draw is the wanted token; the drafter-side pointers are unused.
-int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = false) {
+// no_workspace: the call has no workspace (the simple forms): only the single-launch path, which keeps
+// nothing in global memory, can serve it; otherwise CSD_ERR_ALIGN.
+int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = false, bool no_workspace = false) {
   if (sampling) {
     if (!p.target_logits || !p.uniforms || !p.out_tokens) return CSD_ERR_NULL;
   } else if (!p.target_logits || !p.draft_logits || !p.draft_tokens || !p.uniforms || !p.relax_schedule ||
@@ -247,7 +220,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
   if (cfg && !isfinite(p.cfg_scale)) return CSD_ERR_ARG;
   const bool topk = p.top_k > 0 && p.top_k < p.V;
   const Layout lay = layout_for(p.B, p.gamma, p.V, p.dtype);
-  if (!p.workspace || ((uintptr_t)p.workspace % kAlign) != 0 || p.workspace_bytes < lay.total)
+  if (!no_workspace && (!p.workspace || ((uintptr_t)p.workspace % kAlign) != 0 || p.workspace_bytes < lay.total))
     return CSD_ERR_WORKSPACE;
   int dev = 0;
   const int sms = device_sms(&dev);
@@ -279,8 +252,9 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
   sa.part_elems = kStatsThreads * U * vw;
   sa.n_items = (int)(rows * sa.parts);
   sa.vec_ok = vec_ok ? 1 : 0;
-  sa.partials = reinterpret_cast<float2*>((char*)p.workspace + lay.partials_off);
-  sa.thresholds = reinterpret_cast<const float*>((char*)p.workspace + lay.thresholds_off);
+  char* const ws = no_workspace ? nullptr : (char*)p.workspace;   // (the single-launch path never touches these)
+  sa.partials = ws ? reinterpret_cast<float2*>(ws + lay.partials_off) : nullptr;
+  sa.thresholds = ws ? reinterpret_cast<const float*>(ws + lay.thresholds_off) : nullptr;
 
   SelectArgs se;
   se.target = p.target_logits; se.draft = p.draft_logits;
@@ -290,7 +264,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
   se.tstride = tstride; se.dstride = dstride;
   se.vec_ok = sa.vec_ok;
   se.top_k = p.top_k;
-  se.thresholds = reinterpret_cast<float*>((char*)p.workspace + lay.thresholds_off);
+  se.thresholds = ws ? reinterpret_cast<float*>(ws + lay.thresholds_off) : nullptr;
 
   FinishArgs fa;
   fa.target = p.target_logits; fa.draft = p.draft_logits;
@@ -302,7 +276,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
   fa.vec_ok = sa.vec_ok;
   fa.use_topk = topk ? 1 : 0;
   fa.partials = sa.partials;
-  fa.thresholds = reinterpret_cast<const float*>((char*)p.workspace + lay.thresholds_off);
+  fa.thresholds = sa.thresholds;
   fa.tokens = p.draft_tokens; fa.uniforms = p.uniforms; fa.schedule = p.relax_schedule;
   fa.out_tokens = p.out_tokens; fa.out_accept_len = p.out_accept_len; fa.out_status = p.out_status;
   fa.dbg_p = p.dbg_p; fa.dbg_q = p.dbg_q; fa.dbg_f = p.dbg_f; fa.dbg_G = p.dbg_G;
@@ -310,6 +284,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
 
   // ---- fused single-launch path: aligned rows of at least 512 bytes; with top-k, rows that fit the registers
   const bool fused = vec_ok && (size_t)p.V * es >= 512 && (p.V + 32 * vw - 1) / (32 * vw) <= kFinTiles;
+  if (no_workspace && !fused) return CSD_ERR_ALIGN;
   if (plan_only) {  // number of kernels this call would enqueue
     *plan_only = fused ? 1 : (topk ? 3 : 2);
     return CSD_OK;
@@ -320,7 +295,9 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
     ua.top_k = p.top_k;
     ua.lo_sigmas = nanf("");
     ua.lo_delta = 0.0f;
-    ua.error_flag = reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
+    ua.error_flag = no_workspace ? nullptr : reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
+    ua.wait_limit = g_wait_limit;
+    ua.drop_first_copy = g_drop_first_copy;
     // Blocks are aligned with sequences and positions.  For calls enqueued back to back a block owns a
     // whole sequence (for very large batches seqs_per_cta of them): such calls overlap on the GPU as
     // deeply as their grids allow (a call may start once every block of its predecessor has started),
@@ -399,13 +376,6 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
   return e == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
 }
 
-// internal workspace of the simple form, one per device
-struct OwnedWorkspace {
-  void* ptr = nullptr;
-  size_t bytes = 0;
-};
-OwnedWorkspace g_ws[kMaxDevices];
-
 }  // namespace
 
 extern "C" {
@@ -466,31 +436,6 @@ int csd_verify(const float* target_logits, const float* draft_logits, const int3
                const float* uniforms, const float* relax_schedule, int B, int gamma, int V,
                int32_t* out_tokens, int32_t* out_accept_len, void* stream) {
   if (!shape_ok(B, gamma, V)) return CSD_ERR_SHAPE;
-  const size_t need = csd_workspace_size(B, gamma, V, CSD_F32);
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CSD_ERR_LAUNCH;
-  void* ws = nullptr;
-  {
-    std::lock_guard<std::mutex> lock(g_mutex);
-    OwnedWorkspace& w = g_ws[dev];
-    if (w.bytes < need) {
-      // earlier calls may still be using the old buffer
-      if (w.ptr) {
-        if (cudaDeviceSynchronize() != cudaSuccess) return CSD_ERR_LAUNCH;
-        cudaFree(w.ptr);
-        w.ptr = nullptr;
-        w.bytes = 0;
-      }
-      if (cudaMalloc(&w.ptr, need) != cudaSuccess) {
-        w.ptr = nullptr;
-        (void)cudaGetLastError();
-        return CSD_ERR_ALLOC;
-      }
-      w.bytes = need;
-      if (cudaMemsetAsync(w.ptr, 0, need, (cudaStream_t)stream) != cudaSuccess) return CSD_ERR_LAUNCH;
-    }
-    ws = w.ptr;
-  }
   csd_params p;
   memset(&p, 0, sizeof p);
   p.target_logits = target_logits; p.draft_logits = draft_logits;
@@ -498,9 +443,15 @@ int csd_verify(const float* target_logits, const float* draft_logits, const int3
   p.B = B; p.gamma = gamma; p.V = V; p.target_rows = gamma;
   p.draft_tokens = draft_tokens; p.uniforms = uniforms; p.relax_schedule = relax_schedule;
   p.out_tokens = out_tokens; p.out_accept_len = out_accept_len;
-  p.workspace = ws; p.workspace_bytes = need;
   p.stream = stream;
-  return verify_impl(p);
+  return verify_impl(p, nullptr, false, /*no_workspace=*/true);
+}
+
+int csd_test_hooks(int wait_limit_log2_cycles, int drop_first_copy) {
+  if (wait_limit_log2_cycles != 0 && (wait_limit_log2_cycles < 10 || wait_limit_log2_cycles > 40)) return CSD_ERR_ARG;
+  g_wait_limit = wait_limit_log2_cycles ? (1ll << wait_limit_log2_cycles) : kWaitCycles;
+  g_drop_first_copy = drop_first_copy ? 1 : 0;
+  return CSD_OK;
 }
 
 // ---- allocation-free form -------------------------------------------------------------
@@ -711,12 +662,12 @@ const char* csd_error_string(int code) {
     case CSD_ERR_WORKSPACE: return "workspace missing, not 256-byte aligned, or too small";
     case CSD_ERR_ARG: return "inconsistent or unsupported options";
     case CSD_ERR_LAUNCH: return "CUDA runtime error while enqueueing work";
-    case CSD_ERR_ALLOC: return "could not allocate the internal workspace";
+    case CSD_ERR_ALIGN: return "csd_verify needs 16-byte aligned logits with V a multiple of 4 and at least 128; use csd_verify_ex with a workspace";
     case CSD_ERR_STATIC_LIMIT: return "problem too large for the built-in scratch of csd_verify_static (CSD_STATIC_SCRATCH_BYTES); use csd_verify_ex with a caller workspace";
     default: return "unknown error code";
   }
 }
 
-int csd_version(void) { return 300; }
+int csd_version(void) { return 400; }
 
 }  // extern "C"

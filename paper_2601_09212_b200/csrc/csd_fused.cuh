@@ -60,15 +60,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within about kWaitCycles.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// Bounded wait: false if the phase did not complete within about `limit` cycles.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const long long limit = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (clock64() - t0 > kWaitCycles) return false;
+    if (clock64() - t0 > limit) return false;
   }
 }
 // global -> shared bulk copy of `bytes` (multiple of 16; both addresses 16-byte aligned),
@@ -154,7 +154,10 @@ struct FusedArgs {
   int top_k;
   float lo_sigmas;      // top-k guess: lo = mean + lo_sigmas * deviation (NaN: always select exactly)
   float lo_delta;       // how many deviations below a row's exact threshold the next guess should sit (< 0)
-  int* error_flag;      // set when a bounded wait gave up
+  int* error_flag;      // set when a bounded wait gave up; null: nobody asked for the status
+  long long wait_limit; // cycles a wait on a copy may take (kWaitCycles unless a test shortens it)
+  int drop_first_copy;  // test aid: the first copy of block 0 is announced to its barrier but never issued,
+                        // so that the wait on it runs out (nothing is left in flight)
 };
 
 // ---- a block's share of the work ------------------------------------------------------
@@ -324,31 +327,7 @@ __device__ int draw_token(const FinishArgs& a, const Row<T, CFG>& rt, const Row<
     }
     __syncthreads();
     // ---- locate the tile that holds the crossing C(x) > u Z ---------------------------------
-    if (warp == 0) {
-      const int chunk = (ntiles + 31) / 32;
-      const int t0 = lane * chunk, t1 = min(ntiles, t0 + chunk);
-      double local = 0.0;
-      for (int t = t0; t < t1; ++t) local += tile_sums[t];
-      const double incl = warp_incl_scan_double(local, lane);
-      const double Z = __shfl_sync(0xffffffffu, incl, 31);
-      const double target = (double)u * Z;
-      const bool mine = incl > target && local > 0.0;
-      const unsigned ballot = __ballot_sync(0xffffffffu, mine);
-      if (lane == 0) { sm.Z = Z; sm.pick_tile = -1; }
-      __syncwarp();
-      if (ballot != 0 && lane == __ffs(ballot) - 1) {
-        double c = incl - local, c_pick = c;
-        int pick = t0;
-        for (int t = t0; t < t1; ++t) {
-          const double v = tile_sums[t];
-          if (v > 0.0) { pick = t; c_pick = c; }   // last tile with mass seen so far
-          if (c + v > target && v > 0.0) break;
-          c += v;
-        }
-        sm.pick_tile = pick;
-        sm.pick_prefix = c_pick;
-      }
-    }
+    if (warp == 0) locate_crossing_tile(tile_sums, ntiles, u, lane, sm);
     __syncthreads();
     const double Z = sm.Z;
     if (!(Z > 0.0) || !(Z < (double)CSD_POS_INF)) {
@@ -363,34 +342,18 @@ __device__ int draw_token(const FinishArgs& a, const Row<T, CFG>& rt, const Row<
     // ---- scan inside that tile (its 32 vectors come from global memory again) ------------------
     if (warp == 0) {
       const int tile = sm.pick_tile;
-      const double target = (double)u * Z;
-      const int x0 = tile * TILE + lane * VEC;
-      float zt[VEC], zd[VEC];
-      rt.load_tile(x0, V, 1, zt);
-      if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd);
-      double run[VEC];
-      double acc = 0.0;
-      int last_pos = -1;
-      unsigned posmask = 0;
+      int tok = -1;
+      if (tile >= 0) {   // (the same decision in every lane)
+        const int x0 = tile * TILE + lane * VEC;
+        float zt[VEC], zd[VEC], g[VEC];
+        rt.load_tile(x0, V, 1, zt);
+        if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd);
 #pragma unroll
-      for (int k = 0; k < VEC; ++k) {
-        const float g = weight_of(FILT ? rt.filter(zt[k]) : zt[k], ctx.mode == 0 ? (FILT ? rd.filter(zd[k]) : zd[k]) : 0.0f, ctx);
-        if (g > 0.0f) { last_pos = k; posmask |= 1u << k; }
-        acc += (double)g;
-        run[k] = acc;
+        for (int k = 0; k < VEC; ++k)
+          g[k] = weight_of(FILT ? rt.filter(zt[k]) : zt[k], ctx.mode == 0 ? (FILT ? rd.filter(zd[k]) : zd[k]) : 0.0f, ctx);
+        tok = pick_in_tile<VEC>(g, x0, sm.pick_prefix, (double)u * Z, lane);
       }
-      const double before = sm.pick_prefix + (warp_incl_scan_double(acc, lane) - acc);
-      int first = -1;
-#pragma unroll
-      for (int k = VEC - 1; k >= 0; --k)
-        if (before + run[k] > target && ((posmask >> k) & 1u)) first = k;
-      const unsigned hit = __ballot_sync(0xffffffffu, first >= 0);
-      const unsigned pos = __ballot_sync(0xffffffffu, last_pos >= 0);
-      if (hit != 0) {
-        if (lane == __ffs(hit) - 1) sm.token = x0 + first;
-      } else if (pos != 0) {  // rounding left no crossing: last token with positive weight
-        if (lane == 31 - __clz(pos)) sm.token = x0 + last_pos;
-      } else if (lane == 0) sm.token = -1;
+      if (lane == 0) sm.token = tok;
     }
     __syncthreads();
     token = sm.token;
@@ -726,7 +689,7 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
       if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase, phase2);
       if (sl == 0) {   // before the block's first global write: outputs of consecutive calls stay in order
         pdl_wait();
-        sticky = __ldcg(ua.error_flag) ? 8 : 0;
+        sticky = (ua.error_flag && __ldcg(ua.error_flag)) ? 8 : 0;
       }
       write_pqf(b);
       emit_sequence<T, CFG, NT>(ua, b, st.rec, st.rec.status_any | sticky, tid);
@@ -760,7 +723,7 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
   draw_position<T, CFG, NT, FILT>(ua, sh, 0, j, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
   if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase, phase2);
   pdl_wait();   // the previous call has completed: outputs of consecutive calls stay in order
-  if (__ldcg(ua.error_flag)) any = 8;
+  if (ua.error_flag && __ldcg(ua.error_flag)) any = 8;
   write_pqf(b);
   emit_sequence<T, CFG, NT>(ua, b, st.rec, any, tid);
 }
@@ -824,8 +787,10 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
 
   // producer cursor (meaningful in lane 0): the next chunk to copy
   int p_item = item_begin, p_x = 0, p_xend = 0, p_s = 0;
+  int p_count = 0;   // chunks announced to the barriers so far
   int p_row = item_begin / parts, p_part = item_begin - p_row * parts;   // kept incrementally from here on
   const T *p_cond = nullptr, *p_uncond = nullptr;
+  bool drop_next = a.drop_first_copy != 0 && blockIdx.x == 0 && warp == 0;   // (test aid, see FusedArgs)
   auto producer_open_row = [&]() {    // pointers of row p_row
     int b, which, i;
     local_row(sh, p_row, f.gamma, b, which, i);
@@ -841,8 +806,12 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
     if (p_item >= item_end) return;
     const uint32_t bytes = (uint32_t)(min(EPS, p_xend - p_x) * (int)sizeof(T));
     mbar_expect_tx(&sm.full[warp][p_s], bytes * ARR);
-    bulk_load(&sm.ring[warp][p_s][0], p_cond + p_x, bytes, &sm.full[warp][p_s]);
-    if (CFG) bulk_load(&sm.ring[warp][p_s][kWStageBytes / 2], p_uncond + p_x, bytes, &sm.full[warp][p_s]);
+    if (!drop_next) {
+      bulk_load(&sm.ring[warp][p_s][0], p_cond + p_x, bytes, &sm.full[warp][p_s]);
+      if (CFG) bulk_load(&sm.ring[warp][p_s][kWStageBytes / 2], p_uncond + p_x, bytes, &sm.full[warp][p_s]);
+    }
+    drop_next = false;
+    ++p_count;
     p_s = p_s + 1 == kWStages ? 0 : p_s + 1;
     p_x += EPS;
     if (p_x >= p_xend) {
@@ -869,8 +838,8 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
   {
     int c_s = 0;          // stage the consumer reads next
     uint32_t c_par = 0;   // its parity
-    int issued = 0;       // chunks consumed so far (for the bounded wait after a timeout)
-    bool ok = true;
+    int waited = 0;       // chunks whose copies this lane has seen complete
+    bool ok = true;       // false once a wait has run out: from then on nothing is waited for or issued
     int cur_row = -1, tok_cur = -1, tok_next = -1;
     const int last_row = item_end > item_begin ? (item_end - 1) / parts : -1;
     int row_id = item_begin / parts, part = item_begin - row_id * parts;   // kept incrementally
@@ -899,8 +868,9 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
       float nMwL = CSD_POS_INF, dlt = 0.0f;   // -MwL and dlt of the current reference
       int cnt_run = 0;
       for (int x0 = x_begin; x0 < x_end; x0 += EPS) {
-        if (ok && !mbar_wait(&sm.full[warp][c_s], c_par)) ok = false;
-        ++issued;
+        if (ok) {
+          if (mbar_wait(&sm.full[warp][c_s], c_par, a.wait_limit)) ++waited; else ok = false;
+        }
         const int n = min(EPS, x_end - x0);
         const unsigned char* stage = &sm.ring[warp][c_s][0];
         const bool full = n == EPS;   // (after a timeout the data is garbage anyway: the call is flagged)
@@ -986,7 +956,7 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
           has_tok = true;
         }
         __syncwarp();
-        if (lane == 0) {   // the stage is free again: refill it with the chunk kWStages ahead
+        if (lane == 0 && ok) {   // the stage is free again: refill it with the chunk kWStages ahead
           fence_before_bulk();
           producer_issue();
         }
@@ -1003,12 +973,15 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
         if (has_tok && row_id < kBlockRows) sm.rs.tokz[row_id] = tokz;
       }
     }
-    if (!ok && lane == 0) {
+    if (!ok) {
       sm.abort = 1;
-      atomicExch(a.error_flag, 1);
-      // copies this warp gave up on may still be in flight: wait for them, again bounded
-      for (int s = 0; s < kWStages; ++s)
-        if (issued > s) (void)mbar_wait(&sm.full[warp][s], ((issued - 1 - s) / kWStages) & 1);
+      if (lane == 0) {
+        if (a.error_flag) atomicExch(a.error_flag, 1);
+        // Nothing was issued after lane 0's failed wait, so the copies that may still be in flight are
+        // those of chunks [waited, p_count): at most one per stage.  Wait for each, again bounded.
+        for (int c = waited; c < p_count; ++c)
+          (void)mbar_wait(&sm.full[warp][c % kWStages], (uint32_t)(c / kWStages) & 1u, a.wait_limit);
+      }
     }
   }
 
@@ -1048,6 +1021,7 @@ struct TopkSmem {
   alignas(128) unsigned char ring[kTkStages][kTkStageBytes];
   alignas(8) uint64_t full[kTkStages];
   int readers_done[kTkStages];      // warps that have finished reading the stage's current contents
+  int issued_q;                     // chunks announced to the barriers so far (written by the issuing thread)
   alignas(16) int hist[kLinBins];   // linear histogram; first 256 bins double as the radix histogram
   alignas(8) float list[kTopkWarps][kWarpList];   // per warp: the values >= lo it met (the finish keeps its tile sums here)
   int wpos[kTopkWarps];            // per warp: next free slot of its list (may run past the capacity)
@@ -1196,6 +1170,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
     for (int s = 0; s < kTkStages; ++s) { mbar_init(&sm.full[s], 1); sm.readers_done[s] = 0; }
     mbar_init(&sm.fst.bar, 1); mbar_init(&sm.fst.bar2, 1);
     sm.abort = 0;
+    sm.issued_q = 0;
     sm.n_cand[0] = 0;
     sm.n_cand[1] = 0;
     sm.arrive[0] = 0;
@@ -1233,6 +1208,8 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
     const int x0 = c * EPS;
     const uint32_t bytes = (uint32_t)(min(EPS, V - x0) * (int)sizeof(T));
     mbar_expect_tx(&sm.full[s], bytes * ARR);
+    sm.issued_q = q + 1;
+    if (q == 0 && a.drop_first_copy != 0 && blockIdx.x == 0) return;   // (test aid, see FusedArgs)
     bulk_load(&sm.ring[s][0], row.cond + x0, bytes, &sm.full[s]);
     if (CFG) bulk_load(&sm.ring[s][kTkStageBytes / 2], row.uncond + x0, bytes, &sm.full[s]);
   };
@@ -1258,7 +1235,8 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   int n_my = 0;
   {
     int q = 0;
-    bool ok = true;
+    int waited = 0;   // chunks whose copies this thread has seen complete
+    bool ok = true;   // false once a wait has run out: from then on this thread waits for nothing
     int tok_next = row_begin < row_end ? token_of_row(row_begin) : -1;
     for (int row_id = row_begin; row_id < row_end; ++row_id, ++n_my) {
       const int par = n_my & 1;
@@ -1272,7 +1250,10 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         const int s = q % kTkStages;
         const uint32_t par_s = (uint32_t)(q / kTkStages) & 1u;
         ++q;
-        if (ok && !mbar_wait(&sm.full[s], par_s)) ok = false;
+        if (ok) {
+          if (mbar_wait(&sm.full[s], par_s, a.wait_limit)) ++waited;
+          else { ok = false; *(volatile int*)&sm.abort = 1; }
+        }
         const int x0 = c * EPS;
         const int n = min(EPS, V - x0);
         float z[VPT];
@@ -1322,8 +1303,12 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
           if (atomicAdd(&sm.readers_done[s], 1) == kTopkWarps - 1) {
             sm.readers_done[s] = 0;
             __threadfence_block();
-            fence_before_bulk();
-            issue_chunk(q - 1 + kTkStages, ahead_j, ahead_c);
+            // (a thread that gave up set the flag before it counted itself here: once any wait has
+            // run out, nothing more is issued)
+            if (*(volatile int*)&sm.abort == 0) {
+              fence_before_bulk();
+              issue_chunk(q - 1 + kTkStages, ahead_j, ahead_c);
+            }
           }
         }
         if (++ahead_c == cpr) { ahead_c = 0; ++ahead_j; }
@@ -1567,12 +1552,12 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         sm.rs.thr[r] = thr_e;
       }
     }
-    if (!ok && tid == 0) {
-      sm.abort = 1;
-      atomicExch(a.error_flag, 1);
-      // copies issued for stages this thread gave up on may still be in flight: wait for them, again bounded
-      for (int s = 0; s < kTkStages; ++s)
-        if (q > s) (void)mbar_wait(&sm.full[s], ((q - 1 - s) / kTkStages) & 1);
+    if (sm.abort && tid == 0) {
+      if (a.error_flag) atomicExch(a.error_flag, 1);
+      // Nothing was issued after the first failed wait was seen, so the copies that may still be in
+      // flight are those of chunks [waited, issued_q): at most one per stage.  Wait for each, bounded.
+      for (int c = waited; c < sm.issued_q; ++c)
+        (void)mbar_wait(&sm.full[c % kTkStages], (uint32_t)(c / kTkStages) & 1u, a.wait_limit);
     }
   }
 

@@ -491,6 +491,70 @@ struct FinishSmem {
   double pick_prefix, Z;
 };
 
+// ---- inverse-CDF draw over per-tile sums (one warp) ---------------------------------------------
+// Finds the tile that holds the crossing C(x) > u Z and the sum of the tiles before it; if no tile
+// qualifies (u >= 1 or NaN, or rounding), the last tile with positive mass -- the documented rule
+// "else the last token with positive weight".  Writes sm.Z, sm.pick_tile (-1: no tile has mass)
+// and sm.pick_prefix; every lane of the calling warp takes part.
+__device__ __forceinline__ void locate_crossing_tile(const double* tile_sums, const int ntiles, const float u,
+                                                     const int lane, FinishSmem& sm) {
+  const int chunk = (ntiles + 31) / 32;
+  const int t0 = min(ntiles, lane * chunk), t1 = min(ntiles, t0 + chunk);
+  double local = 0.0;
+  for (int t = t0; t < t1; ++t) local += tile_sums[t];
+  const double incl = warp_incl_scan_double(local, lane);
+  const double Z = __shfl_sync(0xffffffffu, incl, 31);
+  const double target = (double)u * Z;
+  const unsigned crossing = __ballot_sync(0xffffffffu, incl > target && local > 0.0);
+  const unsigned has_mass = __ballot_sync(0xffffffffu, local > 0.0);
+  if (lane == 0) { sm.Z = Z; sm.pick_tile = -1; sm.pick_prefix = 0.0; }
+  __syncwarp();
+  const unsigned from = crossing ? crossing : has_mass;
+  if (from == 0) return;
+  const int owner = crossing ? __ffs(crossing) - 1 : 31 - __clz(has_mass);
+  if (lane == owner) {
+    double c = incl - local, c_pick = c;
+    int pick = -1;
+    for (int t = t0; t < t1; ++t) {
+      const double v = tile_sums[t];
+      if (v > 0.0) { pick = t; c_pick = c; }   // last tile with mass seen so far
+      if (crossing && c + v > target && v > 0.0) break;
+      c += v;
+    }
+    sm.pick_tile = pick;
+    sm.pick_prefix = c_pick;
+  }
+}
+
+// The token inside the picked tile (one warp; lane holds the weights g[0..VEC) of its VEC consecutive
+// tokens starting at x0): the first token whose running sum exceeds u Z, else the tile's last token
+// with positive weight, else -1.
+template <int VEC>
+__device__ __forceinline__ int pick_in_tile(const float (&g)[VEC], const int x0, const double prefix,
+                                            const double target, const int lane) {
+  double run[VEC];
+  double acc = 0.0;
+  int last_pos = -1;
+  unsigned posmask = 0;
+#pragma unroll
+  for (int k = 0; k < VEC; ++k) {
+    if (g[k] > 0.0f) { last_pos = k; posmask |= 1u << k; }
+    acc += (double)g[k];
+    run[k] = acc;
+  }
+  const double before = prefix + (warp_incl_scan_double(acc, lane) - acc);
+  int first = -1;
+#pragma unroll
+  for (int k = VEC - 1; k >= 0; --k)
+    if (before + run[k] > target && ((posmask >> k) & 1u)) first = k;
+  const unsigned hit = __ballot_sync(0xffffffffu, first >= 0);
+  const unsigned pos = __ballot_sync(0xffffffffu, last_pos >= 0);
+  int token = -1;
+  if (hit != 0) token = __shfl_sync(0xffffffffu, x0 + first, __ffs(hit) - 1);
+  else if (pos != 0) token = __shfl_sync(0xffffffffu, x0 + last_pos, 31 - __clz(pos));
+  return token;
+}
+
 // Barrier over the NT threads that run the finish: the whole block (BAR == 0) or
 // a named barrier when other warps of the block do not take part.
 template <int NT, int BAR>
@@ -637,31 +701,7 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
       }
       group_sync<NT, BAR>();
       // ---- 5. locate the tile that holds the crossing C(x) > u Z ------------------
-      if (warp == 0) {
-        const int chunk = (ntiles + 31) / 32;
-        const int t0 = lane * chunk, t1 = min(ntiles, t0 + chunk);
-        double local = 0.0;
-        for (int t = t0; t < t1; ++t) local += tile_sums[t];
-        const double incl = warp_incl_scan_double(local, lane);
-        const double Z = __shfl_sync(0xffffffffu, incl, 31);
-        const double target = (double)u * Z;
-        const bool mine = incl > target && local > 0.0;
-        const unsigned ballot = __ballot_sync(0xffffffffu, mine);
-        if (lane == 0) { sm.Z = Z; sm.pick_tile = -1; }
-        __syncwarp();
-        if (ballot != 0 && lane == __ffs(ballot) - 1) {
-          double c = incl - local, c_pick = c;
-          int pick = t0;
-          for (int t = t0; t < t1; ++t) {
-            const double v = tile_sums[t];
-            if (v > 0.0) { pick = t; c_pick = c; }   // last tile with mass seen so far
-            if (c + v > target && v > 0.0) break;
-            c += v;
-          }
-          sm.pick_tile = pick;
-          sm.pick_prefix = c_pick;
-        }
-      }
+      if (warp == 0) locate_crossing_tile(tile_sums, ntiles, u, lane, sm);
       group_sync<NT, BAR>();
       const double Z = sm.Z;
       if (!(Z > 0.0) || !(Z < (double)CSD_POS_INF)) {
@@ -676,34 +716,18 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
       // ---- 6. scan inside that tile -------------------------------------------------
       if (warp == 0) {
         const int tile = sm.pick_tile;
-        const double target = (double)u * Z;
-        const int x0 = tile * TILE + lane * VEC;
-        float zt[VEC], zd[VEC];
-        rt.load_tile(x0, V, a.vec_ok, zt);
-        if (ctx.mode == 0) rd.load_tile(x0, V, a.vec_ok, zd);
-        double run[VEC];
-        double acc = 0.0;
-        int last_pos = -1;
-        unsigned posmask = 0;
+        int tok = -1;
+        if (tile >= 0) {   // (the same decision in every lane)
+          const int x0 = tile * TILE + lane * VEC;
+          float zt[VEC], zd[VEC], g[VEC];
+          rt.load_tile(x0, V, a.vec_ok, zt);
+          if (ctx.mode == 0) rd.load_tile(x0, V, a.vec_ok, zd);
 #pragma unroll
-        for (int k = 0; k < VEC; ++k) {
-          const float g = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
-          if (g > 0.0f) { last_pos = k; posmask |= 1u << k; }
-          acc += (double)g;
-          run[k] = acc;
+          for (int k = 0; k < VEC; ++k)
+            g[k] = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
+          tok = pick_in_tile<VEC>(g, x0, sm.pick_prefix, (double)u * Z, lane);
         }
-        const double before = sm.pick_prefix + (warp_incl_scan_double(acc, lane) - acc);
-        int first = -1;
-#pragma unroll
-        for (int k = VEC - 1; k >= 0; --k)
-          if (before + run[k] > target && ((posmask >> k) & 1u)) first = k;
-        const unsigned hit = __ballot_sync(0xffffffffu, first >= 0);
-        const unsigned pos = __ballot_sync(0xffffffffu, last_pos >= 0);
-        if (hit != 0) {
-          if (lane == __ffs(hit) - 1) sm.token = x0 + first;
-        } else if (pos != 0) {  // rounding left no crossing: last token with positive weight
-          if (lane == 31 - __clz(pos)) sm.token = x0 + last_pos;
-        } else if (lane == 0) sm.token = -1;
+        if (lane == 0) sm.token = tok;
       }
       group_sync<NT, BAR>();
       token = sm.token;

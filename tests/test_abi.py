@@ -37,7 +37,7 @@ def test_params_struct_matches_header():
 
 
 def test_version_and_error_strings(lib):
-    assert csd.csd_version() == 300
+    assert csd.csd_version() == 400
     for code in range(0, -8, -1):
         assert len(csd.error_string(code)) > 1
     assert "unknown" in csd.error_string(-99)

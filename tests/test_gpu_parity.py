@@ -770,6 +770,72 @@ def _below_resolution(w, got, ref, b):
     return bool(Z < 1e-10) and 0 <= drawn < w.V and P[drawn] > 0.0
 
 
+@pytest.mark.parametrize("kw", [
+    dict(B=6, gamma=3, V=4096, dtype=W.F32), dict(B=6, gamma=3, V=16384, dtype=W.BF16, cfg=True, top_k=500),
+    dict(B=6, gamma=3, V=66, dtype=W.F32), dict(B=40, gamma=4, V=2048, dtype=W.BF16, bonus_row=True)])
+@pytest.mark.parametrize("b2b", [False, True])
+def test_resample_uniform_outside_the_open_interval(kw, b2b):
+    """The draw's uniform is documented as lying in (0, 1).  A generator that can return 1.0, or a NaN,
+    must still give the documented result -- no crossing C(x) > u Z exists, so the last token with
+    positive weight -- and 0 gives the first such token; nothing may be read outside the rows.  The
+    damaged sequences have index > 0.  Every position is made to reject (omega = 0) or to accept
+    (a huge omega, so that the bonus draw is reached where there is a bonus row)."""
+    L = kw["gamma"]
+    for schedule in (np.zeros(L, np.float32), np.full(L, 1e9, np.float32)):
+        w = W.make("t", rho=0.9, schedule=schedule, seed=77, device=DEV, **kw)
+        B = w.B
+        for b, u in ((1, 1.0), (2, float("nan")), (3, 0.0), (B - 1, 1.0), (4, 1.5)):
+            w.uniforms[b, L] = u
+        rep, got, ref = check(w, back_to_back=b2b, want_dbg=B * w.V <= 4e6)
+        assert_ok(rep)
+        for b in (1, 2, B - 1, 4):
+            j = got["accept_len"][b]
+            if got["tokens"][b, j] >= 0:
+                assert got["tokens"][b, j] == ref.tokens[b, j]
+
+
+@pytest.mark.parametrize("kw", [dict(B=20, gamma=4, V=8192, dtype=W.F32),
+                                dict(B=20, gamma=4, V=16384, dtype=W.BF16, cfg=True, top_k=300)])
+@pytest.mark.parametrize("b2b", [False, True])
+def test_wait_that_runs_out_is_reported_not_hung(kw, b2b):
+    """Every wait of a kernel on a copy into shared memory is bounded.  With the testing aid the first
+    copy of block 0 is announced but never issued and the limit is about a millisecond: the call must
+    return, set CSD_STATUS_TIMEOUT for the sequences of the block that gave up, keep the condition in
+    the workspace (later calls on it report it for every sequence) until csd_workspace_init clears it,
+    and leave the context usable."""
+    L = kw["gamma"]
+    w = W.make("t", rho=0.9, schedule=sched(L), seed=31, device=DEV, **kw)
+    ws = csd.new_workspace(w.B, L, w.V, w.dtype)
+    good = run_gpu(w, want_dbg=False, workspace=ws, back_to_back=b2b)
+    assert np.all(good["status"] == 0)
+    csd.csd_test_hooks(21, True)
+    try:
+        bad = run_gpu(w, want_dbg=False, workspace=ws, back_to_back=b2b)
+    finally:
+        csd.csd_test_hooks()
+    assert bad["status"][0] & csd.CSD_STATUS_TIMEOUT
+    assert np.all(bad["accept_len"] >= 0) and np.all(bad["accept_len"] <= L)
+    sticky = run_gpu(w, want_dbg=False, workspace=ws, back_to_back=b2b)     # normal call, same workspace
+    assert np.all(sticky["status"] & csd.CSD_STATUS_TIMEOUT)
+    assert np.array_equal(sticky["tokens"], good["tokens"]) and np.array_equal(sticky["accept_len"], good["accept_len"])
+    csd.csd_workspace_init(ws)
+    clean = run_gpu(w, want_dbg=False, workspace=ws, back_to_back=b2b)
+    for key in ("tokens", "accept_len", "status"):
+        assert np.array_equal(clean[key], good[key]), key
+
+
+def test_multiplier_that_is_negative_or_nan_counts_as_zero():
+    """Eq. relax is stated for omega >= 0; a negative or NaN entry of the schedule is read as 0 on both
+    sides: the position rejects (for q > 0) and the draw is from the target distribution."""
+    L = 4
+    schedule = np.array([50.0, float("nan"), -2.0, 1.0], np.float32)
+    for kw in (dict(V=4096, dtype=W.F32), dict(V=66, dtype=W.F32), dict(V=8192, dtype=W.BF16, cfg=True, top_k=100)):
+        w = W.make("t", B=12, gamma=L, rho=0.95, schedule=schedule, seed=12, device=DEV, **kw)
+        rep, got, ref = check(w)
+        assert_ok(rep)
+        assert np.all(got["accept_len"] <= 1) and np.all(got["f"][:, 1:3] == 0.0)
+
+
 def test_identical_models_and_zero_omega():
     L = 3
     w = W.make("t", B=16, gamma=L, V=512, rho=1.0, schedule=np.array([1.0, 0.3, 0.0], np.float32),
@@ -794,7 +860,7 @@ def test_simple_form_and_determinism():
     for _ in range(3):      # same inputs, same outputs
         again = run_gpu(w, want_dbg=False)
         assert np.array_equal(again["tokens"], got["tokens"])
-    # a second, larger problem grows the internal workspace
+    # a second, larger problem (the simple form keeps no state between calls)
     w2 = W.make("t", B=40, gamma=8, V=16384, rho=0.9, schedule=sched(8), seed=9, device=DEV)
     out_t2 = torch.empty(40, 9, dtype=torch.int32, device=DEV)
     out_l2 = torch.empty(40, dtype=torch.int32, device=DEV)
@@ -803,6 +869,12 @@ def test_simple_form_and_determinism():
     torch.cuda.synchronize()
     got2 = run_gpu(w2, want_dbg=False)
     assert np.array_equal(out_t2.cpu().numpy(), got2["tokens"])
+    # rows the single-launch path cannot take need a workspace, which this form does not have
+    w3 = W.make("t", B=3, gamma=2, V=66, rho=0.9, schedule=sched(2), seed=10, device=DEV)
+    with pytest.raises(csd.CsdError) as err:
+        csd.csd_verify(w3.target_logits, w3.draft_logits, w3.draft_tokens, w3.uniforms, w3.relax_schedule,
+                       torch.empty(3, 3, dtype=torch.int32, device=DEV), torch.empty(3, dtype=torch.int32, device=DEV))
+    assert err.value.code == -7
 
 
 def test_host_buffer_form():

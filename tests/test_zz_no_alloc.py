@@ -5,8 +5,9 @@ that must never hit cudaMalloc's implicit synchronisation, uses csd_verify_stati
 is a fixed array inside the library.  The check here: called through the C ABI twice in a row
 (a larger problem, then a smaller one, so the second call runs over whatever the first left in
 the shared scratch), it must give exactly the accepted lengths and tokens of csd_verify, the
-allocating entry point.  These are integer outputs, so the comparison is exact.  The file name
-makes pytest collect it last.
+simple entry point that takes the same arguments, and of the fp64 oracle on the same inputs (up
+to decisions the oracle flags as within 1e-6 of a threshold).  These are integer outputs, so the
+comparison is exact.  The file name makes pytest collect it last.
 """
 import numpy as np
 import pytest
@@ -19,6 +20,8 @@ if not torch.cuda.is_available():
 
 import paper_2601_09212_b200 as csd
 from paper_2601_09212_b200 import workloads as W
+from gpu_util import run_oracle
+from oracle.compare import compare
 
 DEV = "cuda"
 
@@ -46,6 +49,9 @@ def test_static_scratch_matches_allocating_entry_point_twice_in_a_row():
         assert np.array_equal(tok_s, tok_a)
         assert tau_s.min() >= 0 and tau_s.max() <= w.gamma
         assert (tok_s[np.arange(w.B), tau_s] >= 0).sum() > 0 or (tau_s == w.gamma).all()
+        h, ref = run_oracle(w, want_G=True)
+        rep = compare(ref, tok_s, tau_s, h["draft_tokens"], h["uniforms"])
+        assert rep.ok and rep.tau_mismatch_near + rep.token_mismatch_near <= 1, rep.summary()
 
 
 def test_static_scratch_refuses_what_does_not_fit():
