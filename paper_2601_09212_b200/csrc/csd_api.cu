@@ -79,11 +79,13 @@ double normal_upper_quantile(double tail) {
   return 0.5 * (lo + hi);
 }
 
-// Launches one of the two single-launch kernels (KERNEL: 0 plain, 1 top-k) with its shared-memory
-// size, optionally with programmatic stream serialisation and as clusters of ctas_per_seq blocks.
+// Launches one of the single-launch kernels (KERNEL: 0 plain, 1 top-k on rows that are a whole
+// number of stages, 2 top-k on any row length) with its shared-memory size, optionally with
+// programmatic stream serialisation and as clusters of ctas_per_seq blocks.
 template <typename T, bool CFG, int KERNEL>
 cudaError_t launch_fused(const FusedArgs& a, int grid, bool overlap, cudaStream_t stream) {
-  auto kern = KERNEL ? verify_topk_kernel<T, CFG> : verify_plain_kernel<T, CFG>;
+  auto kern = KERNEL == 0 ? verify_plain_kernel<T, CFG>
+                          : (KERNEL == 1 ? verify_topk_kernel<T, CFG, false> : verify_topk_kernel<T, CFG, true>);
   constexpr size_t kSmem = KERNEL ? sizeof(TopkSmem) : sizeof(PlainSmem);
   constexpr int kThreads = KERNEL ? kTopkThreads : kPlainThreads;
   // the attribute belongs to (function, device): set it once per device (setting it twice is harmless)
@@ -122,7 +124,10 @@ cudaError_t launch_fused(const FusedArgs& a, int grid, bool overlap, cudaStream_
 
 template <typename T, bool CFG>
 cudaError_t launch_fused_t(const FusedArgs& a, bool topk, int grid, bool overlap, cudaStream_t stream) {
-  return topk ? launch_fused<T, CFG, 1>(a, grid, overlap, stream) : launch_fused<T, CFG, 0>(a, grid, overlap, stream);
+  if (!topk) return launch_fused<T, CFG, 0>(a, grid, overlap, stream);
+  constexpr int kStageElems = kTkStageBytes / ((int)sizeof(T) * (CFG ? 2 : 1));
+  return a.fin.V % kStageElems == 0 ? launch_fused<T, CFG, 1>(a, grid, overlap, stream)
+                                    : launch_fused<T, CFG, 2>(a, grid, overlap, stream);
 }
 
 template <typename T, bool CFG, int U, bool TOPK>
@@ -295,6 +300,7 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
     ua.top_k = p.top_k;
     ua.lo_sigmas = nanf("");
     ua.lo_delta = 0.0f;
+    ua.hi_delta = nanf("");
     ua.error_flag = no_workspace ? nullptr : reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
     ua.wait_limit = g_wait_limit;
     ua.drop_first_copy = g_drop_first_copy;
@@ -322,6 +328,13 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
       if (tail < 0.45 && tail * v < 0.8 * kListCap) {
         ua.lo_sigmas = (float)normal_upper_quantile(tail);
         ua.lo_delta = ua.lo_sigmas - (float)normal_upper_quantile(k / v);
+        // a level with, almost surely, fewer than k values above it: the mirror image of the guess.
+        // The short cut it serves keeps lo as the row's threshold, which the diagnostic outputs that
+        // evaluate every token (the distribution drawn from, the monitors) would show in their last
+        // digits: with them requested every row gets its exact threshold.
+        const double tail_hi = 0.75 * k / v - 4.0 * sqrt(k) / v - 16.0 / v;
+        if (tail_hi * v >= 8.0 && !p.dbg_G && !p.diag_accept_mass && !p.diag_bound_term)
+          ua.hi_delta = (float)normal_upper_quantile(tail_hi) - ua.lo_sigmas;
       }
     } else {
       // warp-wide items: parts of rows, sized so that every warp of the grid gets several

@@ -154,6 +154,8 @@ struct FusedArgs {
   int top_k;
   float lo_sigmas;      // top-k guess: lo = mean + lo_sigmas * deviation (NaN: always select exactly)
   float lo_delta;       // how many deviations below a row's exact threshold the next guess should sit (< 0)
+  float hi_delta;       // a level this many deviations above lo has, almost surely, fewer than k values above it
+                        // (NaN: never take the short cut that needs it)
   int* error_flag;      // set when a bounded wait gave up; null: nobody asked for the status
   long long wait_limit; // cycles a wait on a copy may take (kWaitCycles unless a test shortens it)
   int drop_first_copy;  // test aid: the first copy of block 0 is announced to its barrier but never issued,
@@ -229,8 +231,22 @@ constexpr int kBlockRows = 264;   // local rows a block may own (the host keeps 
 struct RowStats {
   float2 ms[kBlockRows];     // (m, s) of the whole row
   float thr[kBlockRows];     // top-k threshold (-inf without top-k)
-  float tokz[kBlockRows];    // logit of the row's drafted token (undefined if the token is out of range)
+  float tokz[kBlockRows];    // logit of the row's drafted token (undefined for a bonus row or a token out of range);
+                             // -inf if the top-k filter is known to drop it
 };
+
+// The logit of every local row's drafted token, by scalar loads straight from global memory (mixed like
+// the rows), when the kernel starts: the loads are long complete when the row's statistics are.
+template <typename T, bool CFG, int NT>
+__device__ __forceinline__ void load_token_logits(const FinishArgs& f, const BlockShare& sh, const int tid, RowStats& rs) {
+  for (int r = tid; r < sh.n_rows && r < kBlockRows; r += NT) {
+    int b, which, i;
+    local_row(sh, r, f.gamma, b, which, i);
+    if (i >= f.gamma) continue;   // the bonus row has no drafted token
+    const int tok = f.tokens[(int64_t)b * f.gamma + i];
+    if (tok >= 0 && tok < f.V) rs.tokz[r] = row_at<T, CFG>(f, b, which, i).load_one(tok);
+  }
+}
 
 // ---- the block's finish on its own positions ----------------------------------------------
 struct FinishStage {
@@ -781,6 +797,7 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
   // the block's items (parts of its local rows, see block_share), split evenly over its warps
   const BlockShare sh = block_share(a);
   stage_inputs(a, sh, 0, tid, sm.fst);
+  load_token_logits<T, CFG, kPlainThreads>(f, sh, tid, sm.rs);
   const int n_block = sh.n_rows * parts;
   const int item_begin = (int)((long long)n_block * warp / kPlainWarps);
   const int item_end = (int)((long long)n_block * (warp + 1) / kPlainWarps);
@@ -826,13 +843,6 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
     for (int s = 0; s < kWStages; ++s) producer_issue();
   }
 
-  // drafted token of a row (-1 for the bonus row), loaded a row ahead of its use
-  auto token_of_row = [&](int row_id) -> int {
-    int b, which, i;
-    local_row(sh, row_id, f.gamma, b, which, i);
-    return i < f.gamma ? __ldg(f.tokens + (int64_t)b * f.gamma + i) : -1;
-  };
-
   // ================================= phase 1 ===========================================
   int n_my = 0;
   {
@@ -840,21 +850,11 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
     uint32_t c_par = 0;   // its parity
     int waited = 0;       // chunks whose copies this lane has seen complete
     bool ok = true;       // false once a wait has run out: from then on nothing is waited for or issued
-    int cur_row = -1, tok_cur = -1, tok_next = -1;
-    const int last_row = item_end > item_begin ? (item_end - 1) / parts : -1;
-    int row_id = item_begin / parts, part = item_begin - row_id * parts;   // kept incrementally
-    if (item_begin < item_end) tok_next = token_of_row(row_id);
+    int part = item_begin % parts;   // kept incrementally
     for (int item = item_begin; item < item_end; ++item, ++n_my, ++part) {
-      if (part == parts) { part = 0; ++row_id; }
+      if (part == parts) part = 0;
       const int x_begin = part * part_elems;
       const int x_end = min(V, x_begin + part_elems);
-      if (row_id != cur_row) {
-        cur_row = row_id;
-        tok_cur = tok_next;
-        if (row_id < last_row) tok_next = token_of_row(row_id + 1);
-      }
-      float tokz = 0.0f;
-      bool has_tok = false;
       // Running statistics of the item, relative to a maximum that is the same in every lane of
       // the warp: Mw = largest value met so far by any lane, s = this lane's sum of
       // exp(z - Mw) over its values below Mw, cnt = this lane's number of values equal to Mw.
@@ -948,13 +948,6 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
             s_run += (acc4[0] + acc4[1]) + (acc4[2] + acc4[3]);
           }
         }
-        const int tl = tok_cur - x0;
-        if (tl >= 0 && tl < n) {   // the drafted token's logit passes by: keep it
-          float zc = load_scalar_smem<T>(stage + tl * (int)sizeof(T));
-          if (CFG) zc = cfg_mix(zc, load_scalar_smem<T>(stage + kWStageBytes / 2 + tl * (int)sizeof(T)), f.cfg_scale);
-          tokz = zc;
-          has_tok = true;
-        }
         __syncwarp();
         if (lane == 0 && ok) {   // the stage is free again: refill it with the chunk kWStages ahead
           fence_before_bulk();
@@ -968,10 +961,7 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
         s_run += __shfl_xor_sync(0xffffffffu, s_run, off);
         cnt_run += __shfl_xor_sync(0xffffffffu, cnt_run, off);
       }
-      if (lane == 0 && item < kBlockStash) {
-        sm.stash[item] = make_float2(Mw, s_run * ex2f(-dlt) + (float)(cnt_run - 1));
-        if (has_tok && row_id < kBlockRows) sm.rs.tokz[row_id] = tokz;
-      }
+      if (lane == 0 && item < kBlockStash) sm.stash[item] = make_float2(Mw, s_run * ex2f(-dlt) + (float)(cnt_run - 1));
     }
     if (!ok) {
       sm.abort = 1;
@@ -1027,14 +1017,18 @@ struct TopkSmem {
   int wpos[kTopkWarps];            // per warp: next free slot of its list (may run past the capacity)
   float cand[kCandCap];             // values in the bin of the k-th largest
   int n_cand[2];                    // by row parity
-  float mom[kTopkWarps][4];        // per warp: sum, sum of squares, count of the sampled values
+  alignas(16) float mom[2][kTopkWarps];   // per warp: sum and sum of squares of its sampled values
   float wmax[kTopkWarps];
   // per warp, by row parity: sum of exp(z - max) over kept non-maximum values and number of kept values
   // equal to the maximum; the extra slot takes the values of the bin that holds the threshold
-  float part_acc[2][kTopkWarps + 1];
-  int part_cmax[2][kTopkWarps + 1];
-  float part_max[2];
-  float part_thr[2];
+  float part_acc[2][kTopkWarps];
+  int part_cmax[2][kTopkWarps];
+  // the short cut (see the kernel): per warp (m, s) of its whole list, its count of values above the
+  // upper level and of values above the drafted token's logit
+  float fw_m[kTopkWarps], fw_s[kTopkWarps];
+  int fw_cgt[kTopkWarps], fw_rk[kTopkWarps];
+  int short_on;                     // cleared once a row has failed the short cut's test: the block stops trying
+  int row_short;                    // this row was settled by the short cut
   int bc_i[4];
   int arrive[2];                    // warps that have finished the first / the second pass over their lists
   float row_mx;                     // set by the warp that picks the bin: the row maximum, and whether the
@@ -1149,13 +1143,62 @@ __device__ void exact_row_from_global(const Row<T, CFG>& row, int V, int k, Topk
   __syncthreads();
 }
 
-template <typename T, bool CFG>
+// One stage of a row as this thread sees it: its NVS 16-byte vectors of the (mixed) row, unpacked
+// to fp32.  `base` is the shared address of the stage plus 16 bytes per thread; vector v of the
+// thread sits 4096 bytes further per v, the unconditional array half a stage further.  n is the
+// number of valid elements in the stage (a multiple of the vector width); what lies beyond reads -inf.
+template <typename T, bool CFG, int NVS, bool RAGGED>
+__device__ __forceinline__ void load_stage(const uint32_t base, const int n, const int tid, const float scale,
+                                           float (&z)[NVS * Elem<T>::kVec]) {
+  constexpr int VEC = Elem<T>::kVec;
+  auto lds128 = [](uint32_t addr, uint32_t (&w)[4]) {
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]) : "r"(addr));
+  };
+  auto unpack = [](const uint32_t (&w)[4], float (&out)[VEC]) {
+    if (sizeof(T) == 4) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) out[k] = __uint_as_float(w[k]);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        out[2 * k] = __uint_as_float(w[k] << 16);
+        out[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+      }
+    }
+  };
+#pragma unroll
+  for (int v = 0; v < NVS; ++v) {
+    float zc[VEC];
+    if (!RAGGED || (v * kTopkThreads + tid) * VEC < n) {
+      uint32_t w[4];
+      lds128(base + v * (kTopkThreads * 16), w);
+      unpack(w, zc);
+      if (CFG) {
+        float zu[VEC];
+        lds128(base + kTkStageBytes / 2 + v * (kTopkThreads * 16), w);
+        unpack(w, zu);
+        cfg_mix_vec<VEC>(zc, zu, scale);
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) zc[e] = CSD_NEG_INF;
+    }
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) z[v * VEC + e] = zc[e];
+  }
+}
+
+// RAGGED: V is not a whole number of stages, so the last stage of a row is partly filled (the host
+// picks the instance; without it the streaming loop has no bounds tests at all).
+template <typename T, bool CFG, bool RAGGED>
 __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const FusedArgs a) {
   constexpr int VEC = Elem<T>::kVec;
   constexpr int ARR = CFG ? 2 : 1;
-  constexpr int EPS = kTkStageBytes / ((int)sizeof(T) * ARR);   // elements of a row per stage
-  constexpr int VPT = EPS / kTopkThreads;                      // values per thread per stage
+  constexpr int ES = (int)sizeof(T);
+  constexpr int EPS = kTkStageBytes / (ES * ARR);               // elements of a row per stage
+  constexpr int VPT = EPS / kTopkThreads;                       // values per thread per stage
   constexpr int NVS = VPT / VEC;                                // 16-byte vectors per thread per stage
+  static_assert(kTkStages == 2, "stage and parity of a chunk are taken from the low bits of its index");
   extern __shared__ __align__(128) unsigned char fused_smem_raw[];
   TopkSmem& sm = *reinterpret_cast<TopkSmem*>(fused_smem_raw);
 
@@ -1178,6 +1221,8 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
     sm.c_kind[0] = a.lo_sigmas;
     sm.c_kind[1] = a.lo_sigmas;
     sm.adapt_on = 0;
+    sm.short_on = (a.hi_delta == a.hi_delta && a.fin.dbg_G == nullptr) ? 1 : 0;
+    sm.row_short = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < (kBlockRows + 31) / 32) sm.need_exact[tid] = 0u;
@@ -1187,225 +1232,224 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   // this block's local rows (see block_share)
   const BlockShare sh = block_share(a);
   stage_inputs(a, sh, 0, tid, sm.fst);
-  const int row_begin = 0, row_end = sh.n_rows;
+  load_token_logits<T, CFG, kTopkThreads>(f, sh, tid, sm.rs);
+  const int n_rows = sh.n_rows;
+  const int n_chunks = n_rows * cpr;
 
   auto row_of = [&](int row_id) -> Row<T, CFG> {
     int b, which, i;
     local_row(sh, row_id, f.gamma, b, which, i);
     return row_at<T, CFG>(f, b, which, i);
   };
-  auto token_of_row = [&](int row_id) -> int {
-    int b, which, i;
-    local_row(sh, row_id, f.gamma, b, which, i);
-    return i < f.gamma ? __ldg(f.tokens + (int64_t)b * f.gamma + i) : -1;
-  };
-  // Issues the copies of chunk c of this block's j-th row (if there is one) into stage q % kTkStages.
-  auto issue_chunk = [&](int q, int j, int c) {
-    const int row_id = row_begin + j;
-    if (row_id >= row_end) return;
-    const Row<T, CFG> row = row_of(row_id);
-    const int s = q % kTkStages;
+  // Issues the copies of chunk q of this block (chunk q % cpr of its local row q / cpr), if there is
+  // one, into stage q % 2.  One thread at a time per stage.
+  auto issue_chunk = [&](int q) {
+    if (q >= n_chunks) return;
+    const int j = q / cpr, c = q - j * cpr;
+    const Row<T, CFG> row = row_of(j);
+    const int s = q & 1;
     const int x0 = c * EPS;
-    const uint32_t bytes = (uint32_t)(min(EPS, V - x0) * (int)sizeof(T));
+    const uint32_t bytes = (uint32_t)(min(EPS, V - x0) * ES);
     mbar_expect_tx(&sm.full[s], bytes * ARR);
-    sm.issued_q = q + 1;
+    atomicMax(&sm.issued_q, q + 1);
     if (q == 0 && a.drop_first_copy != 0 && blockIdx.x == 0) return;   // (test aid, see FusedArgs)
     bulk_load(&sm.ring[s][0], row.cond + x0, bytes, &sm.full[s]);
     if (CFG) bulk_load(&sm.ring[s][kTkStageBytes / 2], row.uncond + x0, bytes, &sm.full[s]);
   };
   if (tid == 0) {
-    for (int q = 0; q < kTkStages; ++q) issue_chunk(q, q / cpr, q % cpr);
+    issue_chunk(0);
+    issue_chunk(1);
   }
-  // (row, chunk) of the chunk kTkStages ahead of the one being read, kept incrementally
-  int ahead_j = kTkStages / cpr, ahead_c = kTkStages % cpr;
-
-  // Merges the per-warp partials of a finished row (parity par) into its stash entry.
-  auto stash_row = [&](int idx, int par) {
-    float tot = 0.0f;
-    int ctot = 0;
-#pragma unroll
-    for (int w = 0; w <= kTopkWarps; ++w) { tot += sm.part_acc[par][w]; ctot += sm.part_cmax[par][w]; }
-    if (idx < kBlockRows) {
-      sm.rs.ms[idx] = make_float2(sm.part_max[par], tot + (float)(ctot - 1));
-      sm.rs.thr[idx] = sm.part_thr[par];
-    }
-  };
 
   // ================================= phase 1 ===========================================
-  int n_my = 0;
   {
-    int q = 0;
+    int q = 0;        // chunks consumed so far
     int waited = 0;   // chunks whose copies this thread has seen complete
     bool ok = true;   // false once a wait has run out: from then on this thread waits for nothing
-    int tok_next = row_begin < row_end ? token_of_row(row_begin) : -1;
-    for (int row_id = row_begin; row_id < row_end; ++row_id, ++n_my) {
-      const int par = n_my & 1;
-      const int tok_cur = tok_next;
-      if (row_id + 1 < row_end) tok_next = token_of_row(row_id + 1);
-      float lo = 0.0f, scale = 0.0f;
-      float mx = CSD_NEG_INF;
+    const uint32_t ring_mine = smem_addr(&sm.ring[0][0]) + (uint32_t)tid * 16u;
+    const uint32_t list_mine = smem_addr(&sm.list[warp][0]);
+    const uint32_t hist_addr = smem_addr(&sm.hist[0]);
+    for (int r = 0; r < n_rows; ++r) {
+      const int par = r & 1;
+      float lo = 0.0f, scale = 0.0f, dev = 0.0f;
       if (lane == 0) sm.wpos[warp] = 0;
-      for (int d = tid; d < kLinBins; d += kTopkThreads) sm.hist[d] = 0;
-      for (int c = 0; c < cpr; ++c) {
-        const int s = q % kTkStages;
-        const uint32_t par_s = (uint32_t)(q / kTkStages) & 1u;
-        ++q;
+      reinterpret_cast<int2*>(sm.hist)[tid] = make_int2(0, 0);
+      static_assert(kLinBins == 2 * kTopkThreads, "every thread clears two bins");
+      for (int c = 0; c < cpr; ++c, ++q) {
+        const int s = q & 1;
         if (ok) {
-          if (mbar_wait(&sm.full[s], par_s, a.wait_limit)) ++waited;
+          if (mbar_wait(&sm.full[s], (uint32_t)(q >> 1) & 1u, a.wait_limit)) ++waited;
           else { ok = false; *(volatile int*)&sm.abort = 1; }
         }
-        const int x0 = c * EPS;
-        const int n = min(EPS, V - x0);
+        const int n = RAGGED ? min(EPS, V - c * EPS) : EPS;
         float z[VPT];
-        if (n == EPS) {   // the common case: a full stage, no bounds to check
-#pragma unroll
-          for (int v = 0; v < NVS; ++v) {
-            const int xo = (v * kTopkThreads + tid) * VEC;
-            float zc[VEC];
-            unpack_vec<T>(&sm.ring[s][xo * (int)sizeof(T)], zc);
-            if (CFG) {
-              float zu[VEC];
-              unpack_vec<T>(&sm.ring[s][kTkStageBytes / 2 + xo * (int)sizeof(T)], zu);
-              cfg_mix_vec<VEC>(zc, zu, f.cfg_scale);
-            }
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) z[v * VEC + e] = zc[e];
-          }
-        } else {
-#pragma unroll
-          for (int v = 0; v < NVS; ++v) {
-            const int xo = (v * kTopkThreads + tid) * VEC;
-            float zc[VEC];
-            if (xo < n) {
-              unpack_vec<T>(&sm.ring[s][xo * (int)sizeof(T)], zc);
-              if (CFG) {
-                float zu[VEC];
-                unpack_vec<T>(&sm.ring[s][kTkStageBytes / 2 + xo * (int)sizeof(T)], zu);
-                cfg_mix_vec<VEC>(zc, zu, f.cfg_scale);
-              }
-            } else {
-#pragma unroll
-              for (int e = 0; e < VEC; ++e) zc[e] = CSD_NEG_INF;
-            }
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) z[v * VEC + e] = zc[e];
-          }
-        }
-        const int tl = tok_cur - x0;
-        if (tid == 0 && tl >= 0 && tl < n) {   // the drafted token's logit passes by: keep it
-          float zc = load_scalar_smem<T>(&sm.ring[s][tl * (int)sizeof(T)]);
-          if (CFG) zc = cfg_mix(zc, load_scalar_smem<T>(&sm.ring[s][kTkStageBytes / 2 + tl * (int)sizeof(T)]), f.cfg_scale);
-          if (n_my < kBlockRows) sm.rs.tokz[n_my] = zc;
-        }
+        load_stage<T, CFG, NVS, RAGGED>(ring_mine + (uint32_t)s * kTkStageBytes, n, tid, f.cfg_scale, z);
         __syncwarp();
         if (lane == 0) {   // this warp is done with the stage; the last one to say so refills it
           __threadfence_block();
-          if (atomicAdd(&sm.readers_done[s], 1) == kTopkWarps - 1) {
+          if (atom_add_shared(&sm.readers_done[s], 1) == kTopkWarps - 1) {
             sm.readers_done[s] = 0;
             __threadfence_block();
             // (a thread that gave up set the flag before it counted itself here: once any wait has
             // run out, nothing more is issued)
             if (*(volatile int*)&sm.abort == 0) {
               fence_before_bulk();
-              issue_chunk(q - 1 + kTkStages, ahead_j, ahead_c);
+              issue_chunk(q + kTkStages);
             }
           }
         }
-        if (++ahead_c == cpr) { ahead_c = 0; ++ahead_j; }
         if (c == 0) {
           // the first stage is the sample for the threshold guess
-          float sum1 = 0.0f, sum2 = 0.0f, cnt = 0.0f;
+          float sum1 = 0.0f, sum2 = 0.0f;
 #pragma unroll
           for (int v = 0; v < NVS; ++v) {
-            if ((v * kTopkThreads + tid) * VEC < n) {
+            if (!RAGGED || (v * kTopkThreads + tid) * VEC < n) {
 #pragma unroll
               for (int e = 0; e < VEC; ++e) { sum1 += z[v * VEC + e]; sum2 = fmaf(z[v * VEC + e], z[v * VEC + e], sum2); }
-              cnt += (float)VEC;
             }
           }
 #pragma unroll
           for (int off = 16; off > 0; off >>= 1) {
             sum1 += __shfl_xor_sync(0xffffffffu, sum1, off);
             sum2 += __shfl_xor_sync(0xffffffffu, sum2, off);
-            cnt += __shfl_xor_sync(0xffffffffu, cnt, off);
           }
-          if (lane == 0) { sm.mom[warp][0] = sum1; sm.mom[warp][1] = sum2; sm.mom[warp][2] = cnt; }
+          if (lane == 0) { sm.mom[0][warp] = sum1; sm.mom[1][warp] = sum2; }
           __syncthreads();   // ---- S0: moments, cleared histogram and list cursors; the previous row is complete
-          if (tid == 0) {
-            sm.n_cand[par ^ 1] = 0;   // for the next row; nobody reads the previous row's count any more
-            if (n_my > 0) stash_row(n_my - 1, par ^ 1);
+          if (tid == 0) sm.n_cand[par ^ 1] = 0;   // for the next row; nobody reads the previous row's count any more
+          float s1 = 0.0f, s2 = 0.0f;
+          {
+            const float4* m4 = reinterpret_cast<const float4*>(&sm.mom[0][0]);
+            static_assert(kTopkWarps == 8, "the moments of eight warps are four 16-byte loads");
+            const float4 a0 = m4[0], a1 = m4[1], b0 = m4[2], b1 = m4[3];
+            s1 = ((a0.x + a0.y) + (a0.z + a0.w)) + ((a1.x + a1.y) + (a1.z + a1.w));
+            s2 = ((b0.x + b0.y) + (b0.z + b0.w)) + ((b1.x + b1.y) + (b1.z + b1.w));
           }
-          float s1 = 0.0f, s2 = 0.0f, nn = 0.0f;
-#pragma unroll
-          for (int w = 0; w < kTopkWarps; ++w) { s1 += sm.mom[w][0]; s2 += sm.mom[w][1]; nn += sm.mom[w][2]; }
-          const float mean = s1 / nn;
-          const float dev = sqrtf(fmaxf(s2 / nn - mean * mean, 0.0f));
+          // (a guess: approximate reciprocal and root are enough, every thread gets the same bits)
+          const float inv_n = RAGGED ? rcp_approx((float)n) : 1.0f / (float)EPS;
+          const float mean = s1 * inv_n;
+          dev = sqrt_approx(fmaxf(s2 * inv_n - mean * mean, 0.0f));
           lo = mean + sm.c_kind[par] * dev;
-          scale = (float)kLinBins / (kLinRangeSigmas * dev);
+          scale = ((float)kLinBins / kLinRangeSigmas) * rcp_approx(dev);
           if (tid == 0) { sm.row_mean[par] = mean; sm.row_dev[par] = dev; }
         }
         // ---- gather this stage's values >= lo into the warp's list -------------------------
         // (the test is "not below lo", so that a NaN lands in the list and marks the row through the
-        // maximum).  Two predicated passes, written out so that they stay free of branches: count,
-        // reserve the slots with one atomic, store.
-        // Four independent chains (every fourth value each), so that neither the counts nor the
-        // addresses form one long dependent sequence.
-        constexpr int NCH = (VPT % 4 == 0) ? 4 : 1;
-        uint32_t cn[NCH];
+        // maximum).  Two predicated passes, free of branches: count, reserve the slots with one
+        // atomic, store.  Four independent chains (every fourth value each), so that neither the
+        // counts nor the addresses form one long dependent sequence.
+        // one bit per value, then the slots are reserved with one atomic and the flagged values stored
+        uint32_t mask = 0;
 #pragma unroll
-        for (int g = 0; g < NCH; ++g) cn[g] = 0;
-        // (count: two comparisons that give all-ones or zero, subtracted by one three-input add)
+        for (int e = 0; e < VPT; ++e) mask |= (z[e] < lo) ? 0u : (1u << e);
+        const uint32_t cnt = (uint32_t)__popc(mask);
+        const uint32_t pos = (uint32_t)atom_add_shared(&sm.wpos[warp], (int)cnt);
+        if (pos + cnt <= (uint32_t)kWarpList) {
+          uint32_t addr = list_mine + 4u * pos;
 #pragma unroll
-        for (int e = 0; e + 2 * NCH <= VPT; e += 2 * NCH) {
-#pragma unroll
-          for (int g = 0; g < NCH; ++g)
-            asm("{\n\t.reg .u32 a, b;\n\tset.geu.u32.f32 a, %1, %3;\n\tset.geu.u32.f32 b, %2, %3;\n\t"
-                "sub.u32 %0, %0, a;\n\tsub.u32 %0, %0, b;\n\t}"
-                : "+r"(cn[g])
-                : "f"(z[e + g]), "f"(z[e + NCH + g]), "f"(lo));
-        }
-        static_assert(VPT % (2 * NCH) == 0, "the count takes the values in pairs per chain");
-        uint32_t cnt = cn[0];
-#pragma unroll
-        for (int g = 1; g < NCH; ++g) cnt += cn[g];
-        if (cnt > 0) {
-          const uint32_t pos = (uint32_t)atomicAdd(&sm.wpos[warp], (int)cnt);
-          if (pos + cnt <= (uint32_t)kWarpList) {
-            uint32_t addr[NCH];
-            addr[0] = smem_addr(&sm.list[warp][pos]);
-#pragma unroll
-            for (int g = 1; g < NCH; ++g) addr[g] = addr[g - 1] + 4u * cn[g - 1];
-#pragma unroll
-            for (int e = 0; e < VPT; ++e)
-              asm volatile(
-                  "{\n\t.reg .pred p;\n\tsetp.geu.f32 p, %1, %2;\n\t@p st.shared.f32 [%0], %1;\n\t@p add.u32 %0, %0, 4;\n\t}"
-                  : "+r"(addr[e % NCH])
-                  : "f"(z[e]), "f"(lo)
-                  : "memory");
+          for (int e = 0; e < VPT; ++e) {
+            if (mask & (1u << e)) {
+              asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(z[e]) : "memory");
+              addr += 4u;
+            }
           }
         }
       }
       // ---- first pass over this warp's list: maximum and histogram -----------------------------
-      // (the row maximum is among the gathered values whenever the lists can be used)
+      // (the row maximum is among the gathered values whenever the lists can be used).  The list is
+      // padded with -inf to a whole number of 32 slots, so that the passes run without bounds tests.
       __syncwarp();
       const int wc = sm.wpos[warp];
-      // Both passes over the list are unrolled over its slots (so that the loads and the bin
-      // arithmetic of all slots overlap), in two versions: three quarters of the capacity, which is
-      // what a list normally holds, and all of it.
-      auto first_pass = [&](auto nslots) {
+      int wcp = 0;   // padded length; 0 if the list overflowed (the row is then selected exactly)
+      if (wc <= kWarpList) {
+        wcp = (wc + 31) & ~31;
+        if (wc + lane < wcp) sm.list[warp][wc + lane] = CSD_NEG_INF;
+      }
+      __syncwarp();
+      // ---- the short cut: no threshold at all --------------------------------------------------
+      // If a level `hi` a little above lo has fewer than k values above it, the k-th largest value lies
+      // in [lo, hi], and the values the filter drops among those gathered all lie there too.  Where
+      // their total weight -- at most (their number) * exp(hi - max) -- is below 2^-26 of the row's
+      // normaliser, dropping them or not changes nothing that fp32 can see: the row's (m, s) is that
+      // of ALL gathered values, lo itself serves as the threshold from here on (for the draw's filter
+      // and the diagnostics: what it lets through beyond the exact filter has weight below 1e-7 of an
+      // ulp), and whether the drafted token survives the exact filter is decided by its exact rank
+      // (fewer than k gathered values above its logit).  One pass over the lists and one barrier
+      // instead of a histogram, a selection and two barriers; rows that fail the test (flat rows,
+      // where the values near the threshold carry weight) take the full selection below, on the same
+      // lists, and the block stops trying.
+      if (sm.short_on) {
+        float mw = CSD_NEG_INF;
+        for (int i = lane; i < wcp; i += 32) mw = max_nan(mw, sm.list[warp][i]);
 #pragma unroll
-        for (int u = 0; u < decltype(nslots)::value; ++u) {
-          const int i = lane + 32 * u;
-          if (i < wc) {
-            const float v = sm.list[warp][i];
-            mx = max_nan(mx, v);
-            atomicAdd(&sm.hist[lin_bin(v, lo, scale)], 1);
+        for (int off = 16; off > 0; off >>= 1) mw = max_nan(mw, __shfl_xor_sync(0xffffffffu, mw, off));
+        const float hi = lo + a.hi_delta * dev;
+        const float ztok = r < kBlockRows ? sm.rs.tokz[r] : 0.0f;
+        float acc = 0.0f;
+        int cmax = 0, cgt = 0, rk = 0;
+        for (int i = lane; i < wcp; i += 32) {
+          const float v = sm.list[warp][i];
+          const float ev = ex2f((v - mw) * kLog2e);   // (0 for the padding)
+          acc += (v != mw) ? ev : 0.0f;
+          cmax += (v == mw) ? 1 : 0;
+          cgt += (v > hi) ? 1 : 0;
+          rk += (v > ztok) ? 1 : 0;
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        cmax = __reduce_add_sync(0xffffffffu, cmax);
+        cgt = __reduce_add_sync(0xffffffffu, cgt);
+        rk = __reduce_add_sync(0xffffffffu, rk);
+        int last_s = 0;
+        if (lane == 0) {
+          sm.fw_m[warp] = mw;
+          sm.fw_s[warp] = wcp > 0 ? acc + (float)(cmax - 1) : -1.0f;   // (an empty list: the identity)
+          sm.fw_cgt[warp] = cgt;
+          sm.fw_rk[warp] = rk;
+          __threadfence_block();
+          last_s = atom_add_shared(&sm.arrive[0], 1) == kTopkWarps - 1 ? 1 : 0;
+        }
+        last_s = __shfl_sync(0xffffffffu, last_s, 0);
+        if (last_s) {
+          if (lane == 0) sm.arrive[0] = 0;
+          __threadfence_block();
+          const bool mine = lane < kTopkWarps;
+          float m = mine ? sm.fw_m[lane] : CSD_NEG_INF, sv = mine ? sm.fw_s[lane] : -1.0f;
+          int n_lo = mine ? sm.wpos[lane] : 0;
+          const bool over = __any_sync(0xffffffffu, n_lo > kWarpList);
+          const bool nan_m = __any_sync(0xffffffffu, m != m);
+          n_lo = __reduce_add_sync(0xffffffffu, n_lo);
+          const int cg = __reduce_add_sync(0xffffffffu, mine ? sm.fw_cgt[lane] : 0);
+          const int rank = __reduce_add_sync(0xffffffffu, mine ? sm.fw_rk[lane] : 0);
+#pragma unroll
+          for (int off = 4; off > 0; off >>= 1) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, m, off), s2 = __shfl_xor_sync(0xffffffffu, sv, off);
+            stat_merge(m, sv, m2, s2);
+          }
+          if (lane == 0) {
+            const float dropped = (float)(n_lo - cg) * ex2f((hi - m) * kLog2e);   // bound on what the filter removes
+            const bool ok = !over && !nan_m && n_lo >= k_top && cg < k_top && m > lo && m < CSD_POS_INF &&
+                            sv >= 0.0f && sv < CSD_POS_INF && dropped <= 1.4901161e-8f;
+            if (ok && r < kBlockRows) {
+              sm.rs.ms[r] = make_float2(m, sv);
+              sm.rs.thr[r] = lo;
+              if (!(rank < k_top)) sm.rs.tokz[r] = CSD_NEG_INF;   // the exact filter drops the drafted token
+            }
+            if (!ok) sm.short_on = 0;
+            sm.row_short = ok ? 1 : 0;
           }
         }
-      };
-      constexpr int kSlotsAll = kWarpList / 32, kSlotsUsual = (3 * kSlotsAll) / 4;
-      if (wc <= 32 * kSlotsUsual) first_pass(std::integral_constant<int, kSlotsUsual>());
-      else if (wc <= kWarpList) first_pass(std::integral_constant<int, kSlotsAll>());
+        __syncthreads();   // ---- D: settled, or on to the full selection
+        if (sm.row_short) continue;
+      }
+      float mx = CSD_NEG_INF;
+      for (int i = lane; i < wcp; i += 32) {
+        const float v = sm.list[warp][i];
+        mx = max_nan(mx, v);
+        const int bv = lin_bin(v, lo, scale);   // (the padding gets a negative bin)
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ge.s32 p, %1, 0;\n\t@p red.shared.add.u32 [%0], 1;\n\t}"
+                     ::"r"(hist_addr + 4u * (uint32_t)bv), "r"(bv)
+                     : "memory");
+      }
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) mx = max_nan(mx, __shfl_xor_sync(0xffffffffu, mx, off));
       __syncwarp();
@@ -1413,7 +1457,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
       if (lane == 0) {
         sm.wmax[warp] = mx;
         __threadfence_block();
-        last = atomicAdd(&sm.arrive[0], 1) == kTopkWarps - 1 ? 1 : 0;
+        last = atom_add_shared(&sm.arrive[0], 1) == kTopkWarps - 1 ? 1 : 0;
       }
       last = __shfl_sync(0xffffffffu, last, 0);
       if (last) {
@@ -1445,7 +1489,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
           else if (!fast && n_lo > kListCap / 2) { sm.c_kind[par] += 0.35f; sm.adapt_on = 1; }
           sm.row_mx = m;
           sm.row_fast = fast ? 1 : 0;
-          if (!fast && n_my < kBlockRows) atomicOr(&sm.need_exact[n_my >> 5], 1u << (n_my & 31));
+          if (!fast && r < kBlockRows) atomicOr(&sm.need_exact[r >> 5], 1u << (r & 31));
         }
       }
       __syncthreads();   // ---- C: decision and bin known
@@ -1456,24 +1500,18 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         const int pick_bin = sm.bc_i[0];
         float acc = 0.0f;
         int cmax = 0;
-        auto second_pass = [&](auto nslots) {   // branch-free but for the rare bin member
-#pragma unroll
-          for (int u = 0; u < decltype(nslots)::value; ++u) {
-            const int i = lane + 32 * u;
-            const float v = i < wc ? sm.list[warp][i] : CSD_NEG_INF;   // -inf: below every bin
-            const int bv = i < wc ? lin_bin(v, lo, scale) : -1;
-            const float ev = ex2f((v - mx) * kLog2e);
-            const bool above = bv > pick_bin;
-            acc += (above && v != mx) ? ev : 0.0f;
-            cmax += (above && v == mx) ? 1 : 0;
-            if (bv == pick_bin) {
-              const int slot = atomicAdd(&sm.n_cand[par], 1);
-              if (slot < kCandCap) sm.cand[slot] = v;
-            }
+        for (int i = lane; i < wcp; i += 32) {
+          const float v = sm.list[warp][i];
+          const int bv = lin_bin(v, lo, scale);   // (-inf, the padding, is below every bin)
+          const float ev = ex2f((v - mx) * kLog2e);
+          const bool above = bv > pick_bin;
+          acc += (above && v != mx) ? ev : 0.0f;
+          cmax += (above && v == mx) ? 1 : 0;
+          if (bv == pick_bin) {
+            const int slot = atomicAdd(&sm.n_cand[par], 1);
+            if (slot < kCandCap) sm.cand[slot] = v;
           }
-        };
-        if (wc <= 32 * kSlotsUsual) second_pass(std::integral_constant<int, kSlotsUsual>());
-        else second_pass(std::integral_constant<int, kSlotsAll>());
+        }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) {
           acc += __shfl_xor_sync(0xffffffffu, acc, off);
@@ -1485,7 +1523,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
           sm.part_acc[par][warp] = acc;
           sm.part_cmax[par][warp] = cmax;
           __threadfence_block();
-          last = atomicAdd(&sm.arrive[1], 1) == kTopkWarps - 1 ? 1 : 0;
+          last = atom_add_shared(&sm.arrive[1], 1) == kTopkWarps - 1 ? 1 : 0;
         }
         last = __shfl_sync(0xffffffffu, last, 0);
         if (last) {
@@ -1521,10 +1559,15 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
               cmax2 += __shfl_xor_sync(0xffffffffu, cmax2, off);
             }
             if (lane == 0) {
-              sm.part_acc[par][kTopkWarps] = acc2;
-              sm.part_cmax[par][kTopkWarps] = cmax2;
-              sm.part_max[par] = mx;
-              sm.part_thr[par] = thr;
+              // every warp published its partials before it counted itself in: the row is complete
+              float tot = acc2;
+              int ctot = cmax2;
+#pragma unroll
+              for (int w = 0; w < kTopkWarps; ++w) { tot += sm.part_acc[par][w]; ctot += sm.part_cmax[par][w]; }
+              if (r < kBlockRows) {
+                sm.rs.ms[r] = make_float2(mx, tot + (float)(ctot - 1));
+                sm.rs.thr[r] = thr;
+              }
               // where the threshold really sat, in deviations from the mean: the next row of this kind
               // guesses a little below that (half-way from the current multiplier)
               // (only once the plain guess has missed in this block: data it fits is left alone)
@@ -1533,20 +1576,18 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
                 if (c_seen == c_seen && fabsf(c_seen) < 64.0f) sm.c_kind[par] = 0.5f * (sm.c_kind[par] + c_seen);
               }
             }
-          } else if (lane == 0 && n_my < kBlockRows) {   // crowded bin
-            atomicOr(&sm.need_exact[n_my >> 5], 1u << (n_my & 31));
+          } else if (lane == 0 && r < kBlockRows) {   // crowded bin
+            atomicOr(&sm.need_exact[r >> 5], 1u << (r & 31));
           }
         }
       }
     }
-    __syncthreads();
-    if (tid == 0 && n_my > 0) stash_row(n_my - 1, (n_my - 1) & 1);
     // ---- rows whose lists could not be used: exact select and statistics from global memory (rare) ----
     __syncthreads();
-    for (int r = 0; r < n_my && r < kBlockRows; ++r) {
+    for (int r = 0; r < n_rows && r < kBlockRows; ++r) {
       if (((sm.need_exact[r >> 5] >> (r & 31)) & 1u) == 0u) continue;   // the same decision in every thread
       float m_e = 0.0f, s_e = 0.0f, thr_e = 0.0f;
-      exact_row_from_global<T, CFG>(row_of(row_begin + r), V, k_top, sm, tid, m_e, s_e, thr_e);
+      exact_row_from_global<T, CFG>(row_of(r), V, k_top, sm, tid, m_e, s_e, thr_e);
       if (tid == 0) {
         sm.rs.ms[r] = make_float2(m_e, s_e);
         sm.rs.thr[r] = thr_e;
@@ -1557,7 +1598,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
       // Nothing was issued after the first failed wait was seen, so the copies that may still be in
       // flight are those of chunks [waited, issued_q): at most one per stage.  Wait for each, bounded.
       for (int c = waited; c < sm.issued_q; ++c)
-        (void)mbar_wait(&sm.full[c % kTkStages], (uint32_t)(c / kTkStages) & 1u, a.wait_limit);
+        (void)mbar_wait(&sm.full[c & 1], (uint32_t)(c >> 1) & 1u, a.wait_limit);
     }
   }
 

@@ -44,6 +44,24 @@ __device__ __forceinline__ void pdl_launch_dependents() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Shared-memory atomic add issued as written (the compiler's warp-aggregated form of atomicAdd costs
+// about ten instructions; these are called by one lane per warp)
+__device__ __forceinline__ int atom_add_shared(int* p, int v) {
+  int old;
+  asm volatile("atom.shared.add.u32 %0, [%1], %2;" : "=r"(old) : "r"((uint32_t)__cvta_generic_to_shared(p)), "r"(v) : "memory");
+  return old;
+}
+__device__ __forceinline__ float sqrt_approx(float x) {
+  float y;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float rcp_approx(float x) {
+  float y;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // ---- (m, s) algebra ---------------------------------------------------------
 // identity: m = -inf, s = -1 (so that 1 + s = 0)
 __device__ __forceinline__ void stat_merge(float& m, float& s, float m2, float s2) {
