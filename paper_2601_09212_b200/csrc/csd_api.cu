@@ -312,7 +312,8 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
     // ctas_per_seq blocks of one cluster (each with both rows of its positions; 2, 4 or 8 blocks)
     // until the GPU is full.
     const long long merge_above = 8LL * sms;   // beyond this many sequences a block takes several
-    const long long split_below = p.back_to_back ? 16 : 2LL * sms;
+    // (measured: the top-k kernel, with its longer per-row work, gains from the finer split)
+    const long long split_below = p.back_to_back ? 16 : (topk ? 4LL : 2LL) * sms;
     long long c = 1, spc = 1;
     if (p.B > merge_above) spc = (p.B + merge_above - 1) / merge_above;
     else if (p.B < split_below) {
