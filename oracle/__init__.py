@@ -57,6 +57,19 @@ class _Params(C.Structure):
     ]
 
 
+class _TreeParams(C.Structure):
+    _fields_ = [
+        ("target_logits", C.c_void_p), ("draft_logits", C.c_void_p),
+        ("target_uncond", C.c_void_p), ("draft_uncond", C.c_void_p),
+        ("dtype", C.c_int32), ("cfg_scale", C.c_float), ("top_k", C.c_int32),
+        ("B", C.c_int32), ("N", C.c_int32), ("V", C.c_int32), ("D", C.c_int32),
+        ("parent", C.c_void_p), ("draft_tokens", C.c_void_p), ("uniforms", C.c_void_p),
+        ("relax_schedule", C.c_void_p),
+        ("out_tokens", C.c_void_p), ("out_accept_len", C.c_void_p), ("out_nodes", C.c_void_p),
+        ("out_status", C.c_void_p), ("G", C.c_void_p), ("margin_accept", C.c_void_p), ("margin_cdf", C.c_void_p),
+    ]
+
+
 _lib = None
 
 
@@ -89,6 +102,8 @@ def _load():
         lib.orc_sample_rows.restype = C.c_int
         lib.orc_verify.argtypes = [C.POINTER(_Params)]
         lib.orc_verify.restype = C.c_int
+        lib.orc_verify_tree.argtypes = [C.POINTER(_TreeParams)]
+        lib.orc_verify_tree.restype = C.c_int
         _lib = lib
     return _lib
 
@@ -255,4 +270,62 @@ def verify(target_logits, draft_logits, draft_tokens, uniforms, relax_schedule, 
     rc = _load().orc_verify(C.byref(prm))
     if rc != 0:
         raise RuntimeError(f"orc_verify failed with code {rc}")
+    return res
+
+
+def tree_depth(parent) -> int:
+    """Deepest level of a tree given as parent indices (-1: child of the root)."""
+    parent = np.asarray(parent, dtype=np.int64)
+    level = np.zeros(len(parent), dtype=np.int64)
+    for n, p in enumerate(parent):
+        if p < -1 or p >= n:
+            raise ValueError("parent[n] must be -1 or an earlier node")
+        level[n] = 1 if p < 0 else level[p] + 1
+    return int(level.max()) if len(parent) else 0
+
+
+@dataclass
+class TreeResult:
+    tokens: np.ndarray        # [B, D+1] int32: accepted path, the drawn token, -1 padding
+    accept_len: np.ndarray    # [B] int32
+    nodes: np.ndarray         # [B, D] int32: node accepted at each level, -1 padding
+    status: np.ndarray        # [B] int32
+    G: Optional[np.ndarray]   # [B, V] float64
+    margin_accept: np.ndarray  # [B, N]
+    margin_cdf: np.ndarray     # [B]
+
+
+def verify_tree(target_logits, draft_logits, parent, draft_tokens, uniforms, relax_schedule, *,
+                dtype: int = F32, target_uncond=None, draft_uncond=None, cfg_scale: float = 1.0,
+                top_k: int = 0, want_G: bool = True) -> TreeResult:
+    """One verification round over a static tree of candidates (see orc_verify_tree in csd_oracle.c).
+
+    target_logits, draft_logits [B, N+1, V]: row 0 is the root context, row n+1 the context after node n;
+    parent [N] int32; draft_tokens [B, N] int32; uniforms [B, N+1] float32 (one accept draw per node, then
+    the resample / bonus draw); relax_schedule [D] float32, one multiplier per level."""
+    t = _raw(target_logits, dtype)
+    d = _raw(draft_logits, dtype)
+    B, N1, V = t.shape
+    N = N1 - 1
+    assert d.shape == (B, N1, V)
+    par = np.ascontiguousarray(parent, dtype=np.int32)
+    assert par.shape == (N,)
+    D = tree_depth(par)
+    tu = None if target_uncond is None else _raw(target_uncond, dtype)
+    du = None if draft_uncond is None else _raw(draft_uncond, dtype)
+    tok = np.ascontiguousarray(draft_tokens, dtype=np.int32)
+    uni = np.ascontiguousarray(uniforms, dtype=np.float32)
+    om = np.ascontiguousarray(relax_schedule, dtype=np.float32)
+    assert tok.shape == (B, N) and uni.shape == (B, N + 1) and om.shape == (D,)
+    res = TreeResult(tokens=np.empty((B, D + 1), np.int32), accept_len=np.empty(B, np.int32),
+                     nodes=np.empty((B, D), np.int32), status=np.zeros(B, np.int32),
+                     G=np.zeros((B, V)) if want_G else None,
+                     margin_accept=np.empty((B, N)), margin_cdf=np.empty(B))
+    prm = _TreeParams(_ptr(t), _ptr(d), _ptr(tu), _ptr(du), int(dtype), float(cfg_scale), int(top_k),
+                      B, N, V, D, _ptr(par), _ptr(tok), _ptr(uni), _ptr(om),
+                      _ptr(res.tokens), _ptr(res.accept_len), _ptr(res.nodes), _ptr(res.status),
+                      _ptr(res.G), _ptr(res.margin_accept), _ptr(res.margin_cdf))
+    rc = _load().orc_verify_tree(C.byref(prm))
+    if rc != 0:
+        raise RuntimeError(f"orc_verify_tree failed with code {rc}")
     return res

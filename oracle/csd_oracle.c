@@ -6,7 +6,9 @@
  * paper (verification stage), the relaxed acceptance probability (Eq. relax),
  * the annealing schedules (UniformRSD, Eq. sdar, and the linear variant of the
  * schedule ablation), and the bound-minimising resampling distribution
- * (Eq. opt_G, Theorem 2 / Proposition LP); the drafting stage's token draws
+ * (Eq. opt_G, Theorem 2 / Proposition LP); the same walk over a static tree of
+ * candidates (the draft structure of the paper's experiments; see orc_verify_tree
+ * for the reading of several candidates per node); the drafting stage's token draws
  * x~_i ~ Q(. | prefix) (Algorithm 1, drafting stage); and, per position, the two sums that
  * Theorem 2 is made of: the acceptance mass sum_x Q f (the inner sum of Eq.
  * token_exp) and the bracket of Eq. bd2, sum_x |P - Q f| - sum_x (1 - f) Q.
@@ -436,6 +438,198 @@ static void verify_one(const orc_params *a, int b, double *zt, double *zd, doubl
       }
     }
   }
+}
+
+/* ---- Tree-structured drafts ------------------------------------------------------------------
+ * The paper's experiments draft a static tree of candidates (Experiments, "Implementation Details");
+ * Algorithm 1 states the chain.  The paper gives no rule for several candidate children of one node
+ * under the relaxed test, so this is the build's reading, chosen so that it contains Algorithm 1 and
+ * stays lossless at omega == 1 (Theorem 1):
+ *   - The candidates of a node are drawn independently from the drafter's distribution Q in that
+ *     node's context (with replacement), and are tried in their stored order.
+ *   - With P' the target's distribution in that context, a candidate x at level i is accepted with
+ *     probability f = min{1, omega_i P'(x)/Q(x)} (Eq. relax on the current residual).  On a rejection
+ *     the residual becomes P' <- Norm([P' - Q f(.)]_+), i.e. Eq. opt_G applied to P' (for omega_i = 1
+ *     this is the recursive rejection sampling of multi-candidate speculative decoding), and the next
+ *     sibling is tried against it with the same Q.
+ *   - An accepted candidate becomes the context of the next level; a node without children ends
+ *     the walk with a bonus token from the target's distribution there (Algorithm 1, last step).
+ *   - When every candidate of a node has been rejected, the emitted token is drawn from the final
+ *     residual by inverse CDF with the sequence's one extra uniform.
+ * A chain (every node the only child of the previous one) is Algorithm 1 itself: the arithmetic below
+ * is then, operation for operation, that of verify_one.
+ *
+ * Layout: contexts are numbered 0 (the root: the prefix alone) and n + 1 (after node n); row c of
+ * target_logits / draft_logits is the model's output in context c.  parent[n] is -1 for a child of the
+ * root, else the index of an EARLIER node.  Siblings are tried in increasing node index.
+ */
+typedef struct {
+  const void *target_logits; /* [B, N+1, V] */
+  const void *draft_logits;  /* [B, N+1, V] (rows of contexts without children are not read) */
+  const void *target_uncond; /* NULL: no guidance mix */
+  const void *draft_uncond;
+  int32_t dtype;
+  float cfg_scale;
+  int32_t top_k;
+  int32_t B, N, V, D;          /* N nodes; D = deepest level (the root's children are level 1) */
+  const int32_t *parent;       /* [N] */
+  const int32_t *draft_tokens; /* [B, N] */
+  const float *uniforms;       /* [B, N+1]: the accept draw of every node, then the resample / bonus draw */
+  const float *relax_schedule; /* [D] omega of levels 1..D */
+  int32_t *out_tokens;         /* [B, D+1]: accepted path, then the drawn token, then -1 */
+  int32_t *out_accept_len;     /* [B] number of accepted levels */
+  int32_t *out_nodes;          /* [B, D] or NULL: the node accepted at each level, then -1 */
+  int32_t *out_status;         /* [B] or NULL */
+  double *G;                   /* [B, V] or NULL: distribution the emitted token was drawn from */
+  double *margin_accept;       /* [B, N] or NULL: |r - f| where the test ran on usable data, else +inf */
+  double *margin_cdf;          /* [B] or NULL */
+} orc_tree_params;
+
+static void verify_tree_one(const orc_tree_params *a, int b, double *zt, double *zd, double *P, double *Q,
+                            double *g, double *scratch) {
+  const int N = a->N, V = a->V, D = a->D;
+  const int64_t stride = (int64_t)(N + 1) * V;
+  const int32_t *tok = a->draft_tokens + (int64_t)b * N;
+  const float *unif = a->uniforms + (int64_t)b * (N + 1);
+  int32_t *out = a->out_tokens + (int64_t)b * (D + 1);
+  for (int i = 0; i <= D; ++i) out[i] = -1;
+  if (a->out_nodes)
+    for (int i = 0; i < D; ++i) a->out_nodes[(int64_t)b * D + i] = -1;
+  if (a->margin_accept)
+    for (int n = 0; n < N; ++n) a->margin_accept[(int64_t)b * N + n] = INFINITY;
+  if (a->margin_cdf) a->margin_cdf[b] = INFINITY;
+  if (a->G)
+    for (int x = 0; x < V; ++x) a->G[(int64_t)b * V + x] = 0.0;
+
+  const double u = (double)unif[N];
+  int status = 0, level = 0, ctx = 0; /* ctx: 0 root, n+1 after node n */
+  for (;;) {
+    const int64_t off = (int64_t)b * stride + (int64_t)ctx * V;
+    orc_prepare_row(a->target_logits, a->target_uncond, a->dtype, off, V, a->cfg_scale, a->top_k, zt, scratch);
+    const int t_ok = orc_softmax(zt, V, P);
+    int first_child = -1;
+    for (int n = 0; n < N; ++n)
+      if (a->parent[n] == ctx - 1) { first_child = n; break; }
+    if (first_child < 0 || level >= D) {
+      /* a leaf: bonus token from the target's distribution in this context */
+      if (t_ok) {
+        double Z = 0.0;
+        for (int x = 0; x < V; ++x) Z += P[x];
+        double mg = INFINITY;
+        out[level] = orc_inverse_cdf(P, V, Z, u, &mg);
+        if (a->margin_cdf) a->margin_cdf[b] = mg;
+        if (a->G)
+          for (int x = 0; x < V; ++x) a->G[(int64_t)b * V + x] = P[x] / Z;
+      } else {
+        status |= ORC_STATUS_BADROW;
+        out[level] = -1;
+      }
+      break;
+    }
+    orc_prepare_row(a->draft_logits, a->draft_uncond, a->dtype, off, V, a->cfg_scale, a->top_k, zd, scratch);
+    const int d_ok = orc_softmax(zd, V, Q);
+    const double omega = (double)a->relax_schedule[level];
+    /* the residual starts as the target's distribution; g, Z hold it unnormalised after a rejection */
+    int have_g = 0, accepted = -1;
+    double Z = 1.0;
+    for (int n = first_child; n < N; ++n) {
+      if (a->parent[n] != ctx - 1) continue;
+      const int x_n = tok[n];
+      const int tok_ok = (x_n >= 0 && x_n < V);
+      double f;
+      if (!t_ok || !d_ok) {
+        f = 0.0;
+        status |= ORC_STATUS_BADROW;
+      } else if (!tok_ok) {
+        f = 0.0;
+        status |= ORC_STATUS_BADTOKEN;
+      } else {
+        f = orc_accept_prob(P[x_n], Q[x_n], omega);
+      }
+      const double r = (double)unif[n];
+      if (a->margin_accept && t_ok && d_ok && tok_ok) a->margin_accept[(int64_t)b * N + n] = fabs(r - f);
+      if (r <= f) { accepted = n; break; }
+      if (!t_ok) continue; /* nothing to update: the emitted token will be -1 */
+      /* rejected: the residual becomes Eq. opt_G of the current residual */
+      if (d_ok) {
+        Z = orc_resample_weights(P, Q, omega, V, g);
+      } else { /* f == 0 for every candidate: Eq. opt_G leaves the residual as it is */
+        Z = 0.0;
+        for (int x = 0; x < V; ++x) { g[x] = P[x]; Z += P[x]; }
+      }
+      if (!(Z > 0.0)) {
+        status |= ORC_STATUS_ZFALLBACK;
+        Z = 0.0;
+        for (int x = 0; x < V; ++x) { g[x] = P[x]; Z += P[x]; }
+      }
+      have_g = 1;
+      /* the next sibling is tested against the normalised residual */
+      int more = 0;
+      for (int m = n + 1; m < N; ++m)
+        if (a->parent[m] == ctx - 1) { more = 1; break; }
+      if (more)
+        for (int x = 0; x < V; ++x) P[x] = g[x] / Z;
+    }
+    if (accepted >= 0) {
+      out[level] = tok[accepted];
+      if (a->out_nodes) a->out_nodes[(int64_t)b * D + level] = accepted;
+      ++level;
+      ctx = accepted + 1;
+      continue;
+    }
+    /* every candidate rejected: draw from the residual */
+    if (!t_ok) {
+      out[level] = -1;
+    } else {
+      double mg = INFINITY;
+      (void)have_g; /* at least one candidate was rejected, so g and Z are set */
+      out[level] = orc_inverse_cdf(g, V, Z, u, &mg);
+      if (a->margin_cdf) a->margin_cdf[b] = mg;
+      if (a->G)
+        for (int x = 0; x < V; ++x) a->G[(int64_t)b * V + x] = g[x] / Z;
+    }
+    break;
+  }
+  a->out_accept_len[b] = level;
+  if (a->out_status) a->out_status[b] = status;
+}
+
+/* Batched driver of the tree walk.  Returns 0, -1 on bad shapes or a malformed tree (a parent that is
+ * not an earlier node, a level beyond D), -2 if memory could not be had. */
+int orc_verify_tree(const orc_tree_params *a) {
+  if (!a || a->B < 1 || a->N < 1 || a->V < 2 || a->D < 1 || !a->parent) return -1;
+  for (int n = 0; n < a->N; ++n) {
+    if (a->parent[n] < -1 || a->parent[n] >= n) return -1;
+    int level = 1;
+    for (int p = a->parent[n]; p >= 0; p = a->parent[p]) ++level;
+    if (level > a->D) return -1;
+  }
+  int failed = 0;
+#ifdef _OPENMP
+#pragma omp parallel
+#endif
+  {
+    const size_t V = (size_t)a->V;
+    double *buf = (double *)malloc(6 * V * sizeof(double));
+    if (!buf) {
+#ifdef _OPENMP
+#pragma omp atomic write
+#endif
+      failed = 1;
+    }
+#ifdef _OPENMP
+#pragma omp barrier
+#endif
+    if (!failed) {
+#ifdef _OPENMP
+#pragma omp for schedule(dynamic, 1)
+#endif
+      for (int b = 0; b < a->B; ++b)
+        verify_tree_one(a, b, buf, buf + V, buf + 2 * V, buf + 3 * V, buf + 4 * V, buf + 5 * V);
+    }
+    free(buf);
+  }
+  return failed ? -2 : 0;
 }
 
 /* ---- Algorithm 1, drafting stage: one token per row -------------------------------------------
