@@ -277,6 +277,69 @@ int csd_sample_rows(const void* logits, const void* uncond, float cfg_scale, int
                     void* workspace, size_t workspace_bytes, int back_to_back, void* stream);
 
 /*
+ * Tree-structured verification: the same round over a static TREE of drafted candidates, the draft
+ * structure of the paper's experiments (Experiments, "Implementation Details": the Eagle-1 static
+ * tree); Algorithm 1 states the chain, which is the tree in which every node has one child.
+ * The paper gives no rule for several candidates of one node under the relaxed test; the rule here:
+ *   - the candidates of a node are independent draws from the drafter's distribution Q in that
+ *     node's context, and are tried in increasing node index;
+ *   - with R the target's distribution in that context, a candidate x at level i is accepted with
+ *     probability min{1, omega_i R(x)/Q(x)} (Eq. relax on the current residual); a rejection replaces
+ *     R by Norm([R - Q f(.)]_+) (Eq. opt_G applied to R; the recursive rejection sampling of
+ *     multi-candidate speculative decoding when omega_i = 1, which keeps Theorem 1), and the next
+ *     sibling is tried against that with the same Q;
+ *   - an accepted candidate becomes the context of the next level; a node without children ends the
+ *     walk with a bonus token from the target's distribution there (Algorithm 1, last step);
+ *   - when every candidate of a node is rejected, the emitted token is drawn from the last residual
+ *     by inverse CDF with the sequence's one extra uniform.
+ * Contexts are numbered 0 (the root: the prefix alone) and n + 1 (after node n); row c of
+ * target_logits and of draft_logits is that model's output in context c (the drafter's rows of
+ * contexts without children are read for their statistics but never used).
+ *   parent         HOST [N]: -1 for a child of the root, else the index of an EARLIER node;
+ *                  1 <= N <= 63, at most 8 children per node, at most 32 levels
+ *   draft_tokens   DEVICE [B, N]
+ *   uniforms       DEVICE [B, N + 1] in (0, 1): the accept draw of every node, then the resample /
+ *                  bonus draw
+ *   relax_schedule DEVICE [D], D = csd_tree_depth(parent, N): omega of levels 1..D
+ *   out_tokens     DEVICE [B, D + 1]: the accepted path's tokens, the drawn token, then -1
+ *   out_accept_len DEVICE [B]: number of accepted levels
+ *   out_nodes      DEVICE [B, D] or NULL: the node accepted at each level, then -1
+ *   out_status     DEVICE [B] or NULL: csd_status_bits (over the contexts the walk visited)
+ *   dbg_G          DEVICE [B, V] or NULL: the distribution the emitted token was drawn from
+ *   workspace      DEVICE, >= csd_tree_workspace_size(B, N, V, dtype) bytes, 256-byte aligned
+ * Other fields as in csd_params.  Every rejection costs one more pass over the two rows of the
+ * current context.  Returns CSD_OK or a negative csd_error (CSD_ERR_ARG for a malformed tree);
+ * nothing is enqueued on an error.
+ */
+typedef struct csd_tree_params {
+  const void* target_logits; /* [B, N + 1, V]                                        */
+  const void* draft_logits;  /* [B, N + 1, V]                                        */
+  const void* target_uncond; /* same layouts, or both NULL                           */
+  const void* draft_uncond;
+  float cfg_scale;
+  int32_t top_k;
+  int32_t dtype;
+  int32_t B, N, V;
+  const int32_t* parent;
+  const int32_t* draft_tokens;
+  const float* uniforms;
+  const float* relax_schedule;
+  int32_t* out_tokens;
+  int32_t* out_accept_len;
+  int32_t* out_nodes;
+  int32_t* out_status;
+  float* dbg_G;
+  void* workspace;
+  size_t workspace_bytes;
+  void* stream;
+} csd_tree_params;
+
+int csd_verify_tree(const csd_tree_params* p);
+size_t csd_tree_workspace_size(int B, int N, int V, int dtype);
+/* Deepest level of the tree (the root's children are level 1), or a negative csd_error. */
+int csd_tree_depth(const int32_t* parent_host, int N);
+
+/*
  * Relaxation schedules, written to HOST memory out_host[0..L-1] = omega_1..omega_L.
  *   kind 0  UniformRSD: omega_i = delta.
  *   kind 1  Cool-SD, Eq. sdar: omega_i = delta * exp(-nu*i - mu) with mu fixed by

@@ -22,7 +22,8 @@ CSD_STATUS_BADROW, CSD_STATUS_BADTOKEN, CSD_STATUS_ZFALLBACK, CSD_STATUS_TIMEOUT
 CSD_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
 EXPORTS = ("csd_verify", "csd_verify_static", "csd_verify_ex", "csd_workspace_size", "csd_workspace_init", "csd_launch_count", "csd_verify_host",
            "csd_host_staging_size", "csd_make_schedule", "csd_error_string", "csd_version",
-           "csd_sample_rows", "csd_sample_workspace_size", "csd_test_hooks")
+           "csd_sample_rows", "csd_sample_workspace_size", "csd_test_hooks",
+           "csd_verify_tree", "csd_tree_workspace_size", "csd_tree_depth")
 
 
 class CsdError(RuntimeError):
@@ -45,6 +46,21 @@ class csd_params(C.Structure):
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p),
         ("back_to_back", C.c_int32),
         ("diag_accept_mass", C.c_void_p), ("diag_bound_term", C.c_void_p),
+    ]
+
+
+class csd_tree_params(C.Structure):
+    """Mirror of ``struct csd_tree_params``."""
+    _fields_ = [
+        ("target_logits", C.c_void_p), ("draft_logits", C.c_void_p),
+        ("target_uncond", C.c_void_p), ("draft_uncond", C.c_void_p),
+        ("cfg_scale", C.c_float), ("top_k", C.c_int32), ("dtype", C.c_int32),
+        ("B", C.c_int32), ("N", C.c_int32), ("V", C.c_int32),
+        ("parent", C.c_void_p), ("draft_tokens", C.c_void_p), ("uniforms", C.c_void_p),
+        ("relax_schedule", C.c_void_p),
+        ("out_tokens", C.c_void_p), ("out_accept_len", C.c_void_p), ("out_nodes", C.c_void_p),
+        ("out_status", C.c_void_p), ("dbg_G", C.c_void_p),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p),
     ]
 
 
@@ -83,6 +99,12 @@ def library() -> C.CDLL:
         lib.csd_version.restype = C.c_int
         lib.csd_test_hooks.argtypes = [C.c_int, C.c_int]
         lib.csd_test_hooks.restype = C.c_int
+        lib.csd_verify_tree.argtypes = [C.POINTER(csd_tree_params)]
+        lib.csd_verify_tree.restype = C.c_int
+        lib.csd_tree_workspace_size.argtypes = [C.c_int] * 4
+        lib.csd_tree_workspace_size.restype = C.c_size_t
+        lib.csd_tree_depth.argtypes = [C.c_void_p, C.c_int]
+        lib.csd_tree_depth.restype = C.c_int
         lib.csd_sample_workspace_size.argtypes = [C.c_int] * 3
         lib.csd_sample_workspace_size.restype = C.c_size_t
         lib.csd_sample_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_int, C.c_int, C.c_int, C.c_int,
@@ -326,3 +348,54 @@ def csd_workspace_init(workspace: torch.Tensor, stream=None) -> None:
                                       workspace.numel() * workspace.element_size(), _stream_handle(stream))
     if rc != 0:
         raise CsdError(rc, "csd_workspace_init")
+
+
+def csd_tree_depth(parent) -> int:
+    """Deepest level of a static tree given as parent indices; raises on a malformed tree."""
+    par = np.ascontiguousarray(parent, dtype=np.int32)
+    d = library().csd_tree_depth(par.ctypes.data_as(C.c_void_p), int(par.size))
+    if d < 0:
+        raise CsdError(d, "csd_tree_depth")
+    return int(d)
+
+
+def csd_tree_workspace_size(B: int, N: int, V: int, dtype: int) -> int:
+    return int(library().csd_tree_workspace_size(int(B), int(N), int(V), int(dtype)))
+
+
+def csd_verify_tree(target_logits, draft_logits, parent, draft_tokens, uniforms, relax_schedule, out_tokens,
+                    out_accept_len, *, target_uncond=None, draft_uncond=None, cfg_scale=1.0, top_k=0,
+                    out_nodes=None, out_status=None, dbg_G=None, workspace=None, stream=None) -> None:
+    """Tree-structured verification (see ``csd_verify_tree`` in csd.h): logits [B, N + 1, V] per context,
+    ``parent`` a host array [N], ``draft_tokens`` [B, N], ``uniforms`` [B, N + 1], ``relax_schedule`` [D]."""
+    B, C1, V = target_logits.shape
+    N = C1 - 1
+    par = np.ascontiguousarray(parent, dtype=np.int32)
+    if draft_logits.shape != (B, C1, V) or par.shape != (N,):
+        raise ValueError("shapes: target and draft [B, N + 1, V], parent [N]")
+    dt = _logit_dtype(target_logits)
+    ldt = target_logits.dtype
+    if workspace is None:
+        workspace = torch.zeros(csd_tree_workspace_size(B, N, V, dt), dtype=torch.uint8, device=target_logits.device)
+    p = csd_tree_params()
+    p.target_logits = _dev_ptr(target_logits, "target_logits", ldt)
+    p.draft_logits = _dev_ptr(draft_logits, "draft_logits", ldt)
+    p.target_uncond = _dev_ptr(target_uncond, "target_uncond", ldt)
+    p.draft_uncond = _dev_ptr(draft_uncond, "draft_uncond", ldt)
+    p.cfg_scale, p.top_k, p.dtype = float(cfg_scale), int(top_k), dt
+    p.B, p.N, p.V = B, N, V
+    p.parent = par.ctypes.data
+    p.draft_tokens = _dev_ptr(draft_tokens, "draft_tokens", torch.int32)
+    p.uniforms = _dev_ptr(uniforms, "uniforms", torch.float32)
+    p.relax_schedule = _dev_ptr(relax_schedule, "relax_schedule", torch.float32)
+    p.out_tokens = _dev_ptr(out_tokens, "out_tokens", torch.int32)
+    p.out_accept_len = _dev_ptr(out_accept_len, "out_accept_len", torch.int32)
+    p.out_nodes = _dev_ptr(out_nodes, "out_nodes", torch.int32)
+    p.out_status = _dev_ptr(out_status, "out_status", torch.int32)
+    p.dbg_G = _dev_ptr(dbg_G, "dbg_G", torch.float32)
+    p.workspace = _dev_ptr(workspace, "workspace")
+    p.workspace_bytes = workspace.numel() * workspace.element_size()
+    p.stream = _stream_handle(stream)
+    rc = library().csd_verify_tree(C.byref(p))
+    if rc != 0:
+        raise CsdError(rc, "csd_verify_tree")

@@ -11,6 +11,7 @@
 #include "../../include/csd.h"
 #include "csd_kernels.cuh"
 #include "csd_fused.cuh"
+#include "csd_tree.cuh"
 
 namespace {
 
@@ -466,6 +467,155 @@ int csd_test_hooks(int wait_limit_log2_cycles, int drop_first_copy) {
   g_wait_limit = wait_limit_log2_cycles ? (1ll << wait_limit_log2_cycles) : kWaitCycles;
   g_drop_first_copy = drop_first_copy ? 1 : 0;
   return CSD_OK;
+}
+
+// ---- tree-structured verification ---------------------------------------------------------
+}  // extern "C"
+namespace {
+template <typename T, bool CFG>
+cudaError_t launch_tree_finish(const TreeArgs& a, cudaStream_t stream) {
+  auto kern = tree_finish_kernel<T, CFG>;
+  constexpr int TILE = 32 * Elem<T>::kVec;
+  size_t slots = (size_t)((a.fin.V + TILE - 1) / TILE);
+  if (slots < 64) slots = 64;
+  const size_t smem = slots * sizeof(double);
+  if (smem > 40 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3((unsigned)a.fin.B);
+  cfg.blockDim = dim3(kFinishThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+// Depth of the tree (the root's children are level 1), or a negative csd_error for a malformed one:
+// a parent that is not -1 or an earlier node, more than kMaxSiblings children of one node, a level
+// beyond kMaxTreeDepth.
+int tree_depth_checked(const int32_t* parent, int N) {
+  if (!parent) return CSD_ERR_NULL;
+  if (N < 1 || N > kMaxTreeNodes) return CSD_ERR_SHAPE;
+  int level[kMaxTreeNodes], kids[kMaxTreeNodes + 1];
+  memset(kids, 0, sizeof kids);
+  int D = 0;
+  for (int n = 0; n < N; ++n) {
+    if (parent[n] < -1 || parent[n] >= n) return CSD_ERR_ARG;
+    level[n] = parent[n] < 0 ? 1 : level[parent[n]] + 1;
+    if (level[n] > kMaxTreeDepth) return CSD_ERR_SHAPE;
+    if (++kids[parent[n] + 1] > kMaxSiblings) return CSD_ERR_SHAPE;
+    if (level[n] > D) D = level[n];
+  }
+  return D;
+}
+}  // namespace
+extern "C" {
+
+int csd_tree_depth(const int32_t* parent_host, int N) { return tree_depth_checked(parent_host, N); }
+
+size_t csd_tree_workspace_size(int B, int N, int V, int dtype) {
+  if (B < 1 || N < 1 || N > kMaxTreeNodes || V < 2 || V > kMaxV || (dtype != CSD_F32 && dtype != CSD_BF16)) return 0;
+  return layout_for(B, N + 1, V, dtype).total;
+}
+
+int csd_verify_tree(const csd_tree_params* pp) {
+  if (!pp) return CSD_ERR_NULL;
+  const csd_tree_params& p = *pp;
+  if (!p.target_logits || !p.draft_logits || !p.parent || !p.draft_tokens || !p.uniforms || !p.relax_schedule ||
+      !p.out_tokens || !p.out_accept_len)
+    return CSD_ERR_NULL;
+  if (p.dtype != CSD_F32 && p.dtype != CSD_BF16) return CSD_ERR_DTYPE;
+  if (p.B < 1 || p.V < 2 || p.V > kMaxV) return CSD_ERR_SHAPE;
+  const int D = tree_depth_checked(p.parent, p.N);
+  if (D < 0) return D;
+  if ((p.target_uncond == nullptr) != (p.draft_uncond == nullptr)) return CSD_ERR_ARG;
+  if (p.top_k < 0) return CSD_ERR_ARG;
+  const bool cfg = p.target_uncond != nullptr;
+  if (cfg && !isfinite(p.cfg_scale)) return CSD_ERR_ARG;
+  const bool topk = p.top_k > 0 && p.top_k < p.V;
+  const int C = p.N + 1;
+  const Layout lay = layout_for(p.B, C, p.V, p.dtype);
+  if (!p.workspace || ((uintptr_t)p.workspace % kAlign) != 0 || p.workspace_bytes < lay.total) return CSD_ERR_WORKSPACE;
+  const int sms = device_sms(nullptr);
+  if (sms <= 0) return CSD_ERR_LAUNCH;
+  const int es = elem_size(p.dtype), vw = vec_width(p.dtype);
+  auto aligned16 = [](const void* q) { return ((uintptr_t)q & 15u) == 0; };
+  const int64_t stride = (int64_t)C * p.V;
+  bool vec_ok = (p.V % vw) == 0 && (stride * es) % 16 == 0 && aligned16(p.target_logits) && aligned16(p.draft_logits);
+  if (cfg) vec_ok = vec_ok && aligned16(p.target_uncond) && aligned16(p.draft_uncond);
+  cudaStream_t stream = (cudaStream_t)p.stream;
+  const long long rows = (long long)p.B * 2 * C;
+  int U = (cfg || topk) ? 4 : 8;
+  auto parts_for = [&](int u) { return (p.V + kStatsThreads * u * vw - 1) / (kStatsThreads * u * vw); };
+  while (U > 1 && rows * parts_for(U) < 4LL * sms) U >>= 1;
+  if (topk && U == 2) U = 1;
+  char* const ws = (char*)p.workspace;
+
+  // the row statistics see a chain of C positions with C target rows
+  StatsArgs sa;
+  sa.target = p.target_logits; sa.draft = p.draft_logits;
+  sa.target_uncond = p.target_uncond; sa.draft_uncond = p.draft_uncond;
+  sa.cfg_scale = p.cfg_scale;
+  sa.B = p.B; sa.gamma = C; sa.T = C; sa.V = p.V;
+  sa.tstride = stride; sa.dstride = stride;
+  sa.parts = parts_for(U);
+  sa.part_elems = kStatsThreads * U * vw;
+  sa.n_items = (int)(rows * sa.parts);
+  sa.vec_ok = vec_ok ? 1 : 0;
+  sa.partials = reinterpret_cast<float2*>(ws + lay.partials_off);
+  sa.thresholds = reinterpret_cast<const float*>(ws + lay.thresholds_off);
+  SelectArgs se;
+  se.target = p.target_logits; se.draft = p.draft_logits;
+  se.target_uncond = p.target_uncond; se.draft_uncond = p.draft_uncond;
+  se.cfg_scale = p.cfg_scale;
+  se.B = p.B; se.gamma = C; se.T = C; se.V = p.V;
+  se.tstride = stride; se.dstride = stride;
+  se.vec_ok = sa.vec_ok;
+  se.top_k = p.top_k;
+  se.thresholds = reinterpret_cast<float*>(ws + lay.thresholds_off);
+  TreeArgs ta;
+  memset(&ta, 0, sizeof ta);
+  FinishArgs& fa = ta.fin;
+  fa.target = p.target_logits; fa.draft = p.draft_logits;
+  fa.target_uncond = p.target_uncond; fa.draft_uncond = p.draft_uncond;
+  fa.cfg_scale = p.cfg_scale;
+  fa.B = p.B; fa.gamma = C; fa.T = C; fa.V = p.V;
+  fa.tstride = stride; fa.dstride = stride;
+  fa.parts = sa.parts;
+  fa.vec_ok = sa.vec_ok;
+  fa.use_topk = topk ? 1 : 0;
+  fa.partials = sa.partials;
+  fa.thresholds = sa.thresholds;
+  fa.tokens = p.draft_tokens; fa.uniforms = p.uniforms; fa.schedule = p.relax_schedule;
+  fa.out_tokens = p.out_tokens; fa.out_accept_len = p.out_accept_len; fa.out_status = p.out_status;
+  fa.dbg_G = p.dbg_G;
+  ta.N = p.N; ta.D = D;
+  ta.out_nodes = p.out_nodes;
+  for (int n = 0; n < p.N; ++n) ta.parent[n] = (signed char)p.parent[n];
+
+  cudaError_t e = cudaSuccess;
+  if (p.dtype == CSD_F32) {
+    if (topk) e = cfg ? launch_select<float, true>(se, sms, stream) : launch_select<float, false>(se, sms, stream);
+    if (e == cudaSuccess)
+      e = cfg ? launch_stats_u<float, true>(sa, U, topk, sms, stream) : launch_stats_u<float, false>(sa, U, topk, sms, stream);
+    if (e == cudaSuccess) e = cfg ? launch_tree_finish<float, true>(ta, stream) : launch_tree_finish<float, false>(ta, stream);
+  } else {
+    if (topk)
+      e = cfg ? launch_select<__nv_bfloat16, true>(se, sms, stream) : launch_select<__nv_bfloat16, false>(se, sms, stream);
+    if (e == cudaSuccess)
+      e = cfg ? launch_stats_u<__nv_bfloat16, true>(sa, U, topk, sms, stream)
+              : launch_stats_u<__nv_bfloat16, false>(sa, U, topk, sms, stream);
+    if (e == cudaSuccess)
+      e = cfg ? launch_tree_finish<__nv_bfloat16, true>(ta, stream) : launch_tree_finish<__nv_bfloat16, false>(ta, stream);
+  }
+  return e == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
 }
 
 // ---- allocation-free form -------------------------------------------------------------

@@ -106,6 +106,19 @@ def _sample_tokens(drafter_rows_f32: torch.Tensor, g: torch.Generator) -> torch.
     return torch.multinomial(probs, 1, generator=g).reshape(B, L).to(torch.int32)
 
 
+def _effective_rows(d_c: torch.Tensor, d_u: Optional[torch.Tensor], cfg_scale: float, top_k: int) -> torch.Tensor:
+    """The drafter's effective rows (what it would sample from), in fp32 from the stored values:
+    mixed with the unconditional rows if there are any, then top-k filtered."""
+    eff = d_c.float()
+    if d_u is not None:
+        eff = torch.addcmul(d_u.float(), d_c.float() - d_u.float(), torch.tensor(
+            cfg_scale, device=d_c.device, dtype=torch.float32))
+    if 0 < top_k < eff.shape[-1]:
+        kth = torch.topk(eff, top_k, dim=-1).values[..., -1:]
+        eff = torch.where(eff >= kth, eff, torch.full_like(eff, float("-inf")))
+    return eff
+
+
 def make(name: str, *, B: int, gamma: int, V: int, dtype: int = F32, rho: float = 0.9,
          law: str = "gauss", scale: float = 3.0, bonus_row: bool = False, cfg: bool = False,
          cfg_scale: float = 4.0, top_k: int = 0, schedule: Optional[np.ndarray] = None,
@@ -130,14 +143,7 @@ def make(name: str, *, B: int, gamma: int, V: int, dtype: int = F32, rho: float 
     t_u = d_u = None
     if cfg:
         t_u, d_u = pair()
-    # the drafter's effective row (what it would sample from), in fp32 from stored values
-    eff = d_c.float()
-    if cfg:
-        eff = torch.addcmul(d_u.float(), d_c.float() - d_u.float(), torch.tensor(
-            cfg_scale, device=device, dtype=torch.float32))
-    if 0 < top_k < V:
-        kth = torch.topk(eff, top_k, dim=-1).values[..., -1:]
-        eff = torch.where(eff >= kth, eff, torch.full_like(eff, float("-inf")))
+    eff = _effective_rows(d_c, d_u, cfg_scale, top_k)
     tokens = _sample_tokens(eff, g)
     uni = torch.from_numpy(open_uniforms((B, gamma + 1), seed=(seed * 7919 + step))).to(device)
     if schedule is None:
@@ -169,3 +175,70 @@ def config(name: str, *, step: int = 0, seed: int = 0, device="cpu", **overrides
     kw.pop("steps", None)
     kw.update(overrides)
     return make(name, seed=seed, step=step, device=device, **kw)
+
+
+# ---- static draft trees -----------------------------------------------------------------------------
+@dataclass
+class TreeWorkload:
+    """One batch of inputs for one tree-structured verify call.  Contexts: 0 is the root, n + 1 the
+    context after node n; row c of the logit arrays is the model's output in context c."""
+    dtype: int
+    B: int
+    N: int
+    V: int
+    parent: np.ndarray               # [N] int32, -1 for a child of the root, else an earlier node
+    target_logits: torch.Tensor      # [B, N + 1, V]
+    draft_logits: torch.Tensor       # [B, N + 1, V]
+    draft_tokens: torch.Tensor       # [B, N] int32
+    uniforms: torch.Tensor           # [B, N + 1] float32
+    relax_schedule: torch.Tensor     # [D] float32
+    target_uncond: Optional[torch.Tensor] = None
+    draft_uncond: Optional[torch.Tensor] = None
+    cfg_scale: float = 1.0
+    top_k: int = 0
+
+    def host_arrays(self) -> dict:
+        def conv(t):
+            if t is None:
+                return None
+            t = t.detach().cpu().contiguous()
+            if t.dtype == torch.bfloat16:
+                return t.view(torch.int16).numpy().view(np.uint16).copy()
+            return t.numpy().copy()
+        return dict(target_logits=conv(self.target_logits), draft_logits=conv(self.draft_logits),
+                    target_uncond=conv(self.target_uncond), draft_uncond=conv(self.draft_uncond),
+                    draft_tokens=conv(self.draft_tokens), uniforms=conv(self.uniforms),
+                    relax_schedule=conv(self.relax_schedule), parent=self.parent.copy())
+
+
+def static_tree(widths) -> np.ndarray:
+    """Parent indices of a static tree in which the first node of every level carries the next level
+    (the shape of a top-heavy static draft tree): widths[i] candidates at level i + 1."""
+    parent, first_of_prev = [], -1
+    for w in widths:
+        start = len(parent)
+        parent.extend([first_of_prev] * int(w))
+        first_of_prev = start
+    return np.asarray(parent, dtype=np.int32)
+
+
+def make_tree(parent, *, B: int, V: int, schedule: np.ndarray, dtype: int = F32, rho: float = 0.9,
+              law: str = "gauss", scale: float = 3.0, cfg: bool = False, cfg_scale: float = 4.0, top_k: int = 0,
+              seed: int = 0, step: int = 0, device="cpu") -> TreeWorkload:
+    """Synthetic inputs for a static draft tree: correlated target/drafter rows for every context, and
+    for every node one independent categorical draw from the drafter's effective row of its parent's
+    context (the drafting rule the tree verification assumes)."""
+    parent = np.asarray(parent, dtype=np.int32)
+    N = len(parent)
+    w = make("tree", B=B, gamma=N + 1, V=V, dtype=dtype, rho=rho, law=law, scale=scale, cfg=cfg, cfg_scale=cfg_scale,
+             top_k=top_k, seed=seed, step=step, device=device)
+    eff = _effective_rows(w.draft_logits, w.draft_uncond, cfg_scale, top_k)       # [B, N + 1, V]
+    g = _gen(torch.device(device), seed + 77, step)
+    ctx = torch.from_numpy(parent.astype(np.int64) + 1).to(eff.device)
+    tokens = _sample_tokens(eff[:, ctx, :].contiguous(), g)                         # node n draws in context parent[n] + 1
+    sched = torch.from_numpy(np.asarray(schedule, dtype=np.float32)).to(eff.device)
+    return TreeWorkload(dtype=dtype, B=B, N=N, V=V, parent=parent, target_logits=w.target_logits,
+                        draft_logits=w.draft_logits, draft_tokens=tokens.contiguous(),
+                        uniforms=w.uniforms[:, :N + 1].contiguous(), relax_schedule=sched,
+                        target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
+                        cfg_scale=w.cfg_scale, top_k=top_k)
