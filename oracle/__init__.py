@@ -54,6 +54,7 @@ class _Params(C.Structure):
         ("p", C.c_void_p), ("q", C.c_void_p), ("f", C.c_void_p), ("G", C.c_void_p),
         ("margin_accept", C.c_void_p), ("margin_cdf", C.c_void_p),
         ("accept_mass", C.c_void_p), ("bound_term", C.c_void_p),
+        ("neighbours", C.c_void_p), ("nbr_k", C.c_int32), ("nbr_lambda", C.c_float),
     ]
 
 
@@ -92,6 +93,11 @@ def _load():
         lib.orc_resample_dist.restype = C.c_double
         lib.orc_position_terms.argtypes = [C.c_void_p, C.c_void_p, C.c_double, C.c_int, C.c_void_p, C.c_void_p]
         lib.orc_position_terms.restype = None
+        lib.orc_neighbour_mass.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_double, C.c_int]
+        lib.orc_neighbour_mass.restype = C.c_double
+        lib.orc_resample_weights_nbr.argtypes = [C.c_void_p, C.c_void_p, C.c_double, C.c_int, C.c_void_p, C.c_int,
+                                                 C.c_double, C.c_void_p]
+        lib.orc_resample_weights_nbr.restype = C.c_double
         lib.orc_inverse_cdf.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_double, C.c_void_p]
         lib.orc_inverse_cdf.restype = C.c_int
         lib.orc_prepare_row.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int,
@@ -170,6 +176,23 @@ def position_terms(P, Q, omega: float):
     return a.value, b.value
 
 
+def neighbour_mass(P, nbr_row, lam: float, x: int) -> float:
+    """LANTERN++'s aggregated mass of token x over its selected nearest tokens."""
+    P = _f64(P)
+    nb = np.ascontiguousarray(nbr_row, dtype=np.int32)
+    return float(_load().orc_neighbour_mass(_ptr(P), int(P.size), _ptr(nb), int(nb.size), float(lam), int(x)))
+
+
+def resample_weights_nbr(P, Q, omega: float, neighbours, lam: float):
+    """Unnormalised Eq. opt_G with LANTERN++'s acceptance at every candidate, and its total Z."""
+    P, Q = _f64(P), _f64(Q)
+    nb = np.ascontiguousarray(neighbours, dtype=np.int32)
+    g = np.empty_like(P)
+    Z = _load().orc_resample_weights_nbr(_ptr(P), _ptr(Q), float(omega), int(P.size), _ptr(nb), int(nb.shape[1]),
+                                         float(lam), _ptr(g))
+    return g, float(Z)
+
+
 def inverse_cdf(g, Z: float, u: float):
     g = _f64(g)
     margin = C.c_double(0.0)
@@ -231,7 +254,7 @@ class VerifyResult:
 def verify(target_logits, draft_logits, draft_tokens, uniforms, relax_schedule, *,
            dtype: int = F32, target_uncond=None, draft_uncond=None, cfg_scale: float = 1.0,
            top_k: int = 0, want_G: bool = True, want_pqf: bool = True,
-           want_terms: bool = False) -> VerifyResult:
+           want_terms: bool = False, neighbours=None, nbr_lambda: float = 0.0) -> VerifyResult:
     """One verification round for B sequences (Algorithm 1, verification stage).
 
     target_logits [B, T, V] with T in {gamma, gamma+1}; draft_logits [B, gamma, V];
@@ -266,7 +289,12 @@ def verify(target_logits, draft_logits, draft_tokens, uniforms, relax_schedule, 
         _ptr(res.tokens), _ptr(res.accept_len), _ptr(res.status),
         _ptr(res.p) if want_pqf else None, _ptr(res.q) if want_pqf else None,
         _ptr(res.f) if want_pqf else None, _ptr(res.G),
-        _ptr(res.margin_accept), _ptr(res.margin_cdf), _ptr(res.accept_mass), _ptr(res.bound_term))
+        _ptr(res.margin_accept), _ptr(res.margin_cdf), _ptr(res.accept_mass), _ptr(res.bound_term),
+        None, 0, 0.0)
+    if neighbours is not None:
+        nb = np.ascontiguousarray(neighbours, dtype=np.int32)
+        assert nb.ndim == 2 and nb.shape[0] == V
+        prm.neighbours, prm.nbr_k, prm.nbr_lambda = _ptr(nb), nb.shape[1], float(nbr_lambda)
     rc = _load().orc_verify(C.byref(prm))
     if rc != 0:
         raise RuntimeError(f"orc_verify failed with code {rc}")

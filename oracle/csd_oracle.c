@@ -95,6 +95,11 @@ typedef struct {
   double *margin_cdf;          /* [B] or NULL: distance of u to the nearest CDF boundary of the pick */
   double *accept_mass;         /* [B, gamma] or NULL: sum_x Q_i(x) f_i(x) at every position (NaN: unusable row) */
   double *bound_term;          /* [B, gamma] or NULL: the bracket of Eq. bd2 at every position */
+  /* Similarity relaxation of LANTERN++ with the paper's resampling distribution (Ablation, "Principled
+   * Resampling Strategy"); NULL / 0: off, and nothing above changes. */
+  const int32_t *neighbours;   /* [V, nbr_k]: for every token its nearest tokens, nearest first (-1: none) */
+  int32_t nbr_k;
+  float nbr_lambda;
 } orc_params;
 
 int orc_num_threads(void) {
@@ -227,6 +232,38 @@ void orc_position_terms(const double *P, const double *Q, double omega, int V, d
   *bound_term = abs_sum - rej;
 }
 
+/* LANTERN++'s aggregated mass of candidate x (the first case of its P^{k,lambda}): P(x) plus the mass
+ * of the selected subset A of x's k nearest tokens.  The paper only says that A is "a selected subset"
+ * with sum_{A \ x} P < lambda P(x); the reading here: neighbours are taken nearest first while the
+ * running sum stays strictly below lambda P(x), and the first one that would break it ends the
+ * selection.  Entries that are -1, out of range or x itself are skipped. */
+double orc_neighbour_mass(const double *P, int V, const int32_t *nbr_row, int k, double lambda, int x) {
+  const double own = P[x];
+  double extra = 0.0;
+  for (int j = 0; j < k; ++j) {
+    const int y = nbr_row[j];
+    if (y < 0 || y >= V || y == x) continue;
+    if (extra + P[y] < lambda * own) extra += P[y];
+    else break;
+  }
+  return own + extra;
+}
+
+/* Eq. opt_G with LANTERN++'s acceptance f^{k,lambda} (times the multiplier omega) at every candidate:
+ * g(x) = [P(x) - Q(x) min{1, omega A(x)/Q(x)}]_+ with A(x) the aggregated mass above.  Returns Z. */
+double orc_resample_weights_nbr(const double *P, const double *Q, double omega, int V, const int32_t *nbr, int k,
+                                double lambda, double *g) {
+  double Z = 0.0;
+  for (int x = 0; x < V; ++x) {
+    const double fx = orc_accept_prob(orc_neighbour_mass(P, V, nbr + (int64_t)x * k, k, lambda, x), Q[x], omega);
+    double v = P[x] - Q[x] * fx;
+    if (!(v > 0.0)) v = 0.0;
+    g[x] = v;
+    Z += v;
+  }
+  return Z;
+}
+
 /* Eq. opt_G normalised; falls back to P when Z = 0.  Returns Z. */
 double orc_resample_dist(const double *P, const double *Q, double omega, int V, double *G) {
   double Z = orc_resample_weights(P, Q, omega, V, G);
@@ -347,6 +384,9 @@ static void verify_one(const orc_params *a, int b, double *zt, double *zd, doubl
     } else if (!tok_ok) {
       f = 0.0;
       status |= ORC_STATUS_BADTOKEN;
+    } else if (a->neighbours) {
+      f = orc_accept_prob(orc_neighbour_mass(P, V, a->neighbours + (int64_t)x_i * a->nbr_k, a->nbr_k,
+                                             (double)a->nbr_lambda, x_i), Q[x_i], omega);
     } else {
       f = orc_accept_prob(P[x_i], Q[x_i], omega);
     }
@@ -362,7 +402,9 @@ static void verify_one(const orc_params *a, int b, double *zt, double *zd, doubl
         out[i - 1] = -1;
       } else {
         double Z;
-        if (d_ok) {
+        if (d_ok && a->neighbours) {
+          Z = orc_resample_weights_nbr(P, Q, omega, V, a->neighbours, a->nbr_k, (double)a->nbr_lambda, g);
+        } else if (d_ok) {
           Z = orc_resample_weights(P, Q, omega, V, g);
         } else { /* f == 0 for every candidate: Eq. opt_G gives P */
           Z = 0.0;
@@ -426,7 +468,10 @@ static void verify_one(const orc_params *a, int b, double *zt, double *zd, doubl
       const int x_i = tok[i - 1];
       const int ok = t_ok && d_ok && x_i >= 0 && x_i < V;
       const int64_t o = (int64_t)b * L + (i - 1);
-      const double pv = ok ? P[x_i] : NAN, qv = ok ? Q[x_i] : NAN;
+      double pv = ok ? P[x_i] : NAN;
+      const double qv = ok ? Q[x_i] : NAN;
+      if (ok && a->neighbours) /* the mass the test used */
+        pv = orc_neighbour_mass(P, V, a->neighbours + (int64_t)x_i * a->nbr_k, a->nbr_k, (double)a->nbr_lambda, x_i);
       if (a->p) a->p[o] = pv;
       if (a->q) a->q[o] = qv;
       if (a->f) a->f[o] = ok ? orc_accept_prob(pv, qv, (double)a->relax_schedule[i - 1]) : 0.0;
