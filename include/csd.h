@@ -277,6 +277,26 @@ int csd_sample_rows(const void* logits, const void* uncond, float cfg_scale, int
                     void* workspace, size_t workspace_bytes, int back_to_back, void* stream);
 
 /*
+ * Similarity relaxation with the paper's resampling distribution (Ablation Study, "Principled
+ * Resampling Strategy": LANTERN++'s acceptance f^{k,lambda} of the Speculative Decoding section with
+ * G* of Eq. opt_G in place of LANTERN++'s own G^{k,lambda}).  The round of csd_verify_ex in which the
+ * target mass of a candidate x is aggregated over a selected subset of its k nearest tokens:
+ *   A(x) = P(x) + sum of P(y) over the selected y,
+ *   f_i  = min{1, omega_i A(x~_i) / Q(x~_i)},      G*_j = Norm([P_j - Q_j min{1, omega_j A(.)/Q_j(.)}]_+)
+ * (for omega_j >= 1 this G* is the vanilla Norm([P_j - Q_j]_+), Proposition 2).  The paper says only
+ * that the subset is "selected" with sum_{y} P(y) < lambda P(x); here neighbours are taken in table
+ * order (nearest first) while the running sum stays strictly below lambda P(x), and the first one that
+ * would break it ends the selection.
+ *   neighbours  DEVICE [V, k] int32: row x lists the nearest tokens of x; entries that are -1, out of
+ *               range or x itself are skipped.  1 <= k <= 64.  (The paper's tables come from the image
+ *               tokenizer's codebook, which the caller supplies.)
+ *   lambda      >= 0; 0 selects nothing: the call then equals csd_verify_ex
+ * dbg_p reports A(x~_i).  The Theorem 2 monitors are not available in this form (CSD_ERR_ARG).  The
+ * call always takes the multi-launch path (csd_launch_count does not apply).
+ */
+int csd_verify_similar(const csd_params* p, const int32_t* neighbours, int k, float lambda);
+
+/*
  * Tree-structured verification: the same round over a static TREE of drafted candidates, the draft
  * structure of the paper's experiments (Experiments, "Implementation Details": the Eagle-1 static
  * tree); Algorithm 1 states the chain, which is the tree in which every node has one child.

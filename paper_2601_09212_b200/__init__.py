@@ -23,7 +23,7 @@ CSD_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
 EXPORTS = ("csd_verify", "csd_verify_static", "csd_verify_ex", "csd_workspace_size", "csd_workspace_init", "csd_launch_count", "csd_verify_host",
            "csd_host_staging_size", "csd_make_schedule", "csd_error_string", "csd_version",
            "csd_sample_rows", "csd_sample_workspace_size", "csd_test_hooks",
-           "csd_verify_tree", "csd_tree_workspace_size", "csd_tree_depth")
+           "csd_verify_tree", "csd_tree_workspace_size", "csd_tree_depth", "csd_verify_similar")
 
 
 class CsdError(RuntimeError):
@@ -99,6 +99,8 @@ def library() -> C.CDLL:
         lib.csd_version.restype = C.c_int
         lib.csd_test_hooks.argtypes = [C.c_int, C.c_int]
         lib.csd_test_hooks.restype = C.c_int
+        lib.csd_verify_similar.argtypes = [C.POINTER(csd_params), C.c_void_p, C.c_int, C.c_float]
+        lib.csd_verify_similar.restype = C.c_int
         lib.csd_verify_tree.argtypes = [C.POINTER(csd_tree_params)]
         lib.csd_verify_tree.restype = C.c_int
         lib.csd_tree_workspace_size.argtypes = [C.c_int] * 4
@@ -350,6 +352,9 @@ def csd_workspace_init(workspace: torch.Tensor, stream=None) -> None:
         raise CsdError(rc, "csd_workspace_init")
 
 
+_tree_ws = {}
+
+
 def csd_tree_depth(parent) -> int:
     """Deepest level of a static tree given as parent indices; raises on a malformed tree."""
     par = np.ascontiguousarray(parent, dtype=np.int32)
@@ -376,7 +381,14 @@ def csd_verify_tree(target_logits, draft_logits, parent, draft_tokens, uniforms,
     dt = _logit_dtype(target_logits)
     ldt = target_logits.dtype
     if workspace is None:
-        workspace = torch.zeros(csd_tree_workspace_size(B, N, V, dt), dtype=torch.uint8, device=target_logits.device)
+        # one grow-only buffer per device, kept by the module: the call is asynchronous, so a buffer made
+        # here must outlive this function
+        need = csd_tree_workspace_size(B, N, V, dt)
+        key = target_logits.device
+        workspace = _tree_ws.get(key)
+        if workspace is None or workspace.numel() < need:
+            workspace = torch.zeros(need, dtype=torch.uint8, device=key)
+            _tree_ws[key] = workspace
     p = csd_tree_params()
     p.target_logits = _dev_ptr(target_logits, "target_logits", ldt)
     p.draft_logits = _dev_ptr(draft_logits, "draft_logits", ldt)
@@ -399,3 +411,14 @@ def csd_verify_tree(target_logits, draft_logits, parent, draft_tokens, uniforms,
     rc = library().csd_verify_tree(C.byref(p))
     if rc != 0:
         raise CsdError(rc, "csd_verify_tree")
+
+
+def csd_verify_similar(params: csd_params, neighbours: torch.Tensor, nbr_lambda: float) -> None:
+    """``csd_verify_ex`` with LANTERN++'s similarity-relaxed acceptance and the paper's G* (see csd.h):
+    ``neighbours`` is a device int32 tensor [V, k]."""
+    if neighbours.dim() != 2 or neighbours.shape[0] != params.V:
+        raise ValueError("neighbours must be [V, k]")
+    rc = library().csd_verify_similar(C.byref(params), _dev_ptr(neighbours, "neighbours", torch.int32),
+                                      int(neighbours.shape[1]), float(nbr_lambda))
+    if rc != 0:
+        raise CsdError(rc, "csd_verify_similar")

@@ -203,7 +203,14 @@ int g_drop_first_copy = 0;
 // "target" row per sequence, whose bonus draw is the wanted token; the drafter-side pointers are unused.
 // no_workspace: the call has no workspace (the simple forms): only the single-launch path, which keeps
 // nothing in global memory, can serve it; otherwise CSD_ERR_ALIGN.
-int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = false, bool no_workspace = false) {
+// similar: the similarity relaxation's neighbour table (csd_verify_similar); served by the multi-launch path.
+struct Similar {
+  const int32_t* nbr = nullptr;
+  int k = 0;
+  float lambda = 0.0f;
+};
+int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = false, bool no_workspace = false,
+                const Similar& similar = Similar()) {
   if (sampling) {
     if (!p.target_logits || !p.uniforms || !p.out_tokens) return CSD_ERR_NULL;
   } else if (!p.target_logits || !p.draft_logits || !p.draft_tokens || !p.uniforms || !p.relax_schedule ||
@@ -287,9 +294,11 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
   fa.out_tokens = p.out_tokens; fa.out_accept_len = p.out_accept_len; fa.out_status = p.out_status;
   fa.dbg_p = p.dbg_p; fa.dbg_q = p.dbg_q; fa.dbg_f = p.dbg_f; fa.dbg_G = p.dbg_G;
   fa.diag_am = p.diag_accept_mass; fa.diag_bt = p.diag_bound_term;
+  fa.nbr = similar.nbr; fa.nbr_k = similar.k; fa.nbr_lambda = similar.lambda;
 
   // ---- fused single-launch path: aligned rows of at least 512 bytes; with top-k, rows that fit the registers
-  const bool fused = vec_ok && (size_t)p.V * es >= 512 && (p.V + 32 * vw - 1) / (32 * vw) <= kFinTiles;
+  const bool fused = vec_ok && (size_t)p.V * es >= 512 && (p.V + 32 * vw - 1) / (32 * vw) <= kFinTiles &&
+                     similar.nbr == nullptr;
   if (no_workspace && !fused) return CSD_ERR_ALIGN;
   if (plan_only) {  // number of kernels this call would enqueue
     *plan_only = fused ? 1 : (topk ? 3 : 2);
@@ -460,6 +469,15 @@ int csd_verify(const float* target_logits, const float* draft_logits, const int3
   p.out_tokens = out_tokens; p.out_accept_len = out_accept_len;
   p.stream = stream;
   return verify_impl(p, nullptr, false, /*no_workspace=*/true);
+}
+
+int csd_verify_similar(const csd_params* p, const int32_t* neighbours, int k, float lambda) {
+  if (!p || !neighbours) return CSD_ERR_NULL;
+  if (k < 1 || k > 64 || !(lambda >= 0.0f) || !isfinite(lambda)) return CSD_ERR_ARG;
+  if (p->diag_accept_mass || p->diag_bound_term) return CSD_ERR_ARG;   // (the monitors are those of Eq. relax)
+  Similar sim;
+  sim.nbr = neighbours; sim.k = k; sim.lambda = lambda;
+  return verify_impl(*p, nullptr, false, false, sim);
 }
 
 int csd_test_hooks(int wait_limit_log2_cycles, int drop_first_copy) {

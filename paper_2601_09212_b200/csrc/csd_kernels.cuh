@@ -450,6 +450,10 @@ struct FinishArgs {
   float* dbg_G;
   float* diag_am;   // [B, gamma] or null: sum_x Q f per position (inner sum of Eq. token_exp)
   float* diag_bt;   // [B, gamma] or null: bracket of Eq. bd2 per position
+  // similarity relaxation (LANTERN++'s acceptance with the paper's G*; multi-launch path only)
+  const int32_t* nbr;   // [V, nbr_k] or null: every token's nearest tokens, nearest first (-1: none)
+  int nbr_k;
+  float nbr_lambda;
 };
 
 struct PairCtx {  // what Eq. opt_G needs at one position
@@ -470,6 +474,33 @@ __device__ __forceinline__ float weight_of(float zt, float zd, const PairCtx& c)
   const float pq = ((et - ed) + (et * c.Sd - ed * c.St)) * c.inv_den;  // P - Q
   const float alt = c.one_minus_omega * et * c.inv_t;                    // (1 - omega) P
   return fmaxf(0.0f, fmaxf(pq, alt));
+}
+
+// Similarity relaxation (LANTERN++'s P^{k,lambda} at the candidate): the target mass of the selected
+// subset of token x's nearest tokens -- taken nearest first while the running sum stays strictly below
+// lambda P(x); the first that would break it ends the selection -- to be added to P(x) = own.
+template <typename RowT>
+__device__ __forceinline__ float neighbour_extra(const RowT& rt, const float Mt, const float inv_t, const int32_t* nbr,
+                                                 const int k, const float lambda, const int x, const int V, const float own) {
+  float extra = 0.0f;
+  const float budget = lambda * own;
+  for (int j = 0; j < k; ++j) {
+    const int y = __ldg(nbr + (int64_t)x * k + j);
+    if (y < 0 || y >= V || y == x) continue;
+    const float py = ex2f((rt.filter(rt.load_one(y)) - Mt) * kLog2e) * inv_t;
+    if (extra + py < budget) extra += py;
+    else break;
+  }
+  return extra;
+}
+// Eq. opt_G's weight with that acceptance, g = [P - min{Q, omega (P + extra)}]_+; P - Q in the
+// cancellation-free form of weight_of.
+__device__ __forceinline__ float weight_of_similar(float zt, float zd, const PairCtx& c, const float extra) {
+  const float et = ex2f((zt - c.Mt) * kLog2e), ed = ex2f((zd - c.Md) * kLog2e);
+  const float pq = ((et - ed) + (et * c.Sd - ed * c.St)) * c.inv_den;
+  const float P = et * c.inv_t, Q = ed / (1.0f + c.Sd);
+  const float oa = (1.0f - c.one_minus_omega) * (P + extra);
+  return oa >= Q ? fmaxf(0.0f, pq) : fmaxf(0.0f, P - oa);
 }
 
 // One candidate token's share of the two per-position sums of Theorem 2, with
@@ -638,9 +669,15 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
           const float dd = rd.filter(rd.load_one(tok)) - M[1];
           p = ex2f(dt * kLog2e) / (1.0f + S[0]);
           q = ex2f(dd * kLog2e) / (1.0f + S[1]);
+          float grow = 1.0f;   // (aggregated mass) / (own mass) under the similarity relaxation
+          if (a.nbr && p > 0.0f) {
+            const float extra = neighbour_extra(rt, M[0], 1.0f / (1.0f + S[0]), a.nbr, a.nbr_k, a.nbr_lambda, tok, V, p);
+            grow = 1.0f + extra / p;
+            p += extra;
+          }
           if (dd == CSD_NEG_INF) f = 1.0f;         // q = 0: p/q = +inf, and 0/0 := 1
           else if (dt == CSD_NEG_INF) f = 0.0f;    // p = 0 < q
-          else f = fminf(1.0f, omega * ex2f((dt - dd) * kLog2e) * ((1.0f + S[1]) / (1.0f + S[0])));
+          else f = fminf(1.0f, omega * grow * ex2f((dt - dd) * kLog2e) * ((1.0f + S[1]) / (1.0f + S[0])));
         }
         const float r = a.uniforms[(int64_t)b * (L + 1) + i];
         sm.acc[i] = (r <= f) ? 1 : 0;
@@ -688,6 +725,17 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
     Row<T, CFG> rd = rt;
     if (j < L) rd = Row<T, CFG>{dft + (int64_t)j * V, CFG ? dft_u + (int64_t)j * V : nullptr, a.cfg_scale, sm.thr[1][j]};
     const float u = a.uniforms[(int64_t)b * (L + 1) + L];
+    // (omega >= 1: the aggregated mass only raises f above f_van, and Eq. opt_G is the vanilla residual)
+    const bool similar = a.nbr != nullptr && j < L && omega < 1.0f;
+    auto weight_at = [&](int x, float zt_x, float zd_x) -> float {
+      const float ft = rt.filter(zt_x);
+      if (ctx.mode != 0) return weight_of(ft, 0.0f, ctx);
+      const float fd = rd.filter(zd_x);
+      if (!similar || x >= V) return weight_of(ft, fd, ctx);
+      const float own = ex2f((ft - ctx.Mt) * kLog2e) * ctx.inv_t;
+      const float extra = own > 0.0f ? neighbour_extra(rt, ctx.Mt, ctx.inv_t, a.nbr, a.nbr_k, a.nbr_lambda, x, V, own) : 0.0f;
+      return weight_of_similar(ft, fd, ctx, extra);
+    };
 
     for (int attempt = 0; attempt < 2; ++attempt) {
       // ---- 4. Eq. opt_G weights, one fp64 sum per tile ---------------------------
@@ -708,10 +756,11 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
         for (int r = 0; r < UNR; ++r) {
           const int tile = tile0 + r * (NT / 32);
           if (tile < ntiles) {
+            const int x0 = tile * TILE + lane * VEC;
             float acc = 0.0f;
 #pragma unroll
             for (int k = 0; k < VEC; ++k)
-              acc += weight_of(rt.filter(zt[r][k]), ctx.mode == 0 ? rd.filter(zd[r][k]) : 0.0f, ctx);
+              acc += weight_at(x0 + k, zt[r][k], ctx.mode == 0 ? zd[r][k] : 0.0f);
             const double tsum = warp_sum_double((double)acc);
             if (lane == 0) tile_sums[tile] = tsum;
           }
@@ -742,7 +791,7 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
           if (ctx.mode == 0) rd.load_tile(x0, V, a.vec_ok, zd);
 #pragma unroll
           for (int k = 0; k < VEC; ++k)
-            g[k] = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx);
+            g[k] = weight_at(x0 + k, zt[k], ctx.mode == 0 ? zd[k] : 0.0f);
           tok = pick_in_tile<VEC>(g, x0, sm.pick_prefix, (double)u * Z, lane);
         }
         if (lane == 0) sm.token = tok;
@@ -760,7 +809,7 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
 #pragma unroll
           for (int k = 0; k < VEC; ++k)
             if (x0 + k < V)
-              G_out[x0 + k] = weight_of(rt.filter(zt[k]), ctx.mode == 0 ? rd.filter(zd[k]) : 0.0f, ctx) * invZ;
+              G_out[x0 + k] = weight_at(x0 + k, zt[k], ctx.mode == 0 ? zd[k] : 0.0f) * invZ;
         }
       }
       break;

@@ -109,8 +109,9 @@ def test_chain_shaped_tree_equals_the_chain_entry_point():
     got = run_tree_gpu(w, want_G=False)
     out_t = torch.empty(B, L + 1, dtype=torch.int32, device=DEV)
     out_l = torch.empty(B, dtype=torch.int32, device=DEV)
-    prm = csd.make_params(w.target_logits, w.draft_logits[:, :L].contiguous(), w.draft_tokens, w.uniforms, w.relax_schedule,
-                          out_t, out_l, workspace=csd.new_workspace(B, L, V, w.dtype))
+    ws, chain_draft = csd.new_workspace(B, L, V, w.dtype), w.draft_logits[:, :L].contiguous()
+    prm = csd.make_params(w.target_logits, chain_draft, w.draft_tokens, w.uniforms, w.relax_schedule,
+                          out_t, out_l, workspace=ws)
     csd.csd_verify_ex(prm)
     torch.cuda.synchronize()
     assert np.array_equal(out_l.cpu().numpy(), got["accept_len"])
