@@ -360,6 +360,59 @@ size_t csd_tree_workspace_size(int B, int N, int V, int dtype);
 int csd_tree_depth(const int32_t* parent_host, int N);
 
 /*
+ * Vocabulary-sharded verification: the round for a tensor-parallel LM head, where each of n ranks
+ * holds a contiguous slice [v_offset, v_offset + Vs) of every logit row (Algorithm 1's steps are the
+ * same; only the three reductions over the vocabulary cross the ranks).  A rank calls, in order and on
+ * one stream,
+ *   csd_shard_stats    its slice's softmax statistics per row (Algorithm 1, "calculate P ... in
+ *                      parallel") and the logits of the drafted tokens that lie in the slice: one
+ *                      16-byte record per row, [B * (target_rows + gamma)] of them
+ *        -- all-gather the records, rank-major: records_all [n][rows] --
+ *   csd_shard_partial  the rows' global statistics, the accept tests and tau (Eq. relax; identical on
+ *                      every rank), then the slice's total of Eq. opt_G's weights at position tau + 1
+ *                      (and its share of P_j, which the fall-back of an empty positive part uses):
+ *                      out_totals [B][2] doubles; dbg_p / dbg_q / dbg_f [B, gamma] or NULL (written by
+ *                      the rank with shard == 0)
+ *        -- all-gather the totals: totals_all [n][B][2] --
+ *   csd_shard_pick     the slice holding the crossing C(x) > u Z picks the token (global id), the
+ *                      others report -1: out_candidates [B][2] int32 (token, status bits)
+ *        -- all-gather the candidates: candidates_all [n][B][2] --
+ *   csd_shard_emit     x_{1:tau+1}, tau and the status on every rank.
+ * The exchanges are the caller's (NCCL all-gather of a few KB each); the library never touches a
+ * peer's memory.  Slices must be numbered in vocabulary order (the inverse CDF runs in token-id
+ * order); they may have different sizes.  The workspace carries state from one of the four calls to
+ * the next.  Top-k filtering (its threshold is a k-th largest value over ALL slices) is not available
+ * in this form; the guidance mix is.  All pointers are DEVICE pointers.
+ */
+typedef struct csd_shard_params {
+  const void* target_logits; /* [B, target_rows, Vs]: this rank's slice */
+  const void* draft_logits;  /* [B, gamma, Vs]                          */
+  const void* target_uncond; /* same layouts, or both NULL              */
+  const void* draft_uncond;
+  float cfg_scale;
+  int32_t dtype;
+  int32_t B, gamma, target_rows;
+  int32_t Vs;                /* tokens in this slice                    */
+  int32_t V_total;           /* tokens in all slices                    */
+  int32_t v_offset;          /* global id of this slice's first token   */
+  int32_t n_shards, shard;   /* ranks, and this rank's index in vocabulary order */
+  const int32_t* draft_tokens;
+  const float* uniforms;
+  const float* relax_schedule;
+  void* workspace;           /* >= csd_shard_workspace_size(...) bytes, 256-byte aligned */
+  size_t workspace_bytes;
+  void* stream;
+} csd_shard_params;
+
+size_t csd_shard_workspace_size(int B, int gamma, int target_rows, int Vs, int dtype);
+int csd_shard_stats(const csd_shard_params* p, void* out_records);
+int csd_shard_partial(const csd_shard_params* p, const void* records_all, double* out_totals, float* dbg_p, float* dbg_q,
+                      float* dbg_f);
+int csd_shard_pick(const csd_shard_params* p, const void* records_all, const double* totals_all, int32_t* out_candidates);
+int csd_shard_emit(const csd_shard_params* p, const int32_t* candidates_all, int32_t* out_tokens, int32_t* out_accept_len,
+                   int32_t* out_status);
+
+/*
  * Relaxation schedules, written to HOST memory out_host[0..L-1] = omega_1..omega_L.
  *   kind 0  UniformRSD: omega_i = delta.
  *   kind 1  Cool-SD, Eq. sdar: omega_i = delta * exp(-nu*i - mu) with mu fixed by

@@ -23,7 +23,8 @@ CSD_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
 EXPORTS = ("csd_verify", "csd_verify_static", "csd_verify_ex", "csd_workspace_size", "csd_workspace_init", "csd_launch_count", "csd_verify_host",
            "csd_host_staging_size", "csd_make_schedule", "csd_error_string", "csd_version",
            "csd_sample_rows", "csd_sample_workspace_size", "csd_test_hooks",
-           "csd_verify_tree", "csd_tree_workspace_size", "csd_tree_depth", "csd_verify_similar")
+           "csd_verify_tree", "csd_tree_workspace_size", "csd_tree_depth", "csd_verify_similar",
+           "csd_shard_workspace_size", "csd_shard_stats", "csd_shard_partial", "csd_shard_pick", "csd_shard_emit")
 
 
 class CsdError(RuntimeError):

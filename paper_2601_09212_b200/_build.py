@@ -10,7 +10,7 @@ LIB_DIR = os.path.join(_HERE, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libcsd.so")
 SOURCES = [os.path.join(SRC_DIR, "csd_api.cu")]
 DEPENDS = SOURCES + [os.path.join(SRC_DIR, "csd_kernels.cuh"), os.path.join(SRC_DIR, "csd_fused.cuh"),
-                     os.path.join(SRC_DIR, "csd_tree.cuh"),
+                     os.path.join(SRC_DIR, "csd_tree.cuh"), os.path.join(SRC_DIR, "csd_shard.cuh"),
                      os.path.join(os.path.dirname(_HERE), "include", "csd.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]

@@ -12,6 +12,7 @@
 #include "csd_kernels.cuh"
 #include "csd_fused.cuh"
 #include "csd_tree.cuh"
+#include "csd_shard.cuh"
 
 namespace {
 
@@ -634,6 +635,194 @@ int csd_verify_tree(const csd_tree_params* pp) {
       e = cfg ? launch_tree_finish<__nv_bfloat16, true>(ta, stream) : launch_tree_finish<__nv_bfloat16, false>(ta, stream);
   }
   return e == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
+}
+
+// ---- vocabulary-sharded verification --------------------------------------------------------
+}  // extern "C"
+namespace {
+struct ShardLayout {
+  size_t parts, partials_off, tiles_off, ctx_off, total;
+  int U;
+};
+ShardLayout shard_layout(int B, int gamma, int T, int Vs, int dtype, bool cfg, int sms) {
+  ShardLayout l;
+  const int vw = vec_width(dtype);
+  const long long rows = (long long)B * (T + gamma);
+  int U = cfg ? 4 : 8;
+  auto parts_for = [&](int u) { return (Vs + kStatsThreads * u * vw - 1) / (kStatsThreads * u * vw); };
+  while (U > 1 && sms > 0 && rows * parts_for(U) < 4LL * sms) U >>= 1;
+  l.U = U;
+  l.parts = (size_t)parts_for(1);   // sized for the finest split, whatever the device
+  const size_t ntiles = ((size_t)Vs + 32 * vw - 1) / (32 * vw);
+  l.partials_off = 0;
+  l.tiles_off = align_up((size_t)rows * l.parts * sizeof(float2));
+  l.ctx_off = l.tiles_off + align_up((size_t)B * ntiles * sizeof(double));
+  l.total = l.ctx_off + align_up((size_t)B * 64);
+  return l;
+}
+
+int shard_check(const csd_shard_params& p) {
+  if (!p.target_logits || !p.draft_logits || !p.draft_tokens || !p.uniforms || !p.relax_schedule) return CSD_ERR_NULL;
+  if (p.dtype != CSD_F32 && p.dtype != CSD_BF16) return CSD_ERR_DTYPE;
+  if (p.B < 1 || p.gamma < 1 || p.gamma > kMaxGamma || p.Vs < 1 || p.Vs > kMaxV) return CSD_ERR_SHAPE;
+  if (p.target_rows != p.gamma && p.target_rows != p.gamma + 1) return CSD_ERR_SHAPE;
+  if (p.n_shards < 1 || p.n_shards > 1024 || p.shard < 0 || p.shard >= p.n_shards) return CSD_ERR_SHAPE;
+  if (p.v_offset < 0 || p.V_total < 2 || (long long)p.v_offset + p.Vs > p.V_total) return CSD_ERR_SHAPE;
+  if ((p.target_uncond == nullptr) != (p.draft_uncond == nullptr)) return CSD_ERR_ARG;
+  if (p.target_uncond && !isfinite(p.cfg_scale)) return CSD_ERR_ARG;
+  const ShardLayout lay = shard_layout(p.B, p.gamma, p.target_rows, p.Vs, p.dtype, p.target_uncond != nullptr, 0);
+  if (!p.workspace || ((uintptr_t)p.workspace % kAlign) != 0 || p.workspace_bytes < lay.total) return CSD_ERR_WORKSPACE;
+  return CSD_OK;
+}
+
+// the slice as the kernels see it
+void shard_args(const csd_shard_params& p, int sms, ShardArgs& sa, StatsArgs& st) {
+  const bool cfg = p.target_uncond != nullptr;
+  const ShardLayout lay = shard_layout(p.B, p.gamma, p.target_rows, p.Vs, p.dtype, cfg, sms);
+  const int es = elem_size(p.dtype), vw = vec_width(p.dtype);
+  auto aligned16 = [](const void* q) { return ((uintptr_t)q & 15u) == 0; };
+  const int64_t tstride = (int64_t)p.target_rows * p.Vs, dstride = (int64_t)p.gamma * p.Vs;
+  bool vec_ok = (p.Vs % vw) == 0 && (tstride * es) % 16 == 0 && (dstride * es) % 16 == 0 &&
+                aligned16(p.target_logits) && aligned16(p.draft_logits);
+  if (cfg) vec_ok = vec_ok && aligned16(p.target_uncond) && aligned16(p.draft_uncond);
+  char* ws = (char*)p.workspace;
+  memset(&sa, 0, sizeof sa);
+  FinishArgs& f = sa.fin;
+  f.target = p.target_logits; f.draft = p.draft_logits;
+  f.target_uncond = p.target_uncond; f.draft_uncond = p.draft_uncond;
+  f.cfg_scale = p.cfg_scale;
+  f.B = p.B; f.gamma = p.gamma; f.T = p.target_rows; f.V = p.Vs;
+  f.tstride = tstride; f.dstride = dstride;
+  f.parts = (p.Vs + kStatsThreads * lay.U * vw - 1) / (kStatsThreads * lay.U * vw);
+  f.vec_ok = vec_ok ? 1 : 0;
+  f.partials = reinterpret_cast<const float2*>(ws + lay.partials_off);
+  f.tokens = p.draft_tokens; f.uniforms = p.uniforms; f.schedule = p.relax_schedule;
+  sa.n_shards = p.n_shards; sa.shard = p.shard; sa.v_offset = p.v_offset; sa.V_total = p.V_total;
+  sa.tile_sums = reinterpret_cast<double*>(ws + lay.tiles_off);
+  sa.ctx = reinterpret_cast<float4*>(ws + lay.ctx_off);
+  st.target = p.target_logits; st.draft = p.draft_logits;
+  st.target_uncond = p.target_uncond; st.draft_uncond = p.draft_uncond;
+  st.cfg_scale = p.cfg_scale;
+  st.B = p.B; st.gamma = p.gamma; st.T = p.target_rows; st.V = p.Vs;
+  st.tstride = tstride; st.dstride = dstride;
+  st.parts = f.parts;
+  st.part_elems = kStatsThreads * lay.U * vw;
+  st.n_items = (int)((long long)p.B * (p.target_rows + p.gamma) * st.parts);
+  st.vec_ok = f.vec_ok;
+  st.partials = reinterpret_cast<float2*>(ws + lay.partials_off);
+  st.thresholds = nullptr;
+}
+
+template <typename K>
+cudaError_t launch_after(K kern, const ShardArgs& a, unsigned grid, unsigned block, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, a);
+}
+}  // namespace
+extern "C" {
+
+size_t csd_shard_workspace_size(int B, int gamma, int target_rows, int Vs, int dtype) {
+  if (B < 1 || gamma < 1 || gamma > kMaxGamma || Vs < 1 || Vs > kMaxV || (dtype != CSD_F32 && dtype != CSD_BF16)) return 0;
+  if (target_rows != gamma && target_rows != gamma + 1) return 0;
+  return shard_layout(B, gamma, target_rows, Vs, dtype, false, 0).total;
+}
+
+int csd_shard_stats(const csd_shard_params* pp, void* out_records) {
+  if (!pp || !out_records) return CSD_ERR_NULL;
+  const csd_shard_params& p = *pp;
+  const int rc = shard_check(p);
+  if (rc != CSD_OK) return rc;
+  const int sms = device_sms(nullptr);
+  if (sms <= 0) return CSD_ERR_LAUNCH;
+  ShardArgs sa; StatsArgs st;
+  shard_args(p, sms, sa, st);
+  sa.local = reinterpret_cast<float4*>(out_records);
+  const bool cfg = p.target_uncond != nullptr;
+  const int U = st.part_elems / (kStatsThreads * vec_width(p.dtype));
+  cudaStream_t stream = (cudaStream_t)p.stream;
+  const unsigned grid = (unsigned)((p.B * (p.target_rows + p.gamma) + 7) / 8);
+  cudaError_t e;
+  if (p.dtype == CSD_F32) {
+    e = cfg ? launch_stats_u<float, true>(st, U, false, sms, stream) : launch_stats_u<float, false>(st, U, false, sms, stream);
+    if (e == cudaSuccess)
+      e = cfg ? launch_after(shard_merge_kernel<float, true>, sa, grid, 256, stream)
+              : launch_after(shard_merge_kernel<float, false>, sa, grid, 256, stream);
+  } else {
+    e = cfg ? launch_stats_u<__nv_bfloat16, true>(st, U, false, sms, stream)
+            : launch_stats_u<__nv_bfloat16, false>(st, U, false, sms, stream);
+    if (e == cudaSuccess)
+      e = cfg ? launch_after(shard_merge_kernel<__nv_bfloat16, true>, sa, grid, 256, stream)
+              : launch_after(shard_merge_kernel<__nv_bfloat16, false>, sa, grid, 256, stream);
+  }
+  return e == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
+}
+
+int csd_shard_partial(const csd_shard_params* pp, const void* records_all, double* out_totals, float* dbg_p, float* dbg_q,
+                      float* dbg_f) {
+  if (!pp || !records_all || !out_totals) return CSD_ERR_NULL;
+  const csd_shard_params& p = *pp;
+  const int rc = shard_check(p);
+  if (rc != CSD_OK) return rc;
+  ShardArgs sa; StatsArgs st;
+  shard_args(p, device_sms(nullptr), sa, st);
+  sa.gathered = reinterpret_cast<const float4*>(records_all);
+  sa.z_local = out_totals;
+  sa.fin.dbg_p = dbg_p; sa.fin.dbg_q = dbg_q; sa.fin.dbg_f = dbg_f;
+  const bool cfg = p.target_uncond != nullptr;
+  cudaStream_t stream = (cudaStream_t)p.stream;
+  if (p.dtype == CSD_F32) {
+    if (cfg) shard_partial_kernel<float, true><<<p.B, kFinishThreads, 0, stream>>>(sa);
+    else shard_partial_kernel<float, false><<<p.B, kFinishThreads, 0, stream>>>(sa);
+  } else {
+    if (cfg) shard_partial_kernel<__nv_bfloat16, true><<<p.B, kFinishThreads, 0, stream>>>(sa);
+    else shard_partial_kernel<__nv_bfloat16, false><<<p.B, kFinishThreads, 0, stream>>>(sa);
+  }
+  return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
+}
+
+int csd_shard_pick(const csd_shard_params* pp, const void* records_all, const double* totals_all, int32_t* out_candidates) {
+  if (!pp || !records_all || !totals_all || !out_candidates) return CSD_ERR_NULL;
+  const csd_shard_params& p = *pp;
+  const int rc = shard_check(p);
+  if (rc != CSD_OK) return rc;
+  ShardArgs sa; StatsArgs st;
+  shard_args(p, device_sms(nullptr), sa, st);
+  sa.gathered = reinterpret_cast<const float4*>(records_all);
+  sa.z_all = totals_all;
+  sa.cand_local = out_candidates;
+  const bool cfg = p.target_uncond != nullptr;
+  cudaStream_t stream = (cudaStream_t)p.stream;
+  if (p.dtype == CSD_F32) {
+    if (cfg) shard_pick_kernel<float, true><<<p.B, kFinishThreads, 0, stream>>>(sa);
+    else shard_pick_kernel<float, false><<<p.B, kFinishThreads, 0, stream>>>(sa);
+  } else {
+    if (cfg) shard_pick_kernel<__nv_bfloat16, true><<<p.B, kFinishThreads, 0, stream>>>(sa);
+    else shard_pick_kernel<__nv_bfloat16, false><<<p.B, kFinishThreads, 0, stream>>>(sa);
+  }
+  return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
+}
+
+int csd_shard_emit(const csd_shard_params* pp, const int32_t* candidates_all, int32_t* out_tokens, int32_t* out_accept_len,
+                   int32_t* out_status) {
+  if (!pp || !candidates_all || !out_tokens || !out_accept_len) return CSD_ERR_NULL;
+  const csd_shard_params& p = *pp;
+  const int rc = shard_check(p);
+  if (rc != CSD_OK) return rc;
+  ShardArgs sa; StatsArgs st;
+  shard_args(p, device_sms(nullptr), sa, st);
+  sa.cand_all = candidates_all;
+  sa.fin.out_tokens = out_tokens; sa.fin.out_accept_len = out_accept_len; sa.fin.out_status = out_status;
+  shard_emit_kernel<<<p.B, 64, 0, (cudaStream_t)p.stream>>>(sa);
+  return cudaGetLastError() == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
 }
 
 // ---- allocation-free form -------------------------------------------------------------

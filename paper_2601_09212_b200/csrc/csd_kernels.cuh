@@ -471,7 +471,9 @@ __device__ __forceinline__ float weight_of(float zt, float zd, const PairCtx& c)
   const float et = ex2f((zt - c.Mt) * kLog2e);
   if (c.mode == 1) return et * c.inv_t;
   const float ed = ex2f((zd - c.Md) * kLog2e);
-  const float pq = ((et - ed) + (et * c.Sd - ed * c.St)) * c.inv_den;  // P - Q
+  // P - Q; written with the rounding intrinsics so that no product is contracted into a fused
+  // multiply-add: identical rows must give exactly 0 at every call site
+  const float pq = __fmul_rn(__fadd_rn(__fsub_rn(et, ed), __fsub_rn(__fmul_rn(et, c.Sd), __fmul_rn(ed, c.St))), c.inv_den);
   const float alt = c.one_minus_omega * et * c.inv_t;                    // (1 - omega) P
   return fmaxf(0.0f, fmaxf(pq, alt));
 }
@@ -497,7 +499,7 @@ __device__ __forceinline__ float neighbour_extra(const RowT& rt, const float Mt,
 // cancellation-free form of weight_of.
 __device__ __forceinline__ float weight_of_similar(float zt, float zd, const PairCtx& c, const float extra) {
   const float et = ex2f((zt - c.Mt) * kLog2e), ed = ex2f((zd - c.Md) * kLog2e);
-  const float pq = ((et - ed) + (et * c.Sd - ed * c.St)) * c.inv_den;
+  const float pq = __fmul_rn(__fadd_rn(__fsub_rn(et, ed), __fsub_rn(__fmul_rn(et, c.Sd), __fmul_rn(ed, c.St))), c.inv_den);
   const float P = et * c.inv_t, Q = ed / (1.0f + c.Sd);
   const float oa = (1.0f - c.one_minus_omega) * (P + extra);
   return oa >= Q ? fmaxf(0.0f, pq) : fmaxf(0.0f, P - oa);
@@ -545,15 +547,18 @@ struct FinishSmem {
 // qualifies (u >= 1 or NaN, or rounding), the last tile with positive mass -- the documented rule
 // "else the last token with positive weight".  Writes sm.Z, sm.pick_tile (-1: no tile has mass)
 // and sm.pick_prefix; every lane of the calling warp takes part.
+// With target_abs given, the crossing looked for is C(x) > *target_abs (a vocabulary shard's share of a
+// draw whose total is known from all shards) instead of u times this array's own total.
 __device__ __forceinline__ void locate_crossing_tile(const double* tile_sums, const int ntiles, const float u,
-                                                     const int lane, FinishSmem& sm) {
+                                                     const int lane, FinishSmem& sm,
+                                                     const double* target_abs = nullptr) {
   const int chunk = (ntiles + 31) / 32;
   const int t0 = min(ntiles, lane * chunk), t1 = min(ntiles, t0 + chunk);
   double local = 0.0;
   for (int t = t0; t < t1; ++t) local += tile_sums[t];
   const double incl = warp_incl_scan_double(local, lane);
   const double Z = __shfl_sync(0xffffffffu, incl, 31);
-  const double target = (double)u * Z;
+  const double target = target_abs ? *target_abs : (double)u * Z;
   const unsigned crossing = __ballot_sync(0xffffffffu, incl > target && local > 0.0);
   const unsigned has_mass = __ballot_sync(0xffffffffu, local > 0.0);
   if (lane == 0) { sm.Z = Z; sm.pick_tile = -1; sm.pick_prefix = 0.0; }
