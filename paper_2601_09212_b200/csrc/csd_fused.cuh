@@ -101,6 +101,12 @@ __device__ __forceinline__ void cluster_store(void* local, uint32_t rank, uint32
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_addr(local)), "r"(rank));
   asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"(v) : "memory");
 }
+// the same for a double
+__device__ __forceinline__ void cluster_store_f64(void* local, uint32_t rank, double v) {
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_addr(local)), "r"(rank));
+  asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(remote), "d"(v) : "memory");
+}
 constexpr int kMaxCluster = 8;   // portable cluster size
 
 template <typename T>
@@ -258,6 +264,8 @@ struct FinishStage {
   float mon_am[kMaxGamma], mon_bt[kMaxGamma];   // per-position monitors of Theorem 2, until they are written out
   SeqRecord rec;
   uint32_t xch[kMaxCluster];   // written by the blocks of the cluster: what each found (see finish_block)
+  uint32_t share[12];          // written by the block that draws, into every block of the cluster: what the
+                               // draw's weights need (see cluster_draw)
   alignas(8) uint64_t bar;
   alignas(8) uint64_t bar2;    // second copy barrier of the per-position monitors
 };
@@ -667,6 +675,141 @@ __device__ void emit_sequence(const FusedArgs& ua, const int b, const SeqRecord&
   }
 }
 
+// The draw of a sequence whose blocks form a cluster, shared by all of them.  The block that holds the
+// first rejection (or, with none, the bonus row) knows what the weights need -- the two rows'
+// statistics and thresholds, the multiplier -- and stores that into every block of the cluster; after
+// a cluster barrier each block sums Eq. opt_G over its share of the tiles of the two rows (read from
+// global memory: L2 hits) and stores the tile sums into the drawing block's shared memory; after a
+// second barrier that block locates the crossing, picks the token and leaves the record in st.rec.
+// Every block of the cluster calls this, with the same `owner`; a draw that turns out to have an empty
+// positive part is redone by the drawing block alone (draw_token).  What a block's own positions
+// contributed to the status is passed in `extra_status`.
+template <typename T, bool CFG, int NT, bool FILT>
+__device__ void cluster_draw(const FusedArgs& ua, const BlockShare& sh, int j, const int owner, const int tid,
+                             unsigned char* ring, const int ring_bytes, double* tile_sums, FinishSmem& sm,
+                             FinishStage& st, uint32_t& phase, const int extra_status) {
+  constexpr int VEC = Elem<T>::kVec;
+  constexpr int TILE = 32 * VEC;
+  const FinishArgs& a = ua.fin;
+  const int L = a.gamma, V = a.V, c = ua.ctas_per_seq;
+  const int b = sh.seq_begin;
+  const int lane = tid & 31, warp = tid >> 5;
+  const bool mine = owner == sh.slot;
+  // ---- the drawing block says what is drawn from ---------------------------------------------------
+  int status = extra_status & ~8;
+  bool rejected = false;
+  if (mine) {
+    rejected = j < sh.pos_end;
+    int draw = 0, mode = 1;
+    if (rejected) {
+      status |= sm.flag[j];
+      draw = sm.valid[0][j] != 0;
+      mode = sm.valid[1][j] ? 0 : 1;
+    } else if (sh.bonus) {
+      j = L;
+      draw = sm.valid[0][L] != 0;
+      if (!draw) status |= 1;
+    }
+    if (tid < c) {
+      const uint32_t rank = (uint32_t)tid;
+      const float omo = 1.0f - (j < L ? st.omega[j] : 0.0f);
+      cluster_store(&st.share[0], rank, (uint32_t)draw);
+      cluster_store(&st.share[1], rank, (uint32_t)mode);
+      cluster_store(&st.share[2], rank, (uint32_t)j);
+      cluster_store(&st.share[3], rank, __float_as_uint(sm.M[0][min(j, a.T - 1)]));
+      cluster_store(&st.share[4], rank, __float_as_uint(sm.S[0][min(j, a.T - 1)]));
+      cluster_store(&st.share[5], rank, __float_as_uint(j < L ? sm.M[1][j] : 0.0f));
+      cluster_store(&st.share[6], rank, __float_as_uint(j < L ? sm.S[1][j] : 0.0f));
+      cluster_store(&st.share[7], rank, __float_as_uint(sm.thr[0][min(j, a.T - 1)]));
+      cluster_store(&st.share[8], rank, __float_as_uint(j < L ? sm.thr[1][j] : CSD_NEG_INF));
+      cluster_store(&st.share[9], rank, __float_as_uint(omo));
+    }
+  }
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  // ---- every block: its share of the tile sums -----------------------------------------------------
+  const int draw = (int)st.share[0];
+  const int jj = (int)st.share[2];
+  PairCtx ctx;
+  ctx.mode = (int)st.share[1];
+  ctx.Mt = __uint_as_float(st.share[3]); ctx.St = __uint_as_float(st.share[4]);
+  ctx.Md = __uint_as_float(st.share[5]); ctx.Sd = __uint_as_float(st.share[6]);
+  ctx.inv_t = 1.0f / (1.0f + ctx.St);
+  ctx.inv_den = ctx.inv_t / (1.0f + ctx.Sd);
+  ctx.one_minus_omega = __uint_as_float(st.share[9]);
+  Row<T, CFG> rt = row_at<T, CFG>(a, b, 0, min(jj, a.T - 1));
+  Row<T, CFG> rd = rt;
+  rt.thr = __uint_as_float(st.share[7]);
+  if (jj < L) { rd = row_at<T, CFG>(a, b, 1, jj); rd.thr = __uint_as_float(st.share[8]); }
+  const int ntiles = (V + TILE - 1) / TILE;
+  if (draw) {
+    const int t_begin = (int)((long long)ntiles * sh.slot / c), t_end = (int)((long long)ntiles * (sh.slot + 1) / c);
+    for (int tile = t_begin + warp; tile < t_end; tile += NT / 32) {
+      const int x0 = tile * TILE + lane * VEC;
+      float zt[VEC], zd[VEC];
+      rt.load_tile(x0, V, 1, zt);
+      if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd);
+      float acc = 0.0f;
+#pragma unroll
+      for (int e = 0; e < VEC; ++e)
+        acc += weight_of(FILT ? rt.filter(zt[e]) : zt[e], ctx.mode == 0 ? (FILT ? rd.filter(zd[e]) : zd[e]) : 0.0f, ctx);
+#pragma unroll
+      for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+      if (lane == 0) cluster_store_f64(&tile_sums[tile], (uint32_t)owner, (double)acc);
+    }
+  }
+  __syncthreads();
+  cluster_arrive();
+  cluster_wait();
+  if (!mine) return;
+  // ---- the drawing block: locate, pick, record --------------------------------------------------------
+  int token = -1;
+  double Z = 0.0;
+  if (draw) {
+    const float u = st.uni[L];
+    if (warp == 0) locate_crossing_tile(tile_sums, ntiles, u, lane, sm);
+    __syncthreads();
+    Z = sm.Z;
+    if (!(Z > 0.0) || !(Z < (double)CSD_POS_INF)) {
+      // an empty positive part (or weights that overflowed): the draw is redone from scratch, alone
+      token = draw_token<T, CFG, NT, FILT>(a, rt, rd, ctx, u, tid, ring, ring_bytes, tile_sums, sm, st, phase, status, Z);
+    } else {
+      if (warp == 0) {
+        const int tile = sm.pick_tile;
+        int tok = -1;
+        if (tile >= 0) {
+          const int x0 = tile * TILE + lane * VEC;
+          float zt[VEC], zd[VEC], g[VEC];
+          rt.load_tile(x0, V, 1, zt);
+          if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd);
+#pragma unroll
+          for (int e = 0; e < VEC; ++e)
+            g[e] = weight_of(FILT ? rt.filter(zt[e]) : zt[e], ctx.mode == 0 ? (FILT ? rd.filter(zd[e]) : zd[e]) : 0.0f, ctx);
+          tok = pick_in_tile<VEC>(g, x0, sm.pick_prefix, (double)u * Z, lane);
+        }
+        if (lane == 0) sm.token = tok;
+      }
+      __syncthreads();
+      token = sm.token;
+    }
+  }
+  if (tid == 0) {
+    SeqRecord& rec = st.rec;
+    rec.first_rej = rejected ? jj : -1;
+    rec.token = token;
+    rec.status_at = status;
+    rec.status_any = extra_status & 8;
+    rec.mode = draw ? ctx.mode : 1;
+    rec.Mt = draw ? ctx.Mt : 0.0f; rec.St = draw ? ctx.St : 0.0f;
+    rec.Md = draw ? ctx.Md : 0.0f; rec.Sd = draw ? ctx.Sd : 0.0f;
+    rec.thr_t = rt.thr; rec.thr_d = rd.thr;
+    rec.one_minus_omega = draw ? ctx.one_minus_omega : 1.0f;
+    rec.Z = Z;
+  }
+  __syncthreads();
+}
+
 // Phase 2 of both kernels.  Entered by the whole block when its row statistics are complete in
 // shared memory.  Everything up to the griddepcontrol.wait reads only the call's inputs, so it runs
 // beside the previous call on the stream; after it come the few global writes.
@@ -674,9 +817,11 @@ __device__ void emit_sequence(const FusedArgs& ua, const int b, const SeqRecord&
 // With ctas_per_seq > 1 the blocks of a sequence form one cluster.  Each runs the accept tests of its
 // own positions and stores what it found -- its first rejection, if any -- into a word of every
 // peer's shared memory; after one cluster barrier every block knows which block holds the sequence's
-// first rejection (or that there is none: then the last block, which owns the bonus row).  That block
-// alone draws the token and emits the sequence; the others are done.  No block reads a peer's shared
-// memory, and none writes to it after the barrier, so blocks leave independently.
+// first rejection (or that there is none: then the last block, which owns the bonus row).  The draw
+// is shared (cluster_draw): that block publishes what the weights need, every block sums its share of
+// the tiles into that block's shared memory, and it alone picks the token and emits the sequence.  No
+// block reads a peer's shared memory, and none writes to it after the last barrier, so blocks leave
+// independently.
 template <typename T, bool CFG, int NT, bool FILT>
 __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const RowStats& rs, const int tid,
                              const bool aborted, unsigned char* ring, const int ring_bytes, double* tile_sums,
@@ -728,6 +873,8 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
     if (w & 1u) owner = k;
     if (w & 2u) any = 8;
   }
+  // the draw is shared by all blocks of the cluster
+  cluster_draw<T, CFG, NT, FILT>(ua, sh, j, owner, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
   if (owner != sh.slot) {   // another block decides the sequence
     if (a.dbg_p || a.dbg_q || a.dbg_f || want_terms) {
       if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase, phase2);
@@ -736,7 +883,6 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
     }
     return;
   }
-  draw_position<T, CFG, NT, FILT>(ua, sh, 0, j, tid, ring, ring_bytes, tile_sums, sm, st, phase, extra);
   if (want_terms) position_terms<T, CFG, NT, FILT>(a, sh, b, tid, ring, ring_bytes, tile_sums, sm, st, phase, phase2);
   pdl_wait();   // the previous call has completed: outputs of consecutive calls stay in order
   if (ua.error_flag && __ldcg(ua.error_flag)) any = 8;
