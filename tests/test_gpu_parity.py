@@ -590,8 +590,9 @@ def test_batch_strides_and_unaligned_views():
     big_d[:, :L * V] = w.draft_logits.reshape(B, -1)
     out_t = torch.empty(B, L + 1, dtype=torch.int32, device=DEV)
     out_l = torch.empty(B, dtype=torch.int32, device=DEV)
+    ws = csd.new_workspace(B, L, V, w.dtype)   # (held: the parameter block keeps raw pointers)
     prm = csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
-                          out_t, out_l, workspace=csd.new_workspace(B, L, V, w.dtype))
+                          out_t, out_l, workspace=ws)
     prm.target_logits = big_t.data_ptr()
     prm.draft_logits = big_d.data_ptr()
     prm.target_batch_stride = big_t.shape[1]
@@ -637,10 +638,11 @@ def test_seeded_sweep_of_batch_strides(i):
         out_t = torch.full((B, L + 1), -7, dtype=torch.int32, device=DEV)
         out_l = torch.full((B,), -7, dtype=torch.int32, device=DEV)
         out_s = torch.full((B,), -7, dtype=torch.int32, device=DEV)
+        ws = csd.new_workspace(B, L, V, w.dtype)   # (held: the parameter block keeps raw pointers)
         prm = csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
                               out_t, out_l, target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
                               cfg_scale=w.cfg_scale, top_k=w.top_k, out_status=out_s,
-                              workspace=csd.new_workspace(B, L, V, w.dtype), back_to_back=b2b)
+                              workspace=ws, back_to_back=b2b)
         prm.target_logits, prm.draft_logits = bt.data_ptr(), bd.data_ptr()
         if btu is not None:
             prm.target_uncond, prm.draft_uncond = btu.data_ptr(), bdu.data_ptr()
@@ -983,8 +985,9 @@ def test_argument_errors():
     w = W.make("t", B=2, gamma=2, V=64, schedule=sched(2), device=DEV)
     out_t = torch.empty(2, 3, dtype=torch.int32, device=DEV)
     out_l = torch.empty(2, dtype=torch.int32, device=DEV)
+    ws = csd.new_workspace(2, 2, 64, 0)
     prm = csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule,
-                          out_t, out_l, workspace=csd.new_workspace(2, 2, 64, 0))
+                          out_t, out_l, workspace=ws)
     lib = csd.library()
     import ctypes as C
     bad = csd.csd_params.from_buffer_copy(prm); bad.workspace_bytes = 16
