@@ -436,6 +436,18 @@ int csd_make_schedule(int kind, double delta, double nu_or_ell, int L, float* ou
  */
 int csd_test_hooks(int wait_limit_log2_cycles, int drop_first_copy);
 
+/*
+ * Testing aid: the library can be built with -DCSD_CHECKED (paper_2601_09212_b200/_build.py,
+ * build_checked_library), in which every element access of a logit row whose index comes from the
+ * data -- a drafted token, a neighbour id -- or from the row length is tested against the row's
+ * length first; a bad index is recorded and the access skipped, so nothing can fault.  This call
+ * synchronises the device and copies the record to HOST out_host[4]: number of bad indices seen since
+ * the library was loaded, the first one, the length it was tested against, and a site tag (1 vector
+ * load, 2 scalar load, 3 bulk copy into shared memory).  Returns 1 from a checked build, 0 from the normal build (whose record stays
+ * zero), or a negative csd_error.
+ */
+int csd_checked_report(int32_t* out_host);
+
 /* Static, NUL-terminated description of a csd_error value. */
 const char* csd_error_string(int code);
 

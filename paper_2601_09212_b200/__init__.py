@@ -8,6 +8,7 @@ has not been built, or no CUDA device is present, calls raise.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes as C
 import os
 from typing import Optional
@@ -22,7 +23,7 @@ CSD_STATUS_BADROW, CSD_STATUS_BADTOKEN, CSD_STATUS_ZFALLBACK, CSD_STATUS_TIMEOUT
 CSD_STATIC_SCRATCH_BYTES = 2 * 1024 * 1024
 EXPORTS = ("csd_verify", "csd_verify_static", "csd_verify_ex", "csd_workspace_size", "csd_workspace_init", "csd_launch_count", "csd_verify_host",
            "csd_host_staging_size", "csd_make_schedule", "csd_error_string", "csd_version",
-           "csd_sample_rows", "csd_sample_workspace_size", "csd_test_hooks",
+           "csd_sample_rows", "csd_sample_workspace_size", "csd_test_hooks", "csd_checked_report",
            "csd_verify_tree", "csd_tree_workspace_size", "csd_tree_depth", "csd_verify_similar",
            "csd_shard_workspace_size", "csd_shard_stats", "csd_shard_partial", "csd_shard_pick", "csd_shard_emit")
 
@@ -76,46 +77,76 @@ def library() -> C.CDLL:
             raise RuntimeError(
                 f"{LIB_PATH} is missing: build it with `python -m paper_2601_09212_b200._build` "
                 "(there is no fallback path)")
-        lib = C.CDLL(LIB_PATH)
-        lib.csd_verify.argtypes = [C.c_void_p] * 5 + [C.c_int] * 3 + [C.c_void_p] * 3
-        lib.csd_verify.restype = C.c_int
-        lib.csd_verify_static.argtypes = lib.csd_verify.argtypes
-        lib.csd_verify_static.restype = C.c_int
-        lib.csd_verify_ex.argtypes = [C.POINTER(csd_params)]
-        lib.csd_verify_ex.restype = C.c_int
-        lib.csd_workspace_size.argtypes = [C.c_int] * 4
-        lib.csd_workspace_size.restype = C.c_size_t
-        lib.csd_launch_count.argtypes = [C.POINTER(csd_params)]
-        lib.csd_launch_count.restype = C.c_int
-        lib.csd_workspace_init.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
-        lib.csd_workspace_init.restype = C.c_int
-        lib.csd_verify_host.argtypes = [C.POINTER(csd_params), C.c_void_p, C.c_size_t]
-        lib.csd_verify_host.restype = C.c_int
-        lib.csd_host_staging_size.argtypes = [C.POINTER(csd_params)]
-        lib.csd_host_staging_size.restype = C.c_size_t
-        lib.csd_make_schedule.argtypes = [C.c_int, C.c_double, C.c_double, C.c_int, C.c_void_p]
-        lib.csd_make_schedule.restype = C.c_int
-        lib.csd_error_string.argtypes = [C.c_int]
-        lib.csd_error_string.restype = C.c_char_p
-        lib.csd_version.restype = C.c_int
-        lib.csd_test_hooks.argtypes = [C.c_int, C.c_int]
-        lib.csd_test_hooks.restype = C.c_int
-        lib.csd_verify_similar.argtypes = [C.POINTER(csd_params), C.c_void_p, C.c_int, C.c_float]
-        lib.csd_verify_similar.restype = C.c_int
-        lib.csd_verify_tree.argtypes = [C.POINTER(csd_tree_params)]
-        lib.csd_verify_tree.restype = C.c_int
-        lib.csd_tree_workspace_size.argtypes = [C.c_int] * 4
-        lib.csd_tree_workspace_size.restype = C.c_size_t
-        lib.csd_tree_depth.argtypes = [C.c_void_p, C.c_int]
-        lib.csd_tree_depth.restype = C.c_int
-        lib.csd_sample_workspace_size.argtypes = [C.c_int] * 3
-        lib.csd_sample_workspace_size.restype = C.c_size_t
-        lib.csd_sample_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_int, C.c_int, C.c_int, C.c_int,
-                                        C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
-                                        C.c_int, C.c_void_p]
-        lib.csd_sample_rows.restype = C.c_int
-        _lib = lib
+        _lib = _configure(C.CDLL(LIB_PATH))
     return _lib
+
+
+def _configure(lib: C.CDLL) -> C.CDLL:
+    lib.csd_verify.argtypes = [C.c_void_p] * 5 + [C.c_int] * 3 + [C.c_void_p] * 3
+    lib.csd_verify.restype = C.c_int
+    lib.csd_verify_static.argtypes = lib.csd_verify.argtypes
+    lib.csd_verify_static.restype = C.c_int
+    lib.csd_verify_ex.argtypes = [C.POINTER(csd_params)]
+    lib.csd_verify_ex.restype = C.c_int
+    lib.csd_workspace_size.argtypes = [C.c_int] * 4
+    lib.csd_workspace_size.restype = C.c_size_t
+    lib.csd_launch_count.argtypes = [C.POINTER(csd_params)]
+    lib.csd_launch_count.restype = C.c_int
+    lib.csd_workspace_init.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.csd_workspace_init.restype = C.c_int
+    lib.csd_verify_host.argtypes = [C.POINTER(csd_params), C.c_void_p, C.c_size_t]
+    lib.csd_verify_host.restype = C.c_int
+    lib.csd_host_staging_size.argtypes = [C.POINTER(csd_params)]
+    lib.csd_host_staging_size.restype = C.c_size_t
+    lib.csd_make_schedule.argtypes = [C.c_int, C.c_double, C.c_double, C.c_int, C.c_void_p]
+    lib.csd_make_schedule.restype = C.c_int
+    lib.csd_error_string.argtypes = [C.c_int]
+    lib.csd_error_string.restype = C.c_char_p
+    lib.csd_version.restype = C.c_int
+    lib.csd_test_hooks.argtypes = [C.c_int, C.c_int]
+    lib.csd_test_hooks.restype = C.c_int
+    lib.csd_verify_similar.argtypes = [C.POINTER(csd_params), C.c_void_p, C.c_int, C.c_float]
+    lib.csd_verify_similar.restype = C.c_int
+    lib.csd_verify_tree.argtypes = [C.POINTER(csd_tree_params)]
+    lib.csd_verify_tree.restype = C.c_int
+    lib.csd_tree_workspace_size.argtypes = [C.c_int] * 4
+    lib.csd_tree_workspace_size.restype = C.c_size_t
+    lib.csd_tree_depth.argtypes = [C.c_void_p, C.c_int]
+    lib.csd_tree_depth.restype = C.c_int
+    lib.csd_sample_workspace_size.argtypes = [C.c_int] * 3
+    lib.csd_sample_workspace_size.restype = C.c_size_t
+    lib.csd_sample_rows.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_int, C.c_int, C.c_int, C.c_int,
+                                    C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                    C.c_int, C.c_void_p]
+    lib.csd_sample_rows.restype = C.c_int
+    lib.csd_checked_report.argtypes = [C.c_void_p]
+    lib.csd_checked_report.restype = C.c_int
+    return lib
+
+
+@contextlib.contextmanager
+def checked_library():
+    """Testing aid: inside the block every call of this module goes to the bounds-checked build of the
+    library (csd.h, csd_checked_report), compiled on first use.  Yields a function that returns the
+    record (bad indices seen, first index, row length, site) after synchronising the device."""
+    global _lib
+    from ._build import CHECKED_LIB_PATH, build_checked_library
+    if not os.path.exists(CHECKED_LIB_PATH):
+        build_checked_library()
+    lib = _configure(C.CDLL(CHECKED_LIB_PATH))
+
+    def report():
+        rec = (C.c_int32 * 4)()
+        rc = lib.csd_checked_report(rec)
+        if rc != 1:
+            raise CsdError(rc, "csd_checked_report") if rc < 0 else RuntimeError("not a checked build")
+        return tuple(rec)
+
+    before, _lib = library(), lib
+    try:
+        yield report
+    finally:
+        _lib = before
 
 
 def error_string(code: int) -> str:

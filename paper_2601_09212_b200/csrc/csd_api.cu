@@ -481,6 +481,18 @@ int csd_verify_similar(const csd_params* p, const int32_t* neighbours, int k, fl
   return verify_impl(*p, nullptr, false, false, sim);
 }
 
+int csd_checked_report(int32_t* out_host) {
+  if (!out_host) return CSD_ERR_NULL;
+  int32_t v[4] = {0, 0, 0, 0};
+  if (cudaMemcpyFromSymbol(v, g_checked, sizeof v) != cudaSuccess) return CSD_ERR_LAUNCH;
+  for (int k = 0; k < 4; ++k) out_host[k] = v[k];
+#ifdef CSD_CHECKED
+  return 1;
+#else
+  return 0;
+#endif
+}
+
 int csd_test_hooks(int wait_limit_log2_cycles, int drop_first_copy) {
   if (wait_limit_log2_cycles != 0 && (wait_limit_log2_cycles < 10 || wait_limit_log2_cycles > 40)) return CSD_ERR_ARG;
   g_wait_limit = wait_limit_log2_cycles ? (1ll << wait_limit_log2_cycles) : kWaitCycles;

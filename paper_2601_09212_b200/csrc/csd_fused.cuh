@@ -79,6 +79,15 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                "l"(src), "r"(bytes), "r"(smem_addr(bar))
                : "memory");
 }
+// the same for `bytes` of a logit row of V elements starting at element x0; the checked build tests the
+// range first and leaves a bad copy out (its wait then runs into the limit and reports TIMEOUT)
+template <typename T>
+__device__ __forceinline__ void bulk_load_row(void* dst, const T* row, int x0, uint32_t bytes, int V, uint64_t* bar) {
+#ifdef CSD_CHECKED
+  if (!checked_ok(x0, (int)(bytes / sizeof(T)), V, 3)) return;
+#endif
+  bulk_load(dst, row + x0, bytes, bar);
+}
 // orders this thread's earlier shared-memory accesses before a bulk copy it issues next
 __device__ __forceinline__ void fence_before_bulk() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -220,6 +229,9 @@ __device__ __forceinline__ Row<T, CFG> row_at(const FinishArgs& f, int b, int wh
   Row<T, CFG> row;
   row.scale = f.cfg_scale;
   row.thr = CSD_NEG_INF;
+#ifdef CSD_CHECKED
+  row.n = f.V;
+#endif
   if (which == 0) {
     const int64_t off = (int64_t)b * f.tstride + (int64_t)i * f.V;
     row.cond = reinterpret_cast<const T*>(f.target) + off;
@@ -298,11 +310,11 @@ __device__ int draw_token(const FinishArgs& a, const Row<T, CFG>& rt, const Row<
         fence_before_bulk();
         const uint32_t bytes = (uint32_t)(n * ES);
         mbar_expect_tx(&st.bar, bytes * n_arr);
-        bulk_load(ring, rt.cond + x0, bytes, &st.bar);
-        if (CFG) bulk_load(ring + slot_bytes, rt.uncond + x0, bytes, &st.bar);
+        bulk_load_row(ring, rt.cond, x0, bytes, V, &st.bar);
+        if (CFG) bulk_load_row(ring + slot_bytes, rt.uncond, x0, bytes, V, &st.bar);
         if (ctx.mode == 0) {
-          bulk_load(ring + ARR * slot_bytes, rd.cond + x0, bytes, &st.bar);
-          if (CFG) bulk_load(ring + (ARR + 1) * slot_bytes, rd.uncond + x0, bytes, &st.bar);
+          bulk_load_row(ring + ARR * slot_bytes, rd.cond, x0, bytes, V, &st.bar);
+          if (CFG) bulk_load_row(ring + (ARR + 1) * slot_bytes, rd.uncond, x0, bytes, V, &st.bar);
         }
       }
       if (!mbar_wait(&st.bar, phase)) status |= 8;
@@ -455,10 +467,10 @@ __device__ void position_terms(const FinishArgs& a, const BlockShare& sh, const 
     const Row<T, CFG> rt = row_at<T, CFG>(a, b, 0, i), rd = row_at<T, CFG>(a, b, 1, i);
     fence_before_bulk();
     mbar_expect_tx(bar, bytes * n_arr);
-    bulk_load(buf, rt.cond + x0, bytes, bar);
-    if (CFG) bulk_load(buf + slot_bytes, rt.uncond + x0, bytes, bar);
-    bulk_load(buf + ARR * slot_bytes, rd.cond + x0, bytes, bar);
-    if (CFG) bulk_load(buf + (ARR + 1) * slot_bytes, rd.uncond + x0, bytes, bar);
+    bulk_load_row(buf, rt.cond, x0, bytes, V, bar);
+    if (CFG) bulk_load_row(buf + slot_bytes, rt.uncond, x0, bytes, V, bar);
+    bulk_load_row(buf + ARR * slot_bytes, rd.cond, x0, bytes, V, bar);
+    if (CFG) bulk_load_row(buf + (ARR + 1) * slot_bytes, rd.uncond, x0, bytes, V, bar);
   };
   __syncthreads();   // everybody is done with what the ring held
   if (tid == 0 && njobs > 0) issue(0);
@@ -970,8 +982,8 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
     const uint32_t bytes = (uint32_t)(min(EPS, p_xend - p_x) * (int)sizeof(T));
     mbar_expect_tx(&sm.full[warp][p_s], bytes * ARR);
     if (!drop_next) {
-      bulk_load(&sm.ring[warp][p_s][0], p_cond + p_x, bytes, &sm.full[warp][p_s]);
-      if (CFG) bulk_load(&sm.ring[warp][p_s][kWStageBytes / 2], p_uncond + p_x, bytes, &sm.full[warp][p_s]);
+      bulk_load_row(&sm.ring[warp][p_s][0], p_cond, p_x, bytes, V, &sm.full[warp][p_s]);
+      if (CFG) bulk_load_row(&sm.ring[warp][p_s][kWStageBytes / 2], p_uncond, p_x, bytes, V, &sm.full[warp][p_s]);
     }
     drop_next = false;
     ++p_count;
@@ -1399,8 +1411,8 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
     mbar_expect_tx(&sm.full[s], bytes * ARR);
     atomicMax(&sm.issued_q, q + 1);
     if (q == 0 && a.drop_first_copy != 0 && blockIdx.x == 0) return;   // (test aid, see FusedArgs)
-    bulk_load(&sm.ring[s][0], row.cond + x0, bytes, &sm.full[s]);
-    if (CFG) bulk_load(&sm.ring[s][kTkStageBytes / 2], row.uncond + x0, bytes, &sm.full[s]);
+    bulk_load_row(&sm.ring[s][0], row.cond, x0, bytes, V, &sm.full[s]);
+    if (CFG) bulk_load_row(&sm.ring[s][kTkStageBytes / 2], row.uncond, x0, bytes, V, &sm.full[s]);
   };
   if (tid == 0) {
     issue_chunk(0);

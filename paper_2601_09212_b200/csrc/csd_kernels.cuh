@@ -98,6 +98,23 @@ __device__ __forceinline__ void stat_of_values(const float (&z)[N], float& m, fl
   s = acc + (float)(cnt - 1);
 }
 
+// ---- checked build ------------------------------------------------------------
+// With -DCSD_CHECKED every element access of a logit row whose index comes from the data (a drafted
+// token, a neighbour id) or from the row length is tested against the row's length first; a bad
+// index is recorded (count, first index, the length it was tested against, a site tag) and the access
+// is skipped (it reads -inf), so nothing can fault.  The normal build has none of this.
+__device__ int g_checked[4];
+#ifdef CSD_CHECKED
+#define CSD_ROW_LEN(len) , (len)
+__device__ __forceinline__ bool checked_ok(int idx, int width, int n, int site) {
+  if (idx >= 0 && idx + width <= n) return true;
+  if (atomicAdd(&g_checked[0], 1) == 0) { g_checked[1] = idx; g_checked[2] = n; g_checked[3] = site; }
+  return false;
+}
+#else
+#define CSD_ROW_LEN(len)
+#endif
+
 // ---- element access -----------------------------------------------------------
 template <typename T> struct Elem;
 template <> struct Elem<float> {
@@ -169,9 +186,19 @@ struct Row {
   const T* uncond;
   float scale;
   float thr;  // entries below thr become -inf (thr = -inf: no filter)
+#ifdef CSD_CHECKED
+  int n = 0x7fffffff;   // elements in the row (checked build only)
+#endif
   static constexpr int kVec = Elem<T>::kVec;
 
   __device__ __forceinline__ void load_vec(int x0, float (&z)[Elem<T>::kVec]) const {
+#ifdef CSD_CHECKED
+    if (!checked_ok(x0, kVec, n, 1)) {
+#pragma unroll
+      for (int k = 0; k < kVec; ++k) z[k] = CSD_NEG_INF;
+      return;
+    }
+#endif
     Elem<T>::load_vec(cond + x0, z);
     if (CFG) {
       float u[kVec];
@@ -180,6 +207,9 @@ struct Row {
     }
   }
   __device__ __forceinline__ float load_one(int x) const {
+#ifdef CSD_CHECKED
+    if (!checked_ok(x, 1, n, 2)) return CSD_NEG_INF;
+#endif
     float z = Elem<T>::load_one(cond + x);
     if (CFG) z = cfg_mix(z, Elem<T>::load_one(uncond + x), scale);
     return z;
@@ -236,6 +266,9 @@ __global__ void __launch_bounds__(kStatsThreads) row_stats_kernel(const StatsArg
     Row<T, CFG> row;
     row.scale = a.cfg_scale;
     row.thr = TOPK ? a.thresholds[row_id] : CSD_NEG_INF;
+#ifdef CSD_CHECKED
+    row.n = a.V;
+#endif
     if (r < a.T) {
       const int64_t off = (int64_t)b * a.tstride + (int64_t)r * a.V;
       row.cond = reinterpret_cast<const T*>(a.target) + off;
@@ -379,6 +412,9 @@ __global__ void __launch_bounds__(kSelectThreads) topk_threshold_kernel(const Se
     Row<T, CFG> row;
     row.scale = a.cfg_scale;
     row.thr = CSD_NEG_INF;
+#ifdef CSD_CHECKED
+    row.n = a.V;
+#endif
     if (r < a.T) {
       const int64_t off = (int64_t)b * a.tstride + (int64_t)r * a.V;
       row.cond = reinterpret_cast<const T*>(a.target) + off;
@@ -668,8 +704,8 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
         if (!t_ok || !d_ok) flag = 1;
         else if (!tok_ok) flag = 2;
         else {
-          Row<T, CFG> rt{tgt + (int64_t)i * V, CFG ? tgt_u + (int64_t)i * V : nullptr, a.cfg_scale, thr[0]};
-          Row<T, CFG> rd{dft + (int64_t)i * V, CFG ? dft_u + (int64_t)i * V : nullptr, a.cfg_scale, thr[1]};
+          Row<T, CFG> rt{tgt + (int64_t)i * V, CFG ? tgt_u + (int64_t)i * V : nullptr, a.cfg_scale, thr[0] CSD_ROW_LEN(V)};
+          Row<T, CFG> rd{dft + (int64_t)i * V, CFG ? dft_u + (int64_t)i * V : nullptr, a.cfg_scale, thr[1] CSD_ROW_LEN(V)};
           const float dt = rt.filter(rt.load_one(tok)) - M[0];
           const float dd = rd.filter(rd.load_one(tok)) - M[1];
           p = ex2f(dt * kLog2e) / (1.0f + S[0]);
@@ -726,9 +762,9 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
     float omega = j < L ? a.schedule[j] : 0.0f;
     omega = omega >= 0.0f ? omega : 0.0f;
     ctx.one_minus_omega = 1.0f - omega;
-    Row<T, CFG> rt{tgt + (int64_t)j * V, CFG ? tgt_u + (int64_t)j * V : nullptr, a.cfg_scale, sm.thr[0][j]};
+    Row<T, CFG> rt{tgt + (int64_t)j * V, CFG ? tgt_u + (int64_t)j * V : nullptr, a.cfg_scale, sm.thr[0][j] CSD_ROW_LEN(V)};
     Row<T, CFG> rd = rt;
-    if (j < L) rd = Row<T, CFG>{dft + (int64_t)j * V, CFG ? dft_u + (int64_t)j * V : nullptr, a.cfg_scale, sm.thr[1][j]};
+    if (j < L) rd = Row<T, CFG>{dft + (int64_t)j * V, CFG ? dft_u + (int64_t)j * V : nullptr, a.cfg_scale, sm.thr[1][j] CSD_ROW_LEN(V)};
     const float u = a.uniforms[(int64_t)b * (L + 1) + L];
     // (omega >= 1: the aggregated mass only raises f above f_van, and Eq. opt_G is the vanilla residual)
     const bool similar = a.nbr != nullptr && j < L && omega < 1.0f;
@@ -846,8 +882,8 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
         tc.inv_t = 1.0f / (1.0f + sm.S[0][i]); tc.inv_d = 1.0f / (1.0f + sm.S[1][i]);
         const float om = a.schedule[i];
         tc.omega = om >= 0.0f ? om : 0.0f;
-        const Row<T, CFG> rt{tgt + (int64_t)i * V, CFG ? tgt_u + (int64_t)i * V : nullptr, a.cfg_scale, sm.thr[0][i]};
-        const Row<T, CFG> rd{dft + (int64_t)i * V, CFG ? dft_u + (int64_t)i * V : nullptr, a.cfg_scale, sm.thr[1][i]};
+        const Row<T, CFG> rt{tgt + (int64_t)i * V, CFG ? tgt_u + (int64_t)i * V : nullptr, a.cfg_scale, sm.thr[0][i] CSD_ROW_LEN(V)};
+        const Row<T, CFG> rd{dft + (int64_t)i * V, CFG ? dft_u + (int64_t)i * V : nullptr, a.cfg_scale, sm.thr[1][i] CSD_ROW_LEN(V)};
         for (int tile = warp; tile < (V + TILE - 1) / TILE; tile += NT / 32) {
           const int x0 = tile * TILE + lane * VEC;
           float zt[VEC], zd[VEC];

@@ -63,7 +63,7 @@ __global__ void __launch_bounds__(256) shard_merge_kernel(const ShardArgs a) {
         const T* base = reinterpret_cast<const T*>(which == 0 ? f.target : f.draft);
         const T* ubase = CFG ? reinterpret_cast<const T*>(which == 0 ? f.target_uncond : f.draft_uncond) : nullptr;
         const int64_t off = (int64_t)b * (which == 0 ? f.tstride : f.dstride) + (int64_t)i * f.V;
-        Row<T, CFG> row{base + off, CFG ? ubase + off : nullptr, f.cfg_scale, CSD_NEG_INF};
+        Row<T, CFG> row{base + off, CFG ? ubase + off : nullptr, f.cfg_scale, CSD_NEG_INF CSD_ROW_LEN(f.V)};
         tokz = row.load_one(loc);
       }
     }
@@ -149,12 +149,12 @@ __device__ __forceinline__ void shard_rows(const FinishArgs& f, int b, int j, Ro
   const int jt = min(j, f.T - 1);
   const int64_t toff = (int64_t)b * f.tstride + (int64_t)jt * f.V;
   rt = Row<T, CFG>{reinterpret_cast<const T*>(f.target) + toff,
-                   CFG ? reinterpret_cast<const T*>(f.target_uncond) + toff : nullptr, f.cfg_scale, CSD_NEG_INF};
+                   CFG ? reinterpret_cast<const T*>(f.target_uncond) + toff : nullptr, f.cfg_scale, CSD_NEG_INF CSD_ROW_LEN(f.V)};
   rd = rt;
   if (j < f.gamma) {
     const int64_t doff = (int64_t)b * f.dstride + (int64_t)j * f.V;
     rd = Row<T, CFG>{reinterpret_cast<const T*>(f.draft) + doff,
-                     CFG ? reinterpret_cast<const T*>(f.draft_uncond) + doff : nullptr, f.cfg_scale, CSD_NEG_INF};
+                     CFG ? reinterpret_cast<const T*>(f.draft_uncond) + doff : nullptr, f.cfg_scale, CSD_NEG_INF CSD_ROW_LEN(f.V)};
   }
 }
 

@@ -106,8 +106,8 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
   float omega = 0.0f;
   for (;;) {
     const bool t_ok = sm.valid[0][ctx] != 0;
-    rt = Row<T, CFG>{tgt + (int64_t)ctx * V, CFG ? tgt_u + (int64_t)ctx * V : nullptr, f.cfg_scale, sm.thr[0][ctx]};
-    rd = Row<T, CFG>{dft + (int64_t)ctx * V, CFG ? dft_u + (int64_t)ctx * V : nullptr, f.cfg_scale, sm.thr[1][ctx]};
+    rt = Row<T, CFG>{tgt + (int64_t)ctx * V, CFG ? tgt_u + (int64_t)ctx * V : nullptr, f.cfg_scale, sm.thr[0][ctx] CSD_ROW_LEN(V)};
+    rd = Row<T, CFG>{dft + (int64_t)ctx * V, CFG ? dft_u + (int64_t)ctx * V : nullptr, f.cfg_scale, sm.thr[1][ctx] CSD_ROW_LEN(V)};
     pc.Mt = sm.M[0][ctx]; pc.St = sm.S[0][ctx];
     pc.inv_t = 1.0f / (1.0f + pc.St);
     int first_child = -1;
