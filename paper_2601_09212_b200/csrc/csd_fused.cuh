@@ -1427,10 +1427,11 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
     const uint32_t ring_mine = smem_addr(&sm.ring[0][0]) + (uint32_t)tid * 16u;
     const uint32_t list_mine = smem_addr(&sm.list[warp][0]);
     const uint32_t hist_addr = smem_addr(&sm.hist[0]);
+    const uint32_t lanemask_lt = (1u << lane) - 1u;
     for (int r = 0; r < n_rows; ++r) {
       const int par = r & 1;
       float lo = 0.0f, scale = 0.0f, dev = 0.0f;
-      if (lane == 0) sm.wpos[warp] = 0;
+      uint32_t wcur = 0;   // next free slot of the warp's list (may run past the capacity)
       reinterpret_cast<int2*>(sm.hist)[tid] = make_int2(0, 0);
       static_assert(kLinBins == 2 * kTopkThreads, "every thread clears two bins");
       for (int c = 0; c < cpr; ++c, ++q) {
@@ -1499,8 +1500,20 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         uint32_t mask = 0;
 #pragma unroll
         for (int e = 0; e < VPT; ++e) mask |= (z[e] < lo) ? 0u : (1u << e);
+        // slots: the warp's cursor lives in a register (the list is the warp's own); a lane's offset is
+        // the sum of the counts of the lanes below it, taken bit by bit from a few ballots
         const uint32_t cnt = (uint32_t)__popc(mask);
-        const uint32_t pos = (uint32_t)atom_add_shared(&sm.wpos[warp], (int)cnt);
+        uint32_t below = 0, total = 0;
+        constexpr int kCntBits = VPT <= 15 ? 4 : (VPT <= 31 ? 5 : 6);
+        static_assert(VPT <= 63, "a lane's count fits six bits");
+#pragma unroll
+        for (int bit = 0; bit < kCntBits; ++bit) {
+          const uint32_t bal = __ballot_sync(0xffffffffu, (cnt >> bit) & 1u);
+          below += (uint32_t)__popc(bal & lanemask_lt) << bit;
+          total += (uint32_t)__popc(bal) << bit;
+        }
+        const uint32_t pos = wcur + below;
+        wcur += total;
         if (pos + cnt <= (uint32_t)kWarpList) {
           uint32_t addr = list_mine + 4u * pos;
 #pragma unroll
@@ -1515,8 +1528,9 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
       // ---- first pass over this warp's list: maximum and histogram -----------------------------
       // (the row maximum is among the gathered values whenever the lists can be used).  The list is
       // padded with -inf to a whole number of 32 slots, so that the passes run without bounds tests.
+      if (lane == 0) sm.wpos[warp] = (int)wcur;   // (the warps that settle the row read every warp's count)
       __syncwarp();
-      const int wc = sm.wpos[warp];
+      const int wc = (int)wcur;
       int wcp = 0;   // padded length; 0 if the list overflowed (the row is then selected exactly)
       if (wc <= kWarpList) {
         wcp = (wc + 31) & ~31;
