@@ -1493,13 +1493,23 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         }
         // ---- gather this stage's values >= lo into the warp's list -------------------------
         // (the test is "not below lo", so that a NaN lands in the list and marks the row through the
-        // maximum).  Two predicated passes, free of branches: count, reserve the slots with one
-        // atomic, store.  Four independent chains (every fourth value each), so that neither the
-        // counts nor the addresses form one long dependent sequence.
-        // one bit per value, then the slots are reserved with one atomic and the flagged values stored
-        uint32_t mask = 0;
+        // maximum).  One bit per value in a mask, the slots from a prefix over the lanes' counts, then
+        // the flagged values are stored.
+        // (the bit is the sign of z - lo, taken two values per subtraction and shifted into the mask by a
+        // funnel shift: a NaN difference is the canonical, positive NaN, and x - x is +0, so both count
+        // as "not below")
+        uint32_t below_lo = 0;
+        {
+          const uint64_t nlo2 = pack2(-lo, -lo);
 #pragma unroll
-        for (int e = 0; e < VPT; ++e) mask |= (z[e] < lo) ? 0u : (1u << e);
+          for (int e = VPT - 2; e >= 0; e -= 2) {
+            float d0, d1;
+            unpack2(add2(pack2(z[e], z[e + 1]), nlo2), d0, d1);
+            below_lo = __funnelshift_l(__float_as_uint(d1), below_lo, 1);
+            below_lo = __funnelshift_l(__float_as_uint(d0), below_lo, 1);
+          }
+        }
+        const uint32_t mask = ~below_lo & (VPT == 32 ? 0xffffffffu : ((1u << (VPT & 31)) - 1u));
         // slots: the warp's cursor lives in a register (the list is the warp's own); a lane's offset is
         // the sum of the counts of the lanes below it, taken bit by bit from a few ballots
         const uint32_t cnt = (uint32_t)__popc(mask);

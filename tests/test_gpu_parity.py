@@ -654,6 +654,34 @@ def test_seeded_sweep_of_batch_strides(i):
         assert np.array_equal(out_s.cpu().numpy(), base["status"]), (pad, kw)
 
 
+@pytest.mark.parametrize("kw", [dict(dtype=W.BF16, cfg=True, top_k=1000), dict(dtype=W.F32, top_k=500),
+                                dict(dtype=W.BF16, top_k=700), dict(dtype=W.F32)])
+@pytest.mark.parametrize("b2b", [False, True])
+def test_nan_of_either_sign_marks_its_row(kw, b2b):
+    """A NaN with the sign bit set (0xFFC0... is as much a NaN as 0x7FC0...) must reach the row's
+    statistics like any other: the top-k gather tests values by the sign of a difference."""
+    B, L, V = 6, 4, 16384
+    w = W.make("t", B=B, gamma=L, V=V, rho=0.9, bonus_row=True, schedule=np.full(L, 1e6, np.float32), seed=11,
+               device=DEV, **kw)
+    neg_nan = torch.tensor([-1], dtype=torch.int32).view(torch.float32).item()   # all bits set: a negative NaN
+    assert neg_nan != neg_nan
+    def put(t, b, i, x):
+        if t.dtype == torch.bfloat16:
+            t.view(torch.int16)[b, i, x] = -64          # 0xFFC0
+        else:
+            t.view(torch.int32)[b, i, x] = -4194304     # 0xFFC00000
+    put(w.target_logits, 0, 1, 5)                       # in the first stage (the sample of the guess)
+    put(w.draft_logits, 1, 2, V - 3)                    # in the last stage
+    put(w.target_logits, 2, 0, V // 2 + 1)
+    if w.draft_uncond is not None:
+        put(w.draft_uncond, 3, 1, 9000)
+    rep, got, ref = check(w, back_to_back=b2b)
+    assert_ok(rep)
+    # (a drafted token outside the target's top-k rejects before the bad row is reached: the oracle says which)
+    assert np.array_equal(got["status"], ref.status) and np.array_equal(got["accept_len"], ref.accept_len)
+    assert got["status"][2] & 1 and got["accept_len"][2] == 0 and (ref.status[:4] & 1).sum() >= 2
+
+
 def test_bad_data_is_reported_not_trapped():
     B, L, V = 5, 3, 64
     w = W.make("t", B=B, gamma=L, V=V, rho=0.9, bonus_row=True, schedule=np.full(L, 1e6, np.float32),
