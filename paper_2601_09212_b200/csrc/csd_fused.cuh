@@ -1513,15 +1513,15 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         // slots: the warp's cursor lives in a register (the list is the warp's own); a lane's offset is
         // the sum of the counts of the lanes below it, taken bit by bit from a few ballots
         const uint32_t cnt = (uint32_t)__popc(mask);
-        uint32_t below = 0, total = 0;
+        uint32_t below = 0;
         constexpr int kCntBits = VPT <= 15 ? 4 : (VPT <= 31 ? 5 : 6);
         static_assert(VPT <= 63, "a lane's count fits six bits");
 #pragma unroll
         for (int bit = 0; bit < kCntBits; ++bit) {
           const uint32_t bal = __ballot_sync(0xffffffffu, (cnt >> bit) & 1u);
           below += (uint32_t)__popc(bal & lanemask_lt) << bit;
-          total += (uint32_t)__popc(bal) << bit;
         }
+        const uint32_t total = __reduce_add_sync(0xffffffffu, cnt);
         const uint32_t pos = wcur + below;
         wcur += total;
         if (pos + cnt <= (uint32_t)kWarpList) {
