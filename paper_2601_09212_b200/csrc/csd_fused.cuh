@@ -932,8 +932,7 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
   constexpr int EPS = kWStageBytes / ((int)sizeof(T) * ARR);   // elements of a row per warp stage
   constexpr int VPL = EPS / 32;                                // values per lane per stage
   constexpr int NVS = VPL / VEC;                               // 16-byte vectors per lane per stage
-  constexpr int GV = (NVS % 2 == 0) ? 2 : 1;                   // vectors reduced together (register budget)
-  static_assert(NVS % GV == 0 && NVS >= 1, "a stage is a whole number of groups");
+  static_assert(NVS >= 1, "a stage holds at least one vector per lane");
   extern __shared__ __align__(128) unsigned char fused_smem_raw[];
   PlainSmem& sm = *reinterpret_cast<PlainSmem*>(fused_smem_raw);
 
@@ -1032,85 +1031,119 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
         const int n = min(EPS, x_end - x0);
         const unsigned char* stage = &sm.ring[warp][c_s][0];
         const bool full = n == EPS;   // (after a timeout the data is garbage anyway: the call is flagged)
+        // The whole stage is one group: its values (packed bf16 pairs where nothing has to be mixed) sit
+        // in registers, one reduction gives the warp's largest, and since that result depends on every
+        // lane's loads the stage can be handed back for its refill before the exponentials are taken.
+        constexpr bool PACKED = !CFG && sizeof(T) == 2;
+        constexpr int NW = PACKED ? NVS * 4 : 1;
+        constexpr int NF = PACKED ? 1 : NVS * VEC;
+        uint32_t w[NW];
+        float vals[NF];
+        float gm;   // this lane's largest value of the stage
+        if (PACKED && full) {
 #pragma unroll
-        for (int g0 = 0; g0 < NVS; g0 += GV) {
-          float vals[GV * VEC];
-          float gm;   // this lane's largest value of the group
-          if (!CFG && sizeof(T) == 2 && full) {
-            // bf16, no mix: the maximum is taken on the packed pairs before unpacking
-            uint32_t w[GV * 4];
+          for (int v = 0; v < NVS; ++v) {
+            const uint4 q4 = *reinterpret_cast<const uint4*>(stage + (v * 32 + lane) * VEC * (int)sizeof(T));
+            w[(v * 4 + 0) % NW] = q4.x; w[(v * 4 + 1) % NW] = q4.y; w[(v * 4 + 2) % NW] = q4.z; w[(v * 4 + 3) % NW] = q4.w;
+          }
+          uint32_t m2[4] = {w[0], w[1 % NW], w[2 % NW], w[3 % NW]};
 #pragma unroll
-            for (int v = 0; v < GV; ++v) {
-              const uint4 q4 = *reinterpret_cast<const uint4*>(stage + ((g0 + v) * 32 + lane) * VEC * (int)sizeof(T));
-              w[v * 4 + 0] = q4.x; w[v * 4 + 1] = q4.y; w[v * 4 + 2] = q4.z; w[v * 4 + 3] = q4.w;
-            }
-            uint32_t m2 = w[0];
+          for (int k = 4; k < NW; ++k) asm("max.bf16x2 %0, %0, %1;" : "+r"(m2[k & 3]) : "r"(w[k]));
+          asm("max.bf16x2 %0, %0, %1;" : "+r"(m2[0]) : "r"(m2[1]));
+          asm("max.bf16x2 %0, %0, %1;" : "+r"(m2[2]) : "r"(m2[3]));
+          asm("max.bf16x2 %0, %0, %1;" : "+r"(m2[0]) : "r"(m2[2]));
+          gm = fmaxf(__uint_as_float(m2[0] << 16), __uint_as_float(m2[0] & 0xffff0000u));
+        } else if (PACKED) {
+          // ragged last stage of a packed row: out-of-range pairs read as -inf (0xff80 twice)
 #pragma unroll
-            for (int k = 1; k < GV * 4; ++k) asm("max.bf16x2 %0, %0, %1;" : "+r"(m2) : "r"(w[k]));
-            gm = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xffff0000u));
+          for (int v = 0; v < NVS; ++v) {
+            const int xo = (v * 32 + lane) * VEC;
+            uint4 q4 = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
+            if (xo < n) q4 = *reinterpret_cast<const uint4*>(stage + xo * (int)sizeof(T));
+            w[(v * 4 + 0) % NW] = q4.x; w[(v * 4 + 1) % NW] = q4.y; w[(v * 4 + 2) % NW] = q4.z; w[(v * 4 + 3) % NW] = q4.w;
+          }
+          uint32_t m2 = w[0];
 #pragma unroll
-            for (int k = 0; k < GV * 4; ++k) {
-              vals[2 * k] = __uint_as_float(w[k] << 16);
-              vals[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
-            }
-          } else {
+          for (int k = 1; k < NW; ++k) asm("max.bf16x2 %0, %0, %1;" : "+r"(m2) : "r"(w[k]));
+          gm = fmaxf(__uint_as_float(m2 << 16), __uint_as_float(m2 & 0xffff0000u));
+        } else {
 #pragma unroll
-            for (int v = 0; v < GV; ++v) {
-              const int xo = ((g0 + v) * 32 + lane) * VEC;
-              float zc[VEC];
-              if (full || xo < n) {
-                unpack_vec<T>(stage + xo * (int)sizeof(T), zc);
-                if (CFG) {
-                  float zu[VEC];
-                  unpack_vec<T>(stage + kWStageBytes / 2 + xo * (int)sizeof(T), zu);
-                  cfg_mix_vec<VEC>(zc, zu, f.cfg_scale);
-                }
-              } else {
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) zc[e] = CSD_NEG_INF;
+          for (int v = 0; v < NVS; ++v) {
+            const int xo = (v * 32 + lane) * VEC;
+            float zc[VEC];
+            if (full || xo < n) {
+              unpack_vec<T>(stage + xo * (int)sizeof(T), zc);
+              if (CFG) {
+                float zu[VEC];
+                unpack_vec<T>(stage + kWStageBytes / 2 + xo * (int)sizeof(T), zu);
+                cfg_mix_vec<VEC>(zc, zu, f.cfg_scale);
               }
+            } else {
 #pragma unroll
-              for (int e = 0; e < VEC; ++e) vals[v * VEC + e] = zc[e];
+              for (int e = 0; e < VEC; ++e) zc[e] = CSD_NEG_INF;
             }
-            float m4[4] = {CSD_NEG_INF, CSD_NEG_INF, CSD_NEG_INF, CSD_NEG_INF};
 #pragma unroll
-            for (int e = 0; e < GV * VEC; ++e) m4[e & 3] = fmaxf(m4[e & 3], vals[e]);
-            gm = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+            for (int e = 0; e < VEC; ++e) vals[(v * VEC + e) % NF] = zc[e];
           }
-          // the group's largest value over the warp (one integer reduction on order-preserving keys)
-          int key = __float_as_int(gm);
-          key ^= (key >> 31) & 0x7fffffff;
-          key = __reduce_max_sync(0xffffffffu, key);
-          key ^= (key >> 31) & 0x7fffffff;
-          const float wm = __int_as_float(key);
-          if (wm > Mw) {   // a new maximum: what was counted as "equal to the maximum" becomes ordinary mass
-            const float MwL = wm * kLog2e;
-            const float dlt_new = fmaf(wm, kLog2e, -MwL);
-            s_run = (s_run * ex2f(-dlt) + (float)cnt_run) * ex2f((Mw - wm) * kLog2e) * ex2f(dlt_new);
-            cnt_run = 0;
-            Mw = wm;
-            nMwL = -MwL;
-            dlt = dlt_new;
-          }
-          if (wm == Mw) {
-            // values equal to the reference may be present: they are counted, not summed
+          float m4[4] = {CSD_NEG_INF, CSD_NEG_INF, CSD_NEG_INF, CSD_NEG_INF};
 #pragma unroll
-            for (int e = 0; e < GV * VEC; ++e) {
-              const float ex = ex2f(fmaf(vals[e], kLog2e, nMwL));
-              if (vals[e] == Mw) cnt_run += 1; else s_run += ex;   // NaN values poison s_run, which marks the row
-            }
-          } else {
-            float acc4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-            for (int e = 0; e < GV * VEC; ++e) acc4[e & 3] += ex2f(fmaf(vals[e], kLog2e, nMwL));
-            s_run += (acc4[0] + acc4[1]) + (acc4[2] + acc4[3]);
-          }
+          for (int e = 0; e < NF; ++e) m4[e & 3] = fmaxf(m4[e & 3], vals[e]);
+          gm = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         }
-        __syncwarp();
-        if (lane == 0 && ok) {   // the stage is free again: refill it with the chunk kWStages ahead
+        // the stage's largest value over the warp (one integer reduction on order-preserving keys)
+        int key = __float_as_int(gm);
+        key ^= (key >> 31) & 0x7fffffff;
+        key = __reduce_max_sync(0xffffffffu, key);
+        key ^= (key >> 31) & 0x7fffffff;
+        const float wm = __int_as_float(key);
+        if (lane == 0 && ok) {   // every lane has read the stage: refill it with the chunk kWStages ahead
           fence_before_bulk();
           producer_issue();
         }
+        if (wm > Mw) {   // a new maximum: what was counted as "equal to the maximum" becomes ordinary mass
+          const float MwL = wm * kLog2e;
+          const float dlt_new = fmaf(wm, kLog2e, -MwL);
+          s_run = (s_run * ex2f(-dlt) + (float)cnt_run) * ex2f((Mw - wm) * kLog2e) * ex2f(dlt_new);
+          cnt_run = 0;
+          Mw = wm;
+          nMwL = -MwL;
+          dlt = dlt_new;
+        }
+        float acc4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (wm == Mw) {
+          // values equal to the reference may be present: they are counted, not summed (branch-free:
+          // the exponential of such a value is replaced by 0)
+          int c4[4] = {0, 0, 0, 0};
+          if (PACKED) {
+#pragma unroll
+            for (int k = 0; k < NW; ++k) {
+              const float v0 = __uint_as_float(w[k] << 16), v1 = __uint_as_float(w[k] & 0xffff0000u);
+              const float e0 = ex2f(fmaf(v0, kLog2e, nMwL)), e1 = ex2f(fmaf(v1, kLog2e, nMwL));
+              acc4[(2 * k) & 3] += v0 == Mw ? 0.0f : e0;       // NaN values poison the sum, which marks the row
+              acc4[(2 * k + 1) & 3] += v1 == Mw ? 0.0f : e1;
+              c4[(2 * k) & 3] += v0 == Mw ? 1 : 0;
+              c4[(2 * k + 1) & 3] += v1 == Mw ? 1 : 0;
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < NF; ++e) {
+              const float ex = ex2f(fmaf(vals[e], kLog2e, nMwL));
+              acc4[e & 3] += vals[e] == Mw ? 0.0f : ex;
+              c4[e & 3] += vals[e] == Mw ? 1 : 0;
+            }
+          }
+          cnt_run += (c4[0] + c4[1]) + (c4[2] + c4[3]);
+        } else if (PACKED) {
+#pragma unroll
+          for (int k = 0; k < NW; ++k) {
+            acc4[(2 * k) & 3] += ex2f(fmaf(__uint_as_float(w[k] << 16), kLog2e, nMwL));
+            acc4[(2 * k + 1) & 3] += ex2f(fmaf(__uint_as_float(w[k] & 0xffff0000u), kLog2e, nMwL));
+          }
+        } else {
+#pragma unroll
+          for (int e = 0; e < NF; ++e) acc4[e & 3] += ex2f(fmaf(vals[e], kLog2e, nMwL));
+        }
+        s_run += (acc4[0] + acc4[1]) + (acc4[2] + acc4[3]);
         if (++c_s == kWStages) { c_s = 0; c_par ^= 1u; }
       }
       // the item's pair: m = Mw, s = sum over everything except one entry at the maximum
