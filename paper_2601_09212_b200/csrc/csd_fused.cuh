@@ -1022,7 +1022,8 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
       // the ROUNDED product Mw * log2(e); its rounding error dlt = Mw * log2(e) - MwL (exact, again by
       // a fused multiply-add) is a common factor 2^dlt of the sum and is divided out once per item.
       float Mw = CSD_NEG_INF, s_run = 0.0f;
-      float nMwL = CSD_POS_INF, dlt = 0.0f;   // -MwL and dlt of the current reference
+      float nMwL = 0.0f, dlt = 0.0f;   // -MwL and dlt of the current reference (while Mw is -inf every value is
+                                       // -inf or NaN, and with 0 here its exponential is 0 or NaN as it should be)
       int cnt_run = 0;
       for (int x0 = x_begin; x0 < x_end; x0 += EPS) {
         if (ok) {
@@ -1110,35 +1111,41 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
           dlt = dlt_new;
         }
         float acc4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if (wm == Mw) {
-          // values equal to the reference may be present: they are counted, not summed (branch-free:
-          // the exponential of such a value is replaced by 0)
-          int c4[4] = {0, 0, 0, 0};
-          if (PACKED) {
+        if (PACKED) {
+          if (wm == Mw) {
+            // values equal to the reference may be present: they are counted, not summed.  On the packed
+            // pairs: one compare per pair marks them, the marked halves become -inf (their exponential is
+            // then exactly 0) and are counted, 16 bits of the counter per half.
+            const uint32_t m16 = __float_as_uint(Mw) >> 16;
+            const uint32_t Mw2 = m16 | (m16 << 16);
+            uint32_t c2 = 0;
 #pragma unroll
-            for (int k = 0; k < NW; ++k) {
-              const float v0 = __uint_as_float(w[k] << 16), v1 = __uint_as_float(w[k] & 0xffff0000u);
-              const float e0 = ex2f(fmaf(v0, kLog2e, nMwL)), e1 = ex2f(fmaf(v1, kLog2e, nMwL));
-              acc4[(2 * k) & 3] += v0 == Mw ? 0.0f : e0;       // NaN values poison the sum, which marks the row
-              acc4[(2 * k + 1) & 3] += v1 == Mw ? 0.0f : e1;
-              c4[(2 * k) & 3] += v0 == Mw ? 1 : 0;
-              c4[(2 * k + 1) & 3] += v1 == Mw ? 1 : 0;
+            for (int k = 0; k < NW; k += 2) {
+              uint32_t e0, e1;
+              asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(e0) : "r"(w[k]), "r"(Mw2));
+              asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(e1) : "r"(w[(k + 1) % NW]), "r"(Mw2));
+              w[k] = (w[k] & ~e0) | (0xff80ff80u & e0);
+              w[(k + 1) % NW] = (w[(k + 1) % NW] & ~e1) | (0xff80ff80u & e1);
+              c2 += (e0 & 0x00010001u) + (e1 & 0x00010001u);
             }
-          } else {
-#pragma unroll
-            for (int e = 0; e < NF; ++e) {
-              const float ex = ex2f(fmaf(vals[e], kLog2e, nMwL));
-              acc4[e & 3] += vals[e] == Mw ? 0.0f : ex;
-              c4[e & 3] += vals[e] == Mw ? 1 : 0;
-            }
+            static_assert(NW % 2 == 0 || NW == 1, "pairs of words");
+            cnt_run += (int)((c2 & 0xffffu) + (c2 >> 16));
           }
-          cnt_run += (c4[0] + c4[1]) + (c4[2] + c4[3]);
-        } else if (PACKED) {
 #pragma unroll
           for (int k = 0; k < NW; ++k) {
-            acc4[(2 * k) & 3] += ex2f(fmaf(__uint_as_float(w[k] << 16), kLog2e, nMwL));
-            acc4[(2 * k + 1) & 3] += ex2f(fmaf(__uint_as_float(w[k] & 0xffff0000u), kLog2e, nMwL));
+            acc4[(2 * k) & 3] += ex2f(fmaf(__uint_as_float(w[k] << 16), kLog2e, nMwL));   // NaN values poison the sum,
+            acc4[(2 * k + 1) & 3] += ex2f(fmaf(__uint_as_float(w[k] & 0xffff0000u), kLog2e, nMwL));   // which marks the row
           }
+        } else if (wm == Mw) {
+          // (branch-free: the exponential of a value equal to the reference is replaced by 0)
+          int c4[4] = {0, 0, 0, 0};
+#pragma unroll
+          for (int e = 0; e < NF; ++e) {
+            const float ex = ex2f(fmaf(vals[e], kLog2e, nMwL));
+            acc4[e & 3] += vals[e] == Mw ? 0.0f : ex;
+            c4[e & 3] += vals[e] == Mw ? 1 : 0;
+          }
+          cnt_run += (c4[0] + c4[1]) + (c4[2] + c4[3]);
         } else {
 #pragma unroll
           for (int e = 0; e < NF; ++e) acc4[e & 3] += ex2f(fmaf(vals[e], kLog2e, nMwL));
