@@ -353,10 +353,32 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
       const int eps = kWStageBytes / (es * (cfg ? 2 : 1));
       const long long cpr = (p.V + eps - 1) / eps;
       const long long blocks = c > 1 ? (long long)p.B * c : (p.B + spc - 1) / spc;
-      long long cpp = 2 * rows * cpr / (5 * blocks * kPlainWarps);   // about 2.5 items per warp
-      if (cpp < 1) cpp = 1;
-      if (cpp > 8) cpp = 8;
-      if (cpp > cpr) cpp = cpr;
+      // A row is cut into 1 ... 16 parts; the choice minimises the work of the block's busiest warp
+      // (its items are a contiguous eighth of the block's items; an item costs its stages plus about
+      // half a stage of fixed work).  Long items are better for their own sake -- fewer changes of
+      // the running maximum, fewer reductions -- so ties go to the fewer parts.
+      const long long rows_b = (c > 1) ? (2LL * ((p.gamma + c - 1) / c) + 1) : spc * rows_per_seq;
+      long long cpp = cpr;
+      double best = -1.0;
+      for (long long np = 1; np <= 16 && np <= cpr; ++np) {
+        const long long cand = (cpr + np - 1) / np;          // stages per part
+        const long long parts = (cpr + cand - 1) / cand;
+        if (parts != np && np > 1) continue;                 // (the same cut as a smaller np)
+        const long long n = rows_b * parts;
+        const long long last = cpr - (parts - 1) * cand;      // stages of a row's last part
+        double worst = 0.0;
+        for (int w = 0; w < kPlainWarps; ++w) {
+          const long long b0 = n * w / kPlainWarps, b1 = n * (w + 1) / kPlainWarps;
+          // items b0 .. b1-1; item i is part i % parts of its row
+          const long long full_rows = (b1 - b0) / parts;
+          double load = (double)full_rows * ((double)cpr + 0.5 * (double)parts);
+          for (long long i = b0 + full_rows * parts; i < b1; ++i)
+            load += (double)((i % parts == parts - 1) ? last : cand) + 0.5;
+          if (load > worst) worst = load;
+        }
+        if (best < 0.0 || worst < best * 0.97) { best = worst; cpp = cand; }
+      }
+      (void)blocks;
       // a block keeps one stash entry per item
       for (;;) {
         const long long parts = (cpr + cpp - 1) / cpp;

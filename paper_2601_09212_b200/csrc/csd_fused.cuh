@@ -964,7 +964,8 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
   int p_count = 0;   // chunks announced to the barriers so far
   int p_row = item_begin / parts, p_part = item_begin - p_row * parts;   // kept incrementally from here on
   const T *p_cond = nullptr, *p_uncond = nullptr;
-  bool drop_next = a.drop_first_copy != 0 && blockIdx.x == 0 && warp == 0;   // (test aid, see FusedArgs)
+  // (test aid, see FusedArgs: the warp that owns the block's first item)
+  bool drop_next = a.drop_first_copy != 0 && blockIdx.x == 0 && item_begin == 0 && item_end > 0;
   auto producer_open_row = [&]() {    // pointers of row p_row
     int b, which, i;
     local_row(sh, p_row, f.gamma, b, which, i);
