@@ -549,6 +549,130 @@ def run_drafting_stage(args) -> None:
     }))
 
 
+def run_widened(args) -> None:
+    """Side measurements (not the headline) of the widened entry points on the workload's shapes: tree
+    verification (csd_verify_tree, a static 4-3-2-2 tree), similarity-relaxed acceptance
+    (csd_verify_similar, k = 10 neighbours, lambda = 2) and one rank's four calls of the
+    vocabulary-sharded round (csd_shard_*, with the whole vocabulary or a quarter of it as the slice;
+    the all-gathers are replaced by views of the rank's own buffers, so this is kernel time only).
+    Timed like the round: resident inputs larger than L2, a CUDA graph of calls replayed, CUDA events on
+    the launching stream, calls in stream order.  One GPU."""
+    import numpy as np
+    import torch
+    from paper_2601_09212_b200 import _build, workloads as W
+    import paper_2601_09212_b200 as csd
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    _build.build_library()
+    kind, name = args.widened, args.workload
+    kw = workload_kwargs(name)
+    B, L, V, dtype = kw["B"], kw["gamma"], kw["V"], kw.get("dtype", W.F32)
+    es = 2 if dtype == W.BF16 else 4
+    arrays = 2 if kw.get("cfg") else 1
+    stream = torch.cuda.Stream(device=dev)
+    keep = []
+    if kind == "tree":
+        parent = W.static_tree([4, 3, 2, 2])
+        N, D = len(parent), csd.csd_tree_depth(parent)
+        sched = csd.csd_make_schedule(1, 1.1, 0.7, D)
+        step_bytes = 2 * arrays * (N + 1) * V * es * B
+        units, unit_name, op = B * N, "verified_tree_nodes_per_sec", f"csd_verify_tree, static tree 4-3-2-2 ({N} nodes, depth {D})"
+        ring_n = max(2, -(-2 * L2_BYTES // step_bytes))
+        tkw = {k: v for k, v in kw.items() if k not in ("B", "gamma", "V", "bonus_row")}
+        for s_ in range(ring_n):
+            w = W.make_tree(parent, B=B, V=V, schedule=sched, seed=1, step=s_, device=dev, **tkw)
+            out = (torch.empty(B, D + 1, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev))
+            ws = torch.zeros(csd.csd_tree_workspace_size(B, N, V, dtype), dtype=torch.uint8, device=dev)
+            keep.append((w, out, ws))
+
+        def enqueue(i):
+            w, out, ws = keep[i % ring_n]
+            csd.csd_verify_tree(w.target_logits, w.draft_logits, w.parent, w.draft_tokens, w.uniforms, w.relax_schedule,
+                                out[0], out[1], target_uncond=w.target_uncond, draft_uncond=w.draft_uncond,
+                                cfg_scale=w.cfg_scale, top_k=w.top_k, workspace=ws, stream=stream)
+
+    elif kind == "similar":
+        sched = csd.csd_make_schedule(1, 1.1, 0.7, L)
+        step_bytes = algorithmic_bytes(kw)
+        units, unit_name, op = B * L, "verified_draft_tokens_per_sec", "csd_verify_similar, k = 10 neighbours, lambda = 2"
+        ring_n = max(2, -(-2 * L2_BYTES // step_bytes))
+        r = np.random.default_rng(5)
+        nb = ((np.arange(V)[:, None] + 1 + r.integers(0, V - 1, size=(V, 10))) % V).astype(np.int32)   # never the token itself
+        table = torch.from_numpy(nb).to(dev)
+        for s_ in range(ring_n):
+            w = W.make(name, seed=1, step=s_, schedule=sched, device=dev, **kw)
+            out = (torch.empty(B, L + 1, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev))
+            ws = csd.new_workspace(B, L, V, dtype, dev)
+            prm = csd.make_params(w.target_logits, w.draft_logits, w.draft_tokens, w.uniforms, w.relax_schedule, out[0], out[1],
+                                  target_uncond=w.target_uncond, draft_uncond=w.draft_uncond, cfg_scale=w.cfg_scale,
+                                  top_k=w.top_k, workspace=ws, stream=stream)
+            keep.append((w, out, ws, prm))
+
+        def enqueue(i):
+            csd.csd_verify_similar(keep[i % ring_n][3], table, 2.0)
+    else:
+        from paper_2601_09212_b200.vocab_sharded import ShardedRound, csd_verify_sharded
+        n_sh = 4 if kind == "sharded4" else 1
+        Vs = V // n_sh
+        sched = csd.csd_make_schedule(1, 1.1, 0.7, L)
+        step_bytes = 2 * arrays * L * Vs * es * B
+        units, unit_name = B * L, "verified_draft_tokens_per_sec"
+        op = f"csd_shard_stats/partial/pick/emit on one rank's slice of {Vs} of {V} tokens ({n_sh} slices; gathers are views)"
+        ring_n = max(2, -(-2 * L2_BYTES // step_bytes))
+        skw = {k: v for k, v in kw.items() if k != "top_k"}   # (top-k is not part of the sharded round)
+        for s_ in range(ring_n):
+            w = W.make(name, seed=1, step=s_, schedule=sched, device=dev, **skw)
+            cut = lambda t: None if t is None else t[:, :, :Vs].contiguous()
+            rd = ShardedRound(cut(w.target_logits), cut(w.draft_logits), w.draft_tokens, w.uniforms, w.relax_schedule,
+                              v_offset=0, V_total=V, shard=0, n_shards=n_sh, target_uncond=cut(w.target_uncond),
+                              draft_uncond=cut(w.draft_uncond), cfg_scale=w.cfg_scale, stream=stream)
+            out = (torch.empty(B, L + 1, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.int32, device=dev))
+            keep.append((w, rd, out))
+        # every "rank" of the stand-in gather holds this rank's buffer: shapes and kernels are those of n_sh ranks
+        gather = lambda t: t.unsqueeze(0).expand((n_sh,) + tuple(t.shape)).contiguous() if n_sh > 1 else t.unsqueeze(0)
+
+        def enqueue(i):
+            _, rd, out = keep[i % ring_n]
+            csd_verify_sharded(rd, out[0], out[1], gather=gather)
+
+    graph_steps = ring_n * max(1, -(-32 // ring_n))
+    with torch.cuda.stream(stream):
+        for i in range(ring_n):
+            enqueue(i)
+    stream.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        for i in range(graph_steps):
+            enqueue(i)
+    replays = max(1, min(args.steps, 512) // graph_steps)
+    with torch.cuda.stream(stream):
+        graph.replay()
+    stream.synchronize()
+    reps = []
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _r in range(replays):
+                graph.replay()
+            e1.record(stream)
+        stream.synchronize()
+        reps.append(e0.elapsed_time(e1))
+    reps.sort()
+    steps = replays * graph_steps
+    ms = reps[len(reps) // 2]
+    peak, peak_kind = measured_peak()
+    achieved = step_bytes / (ms * 1e-3 / steps) / 1e9
+    print(json.dumps({
+        "metric": unit_name, "value": units * steps / (ms * 1e-3), "unit": "1/s", "n_gpus": 1,
+        "steps": steps, "reps": len(reps), "ms_per_step": ms / steps, "higher_is_better": True, "data": "synthetic",
+        "config": dict(describe(name, kw, "exp delta=1.1 nu=0.7"), op=op,
+                       launch=f"CUDA graph of {graph_steps} calls in stream order, {replays} replays, median of {len(reps)}"),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": peak_kind, "bytes_per_launch": step_bytes, "traffic": None},
+    }))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -563,9 +687,13 @@ def main() -> None:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--drafting-stage", action="store_true",
                     help="side measurement: time csd_sample_rows on the workload's drafter rows instead of the round")
+    ap.add_argument("--widened", default=None, choices=["tree", "similar", "sharded", "sharded4"],
+                    help="side measurement of a widened entry point on the workload's shapes (see run_widened)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.widened:
+        run_widened(args)
     elif args.drafting_stage:
         run_drafting_stage(args)
     else:

@@ -200,6 +200,130 @@ cudaError_t launch_finish(const FinishArgs& a, cudaStream_t stream) {
 long long g_wait_limit = kWaitCycles;
 int g_drop_first_copy = 0;
 
+// The single-launch path's partition and launch (see the comments inside).  With stats_out set the
+// kernels stop after their streaming phase and write every row's (m, s) -- and, with top-k, its exact
+// threshold -- to global memory in the row order of the multi-launch kernels (one part per row), for a
+// finishing kernel of that path to consume (tree drafts, the similarity relaxation).
+struct FusedPlan {
+  FinishArgs fa;
+  int B, gamma, V, top_k, dtype;
+  int rows_per_seq;
+  long long rows;
+  int sms, es;
+  bool cfg, topk, back_to_back, allow_short_cut;
+  int* error_flag;
+  float2* stats_out;
+  float* thr_out;
+  cudaStream_t stream;
+};
+cudaError_t plan_and_launch_fused(const FusedPlan& in) {
+  const int sms = in.sms, es = in.es, rows_per_seq = in.rows_per_seq;
+  const long long rows = in.rows;
+  const bool cfg = in.cfg, topk = in.topk;
+  cudaStream_t stream = in.stream;
+  {
+    FusedArgs ua;
+    ua.fin = in.fa;
+    ua.top_k = in.top_k;
+    ua.lo_sigmas = nanf("");
+    ua.lo_delta = 0.0f;
+    ua.hi_delta = nanf("");
+    ua.error_flag = in.error_flag;
+    ua.stats_out = in.stats_out;
+    ua.thr_out = in.thr_out;
+    ua.wait_limit = g_wait_limit;
+    ua.drop_first_copy = g_drop_first_copy;
+    // Blocks are aligned with sequences and positions.  For calls enqueued back to back a block owns a
+    // whole sequence (for very large batches seqs_per_cta of them): such calls overlap on the GPU as
+    // deeply as their grids allow (a call may start once every block of its predecessor has started),
+    // so few long-lived blocks per call are best, split only when the batch is too small to give 16
+    // blocks.  Otherwise the call runs alone, and a sequence's draft positions are split over the
+    // ctas_per_seq blocks of one cluster (each with both rows of its positions; 2, 4 or 8 blocks)
+    // until the GPU is full.
+    const long long merge_above = 8LL * sms;   // beyond this many sequences a block takes several
+    // (measured: the top-k kernel, with its longer per-row work, gains from the finer split)
+    const long long split_below = in.back_to_back ? 16 : (topk ? 4LL : 2LL) * sms;
+    long long c = 1, spc = 1;
+    if (in.B > merge_above) spc = (in.B + merge_above - 1) / merge_above;
+    else if (in.B < split_below) {
+      const long long want = split_below / in.B;
+      while (2 * c <= want && 2 * c <= in.gamma && 2 * c <= kMaxCluster) c *= 2;
+    }
+    while (spc > 1 && spc * rows_per_seq > kBlockRows) --spc;   // rows_per_seq <= 65 < kBlockRows
+    if (topk) {
+      ua.chunks_per_part = 0;
+      ua.parts_per_row = 1;
+      const double k = in.top_k, v = in.V;
+      const double tail = 1.25 * k / v + 4.0 * sqrt(k) / v + 16.0 / v;
+      if (tail < 0.45 && tail * v < 0.8 * kListCap) {
+        ua.lo_sigmas = (float)normal_upper_quantile(tail);
+        ua.lo_delta = ua.lo_sigmas - (float)normal_upper_quantile(k / v);
+        // a level with, almost surely, fewer than k values above it: the mirror image of the guess.
+        // The short cut it serves keeps lo as the row's threshold, which the diagnostic outputs that
+        // evaluate every token (the distribution drawn from, the monitors) would show in their last
+        // digits: with them requested every row gets its exact threshold.
+        const double tail_hi = 0.75 * k / v - 4.0 * sqrt(k) / v - 16.0 / v;
+        if (tail_hi * v >= 8.0 && in.allow_short_cut)
+          ua.hi_delta = (float)normal_upper_quantile(tail_hi) - ua.lo_sigmas;
+      }
+    } else {
+      // warp-wide items: parts of rows, sized so that every warp of the grid gets several
+      const int eps = kWStageBytes / (es * (cfg ? 2 : 1));
+      const long long cpr = (in.V + eps - 1) / eps;
+      const long long blocks = c > 1 ? (long long)in.B * c : (in.B + spc - 1) / spc;
+      // A row is cut into 1 ... 16 parts; the choice minimises the work of the block's busiest warp
+      // (its items are a contiguous eighth of the block's items; an item costs its stages plus about
+      // half a stage of fixed work).  Long items are better for their own sake -- fewer changes of
+      // the running maximum, fewer reductions -- so ties go to the fewer parts.
+      const long long rows_b = (c > 1) ? (2LL * ((in.gamma + c - 1) / c) + 1) : spc * rows_per_seq;
+      long long cpp = cpr;
+      double best = -1.0;
+      for (long long np = 1; np <= 16 && np <= cpr; ++np) {
+        const long long cand = (cpr + np - 1) / np;          // stages per part
+        const long long parts = (cpr + cand - 1) / cand;
+        if (parts != np && np > 1) continue;                 // (the same cut as a smaller np)
+        const long long n = rows_b * parts;
+        const long long last = cpr - (parts - 1) * cand;      // stages of a row's last part
+        double worst = 0.0;
+        for (int w = 0; w < kPlainWarps; ++w) {
+          const long long b0 = n * w / kPlainWarps, b1 = n * (w + 1) / kPlainWarps;
+          // items b0 .. b1-1; item i is part i % parts of its row
+          const long long full_rows = (b1 - b0) / parts;
+          double load = (double)full_rows * ((double)cpr + 0.5 * (double)parts);
+          for (long long i = b0 + full_rows * parts; i < b1; ++i)
+            load += (double)((i % parts == parts - 1) ? last : cand) + 0.5;
+          if (load > worst) worst = load;
+        }
+        if (best < 0.0 || worst < best * 0.97) { best = worst; cpp = cand; }
+      }
+      (void)blocks;
+      // a block keeps one stash entry per item
+      for (;;) {
+        const long long parts = (cpr + cpp - 1) / cpp;
+        const long long rows_block = (c > 1) ? (2LL * ((in.gamma + c - 1) / c) + 1) : spc * rows_per_seq;
+        if (rows_block * parts <= kBlockStash) break;
+        if (cpp < cpr) cpp = (cpp * 2 < cpr) ? cpp * 2 : cpr;
+        else if (spc > 1) --spc;
+        else break;   // one sequence per block, one part per row: at most 65 items
+      }
+      ua.chunks_per_part = (int)cpp;
+      ua.parts_per_row = (int)((cpr + cpp - 1) / cpp);
+    }
+    const long long grid = c > 1 ? (long long)in.B * c : (in.B + spc - 1) / spc;
+    ua.ctas_per_seq = (int)c;
+    ua.seqs_per_cta = (int)spc;
+    cudaError_t fe;
+    const bool overlap = in.back_to_back != 0;
+    if (in.dtype == CSD_F32)
+      fe = cfg ? launch_fused_t<float, true>(ua, topk, (int)grid, overlap, stream)
+               : launch_fused_t<float, false>(ua, topk, (int)grid, overlap, stream);
+    else
+      fe = cfg ? launch_fused_t<__nv_bfloat16, true>(ua, topk, (int)grid, overlap, stream)
+               : launch_fused_t<__nv_bfloat16, false>(ua, topk, (int)grid, overlap, stream);
+    return fe;
+  }
+}
+
 // sampling: the degenerate round used by csd_sample_rows -- no draft positions (gamma = 0), one
 // "target" row per sequence, whose bonus draw is the wanted token; the drafter-side pointers are unused.
 // no_workspace: the call has no workspace (the simple forms): only the single-launch path, which keeps
@@ -301,112 +425,46 @@ int verify_impl(const csd_params& p, int* plan_only = nullptr, bool sampling = f
   const bool fused = vec_ok && (size_t)p.V * es >= 512 && (p.V + 32 * vw - 1) / (32 * vw) <= kFinTiles &&
                      similar.nbr == nullptr;
   if (no_workspace && !fused) return CSD_ERR_ALIGN;
+  // the similarity relaxation finishes in the multi-launch path's kernel; where the rows qualify, their
+  // statistics still come from the streaming kernels (one launch, every logit read once)
+  const bool stream_stats = !fused && similar.nbr != nullptr && !no_workspace && vec_ok && (size_t)p.V * es >= 512 &&
+                            (p.V + 32 * vw - 1) / (32 * vw) <= kFinTiles;
   if (plan_only) {  // number of kernels this call would enqueue
-    *plan_only = fused ? 1 : (topk ? 3 : 2);
+    *plan_only = fused ? 1 : (stream_stats ? 2 : (topk ? 3 : 2));
     return CSD_OK;
   }
   if (fused) {
-    FusedArgs ua;
-    ua.fin = fa;
-    ua.top_k = p.top_k;
-    ua.lo_sigmas = nanf("");
-    ua.lo_delta = 0.0f;
-    ua.hi_delta = nanf("");
-    ua.error_flag = no_workspace ? nullptr : reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
-    ua.wait_limit = g_wait_limit;
-    ua.drop_first_copy = g_drop_first_copy;
-    // Blocks are aligned with sequences and positions.  For calls enqueued back to back a block owns a
-    // whole sequence (for very large batches seqs_per_cta of them): such calls overlap on the GPU as
-    // deeply as their grids allow (a call may start once every block of its predecessor has started),
-    // so few long-lived blocks per call are best, split only when the batch is too small to give 16
-    // blocks.  Otherwise the call runs alone, and a sequence's draft positions are split over the
-    // ctas_per_seq blocks of one cluster (each with both rows of its positions; 2, 4 or 8 blocks)
-    // until the GPU is full.
-    const long long merge_above = 8LL * sms;   // beyond this many sequences a block takes several
-    // (measured: the top-k kernel, with its longer per-row work, gains from the finer split)
-    const long long split_below = p.back_to_back ? 16 : (topk ? 4LL : 2LL) * sms;
-    long long c = 1, spc = 1;
-    if (p.B > merge_above) spc = (p.B + merge_above - 1) / merge_above;
-    else if (p.B < split_below) {
-      const long long want = split_below / p.B;
-      while (2 * c <= want && 2 * c <= p.gamma && 2 * c <= kMaxCluster) c *= 2;
-    }
-    while (spc > 1 && spc * rows_per_seq > kBlockRows) --spc;   // rows_per_seq <= 65 < kBlockRows
-    if (topk) {
-      ua.chunks_per_part = 0;
-      ua.parts_per_row = 1;
-      const double k = p.top_k, v = p.V;
-      const double tail = 1.25 * k / v + 4.0 * sqrt(k) / v + 16.0 / v;
-      if (tail < 0.45 && tail * v < 0.8 * kListCap) {
-        ua.lo_sigmas = (float)normal_upper_quantile(tail);
-        ua.lo_delta = ua.lo_sigmas - (float)normal_upper_quantile(k / v);
-        // a level with, almost surely, fewer than k values above it: the mirror image of the guess.
-        // The short cut it serves keeps lo as the row's threshold, which the diagnostic outputs that
-        // evaluate every token (the distribution drawn from, the monitors) would show in their last
-        // digits: with them requested every row gets its exact threshold.
-        const double tail_hi = 0.75 * k / v - 4.0 * sqrt(k) / v - 16.0 / v;
-        if (tail_hi * v >= 8.0 && !p.dbg_G && !p.diag_accept_mass && !p.diag_bound_term)
-          ua.hi_delta = (float)normal_upper_quantile(tail_hi) - ua.lo_sigmas;
-      }
-    } else {
-      // warp-wide items: parts of rows, sized so that every warp of the grid gets several
-      const int eps = kWStageBytes / (es * (cfg ? 2 : 1));
-      const long long cpr = (p.V + eps - 1) / eps;
-      const long long blocks = c > 1 ? (long long)p.B * c : (p.B + spc - 1) / spc;
-      // A row is cut into 1 ... 16 parts; the choice minimises the work of the block's busiest warp
-      // (its items are a contiguous eighth of the block's items; an item costs its stages plus about
-      // half a stage of fixed work).  Long items are better for their own sake -- fewer changes of
-      // the running maximum, fewer reductions -- so ties go to the fewer parts.
-      const long long rows_b = (c > 1) ? (2LL * ((p.gamma + c - 1) / c) + 1) : spc * rows_per_seq;
-      long long cpp = cpr;
-      double best = -1.0;
-      for (long long np = 1; np <= 16 && np <= cpr; ++np) {
-        const long long cand = (cpr + np - 1) / np;          // stages per part
-        const long long parts = (cpr + cand - 1) / cand;
-        if (parts != np && np > 1) continue;                 // (the same cut as a smaller np)
-        const long long n = rows_b * parts;
-        const long long last = cpr - (parts - 1) * cand;      // stages of a row's last part
-        double worst = 0.0;
-        for (int w = 0; w < kPlainWarps; ++w) {
-          const long long b0 = n * w / kPlainWarps, b1 = n * (w + 1) / kPlainWarps;
-          // items b0 .. b1-1; item i is part i % parts of its row
-          const long long full_rows = (b1 - b0) / parts;
-          double load = (double)full_rows * ((double)cpr + 0.5 * (double)parts);
-          for (long long i = b0 + full_rows * parts; i < b1; ++i)
-            load += (double)((i % parts == parts - 1) ? last : cand) + 0.5;
-          if (load > worst) worst = load;
-        }
-        if (best < 0.0 || worst < best * 0.97) { best = worst; cpp = cand; }
-      }
-      (void)blocks;
-      // a block keeps one stash entry per item
-      for (;;) {
-        const long long parts = (cpr + cpp - 1) / cpp;
-        const long long rows_block = (c > 1) ? (2LL * ((p.gamma + c - 1) / c) + 1) : spc * rows_per_seq;
-        if (rows_block * parts <= kBlockStash) break;
-        if (cpp < cpr) cpp = (cpp * 2 < cpr) ? cpp * 2 : cpr;
-        else if (spc > 1) --spc;
-        else break;   // one sequence per block, one part per row: at most 65 items
-      }
-      ua.chunks_per_part = (int)cpp;
-      ua.parts_per_row = (int)((cpr + cpp - 1) / cpp);
-    }
-    const long long grid = c > 1 ? (long long)p.B * c : (p.B + spc - 1) / spc;
-    ua.ctas_per_seq = (int)c;
-    ua.seqs_per_cta = (int)spc;
-    cudaError_t fe;
-    const bool overlap = p.back_to_back != 0;
-    if (p.dtype == CSD_F32)
-      fe = cfg ? launch_fused_t<float, true>(ua, topk, (int)grid, overlap, stream)
-               : launch_fused_t<float, false>(ua, topk, (int)grid, overlap, stream);
-    else
-      fe = cfg ? launch_fused_t<__nv_bfloat16, true>(ua, topk, (int)grid, overlap, stream)
-               : launch_fused_t<__nv_bfloat16, false>(ua, topk, (int)grid, overlap, stream);
-    return fe == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
+    FusedPlan fp;
+    fp.fa = fa;
+    fp.B = p.B; fp.gamma = p.gamma; fp.V = p.V; fp.top_k = p.top_k; fp.dtype = p.dtype;
+    fp.rows_per_seq = rows_per_seq; fp.rows = rows; fp.sms = sms; fp.es = es;
+    fp.cfg = cfg; fp.topk = topk; fp.back_to_back = p.back_to_back != 0;
+    fp.allow_short_cut = !p.dbg_G && !p.diag_accept_mass && !p.diag_bound_term;
+    fp.error_flag = no_workspace ? nullptr : reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
+    fp.stats_out = nullptr; fp.thr_out = nullptr;
+    fp.stream = stream;
+    return plan_and_launch_fused(fp) == cudaSuccess ? CSD_OK : CSD_ERR_LAUNCH;
   }
 
   cudaError_t e = cudaSuccess;
-  if (p.dtype == CSD_F32) {
+  if (stream_stats) {
+    FusedPlan fp;
+    fa.parts = 1;
+    fp.fa = fa;
+    fp.B = p.B; fp.gamma = p.gamma; fp.V = p.V; fp.top_k = p.top_k; fp.dtype = p.dtype;
+    fp.rows_per_seq = rows_per_seq; fp.rows = rows; fp.sms = sms; fp.es = es;
+    fp.cfg = cfg; fp.topk = topk; fp.back_to_back = false;
+    fp.allow_short_cut = false;   // the finishing kernel filters by the exact threshold
+    fp.error_flag = reinterpret_cast<int*>((char*)p.workspace + lay.header_off);
+    fp.stats_out = sa.partials;
+    fp.thr_out = topk ? se.thresholds : nullptr;
+    fp.stream = stream;
+    e = plan_and_launch_fused(fp);
+    if (e == cudaSuccess) {
+      if (p.dtype == CSD_F32) e = cfg ? launch_finish<float, true>(fa, stream) : launch_finish<float, false>(fa, stream);
+      else e = cfg ? launch_finish<__nv_bfloat16, true>(fa, stream) : launch_finish<__nv_bfloat16, false>(fa, stream);
+    }
+  } else if (p.dtype == CSD_F32) {
     if (topk) e = cfg ? launch_select<float, true>(se, sms, stream) : launch_select<float, false>(se, sms, stream);
     if (e == cudaSuccess)
       e = cfg ? launch_stats_u<float, true>(sa, U, topk, sms, stream) : launch_stats_u<float, false>(sa, U, topk, sms, stream);
@@ -654,7 +712,30 @@ int csd_verify_tree(const csd_tree_params* pp) {
   for (int n = 0; n < p.N; ++n) ta.parent[n] = (signed char)p.parent[n];
 
   cudaError_t e = cudaSuccess;
-  if (p.dtype == CSD_F32) {
+  // Row statistics (and thresholds) of all 2 C rows: by the streaming kernels of the single-launch path
+  // where the rows qualify for them (aligned, at least 512 bytes, within the draw's tile table), one
+  // launch that reads every logit once; otherwise by the select and statistics kernels.
+  const bool stream_stats = vec_ok && (size_t)p.V * es >= 512 && (p.V + 32 * vw - 1) / (32 * vw) <= kFinTiles &&
+                            2 * C <= kBlockRows;
+  if (stream_stats) {
+    FusedPlan fp;
+    fp.fa = fa;
+    fp.fa.parts = 1;
+    fp.B = p.B; fp.gamma = C; fp.V = p.V; fp.top_k = p.top_k; fp.dtype = p.dtype;
+    fp.rows_per_seq = 2 * C; fp.rows = rows; fp.sms = sms; fp.es = es;
+    fp.cfg = cfg; fp.topk = topk; fp.back_to_back = false;
+    fp.allow_short_cut = false;   // the finishing kernel filters by the exact threshold
+    fp.error_flag = reinterpret_cast<int*>(ws + lay.header_off);
+    fp.stats_out = sa.partials;
+    fp.thr_out = topk ? se.thresholds : nullptr;
+    fp.stream = stream;
+    e = plan_and_launch_fused(fp);
+    fa.parts = 1;
+    if (e == cudaSuccess) {
+      if (p.dtype == CSD_F32) e = cfg ? launch_tree_finish<float, true>(ta, stream) : launch_tree_finish<float, false>(ta, stream);
+      else e = cfg ? launch_tree_finish<__nv_bfloat16, true>(ta, stream) : launch_tree_finish<__nv_bfloat16, false>(ta, stream);
+    }
+  } else if (p.dtype == CSD_F32) {
     if (topk) e = cfg ? launch_select<float, true>(se, sms, stream) : launch_select<float, false>(se, sms, stream);
     if (e == cudaSuccess)
       e = cfg ? launch_stats_u<float, true>(sa, U, topk, sms, stream) : launch_stats_u<float, false>(sa, U, topk, sms, stream);

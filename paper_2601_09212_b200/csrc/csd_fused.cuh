@@ -173,6 +173,8 @@ struct FusedArgs {
                         // (NaN: never take the short cut that needs it)
   int* error_flag;      // set when a bounded wait gave up; null: nobody asked for the status
   long long wait_limit; // cycles a wait on a copy may take (kWaitCycles unless a test shortens it)
+  float2* stats_out;    // not null: stop after the streaming phase and write every local row's (m, s) here,
+  float* thr_out;       //   and its top-k threshold there (may be null), at row b * (T + gamma) + (target ? i : T + i)
   int drop_first_copy;  // test aid: the first copy of block 0 is announced to its barrier but never issued,
                         // so that the wait on it runs out (nothing is left in flight)
 };
@@ -902,6 +904,23 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
   emit_sequence<T, CFG, NT>(ua, b, st.rec, any, tid);
 }
 
+// Stats-only calls (FusedArgs::stats_out): the block's rows go to global memory in the row order of the
+// multi-launch kernels, after the previous operation on the stream has completed (its finishing kernel
+// may still be reading the same arrays).
+__device__ __forceinline__ void write_row_stats(const FusedArgs& a, const BlockShare& sh, const RowStats& rs, const int tid,
+                                                const int nthreads, const bool aborted) {
+  pdl_wait();
+  const FinishArgs& f = a.fin;
+  for (int r = tid; r < sh.n_rows && r < kBlockRows; r += nthreads) {
+    int b, which, i;
+    local_row(sh, r, f.gamma, b, which, i);
+    const int64_t row_id = (int64_t)b * (f.T + f.gamma) + (which == 0 ? i : f.T + i);
+    a.stats_out[row_id] = aborted ? make_float2(__int_as_float(0x7fc00000), 0.0f) : rs.ms[r];   // (a row of a call that
+    if (a.thr_out) a.thr_out[row_id] = rs.thr[r];                                              //  gave up reads as unusable)
+  }
+  if (a.ctas_per_seq > 1) cluster_wait();   // second half of the barrier begun at kernel start
+}
+
 // ======================= plain kernel: one pipeline per warp ============================
 // A warp owns a contiguous range of items (an item is a part of a row: chunks_per_part warp
 // stages), a private ring of kWStages stages of kWStageBytes, issues its own refills, and keeps
@@ -936,7 +955,9 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
   extern __shared__ __align__(128) unsigned char fused_smem_raw[];
   PlainSmem& sm = *reinterpret_cast<PlainSmem*>(fused_smem_raw);
 
-  pdl_launch_dependents();   // the next call on the stream may start: see the head of this file
+  // the next call on the stream may start: see the head of this file (a stats-only call is followed by
+  // its finishing kernel, whose large blocks would only sit on SMs this kernel needs: it follows at exit)
+  if (a.stats_out == nullptr) pdl_launch_dependents();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const FinishArgs& f = a.fin;
   const int V = f.V;
@@ -953,8 +974,11 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
 
   // the block's items (parts of its local rows, see block_share), split evenly over its warps
   const BlockShare sh = block_share(a);
-  stage_inputs(a, sh, 0, tid, sm.fst);
-  load_token_logits<T, CFG, kPlainThreads>(f, sh, tid, sm.rs);
+  const bool stats_only = a.stats_out != nullptr;
+  if (!stats_only) {
+    stage_inputs(a, sh, 0, tid, sm.fst);
+    load_token_logits<T, CFG, kPlainThreads>(f, sh, tid, sm.rs);
+  }
   const int n_block = sh.n_rows * parts;
   const int item_begin = (int)((long long)n_block * warp / kPlainWarps);
   const int item_end = (int)((long long)n_block * (warp + 1) / kPlainWarps);
@@ -1187,6 +1211,10 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
     if (lane == 0) { sm.rs.ms[r] = make_float2(m, s_acc); sm.rs.thr[r] = CSD_NEG_INF; }
   }
   __syncthreads();
+  if (stats_only) {
+    write_row_stats(a, sh, sm.rs, tid, kPlainThreads, sm.abort != 0);
+    return;
+  }
   finish_block<T, CFG, kPlainThreads, false>(a, sh, sm.rs, tid, sm.abort != 0, &sm.ring[0][0][0], kPlainRingBytes,
                                       reinterpret_cast<double*>(&sm.stash[0]), sm.fin, sm.fst);
 }
@@ -1401,7 +1429,9 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   extern __shared__ __align__(128) unsigned char fused_smem_raw[];
   TopkSmem& sm = *reinterpret_cast<TopkSmem*>(fused_smem_raw);
 
-  pdl_launch_dependents();   // the next call on the stream may start: see the head of this file
+  // the next call on the stream may start: see the head of this file (a stats-only call is followed by
+  // its finishing kernel, whose large blocks would only sit on SMs this kernel needs: it follows at exit)
+  if (a.stats_out == nullptr) pdl_launch_dependents();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const FinishArgs& f = a.fin;
   const int V = f.V;
@@ -1430,8 +1460,13 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
 
   // this block's local rows (see block_share)
   const BlockShare sh = block_share(a);
-  stage_inputs(a, sh, 0, tid, sm.fst);
-  load_token_logits<T, CFG, kTopkThreads>(f, sh, tid, sm.rs);
+  const bool stats_only = a.stats_out != nullptr;
+  if (!stats_only) {
+    stage_inputs(a, sh, 0, tid, sm.fst);
+    load_token_logits<T, CFG, kTopkThreads>(f, sh, tid, sm.rs);
+  } else {
+    for (int r = tid; r < kBlockRows; r += kTopkThreads) sm.rs.tokz[r] = 0.0f;   // (read by the short cut's rank, unused here)
+  }
   const int n_rows = sh.n_rows;
   const int n_chunks = n_rows * cpr;
 
@@ -1827,6 +1862,10 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
 
   // ================================= phase 2 ===========================================
   __syncthreads();
+  if (stats_only) {
+    write_row_stats(a, sh, sm.rs, tid, kTopkThreads, sm.abort != 0);
+    return;
+  }
   static_assert(sizeof(sm.list) >= kFinTiles * sizeof(double), "tile sums live in the list area");
   finish_block<T, CFG, kTopkThreads, true>(a, sh, sm.rs, tid, sm.abort != 0, &sm.ring[0][0], kTkRingBytes,
                                      reinterpret_cast<double*>(&sm.list[0][0]), sm.fin, sm.fst);
