@@ -292,7 +292,8 @@ int csd_sample_rows(const void* logits, const void* uncond, float cfg_scale, int
  *               tokenizer's codebook, which the caller supplies.)
  *   lambda      >= 0; 0 selects nothing: the call then equals csd_verify_ex
  * dbg_p reports A(x~_i).  The Theorem 2 monitors are not available in this form (CSD_ERR_ARG).  The
- * call always takes the multi-launch path (csd_launch_count does not apply).
+ * call enqueues two kernels (statistics of every row, then one block per sequence for the tests and the
+ * draw), three for rows that are unaligned or shorter than 512 bytes; csd_launch_count does not apply.
  */
 int csd_verify_similar(const csd_params* p, const int32_t* neighbours, int k, float lambda);
 

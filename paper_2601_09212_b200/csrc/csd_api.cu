@@ -218,7 +218,6 @@ struct FusedPlan {
 };
 cudaError_t plan_and_launch_fused(const FusedPlan& in) {
   const int sms = in.sms, es = in.es, rows_per_seq = in.rows_per_seq;
-  const long long rows = in.rows;
   const bool cfg = in.cfg, topk = in.topk;
   cudaStream_t stream = in.stream;
   {
@@ -270,7 +269,6 @@ cudaError_t plan_and_launch_fused(const FusedPlan& in) {
       // warp-wide items: parts of rows, sized so that every warp of the grid gets several
       const int eps = kWStageBytes / (es * (cfg ? 2 : 1));
       const long long cpr = (in.V + eps - 1) / eps;
-      const long long blocks = c > 1 ? (long long)in.B * c : (in.B + spc - 1) / spc;
       // A row is cut into 1 ... 16 parts; the choice minimises the work of the block's busiest warp
       // (its items are a contiguous eighth of the block's items; an item costs its stages plus about
       // half a stage of fixed work).  Long items are better for their own sake -- fewer changes of
@@ -296,7 +294,6 @@ cudaError_t plan_and_launch_fused(const FusedPlan& in) {
         }
         if (best < 0.0 || worst < best * 0.97) { best = worst; cpp = cand; }
       }
-      (void)blocks;
       // a block keeps one stash entry per item
       for (;;) {
         const long long parts = (cpr + cpp - 1) / cpp;
