@@ -278,8 +278,9 @@ struct FinishStage {
   float mon_am[kMaxGamma], mon_bt[kMaxGamma];   // per-position monitors of Theorem 2, until they are written out
   SeqRecord rec;
   uint32_t xch[kMaxCluster];   // written by the blocks of the cluster: what each found (see finish_block)
-  uint32_t share[12];          // written by the block that draws, into every block of the cluster: what the
-                               // draw's weights need (see cluster_draw)
+  uint32_t share[kMaxCluster][12];   // written by every block of the cluster into every block, together with xch:
+                                     // what the draw's weights need if that block turns out to hold the
+                                     // sequence's first rejection (see finish_block, cluster_draw)
   alignas(8) uint64_t bar;
   alignas(8) uint64_t bar2;    // second copy barrier of the per-position monitors
 };
@@ -709,68 +710,59 @@ __device__ void cluster_draw(const FusedArgs& ua, const BlockShare& sh, int j, c
   const int b = sh.seq_begin;
   const int lane = tid & 31, warp = tid >> 5;
   const bool mine = owner == sh.slot;
-  // ---- the drawing block says what is drawn from ---------------------------------------------------
+  // ---- what is drawn from: published by the drawing block before the exchange's barrier -----------------
   int status = extra_status & ~8;
   bool rejected = false;
   if (mine) {
     rejected = j < sh.pos_end;
-    int draw = 0, mode = 1;
-    if (rejected) {
-      status |= sm.flag[j];
-      draw = sm.valid[0][j] != 0;
-      mode = sm.valid[1][j] ? 0 : 1;
-    } else if (sh.bonus) {
-      j = L;
-      draw = sm.valid[0][L] != 0;
-      if (!draw) status |= 1;
-    }
-    if (tid < c) {
-      const uint32_t rank = (uint32_t)tid;
-      const float omo = 1.0f - (j < L ? st.omega[j] : 0.0f);
-      cluster_store(&st.share[0], rank, (uint32_t)draw);
-      cluster_store(&st.share[1], rank, (uint32_t)mode);
-      cluster_store(&st.share[2], rank, (uint32_t)j);
-      cluster_store(&st.share[3], rank, __float_as_uint(sm.M[0][min(j, a.T - 1)]));
-      cluster_store(&st.share[4], rank, __float_as_uint(sm.S[0][min(j, a.T - 1)]));
-      cluster_store(&st.share[5], rank, __float_as_uint(j < L ? sm.M[1][j] : 0.0f));
-      cluster_store(&st.share[6], rank, __float_as_uint(j < L ? sm.S[1][j] : 0.0f));
-      cluster_store(&st.share[7], rank, __float_as_uint(sm.thr[0][min(j, a.T - 1)]));
-      cluster_store(&st.share[8], rank, __float_as_uint(j < L ? sm.thr[1][j] : CSD_NEG_INF));
-      cluster_store(&st.share[9], rank, __float_as_uint(omo));
-    }
+    if (rejected) status |= sm.flag[j];
+    else if (sh.bonus && !sm.valid[0][L]) status |= 1;
   }
-  __syncthreads();
-  cluster_arrive();
-  cluster_wait();
+  const uint32_t* share = st.share[owner];
   // ---- every block: its share of the tile sums -----------------------------------------------------
-  const int draw = (int)st.share[0];
-  const int jj = (int)st.share[2];
+  const int draw = (int)share[0];
+  const int jj = (int)share[2];
   PairCtx ctx;
-  ctx.mode = (int)st.share[1];
-  ctx.Mt = __uint_as_float(st.share[3]); ctx.St = __uint_as_float(st.share[4]);
-  ctx.Md = __uint_as_float(st.share[5]); ctx.Sd = __uint_as_float(st.share[6]);
+  ctx.mode = (int)share[1];
+  ctx.Mt = __uint_as_float(share[3]); ctx.St = __uint_as_float(share[4]);
+  ctx.Md = __uint_as_float(share[5]); ctx.Sd = __uint_as_float(share[6]);
   ctx.inv_t = 1.0f / (1.0f + ctx.St);
   ctx.inv_den = ctx.inv_t / (1.0f + ctx.Sd);
-  ctx.one_minus_omega = __uint_as_float(st.share[9]);
+  ctx.one_minus_omega = __uint_as_float(share[9]);
   Row<T, CFG> rt = row_at<T, CFG>(a, b, 0, min(jj, a.T - 1));
   Row<T, CFG> rd = rt;
-  rt.thr = __uint_as_float(st.share[7]);
-  if (jj < L) { rd = row_at<T, CFG>(a, b, 1, jj); rd.thr = __uint_as_float(st.share[8]); }
+  rt.thr = __uint_as_float(share[7]);
+  if (jj < L) { rd = row_at<T, CFG>(a, b, 1, jj); rd.thr = __uint_as_float(share[8]); }
   const int ntiles = (V + TILE - 1) / TILE;
   if (draw) {
     const int t_begin = (int)((long long)ntiles * sh.slot / c), t_end = (int)((long long)ntiles * (sh.slot + 1) / c);
-    for (int tile = t_begin + warp; tile < t_end; tile += NT / 32) {
-      const int x0 = tile * TILE + lane * VEC;
-      float zt[VEC], zd[VEC];
-      rt.load_tile(x0, V, 1, zt);
-      if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd);
-      float acc = 0.0f;
+    // (tiles per warp and trip: two, with all loads issued before the first use, measured no faster here and
+    // cost the streaming loops registers)
+    constexpr int UNR = 1;
+    for (int tile0 = t_begin + warp; tile0 < t_end; tile0 += UNR * (NT / 32)) {
+      float zt[UNR][VEC], zd[UNR][VEC];
 #pragma unroll
-      for (int e = 0; e < VEC; ++e)
-        acc += weight_of(FILT ? rt.filter(zt[e]) : zt[e], ctx.mode == 0 ? (FILT ? rd.filter(zd[e]) : zd[e]) : 0.0f, ctx);
+      for (int r = 0; r < UNR; ++r) {
+        const int tile = tile0 + r * (NT / 32);
+        if (tile < t_end) {
+          const int x0 = tile * TILE + lane * VEC;
+          rt.load_tile(x0, V, 1, zt[r]);
+          if (ctx.mode == 0) rd.load_tile(x0, V, 1, zd[r]);
+        }
+      }
 #pragma unroll
-      for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-      if (lane == 0) cluster_store_f64(&tile_sums[tile], (uint32_t)owner, (double)acc);
+      for (int r = 0; r < UNR; ++r) {
+        const int tile = tile0 + r * (NT / 32);
+        if (tile < t_end) {
+          float acc = 0.0f;
+#pragma unroll
+          for (int e = 0; e < VEC; ++e)
+            acc += weight_of(FILT ? rt.filter(zt[r][e]) : zt[r][e], ctx.mode == 0 ? (FILT ? rd.filter(zd[r][e]) : zd[r][e]) : 0.0f, ctx);
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+          if (lane == 0) cluster_store_f64(&tile_sums[tile], (uint32_t)owner, (double)acc);
+        }
+      }
     }
   }
   __syncthreads();
@@ -877,7 +869,33 @@ __device__ void finish_block(const FusedArgs& ua, const BlockShare& sh, const Ro
   const int j = accept_positions<T, CFG, NT>(ua, sh, 0, rs, tid, sm, st);
   // ---- tell every block of the sequence: bit 0 rejected, bit 1 a bounded wait gave up ------------
   cluster_wait();   // second half of the barrier begun at kernel start: every peer is running
-  if (tid < c) cluster_store(&st.xch[sh.slot], (uint32_t)tid, (j < sh.pos_end ? 1u : 0u) | (aborted ? 2u : 0u));
+  if (tid < c) {
+    const uint32_t rank = (uint32_t)tid;
+    cluster_store(&st.xch[sh.slot], rank, (j < sh.pos_end ? 1u : 0u) | (aborted ? 2u : 0u));
+    // ... and, in the same exchange, what the draw's weights need should this block turn out to decide
+    // the sequence: the position drawn at (its first rejection, or the bonus row), the two rows'
+    // statistics and filter levels, 1 - omega
+    int jd = j, draw = 0, mode = 1;
+    if (j < sh.pos_end) {
+      draw = sm.valid[0][j] != 0;
+      mode = sm.valid[1][j] ? 0 : 1;
+    } else if (sh.bonus) {
+      jd = L;
+      draw = sm.valid[0][L] != 0;
+    }
+    const int jt = min(jd, a.T - 1);
+    uint32_t* mine_at = st.share[sh.slot];
+    cluster_store(&mine_at[0], rank, (uint32_t)draw);
+    cluster_store(&mine_at[1], rank, (uint32_t)mode);
+    cluster_store(&mine_at[2], rank, (uint32_t)jd);
+    cluster_store(&mine_at[3], rank, __float_as_uint(sm.M[0][jt]));
+    cluster_store(&mine_at[4], rank, __float_as_uint(sm.S[0][jt]));
+    cluster_store(&mine_at[5], rank, __float_as_uint(jd < L ? sm.M[1][jd] : 0.0f));
+    cluster_store(&mine_at[6], rank, __float_as_uint(jd < L ? sm.S[1][jd] : 0.0f));
+    cluster_store(&mine_at[7], rank, __float_as_uint(sm.thr[0][jt]));
+    cluster_store(&mine_at[8], rank, __float_as_uint(jd < L ? sm.thr[1][jd] : CSD_NEG_INF));
+    cluster_store(&mine_at[9], rank, __float_as_uint(1.0f - (jd < L ? st.omega[jd] : 0.0f)));
+  }
   __syncthreads();
   cluster_arrive();
   cluster_wait();
