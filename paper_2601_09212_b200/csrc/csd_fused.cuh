@@ -1174,11 +1174,18 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
             static_assert(NW % 2 == 0 || NW == 1, "pairs of words");
             cnt_run += (int)((c2 & 0xffffu) + (c2 >> 16));
           }
+          // exponents and sums two values per instruction (each half the IEEE operation: the same bits as
+          // the scalar form); NaN values poison the sum, which marks the row
+          const uint64_t l2e2 = pack2(kLog2e, kLog2e), nm2 = pack2(nMwL, nMwL);
+          uint64_t accp[2] = {pack2(0.0f, 0.0f), pack2(0.0f, 0.0f)};
 #pragma unroll
           for (int k = 0; k < NW; ++k) {
-            acc4[(2 * k) & 3] += ex2f(fmaf(__uint_as_float(w[k] << 16), kLog2e, nMwL));   // NaN values poison the sum,
-            acc4[(2 * k + 1) & 3] += ex2f(fmaf(__uint_as_float(w[k] & 0xffff0000u), kLog2e, nMwL));   // which marks the row
+            float x0, x1;
+            unpack2(fma2(pack2(__uint_as_float(w[k] << 16), __uint_as_float(w[k] & 0xffff0000u)), l2e2, nm2), x0, x1);
+            accp[k & 1] = add2(accp[k & 1], pack2(ex2f(x0), ex2f(x1)));
           }
+          unpack2(accp[0], acc4[0], acc4[1]);
+          unpack2(accp[1], acc4[2], acc4[3]);
         } else if (wm == Mw) {
           // (branch-free: the exponential of a value equal to the reference is replaced by 0)
           int c4[4] = {0, 0, 0, 0};
