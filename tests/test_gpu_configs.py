@@ -58,3 +58,31 @@ def test_c3_sixteen_steps():
 
 def test_c4_all_sequences_of_two_steps():
     _run("C4", 2, schedule=_sched(16))
+
+
+def test_widened_rounds_on_c3_shapes():
+    """The tree and the similarity-relaxed rounds at the shapes bench.py times them on (C3: 64 sequences,
+    V = 16384, bf16, guidance mix, top-k 1000): their row statistics come from the streaming kernels'
+    stats-only mode there.  Every output against the oracle."""
+    from oracle.compare import compare
+    from gpu_util import run_oracle
+    from test_gpu_similar import run_similar
+    from test_gpu_tree import compare_tree, run_tree_gpu, run_tree_oracle
+    kw = {k: v for k, v in W.CONFIGS["C3"].items() if k not in ("B", "gamma", "V", "bonus_row", "steps")}
+    B, V = W.CONFIGS["C3"]["B"], W.CONFIGS["C3"]["V"]
+    parent = W.static_tree([4, 3, 2, 2])
+    D = csd.csd_tree_depth(parent)
+    for step in range(2):
+        wt = W.make_tree(parent, B=B, V=V, schedule=_sched(D), seed=21, step=step, device=DEV, **kw)
+        n_near, bad = compare_tree(wt, run_tree_gpu(wt, want_G=False), run_tree_oracle(wt))
+        assert not bad, bad[:4]
+        assert n_near <= 2
+        w = W.config("C3", step=step, schedule=_sched(8), device=DEV)
+        r = np.random.default_rng(step)
+        nbr = ((np.arange(V)[:, None] + 1 + r.integers(0, V - 1, size=(V, 10))) % V).astype(np.int32)
+        got = run_similar(w, nbr, 2.0)
+        h, ref = run_oracle(w, neighbours=nbr, nbr_lambda=2.0)
+        rep = compare(ref, got["tokens"], got["accept_len"], h["draft_tokens"], h["uniforms"], status=got["status"],
+                      p=got["p"], q=got["q"], f=got["f"], tol=2e-3)
+        assert rep.ok, rep.summary() + " :: " + str(rep.unexplained[:4])
+        assert rep.tau_mismatch_near + rep.token_mismatch_near <= 2, rep.summary()
