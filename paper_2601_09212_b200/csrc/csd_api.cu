@@ -19,6 +19,7 @@ namespace {
 using namespace csd;
 
 static_assert(sizeof(TopkSmem) <= 55 * 1024, "four blocks of the top-k kernel per SM must fit");
+static_assert(sizeof(TopkSmemT<kWarpListLarge>) <= 74 * 1024, "three blocks of its large-list instance per SM must fit");
 static_assert(sizeof(PlainSmem) <= 75 * 1024, "three blocks of the plain kernel per SM must fit");
 
 constexpr int kMaxV = 1 << 20;
@@ -82,13 +83,16 @@ double normal_upper_quantile(double tail) {
 }
 
 // Launches one of the single-launch kernels (KERNEL: 0 plain, 1 top-k on rows that are a whole
-// number of stages, 2 top-k on any row length) with its shared-memory size, optionally with
+// number of stages, 2 top-k on any row length, 3 and 4 the same two with the large candidate lists) with its shared-memory size, optionally with
 // programmatic stream serialisation and as clusters of ctas_per_seq blocks.
 template <typename T, bool CFG, int KERNEL>
 cudaError_t launch_fused(const FusedArgs& a, int grid, bool overlap, cudaStream_t stream) {
   auto kern = KERNEL == 0 ? verify_plain_kernel<T, CFG>
-                          : (KERNEL == 1 ? verify_topk_kernel<T, CFG, false> : verify_topk_kernel<T, CFG, true>);
-  constexpr size_t kSmem = KERNEL ? sizeof(TopkSmem) : sizeof(PlainSmem);
+              : KERNEL == 1 ? verify_topk_kernel<T, CFG, false, kWarpList>
+              : KERNEL == 2 ? verify_topk_kernel<T, CFG, true, kWarpList>
+              : KERNEL == 3 ? verify_topk_kernel<T, CFG, false, kWarpListLarge>
+                            : verify_topk_kernel<T, CFG, true, kWarpListLarge>;
+  constexpr size_t kSmem = KERNEL == 0 ? sizeof(PlainSmem) : (KERNEL <= 2 ? sizeof(TopkSmem) : sizeof(TopkSmemT<kWarpListLarge>));
   constexpr int kThreads = KERNEL ? kTopkThreads : kPlainThreads;
   // the attribute belongs to (function, device): set it once per device (setting it twice is harmless)
   static bool configured[kMaxDevices] = {};
@@ -128,8 +132,9 @@ template <typename T, bool CFG>
 cudaError_t launch_fused_t(const FusedArgs& a, bool topk, int grid, bool overlap, cudaStream_t stream) {
   if (!topk) return launch_fused<T, CFG, 0>(a, grid, overlap, stream);
   constexpr int kStageElems = kTkStageBytes / ((int)sizeof(T) * (CFG ? 2 : 1));
-  return a.fin.V % kStageElems == 0 ? launch_fused<T, CFG, 1>(a, grid, overlap, stream)
-                                    : launch_fused<T, CFG, 2>(a, grid, overlap, stream);
+  const bool whole = a.fin.V % kStageElems == 0;
+  if (a.large_lists) return whole ? launch_fused<T, CFG, 3>(a, grid, overlap, stream) : launch_fused<T, CFG, 4>(a, grid, overlap, stream);
+  return whole ? launch_fused<T, CFG, 1>(a, grid, overlap, stream) : launch_fused<T, CFG, 2>(a, grid, overlap, stream);
 }
 
 template <typename T, bool CFG, int U, bool TOPK>
@@ -227,6 +232,7 @@ cudaError_t plan_and_launch_fused(const FusedPlan& in) {
     ua.lo_sigmas = nanf("");
     ua.lo_delta = 0.0f;
     ua.hi_delta = nanf("");
+    ua.large_lists = 0;
     ua.error_flag = in.error_flag;
     ua.stats_out = in.stats_out;
     ua.thr_out = in.thr_out;
@@ -240,8 +246,12 @@ cudaError_t plan_and_launch_fused(const FusedPlan& in) {
     // ctas_per_seq blocks of one cluster (each with both rows of its positions; 2, 4 or 8 blocks)
     // until the GPU is full.
     const long long merge_above = 8LL * sms;   // beyond this many sequences a block takes several
-    // (measured: the top-k kernel, with its longer per-row work, gains from the finer split)
-    const long long split_below = in.back_to_back ? 16 : (topk ? 4LL : 2LL) * sms;
+    // (measured: the top-k kernel, with its longer per-row work, gains from the finer split; its
+    // large-list instance has three blocks per SM, and a lone call should fit one wave)
+    const double tk_k = in.top_k, tk_v = in.V;
+    const double tk_tail = 1.25 * tk_k / tk_v + 4.0 * sqrt(tk_k) / tk_v + 16.0 / tk_v;
+    const bool tk_large = topk && tk_tail * tk_v >= 0.8 * (kTopkWarps * kWarpList);
+    const long long split_below = in.back_to_back ? 16 : (topk ? (tk_large ? 3LL : 4LL) : 2LL) * sms;
     long long c = 1, spc = 1;
     if (in.B > merge_above) spc = (in.B + merge_above - 1) / merge_above;
     else if (in.B < split_below) {
@@ -252,9 +262,11 @@ cudaError_t plan_and_launch_fused(const FusedPlan& in) {
     if (topk) {
       ua.chunks_per_part = 0;
       ua.parts_per_row = 1;
-      const double k = in.top_k, v = in.V;
-      const double tail = 1.25 * k / v + 4.0 * sqrt(k) / v + 16.0 / v;
-      if (tail < 0.45 && tail * v < 0.8 * kListCap) {
+      const double k = tk_k, v = tk_v, tail = tk_tail;
+      // the candidates must fit the per-warp lists with room to spare: the small lists (four blocks per SM)
+      // where they do, else the large ones (three blocks per SM), else every row is selected exactly
+      ua.large_lists = tk_large ? 1 : 0;
+      if (tail < 0.45 && tail * v < 0.8 * (kTopkWarps * kWarpListLarge)) {
         ua.lo_sigmas = (float)normal_upper_quantile(tail);
         ua.lo_delta = ua.lo_sigmas - (float)normal_upper_quantile(k / v);
         // a level with, almost surely, fewer than k values above it: the mirror image of the guess.

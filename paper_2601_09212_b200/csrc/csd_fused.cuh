@@ -173,6 +173,7 @@ struct FusedArgs {
                         // (NaN: never take the short cut that needs it)
   int* error_flag;      // set when a bounded wait gave up; null: nobody asked for the status
   long long wait_limit; // cycles a wait on a copy may take (kWaitCycles unless a test shortens it)
+  int large_lists;      // top-k: the instance with the large candidate lists (set by the host from k and V)
   float2* stats_out;    // not null: stop after the streaming phase and write every local row's (m, s) here,
   float* thr_out;       //   and its top-k threshold there (may be null), at row b * (T + gamma) + (target ? i : T + i)
   int drop_first_copy;  // test aid: the first copy of block 0 is announced to its barrier but never issued,
@@ -1248,8 +1249,9 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
 constexpr int kTkStages = 2;
 constexpr int kTkStageBytes = 16384;
 constexpr int kTkRingBytes = kTkStages * kTkStageBytes;
-constexpr int kWarpList = 256;                // per-warp capacity of the list of values >= lo
-constexpr int kListCap = kTopkWarps * kWarpList;
+constexpr int kWarpList = 256;                // per-warp capacity of the list of values >= lo: the instance that
+                                              // leaves room for four blocks per SM ...
+constexpr int kWarpListLarge = 512;           // ... and the one for larger k (three blocks per SM)
 constexpr int kLinBins = 512;
 constexpr int kCandCap = 64;
 constexpr float kLinRangeSigmas = 4.75f;      // the histogram spans [lo, lo + this many deviations)
@@ -1259,13 +1261,14 @@ __device__ __forceinline__ int lin_bin(float v, float lo, float scale) {
   return min(kLinBins - 1, (int)__fmul_rn(__fsub_rn(v, lo), scale));
 }
 
-struct TopkSmem {
+template <int WL>
+struct TopkSmemT {
   alignas(128) unsigned char ring[kTkStages][kTkStageBytes];
   alignas(8) uint64_t full[kTkStages];
   int readers_done[kTkStages];      // warps that have finished reading the stage's current contents
   int issued_q;                     // chunks announced to the barriers so far (written by the issuing thread)
   alignas(16) int hist[kLinBins];   // linear histogram; first 256 bins double as the radix histogram
-  alignas(8) float list[kTopkWarps][kWarpList];   // per warp: the values >= lo it met (the finish keeps its tile sums here)
+  alignas(8) float list[kTopkWarps][WL];   // per warp: the values >= lo it met (the finish keeps its tile sums here)
   int wpos[kTopkWarps];            // per warp: next free slot of its list (may run past the capacity)
   float cand[kCandCap];             // values in the bin of the k-th largest
   int n_cand[2];                    // by row parity
@@ -1296,6 +1299,7 @@ struct TopkSmem {
   float row_mean[2], row_dev[2];    // by row parity: the sample's moments (for that adaptation)
   int adapt_on;                     // set once a guess has missed: from then on every row adapts the multiplier
 };
+using TopkSmem = TopkSmemT<kWarpList>;
 
 // Bin (of kLinBins, counted in `hist`) that holds the k-th largest value, found by one warp:
 // 16 bins per lane from the top, a warp scan, then a second scan inside the owner's 16 bins.
@@ -1340,8 +1344,8 @@ __device__ __forceinline__ int warp_pick_bin(const int* hist, int k, int lane, i
 // Exact threshold and filtered statistics of one row read again from global memory: radix
 // select over order-preserving keys (four 8-bit digits), then one pass for (m, s).  All
 // threads of the block take part; the results are valid in thread 0.
-template <typename T, bool CFG>
-__device__ void exact_row_from_global(const Row<T, CFG>& row, int V, int k, TopkSmem& sm, int tid, float& out_m,
+template <typename T, bool CFG, typename SM>
+__device__ void exact_row_from_global(const Row<T, CFG>& row, int V, int k, SM& sm, int tid, float& out_m,
                                       float& out_s, float& out_thr) {
   constexpr int VEC = Elem<T>::kVec;
   const int lane = tid & 31, warp = tid >> 5;
@@ -1442,8 +1446,8 @@ __device__ __forceinline__ void load_stage(const uint32_t base, const int n, con
 
 // RAGGED: V is not a whole number of stages, so the last stage of a row is partly filled (the host
 // picks the instance; without it the streaming loop has no bounds tests at all).
-template <typename T, bool CFG, bool RAGGED>
-__global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const FusedArgs a) {
+template <typename T, bool CFG, bool RAGGED, int WL>
+__global__ void __launch_bounds__(kTopkThreads, WL == kWarpList ? 4 : 3) verify_topk_kernel(const FusedArgs a) {
   constexpr int VEC = Elem<T>::kVec;
   constexpr int ARR = CFG ? 2 : 1;
   constexpr int ES = (int)sizeof(T);
@@ -1452,7 +1456,9 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   constexpr int NVS = VPT / VEC;                                // 16-byte vectors per thread per stage
   static_assert(kTkStages == 2, "stage and parity of a chunk are taken from the low bits of its index");
   extern __shared__ __align__(128) unsigned char fused_smem_raw[];
-  TopkSmem& sm = *reinterpret_cast<TopkSmem*>(fused_smem_raw);
+  using Smem = TopkSmemT<WL>;
+  constexpr int kListCap = kTopkWarps * WL;
+  Smem& sm = *reinterpret_cast<Smem*>(fused_smem_raw);
 
   // the next call on the stream may start: see the head of this file (a stats-only call is followed by
   // its finishing kernel, whose large blocks would only sit on SMs this kernel needs: it follows at exit)
@@ -1625,7 +1631,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
         const uint32_t total = __reduce_add_sync(0xffffffffu, cnt);
         const uint32_t pos = wcur + below;
         wcur += total;
-        if (pos + cnt <= (uint32_t)kWarpList) {
+        if (pos + cnt <= (uint32_t)WL) {
           uint32_t addr = list_mine + 4u * pos;
 #pragma unroll
           for (int e = 0; e < VPT; ++e) {
@@ -1643,7 +1649,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
       __syncwarp();
       const int wc = (int)wcur;
       int wcp = 0;   // padded length; 0 if the list overflowed (the row is then selected exactly)
-      if (wc <= kWarpList) {
+      if (wc <= WL) {
         wcp = (wc + 31) & ~31;
         if (wc + lane < wcp) sm.list[warp][wc + lane] = CSD_NEG_INF;
       }
@@ -1698,7 +1704,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
           const bool mine = lane < kTopkWarps;
           float m = mine ? sm.fw_m[lane] : CSD_NEG_INF, sv = mine ? sm.fw_s[lane] : -1.0f;
           int n_lo = mine ? sm.wpos[lane] : 0;
-          const bool over = __any_sync(0xffffffffu, n_lo > kWarpList);
+          const bool over = __any_sync(0xffffffffu, n_lo > WL);
           const bool nan_m = __any_sync(0xffffffffu, m != m);
           n_lo = __reduce_add_sync(0xffffffffu, n_lo);
           const int cg = __reduce_add_sync(0xffffffffu, mine ? sm.fw_cgt[lane] : 0);
@@ -1754,7 +1760,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
 #pragma unroll
         for (int w = 0; w < kTopkWarps; ++w) {
           const int cw = sm.wpos[w];
-          if (cw > kWarpList) fast = false;
+          if (cw > WL) fast = false;
           n_lo += cw;
           m = max_nan(m, sm.wmax[w]);
         }
@@ -1870,7 +1876,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
     for (int r = 0; r < n_rows && r < kBlockRows; ++r) {
       if (((sm.need_exact[r >> 5] >> (r & 31)) & 1u) == 0u) continue;   // the same decision in every thread
       float m_e = 0.0f, s_e = 0.0f, thr_e = 0.0f;
-      exact_row_from_global<T, CFG>(row_of(r), V, k_top, sm, tid, m_e, s_e, thr_e);
+      exact_row_from_global<T, CFG, Smem>(row_of(r), V, k_top, sm, tid, m_e, s_e, thr_e);
       if (tid == 0) {
         sm.rs.ms[r] = make_float2(m_e, s_e);
         sm.rs.thr[r] = thr_e;

@@ -195,6 +195,25 @@ def test_topk_with_masked_and_tied_rows():
     assert_ok(rep)
 
 
+@pytest.mark.parametrize("kw", [dict(V=65536, dtype=W.BF16, cfg=True, cfg_scale=3.0, top_k=2000),
+                                dict(V=32768, dtype=W.F32, top_k=2400),
+                                dict(V=50000, dtype=W.BF16, cfg=True, top_k=1800),
+                                dict(V=65536, dtype=W.BF16, top_k=2000, law="student3"),
+                                dict(V=20000, dtype=W.F32, cfg=True, top_k=1400)])
+@pytest.mark.parametrize("b2b", [False, True])
+def test_topk_beyond_the_small_lists(kw, b2b):
+    """k between about 1200 and 2400 (a 65536-token vocabulary filtered to its 2000 best, say): the
+    streaming selection runs on the instance of the kernel with the larger candidate lists; whole and
+    ragged rows, Gaussian and heavy-tailed logits."""
+    L = 4
+    w = W.make("t", B=10, gamma=L, rho=0.9, bonus_row=True, schedule=sched(L), seed=kw["V"] % 97, device=DEV, **kw)
+    w.target_logits[1, 0, :] = torch.round(w.target_logits[1, 0, :])     # heavy ties around the threshold
+    rep, got, ref = check(w, back_to_back=b2b, want_dbg=False)
+    assert_ok(rep)
+    rep, got, ref = check(w, back_to_back=b2b)                            # with G: the full selection, exact thresholds
+    assert_ok(rep)
+
+
 @pytest.mark.parametrize("kw", [
     dict(B=64, gamma=8, V=16384, dtype=W.F32),
     dict(B=64, gamma=8, V=16384, dtype=W.BF16, cfg=True, top_k=1000),
