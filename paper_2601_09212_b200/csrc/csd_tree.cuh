@@ -39,6 +39,11 @@ struct TreeSmem {
   FinishSmem pick;             // Z, tile and prefix of the draw
   int path_tok[kMaxTreeDepth + 1];
   int path_node[kMaxTreeDepth];
+  // fetched for all nodes at once before the walk, so that its accept tests wait for no memory: every
+  // node's token, that token's (filtered) logits in the two rows of its parent's context, its uniform
+  int tok[kMaxTreeNodes];
+  float tokz[2][kMaxTreeNodes];
+  float uni[kMaxTreeNodes];
 };
 
 // Unnormalised residual after `k` rejections at one token: g_k(x), where g_1 = [P - min{Q, omega P}]_+
@@ -96,6 +101,23 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
   }
   __syncthreads();
 
+  if (tid < N) {
+    const int n = tid, c = a.parent[n] + 1;
+    const int tok = f.tokens[(int64_t)b * N + n];
+    sm.tok[n] = tok;
+    sm.uni[n] = f.uniforms[(int64_t)b * (N + 1) + n];
+    float zt = 0.0f, zd = 0.0f;
+    if (tok >= 0 && tok < V && sm.valid[0][c] && sm.valid[1][c]) {
+      const Row<T, CFG> qt{tgt + (int64_t)c * V, CFG ? tgt_u + (int64_t)c * V : nullptr, f.cfg_scale, sm.thr[0][c] CSD_ROW_LEN(V)};
+      const Row<T, CFG> qd{dft + (int64_t)c * V, CFG ? dft_u + (int64_t)c * V : nullptr, f.cfg_scale, sm.thr[1][c] CSD_ROW_LEN(V)};
+      zt = qt.filter(qt.load_one(tok));
+      zd = qd.filter(qd.load_one(tok));
+    }
+    sm.tokz[0][n] = zt;
+    sm.tokz[1][n] = zd;
+  }
+  __syncthreads();
+
   // ---- the walk (every thread follows it; thread 0 takes the accept decisions) ---------------
   const float u = f.uniforms[(int64_t)b * (N + 1) + N];
   int status = 0, level = 0, ctx = 0, token = -1;
@@ -132,14 +154,14 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
       if (a.parent[n] != ctx - 1) continue;
       // ---- accept test of candidate n against the residual after k rejections -------------------
       if (tid == 0) {
-        const int tok = f.tokens[(int64_t)b * N + n];
+        const int tok = sm.tok[n];
         const bool tok_ok = tok >= 0 && tok < V;
         float fa = 0.0f;
         int flag = 0;
         if (!t_ok || !d_ok) flag = 1;
         else if (!tok_ok) flag = 2;
         else {
-          const float zt = rt.filter(rt.load_one(tok)), zd = rd.filter(rd.load_one(tok));
+          const float zt = sm.tokz[0][n], zd = sm.tokz[1][n];
           const float dt = zt - pc.Mt, dd = zd - pc.Md;
           if (dd == CSD_NEG_INF) fa = 1.0f;            // q = 0: p/q = +inf, and 0/0 := 1
           else if (k == 0) {
@@ -151,7 +173,7 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
             fa = R > 0.0f ? fminf(1.0f, omega * R / Q) : 0.0f;
           }
         }
-        const float r = f.uniforms[(int64_t)b * (N + 1) + n];
+        const float r = sm.uni[n];
         sm.decision = ((r <= fa) ? 1 : 0) | (flag << 1);
       }
       __syncthreads();
