@@ -2,6 +2,8 @@
 seeded inputs and the same supplied uniforms.  Accepted lengths and tokens must be identical
 except for decisions the oracle flags as within 1e-6 of a threshold (counted); probabilities and
 the resampling distribution within 1e-5 (fp32 logits) / 2e-3 (bf16 logits) absolute."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -286,10 +288,15 @@ def _random_case(i):
         kw["top_k"] = int(min(V - 1, r.choice([1, 7, 100, 1000])))
     if r.integers(4) == 0:
         kw["law"] = "student3"                     # heavy tails: the selection's guess misses and adapts
-    return kw, bool(r.integers(2))
+    b2b = bool(r.integers(2))
+    r2 = np.random.default_rng(7000 + i)           # (a second stream, so that the cases above stay what they were)
+    if r2.integers(4) == 0 and V >= 8192:          # k beyond the small candidate lists, and beyond the large ones
+        kw["top_k"] = int(min(V - 1, r2.choice([1200, 1500, 2000, 2400, 3000])))
+    return kw, b2b
 
 
-@pytest.mark.parametrize("i", range(96))
+# CSD_SWEEP_CASES=8000 runs the same sweep over that many cases (about six minutes on a B200)
+@pytest.mark.parametrize("i", range(int(os.environ.get("CSD_SWEEP_CASES", "96"))))
 def test_seeded_sweep_of_partitions(i):
     kw, b2b = _random_case(i)
     L = kw["gamma"]
