@@ -144,3 +144,37 @@ def test_tree_argument_errors():
     assert lib.csd_tree_depth(many.ctypes.data_as(C.c_void_p), 9) == -2     # more than 8 candidates of one node
     assert lib.csd_verify_tree(None) == -1
     assert csd.csd_tree_workspace_size(4, 64, 1000, 0) == 0 and csd.csd_tree_workspace_size(4, 63, 1000, 0) > 0
+
+
+@pytest.mark.parametrize("i", range(24))
+def test_seeded_sweep_of_random_trees(i):
+    """Random trees (up to 39 nodes, up to 8 candidates per node, any depth the limits allow), vocabularies
+    with and without a ragged tail, both dtypes, guidance mix, top-k below and above the small candidate
+    lists, heavy-tailed logits, batch sizes 1 - 40, multipliers on both sides of 1."""
+    r = np.random.default_rng(50000 + i)
+    N = int(r.integers(1, 40))
+    parent, kids, depth = [], {}, {}
+    for n in range(N):
+        while True:
+            p = int(r.integers(-1, n))
+            d = 0 if p < 0 else depth[p] + 1
+            if kids.get(p, 0) < 8 and d < 31:
+                break
+        parent.append(p); kids[p] = kids.get(p, 0) + 1; depth[n] = d
+    parent = np.array(parent, np.int32)
+    D = oracle.tree_depth(parent)
+    V = int(r.choice([66, 1000, 2048, 4100, 8192, 16384, 20000]))
+    kw = dict(V=V, dtype=[W.F32, W.BF16][int(r.integers(2))])
+    if r.integers(3) == 0:
+        kw["cfg"] = True
+    if r.integers(2) == 0:
+        kw["top_k"] = int(min(V - 1, r.choice([5, 100, 1000, 1500])))
+    if r.integers(5) == 0:
+        kw["law"] = "student3"
+    B = int(r.choice([1, 3, 17, 40]))
+    sched = (np.exp(-0.3 * np.arange(D)) * r.choice([1.0, 1.5, 3.0])).astype(np.float32)
+    w = W.make_tree(parent, B=B, rho=float(r.choice([0.7, 0.9, 0.99])), schedule=sched, seed=i, device=DEV, **kw)
+    got, ref = run_tree_gpu(w, want_G=B * V <= 2e6), run_tree_oracle(w)
+    n_near, bad = compare_tree(w, got, ref)
+    assert not bad, (N, D, kw, B, bad[:3])
+    assert n_near <= 2
