@@ -1565,19 +1565,54 @@ __global__ void __launch_bounds__(kTopkThreads, WL == kWarpList ? 4 : 3) verify_
           }
         }
         if (c == 0) {
-          // the first stage is the sample for the threshold guess
-          float sum1 = 0.0f, sum2 = 0.0f;
+          // The first stage is the sample for the threshold guess: its mean, and as its scale the mean
+          // ABSOLUTE deviation (each warp about its own mean, over every other 16-byte vector of the
+          // sample), which heavy-tailed logits do not throw about from row to row the way they do the
+          // standard deviation -- and in whose units the upper quantiles of a Gaussian and of a
+          // Student-t with three degrees of freedom nearly coincide, so one multiplier serves both.
+          float sum1 = 0.0f, sum2 = 0.0f, sum2b = 0.0f;
+          uint64_t sum1p = pack2(0.0f, 0.0f);   // (two values per addition)
+          int mine_n = 0;
 #pragma unroll
           for (int v = 0; v < NVS; ++v) {
             if (!RAGGED || (v * kTopkThreads + tid) * VEC < n) {
 #pragma unroll
-              for (int e = 0; e < VEC; ++e) { sum1 += z[v * VEC + e]; sum2 = fmaf(z[v * VEC + e], z[v * VEC + e], sum2); }
+              for (int e = 0; e < VEC; e += 2) sum1p = add2(sum1p, pack2(z[v * VEC + e], z[v * VEC + e + 1]));
+              mine_n += VEC;
             }
           }
+          { float s_lo, s_hi; unpack2(sum1p, s_lo, s_hi); sum1 = s_lo + s_hi; }
 #pragma unroll
-          for (int off = 16; off > 0; off >>= 1) {
-            sum1 += __shfl_xor_sync(0xffffffffu, sum1, off);
-            sum2 += __shfl_xor_sync(0xffffffffu, sum2, off);
+          for (int off = 16; off > 0; off >>= 1) sum1 += __shfl_xor_sync(0xffffffffu, sum1, off);
+          const float wmean = RAGGED ? sum1 * rcp_approx((float)max(1, __reduce_add_sync(0xffffffffu, mine_n)))
+                                     : sum1 * (1.0f / (float)(32 * VPT));
+          const uint64_t nwm2 = pack2(-wmean, -wmean);
+          int dev_n = 0;   // values this thread put into the deviation sum
+#pragma unroll
+          for (int v = 0; v < NVS; v += 2) {
+            if (!RAGGED || (v * kTopkThreads + tid) * VEC < n) {
+#pragma unroll
+              for (int e = 0; e < VEC; e += 2) {
+                float d0, d1;
+                unpack2(add2(pack2(z[v * VEC + e], z[v * VEC + e + 1]), nwm2), d0, d1);
+                sum2 += fabsf(d0);
+                sum2b += fabsf(d1);
+              }
+              dev_n += VEC;
+            }
+          }
+          sum2 += sum2b;
+          // (the sum goes to the block as a mean over the warp's share, scaled back to the sample's size)
+          {
+            float cntf = RAGGED ? (float)dev_n : (float)(VEC * ((NVS + 1) / 2));
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+              sum2 += __shfl_xor_sync(0xffffffffu, sum2, off);
+              if (RAGGED) cntf += __shfl_xor_sync(0xffffffffu, cntf, off);
+            }
+            if (!RAGGED) cntf *= 32.0f;
+            const float warp_n = RAGGED ? (float)__reduce_add_sync(0xffffffffu, mine_n) : (float)(32 * VPT);
+            sum2 = cntf > 0.0f ? sum2 * (warp_n * rcp_approx(cntf)) : 0.0f;
           }
           if (lane == 0) { sm.mom[0][warp] = sum1; sm.mom[1][warp] = sum2; }
           __syncthreads();   // ---- S0: moments, cleared histogram and list cursors; the previous row is complete
@@ -1593,7 +1628,8 @@ __global__ void __launch_bounds__(kTopkThreads, WL == kWarpList ? 4 : 3) verify_
           // (a guess: approximate reciprocal and root are enough, every thread gets the same bits)
           const float inv_n = RAGGED ? rcp_approx((float)n) : 1.0f / (float)EPS;
           const float mean = s1 * inv_n;
-          dev = sqrt_approx(fmaxf(s2 * inv_n - mean * mean, 0.0f));
+          // (sqrt(pi / 2) x mean absolute deviation is the standard deviation, were the row Gaussian)
+          dev = 1.2533141f * (s2 * inv_n);
           lo = mean + sm.c_kind[par] * dev;
           scale = ((float)kLinBins / kLinRangeSigmas) * rcp_approx(dev);
           if (tid == 0) { sm.row_mean[par] = mean; sm.row_dev[par] = dev; }
