@@ -177,12 +177,18 @@ cudaError_t launch_select(const SelectArgs& a, int sms, cudaStream_t stream) {
 }
 
 template <typename T, bool CFG>
-cudaError_t launch_finish(const FinishArgs& a, cudaStream_t stream) {
+cudaError_t launch_finish(const FinishArgs& a_in, cudaStream_t stream) {
   auto kern = finish_kernel<T, CFG>;
   constexpr int TILE = 32 * Elem<T>::kVec;
+  FinishArgs a = a_in;
   size_t slots = (size_t)((a.V + TILE - 1) / TILE);
   if (slots < 2 * (kFinishThreads / 32)) slots = 2 * (kFinishThreads / 32);   // the monitors' two sums per warp
-  const size_t smem = slots * sizeof(double);
+  size_t smem = slots * sizeof(double);
+  a.nbr_table_off = 0;
+  if (a.nbr != nullptr && smem + (size_t)a.V * sizeof(float) <= 200 * 1024) {   // the similarity relaxation's table of P
+    a.nbr_table_off = (int)slots;
+    smem += (size_t)a.V * sizeof(float);
+  }
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

@@ -490,6 +490,8 @@ struct FinishArgs {
   const int32_t* nbr;   // [V, nbr_k] or null: every token's nearest tokens, nearest first (-1: none)
   int nbr_k;
   float nbr_lambda;
+  int nbr_table_off;    // > 0: the block's dynamic shared memory has room for a float[V] table of the target's
+                        //      probabilities at this offset (in doubles, after the tile sums); 0: look them up in global memory
 };
 
 struct PairCtx {  // what Eq. opt_G needs at one position
@@ -526,6 +528,20 @@ __device__ __forceinline__ float neighbour_extra(const RowT& rt, const float Mt,
     const int y = __ldg(nbr + (int64_t)x * k + j);
     if (y < 0 || y >= V || y == x) continue;
     const float py = ex2f((rt.filter(rt.load_one(y)) - Mt) * kLog2e) * inv_t;
+    if (extra + py < budget) extra += py;
+    else break;
+  }
+  return extra;
+}
+// The same selection with the target's probabilities read from a table (shared memory).
+__device__ __forceinline__ float neighbour_extra_table(const float* tP, const int32_t* nbr, const int k, const float lambda,
+                                                       const int x, const int V, const float own) {
+  float extra = 0.0f;
+  const float budget = lambda * own;
+  for (int j = 0; j < k; ++j) {
+    const int y = __ldg(nbr + (int64_t)x * k + j);
+    if (y < 0 || y >= V || y == x) continue;
+    const float py = tP[y];
     if (extra + py < budget) extra += py;
     else break;
   }
@@ -767,14 +783,32 @@ __device__ void finish_sequence(const FinishArgs& a, const int b, const int tid,
     if (j < L) rd = Row<T, CFG>{dft + (int64_t)j * V, CFG ? dft_u + (int64_t)j * V : nullptr, a.cfg_scale, sm.thr[1][j] CSD_ROW_LEN(V)};
     const float u = a.uniforms[(int64_t)b * (L + 1) + L];
     // (omega >= 1: the aggregated mass only raises f above f_van, and Eq. opt_G is the vanilla residual)
-    const bool similar = a.nbr != nullptr && j < L && omega < 1.0f;
+    const bool similar = a.nbr != nullptr && j < L && omega < 1.0f && ctx.mode == 0;
+    // Every candidate with target mass then needs the mass of up to k neighbours: where the block's shared
+    // memory has room, the target's probabilities are tabulated there once (the same expression, hence the
+    // same bits, as a lookup in global memory would evaluate) and the lookups stay on the SM.
+    float* const tP = (similar && a.nbr_table_off > 0) ? reinterpret_cast<float*>(tile_sums + a.nbr_table_off) : nullptr;
+    if (tP) {
+      for (int tile = warp; tile < ntiles; tile += NT / 32) {
+        const int x0 = tile * TILE + lane * VEC;
+        float zt[VEC];
+        rt.load_tile(x0, V, a.vec_ok, zt);
+#pragma unroll
+        for (int k = 0; k < VEC; ++k)
+          if (x0 + k < V) tP[x0 + k] = ex2f((rt.filter(zt[k]) - ctx.Mt) * kLog2e) * ctx.inv_t;
+      }
+      group_sync<NT, BAR>();
+    }
     auto weight_at = [&](int x, float zt_x, float zd_x) -> float {
       const float ft = rt.filter(zt_x);
       if (ctx.mode != 0) return weight_of(ft, 0.0f, ctx);
       const float fd = rd.filter(zd_x);
       if (!similar || x >= V) return weight_of(ft, fd, ctx);
       const float own = ex2f((ft - ctx.Mt) * kLog2e) * ctx.inv_t;
-      const float extra = own > 0.0f ? neighbour_extra(rt, ctx.Mt, ctx.inv_t, a.nbr, a.nbr_k, a.nbr_lambda, x, V, own) : 0.0f;
+      float extra = 0.0f;
+      if (own > 0.0f)
+        extra = tP ? neighbour_extra_table(tP, a.nbr, a.nbr_k, a.nbr_lambda, x, V, own)
+                   : neighbour_extra(rt, ctx.Mt, ctx.inv_t, a.nbr, a.nbr_k, a.nbr_lambda, x, V, own);
       return weight_of_similar(ft, fd, ctx, extra);
     };
 
