@@ -599,12 +599,18 @@ int csd_test_hooks(int wait_limit_log2_cycles, int drop_first_copy) {
 }  // extern "C"
 namespace {
 template <typename T, bool CFG>
-cudaError_t launch_tree_finish(const TreeArgs& a, cudaStream_t stream) {
+cudaError_t launch_tree_finish(const TreeArgs& a_in, cudaStream_t stream) {
   auto kern = tree_finish_kernel<T, CFG>;
   constexpr int TILE = 32 * Elem<T>::kVec;
+  TreeArgs a = a_in;
   size_t slots = (size_t)((a.fin.V + TILE - 1) / TILE);
   if (slots < 64) slots = 64;
-  const size_t smem = slots * sizeof(double);
+  size_t smem = slots * sizeof(double);
+  a.tab_off = 0;
+  if (smem + 2 * (size_t)a.fin.V * sizeof(float) <= 200 * 1024) {   // the walk's tables of the residual and of Q
+    a.tab_off = (int)slots;
+    smem += 2 * (size_t)a.fin.V * sizeof(float);
+  }
   if (smem > 40 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

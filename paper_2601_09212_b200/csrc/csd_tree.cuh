@@ -27,6 +27,8 @@ struct TreeArgs {
                          // out_tokens [B, D + 1]
   int N, D;
   int32_t* out_nodes;    // [B, D] or null
+  int tab_off;           // > 0: the block's dynamic shared memory holds, at this offset (in doubles, after the tile
+                         //      sums), two float[V] tables (see the kernel); 0: no room for them
   signed char parent[kMaxTreeNodes + 1];
 };
 
@@ -77,6 +79,12 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
   const int N = a.N, C = N + 1, V = f.V, D = a.D;
   const int rows_per_seq = 2 * C;
   const int ntiles = (V + TILE - 1) / TILE;
+  // Where they fit, two tables over the vocabulary live in shared memory while the walk stays in one
+  // context: the current residual g_k(x) and the drafter's Q(x).  A rejection then updates the residual
+  // in place (a few operations per token) instead of running the k-step recursion from the logits again;
+  // the values are the same bits either way.
+  float* const tabG = a.tab_off > 0 ? reinterpret_cast<float*>(tile_sums + a.tab_off) : nullptr;
+  float* const tabQ = tabG ? tabG + V : nullptr;
   const T* tgt = reinterpret_cast<const T*>(f.target) + (int64_t)b * f.tstride;
   const T* dft = reinterpret_cast<const T*>(f.draft) + (int64_t)b * f.dstride;
   const T* tgt_u = CFG ? reinterpret_cast<const T*>(f.target_uncond) + (int64_t)b * f.tstride : nullptr;
@@ -126,6 +134,7 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
   PairCtx pc;
   Row<T, CFG> rt, rd;
   float omega = 0.0f;
+  bool use_tab = false;   // the current context's residual and Q are tabulated (once it has had a rejection)
   for (;;) {
     const bool t_ok = sm.valid[0][ctx] != 0;
     rt = Row<T, CFG>{tgt + (int64_t)ctx * V, CFG ? tgt_u + (int64_t)ctx * V : nullptr, f.cfg_scale, sm.thr[0][ctx] CSD_ROW_LEN(V)};
@@ -137,6 +146,7 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
       if (a.parent[n] == ctx - 1) { first_child = n; break; }
     k = 0;
     if (first_child < 0 || level >= D) {   // a leaf: bonus token from the target's distribution here
+      use_tab = false;
       pc.mode = 1; pc.Md = 0.0f; pc.Sd = 0.0f; pc.inv_den = pc.inv_t; pc.one_minus_omega = 1.0f;
       if (!t_ok) status |= 1;
       drew = t_ok;
@@ -150,6 +160,7 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
     omega = omega >= 0.0f ? omega : 0.0f;
     pc.one_minus_omega = 1.0f - omega;
     int accepted = -1;
+    use_tab = tabG != nullptr && pc.mode == 0 && t_ok;   // (the same in every thread; tables are filled by this context's first rejection)
     for (int n = first_child; n < N; ++n) {
       if (a.parent[n] != ctx - 1) continue;
       // ---- accept test of candidate n against the residual after k rejections -------------------
@@ -168,7 +179,7 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
             if (dt == CSD_NEG_INF) fa = 0.0f;          // p = 0 < q
             else fa = fminf(1.0f, omega * ex2f((dt - dd) * kLog2e) * ((1.0f + pc.Sd) / (1.0f + pc.St)));
           } else {
-            const float R = residual_of(zt, zd, pc, omega, k, sm.inv_z, sm.keep) * sm.inv_z[k - 1];
+            const float R = (use_tab ? tabG[tok] : residual_of(zt, zd, pc, omega, k, sm.inv_z, sm.keep)) * sm.inv_z[k - 1];
             const float Q = ex2f(dd * kLog2e) / (1.0f + pc.Sd);
             fa = R > 0.0f ? fminf(1.0f, omega * R / Q) : 0.0f;
           }
@@ -187,15 +198,50 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
       if (tid == 0) sm.keep[k] = 0;
       __syncthreads();
       for (int attempt = 0; attempt < 2; ++attempt) {
+        if (use_tab && k >= 1 && attempt == 1) {
+          // the update found an empty positive part and has overwritten the table: bring g_k back from the logits
+          for (int tile = warp; tile < ntiles; tile += NT / 32) {
+            const int x0 = tile * TILE + lane * VEC;
+            float zt[VEC], zd[VEC];
+            rt.load_tile(x0, V, f.vec_ok, zt);
+            rd.load_tile(x0, V, f.vec_ok, zd);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e)
+              if (x0 + e < V) tabG[x0 + e] = residual_of(rt.filter(zt[e]), rd.filter(zd[e]), pc, omega, k, sm.inv_z, sm.keep);
+          }
+          __syncthreads();
+        }
         for (int tile = warp; tile < ntiles; tile += NT / 32) {
           const int x0 = tile * TILE + lane * VEC;
-          float zt[VEC], zd[VEC];
-          rt.load_tile(x0, V, f.vec_ok, zt);
-          if (pc.mode == 0) rd.load_tile(x0, V, f.vec_ok, zd);
           float acc = 0.0f;
+          if (use_tab && k >= 1) {
+            // g_{k+1} from the tabulated g_k and Q: the last step of residual_of's recursion
+            const float iz = sm.inv_z[k - 1];
+            const bool kp = sm.keep[k] != 0;
 #pragma unroll
-          for (int e = 0; e < VEC; ++e)
-            acc += residual_of(rt.filter(zt[e]), pc.mode == 0 ? rd.filter(zd[e]) : 0.0f, pc, omega, k + 1, sm.inv_z, sm.keep);
+            for (int e = 0; e < VEC; ++e) {
+              if (x0 + e < V) {
+                const float R = tabG[x0 + e] * iz;
+                const float gn = kp ? R : fmaxf(0.0f, R - fminf(tabQ[x0 + e], omega * R));
+                tabG[x0 + e] = gn;
+                acc += gn;
+              }
+            }
+          } else {
+            float zt[VEC], zd[VEC];
+            rt.load_tile(x0, V, f.vec_ok, zt);
+            if (pc.mode == 0) rd.load_tile(x0, V, f.vec_ok, zd);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+              const float ft = rt.filter(zt[e]), fd = pc.mode == 0 ? rd.filter(zd[e]) : 0.0f;
+              const float gn = residual_of(ft, fd, pc, omega, k + 1, sm.inv_z, sm.keep);
+              if (use_tab && x0 + e < V) {   // (k == 0: the tables are filled here)
+                tabG[x0 + e] = gn;
+                tabQ[x0 + e] = ex2f((fd - pc.Md) * kLog2e) / (1.0f + pc.Sd);
+              }
+              acc += gn;
+            }
+          }
           const double tsum = warp_sum_double((double)acc);
           if (lane == 0) tile_sums[tile] = tsum;
         }
@@ -255,11 +301,16 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
         if (tile >= 0) {
           const int x0 = tile * TILE + lane * VEC;
           float zt[VEC], zd[VEC], g[VEC];
-          rt.load_tile(x0, V, f.vec_ok, zt);
-          if (pc.mode == 0 && k > 0) rd.load_tile(x0, V, f.vec_ok, zd);
+          if (use_tab && k > 0) {
 #pragma unroll
-          for (int e = 0; e < VEC; ++e)
-            g[e] = residual_of(rt.filter(zt[e]), (pc.mode == 0 && k > 0) ? rd.filter(zd[e]) : 0.0f, pc, omega, k, sm.inv_z, sm.keep);
+            for (int e = 0; e < VEC; ++e) g[e] = x0 + e < V ? tabG[x0 + e] : 0.0f;
+          } else {
+            rt.load_tile(x0, V, f.vec_ok, zt);
+            if (pc.mode == 0 && k > 0) rd.load_tile(x0, V, f.vec_ok, zd);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e)
+              g[e] = residual_of(rt.filter(zt[e]), (pc.mode == 0 && k > 0) ? rd.filter(zd[e]) : 0.0f, pc, omega, k, sm.inv_z, sm.keep);
+          }
           tok = pick_in_tile<VEC>(g, x0, sm.pick.pick_prefix, (double)u * Z, lane);
         }
         if (lane == 0) sm.pick.token = tok;
@@ -276,6 +327,12 @@ __global__ void __launch_bounds__(kFinishThreads, 1) tree_finish_kernel(const Tr
       for (int tile = warp; tile < ntiles; tile += NT / 32) {
         const int x0 = tile * TILE + lane * VEC;
         float zt[VEC], zd[VEC];
+        if (use_tab && k > 0) {
+#pragma unroll
+          for (int e = 0; e < VEC; ++e)
+            if (x0 + e < V) G_out[x0 + e] = tabG[x0 + e] * invZ;
+          continue;
+        }
         rt.load_tile(x0, V, f.vec_ok, zt);
         if (pc.mode == 0 && k > 0) rd.load_tile(x0, V, f.vec_ok, zd);
 #pragma unroll
