@@ -11,8 +11,9 @@
 // model's output in context c.  The row statistics of all 2 (N + 1) rows come from the kernels of
 // csd_kernels.cuh (a call looks to them like a chain of N + 1 positions); tree_finish_kernel, one
 // block per sequence, then walks the tree.  Every rejection costs one pass over the two rows of the
-// current context (its normaliser Z), and the residual after k rejections is evaluated token by
-// token by running the k-step recursion, so nothing of length V is ever stored.
+// current context (its normaliser Z).  The residual after k rejections is evaluated token by token
+// by running the k-step recursion from the two logits; where two float[V] tables fit the block's shared
+// memory, the residual and Q of the current context are kept there instead and updated in place.
 #pragma once
 #include "csd_kernels.cuh"
 
