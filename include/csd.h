@@ -172,7 +172,9 @@ typedef struct csd_params {
   const void* target_uncond; /* same layout as target_logits, or NULL               */
   const void* draft_uncond;  /* same layout as draft_logits; NULL iff target_uncond */
   float cfg_scale;           /* s in uncond + s*(cond - uncond); unused without uncond */
-  int32_t top_k;             /* 0 or >= V: off                                      */
+  int32_t top_k;             /* 0 or >= V: off.  Any k gives the exact filter (every logit >= the k-th
+                                largest of its row is kept); k up to about 2400 runs at streaming speed,
+                                larger k selects every row by radix, several times slower */
   int32_t dtype;             /* csd_dtype of all four logit arrays                  */
   int32_t B, gamma, V;
   int32_t target_rows;         /* gamma or gamma + 1                                */
