@@ -19,7 +19,7 @@ namespace {
 using namespace csd;
 
 static_assert(sizeof(TopkSmem) <= 55 * 1024, "four blocks of the top-k kernel per SM must fit");
-static_assert(sizeof(TopkSmemT<kWarpListLarge>) <= 74 * 1024, "three blocks of its large-list instance per SM must fit");
+static_assert(sizeof(TopkSmemT<kWarpListLarge>) <= 56 * 1024, "four blocks of its large-list instance per SM must fit");
 static_assert(sizeof(PlainSmem) <= 75 * 1024, "three blocks of the plain kernel per SM must fit");
 
 constexpr int kMaxV = 1 << 20;
@@ -252,12 +252,11 @@ cudaError_t plan_and_launch_fused(const FusedPlan& in) {
     // ctas_per_seq blocks of one cluster (each with both rows of its positions; 2, 4 or 8 blocks)
     // until the GPU is full.
     const long long merge_above = 8LL * sms;   // beyond this many sequences a block takes several
-    // (measured: the top-k kernel, with its longer per-row work, gains from the finer split; its
-    // large-list instance has three blocks per SM, and a lone call should fit one wave)
+    // (measured: the top-k kernel, with its longer per-row work, gains from the finer split)
     const double tk_k = in.top_k, tk_v = in.V;
     const double tk_tail = 1.25 * tk_k / tk_v + 4.0 * sqrt(tk_k) / tk_v + 16.0 / tk_v;
     const bool tk_large = topk && tk_tail * tk_v >= 0.8 * (kTopkWarps * kWarpList);
-    const long long split_below = in.back_to_back ? 16 : (topk ? (tk_large ? 3LL : 4LL) : 2LL) * sms;
+    const long long split_below = in.back_to_back ? 16 : (topk ? 4LL : 2LL) * sms;
     long long c = 1, spc = 1;
     if (in.B > merge_above) spc = (in.B + merge_above - 1) / merge_above;
     else if (in.B < split_below) {

@@ -246,7 +246,8 @@ __device__ __forceinline__ Row<T, CFG> row_at(const FinishArgs& f, int b, int wh
   }
   return row;
 }
-constexpr int kBlockRows = 264;   // local rows a block may own (the host keeps it within this)
+constexpr int kBlockRows = 128;   // local rows a block may own (the host keeps it within this; a tree's 64 contexts
+                                  // are 128 rows)
 
 // Per-row results of phase 1, in shared memory until the block's own finish consumes them.
 struct RowStats {
@@ -1251,7 +1252,7 @@ constexpr int kTkStageBytes = 16384;
 constexpr int kTkRingBytes = kTkStages * kTkStageBytes;
 constexpr int kWarpList = 256;                // per-warp capacity of the list of values >= lo: the instance that
                                               // leaves room for four blocks per SM ...
-constexpr int kWarpListLarge = 512;           // ... and the one for larger k (three blocks per SM)
+constexpr int kWarpListLarge = 512;           // ... and the one for larger k (four as well, with 300 bytes to spare)
 constexpr int kLinBins = 512;
 constexpr int kCandCap = 64;
 constexpr float kLinRangeSigmas = 4.75f;      // the histogram spans [lo, lo + this many deviations)
@@ -1284,6 +1285,7 @@ struct TopkSmemT {
   int fw_cgt[kTopkWarps], fw_rk[kTopkWarps];
   int short_on;                     // cleared once a row has failed the short cut's test: the block stops trying
   int row_short;                    // this row was settled by the short cut
+  int short_fail;                   // rows that failed the short cut's test so far
   int bc_i[4];
   int arrive[2];                    // warps that have finished the first / the second pass over their lists
   float row_mx;                     // set by the warp that picks the bin: the row maximum, and whether the
@@ -1447,7 +1449,7 @@ __device__ __forceinline__ void load_stage(const uint32_t base, const int n, con
 // RAGGED: V is not a whole number of stages, so the last stage of a row is partly filled (the host
 // picks the instance; without it the streaming loop has no bounds tests at all).
 template <typename T, bool CFG, bool RAGGED, int WL>
-__global__ void __launch_bounds__(kTopkThreads, WL == kWarpList ? 4 : 3) verify_topk_kernel(const FusedArgs a) {
+__global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const FusedArgs a) {
   constexpr int VEC = Elem<T>::kVec;
   constexpr int ARR = CFG ? 2 : 1;
   constexpr int ES = (int)sizeof(T);
@@ -1483,6 +1485,7 @@ __global__ void __launch_bounds__(kTopkThreads, WL == kWarpList ? 4 : 3) verify_
     sm.adapt_on = 0;
     sm.short_on = (a.hi_delta == a.hi_delta && a.fin.dbg_G == nullptr) ? 1 : 0;
     sm.row_short = 0;
+    sm.short_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < (kBlockRows + 31) / 32) sm.need_exact[tid] = 0u;
@@ -1701,7 +1704,7 @@ __global__ void __launch_bounds__(kTopkThreads, WL == kWarpList ? 4 : 3) verify_
       // (fewer than k gathered values above its logit).  One pass over the lists and one barrier
       // instead of a histogram, a selection and two barriers; rows that fail the test (flat rows,
       // where the values near the threshold carry weight) take the full selection below, on the same
-      // lists, and the block stops trying.
+      // lists; after three such rows the block stops trying.
       if (sm.short_on) {
         float mw = CSD_NEG_INF;
         for (int i = lane; i < wcp; i += 32) mw = max_nan(mw, sm.list[warp][i]);
@@ -1759,7 +1762,9 @@ __global__ void __launch_bounds__(kTopkThreads, WL == kWarpList ? 4 : 3) verify_
               sm.rs.thr[r] = lo;
               if (!(rank < k_top)) sm.rs.tokz[r] = CSD_NEG_INF;   // the exact filter drops the drafted token
             }
-            if (!ok) sm.short_on = 0;
+            // (a single row can fail -- a row maximum on the low side leaves the bound short -- without the
+            // next ones doing so; rows that are flat keep failing, and after three such the block stops trying)
+            if (!ok && ++sm.short_fail >= 3) sm.short_on = 0;
             sm.row_short = ok ? 1 : 0;
           }
         }
