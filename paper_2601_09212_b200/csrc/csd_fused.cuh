@@ -1696,7 +1696,7 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
       // ---- the short cut: no threshold at all --------------------------------------------------
       // If a level `hi` a little above lo has fewer than k values above it, the k-th largest value lies
       // in [lo, hi], and the values the filter drops among those gathered all lie there too.  Where
-      // their total weight -- at most (their number) * exp(hi - max) -- is below 2^-26 of the row's
+      // their total weight -- at most (gathered - k) * exp(hi - max) -- is below 2^-26 of the row's
       // normaliser, dropping them or not changes nothing that fp32 can see: the row's (m, s) is that
       // of ALL gathered values, lo itself serves as the threshold from here on (for the draw's filter
       // and the diagnostics: what it lets through beyond the exact filter has weight below 1e-7 of an
@@ -1754,7 +1754,9 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
             stat_merge(m, sv, m2, s2);
           }
           if (lane == 0) {
-            const float dropped = (float)(n_lo - cg) * ex2f((hi - m) * kLog2e);   // bound on what the filter removes
+            // bound on what the filter removes: at least k of the gathered values are kept, and with fewer than k
+            // values above hi every one it removes lies at or below hi
+            const float dropped = (float)(n_lo - k_top) * ex2f((hi - m) * kLog2e);
             const bool ok = !over && !nan_m && n_lo >= k_top && cg < k_top && m > lo && m < CSD_POS_INF &&
                             sv >= 0.0f && sv < CSD_POS_INF && dropped <= 1.4901161e-8f;
             if (ok && r < kBlockRows) {
