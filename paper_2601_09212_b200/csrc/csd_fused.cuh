@@ -347,10 +347,16 @@ __device__ int draw_token(const FinishArgs& a, const Row<T, CFG>& rt, const Row<
                 cfg_mix_vec<VEC>(zd, zu, a.cfg_scale);
               }
             }
-            float acc = 0.0f;
+            float acc = 0.0f;   // (summed in the order of the scalar form)
 #pragma unroll
-            for (int k = 0; k < VEC; ++k)
-              acc += weight_of(FILT ? rt.filter(zt[k]) : zt[k], ctx.mode == 0 ? (FILT ? rd.filter(zd[k]) : zd[k]) : 0.0f, ctx);
+            for (int k = 0; k < VEC; k += 2) {
+              float g0, g1;
+              weight_of_pair(FILT ? rt.filter(zt[k]) : zt[k], FILT ? rt.filter(zt[k + 1]) : zt[k + 1],
+                             ctx.mode == 0 ? (FILT ? rd.filter(zd[k]) : zd[k]) : 0.0f,
+                             ctx.mode == 0 ? (FILT ? rd.filter(zd[k + 1]) : zd[k + 1]) : 0.0f, ctx, g0, g1);
+              acc += g0;
+              acc += g1;
+            }
             acc2[r] = acc;
           }
         }
@@ -758,8 +764,14 @@ __device__ void cluster_draw(const FusedArgs& ua, const BlockShare& sh, int j, c
         if (tile < t_end) {
           float acc = 0.0f;
 #pragma unroll
-          for (int e = 0; e < VEC; ++e)
-            acc += weight_of(FILT ? rt.filter(zt[r][e]) : zt[r][e], ctx.mode == 0 ? (FILT ? rd.filter(zd[r][e]) : zd[r][e]) : 0.0f, ctx);
+          for (int e = 0; e < VEC; e += 2) {
+            float g0, g1;
+            weight_of_pair(FILT ? rt.filter(zt[r][e]) : zt[r][e], FILT ? rt.filter(zt[r][e + 1]) : zt[r][e + 1],
+                           ctx.mode == 0 ? (FILT ? rd.filter(zd[r][e]) : zd[r][e]) : 0.0f,
+                           ctx.mode == 0 ? (FILT ? rd.filter(zd[r][e + 1]) : zd[r][e + 1]) : 0.0f, ctx, g0, g1);
+            acc += g0;
+            acc += g1;
+          }
 #pragma unroll
           for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
           if (lane == 0) cluster_store_f64(&tile_sums[tile], (uint32_t)owner, (double)acc);

@@ -166,6 +166,11 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 // cfg_mix of VEC values in pairs: c - u as fma(u, -1, c) (one rounding, like the subtraction)
 template <int VEC>
 __device__ __forceinline__ void cfg_mix_vec(float (&c)[VEC], const float (&u)[VEC], float s) {
@@ -514,6 +519,30 @@ __device__ __forceinline__ float weight_of(float zt, float zd, const PairCtx& c)
   const float pq = __fmul_rn(__fadd_rn(__fsub_rn(et, ed), __fsub_rn(__fmul_rn(et, c.Sd), __fmul_rn(ed, c.St))), c.inv_den);
   const float alt = c.one_minus_omega * et * c.inv_t;                    // (1 - omega) P
   return fmaxf(0.0f, fmaxf(pq, alt));
+}
+
+// weight_of for two candidates at once, two values per instruction: the same operations in the same
+// order, each half the IEEE operation, so the results are weight_of's bit for bit (a - b is taken as
+// fma(b, -1, a), which rounds once like the subtraction).
+__device__ __forceinline__ void weight_of_pair(float zt0, float zt1, float zd0, float zd1, const PairCtx& c, float& g0, float& g1) {
+  const uint64_t l2e = pack2(kLog2e, kLog2e), m1 = pack2(-1.0f, -1.0f);
+  float xt0, xt1;
+  unpack2(mul2(add2(pack2(zt0, zt1), pack2(-c.Mt, -c.Mt)), l2e), xt0, xt1);
+  const uint64_t et = pack2(ex2f(xt0), ex2f(xt1));
+  if (c.mode == 1) {
+    unpack2(mul2(et, pack2(c.inv_t, c.inv_t)), g0, g1);
+    return;
+  }
+  float xd0, xd1;
+  unpack2(mul2(add2(pack2(zd0, zd1), pack2(-c.Md, -c.Md)), l2e), xd0, xd1);
+  const uint64_t ed = pack2(ex2f(xd0), ex2f(xd1));
+  const uint64_t diff = fma2(ed, m1, et);                                                   // et - ed
+  const uint64_t cross = fma2(mul2(ed, pack2(c.St, c.St)), m1, mul2(et, pack2(c.Sd, c.Sd)));   // et Sd - ed St
+  float pq0, pq1, a0, a1;
+  unpack2(mul2(add2(diff, cross), pack2(c.inv_den, c.inv_den)), pq0, pq1);
+  unpack2(mul2(mul2(pack2(c.one_minus_omega, c.one_minus_omega), et), pack2(c.inv_t, c.inv_t)), a0, a1);
+  g0 = fmaxf(0.0f, fmaxf(pq0, a0));
+  g1 = fmaxf(0.0f, fmaxf(pq1, a1));
 }
 
 // Similarity relaxation (LANTERN++'s P^{k,lambda} at the candidate): the target mass of the selected
