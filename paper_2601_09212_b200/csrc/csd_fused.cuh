@@ -1007,10 +1007,6 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
   // the block's items (parts of its local rows, see block_share), split evenly over its warps
   const BlockShare sh = block_share(a);
   const bool stats_only = a.stats_out != nullptr;
-  if (!stats_only) {
-    stage_inputs(a, sh, 0, tid, sm.fst);
-    load_token_logits<T, CFG, kPlainThreads>(f, sh, tid, sm.rs);
-  }
   const int n_block = sh.n_rows * parts;
   const int item_begin = (int)((long long)n_block * warp / kPlainWarps);
   const int item_end = (int)((long long)n_block * (warp + 1) / kPlainWarps);
@@ -1055,6 +1051,12 @@ __global__ void __launch_bounds__(kPlainThreads, 3) verify_plain_kernel(const Fu
     producer_open_row();
     producer_open_item();
     for (int s = 0; s < kWStages; ++s) producer_issue();
+  }
+  // (the first copies are under way: the block's small inputs and the drafted tokens' logits -- two dependent
+  // trips to memory -- are fetched in their shadow)
+  if (!stats_only) {
+    stage_inputs(a, sh, 0, tid, sm.fst);
+    load_token_logits<T, CFG, kPlainThreads>(f, sh, tid, sm.rs);
   }
 
   // ================================= phase 1 ===========================================
@@ -1507,12 +1509,6 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   // this block's local rows (see block_share)
   const BlockShare sh = block_share(a);
   const bool stats_only = a.stats_out != nullptr;
-  if (!stats_only) {
-    stage_inputs(a, sh, 0, tid, sm.fst);
-    load_token_logits<T, CFG, kTopkThreads>(f, sh, tid, sm.rs);
-  } else {
-    for (int r = tid; r < kBlockRows; r += kTopkThreads) sm.rs.tokz[r] = 0.0f;   // (read by the short cut's rank, unused here)
-  }
   const int n_rows = sh.n_rows;
   const int n_chunks = n_rows * cpr;
 
@@ -1539,6 +1535,14 @@ __global__ void __launch_bounds__(kTopkThreads, 4) verify_topk_kernel(const Fuse
   if (tid == 0) {
     issue_chunk(0);
     issue_chunk(1);
+  }
+  // (the first copies are under way: the block's small inputs and the drafted tokens' logits -- two dependent
+  // trips to memory -- are fetched in their shadow)
+  if (!stats_only) {
+    stage_inputs(a, sh, 0, tid, sm.fst);
+    load_token_logits<T, CFG, kTopkThreads>(f, sh, tid, sm.rs);
+  } else {
+    for (int r = tid; r < kBlockRows; r += kTopkThreads) sm.rs.tokz[r] = 0.0f;   // (read by the short cut's rank, unused here)
   }
 
   // ================================= phase 1 ===========================================
